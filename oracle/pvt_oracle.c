@@ -1,0 +1,376 @@
+/*
+ * CPU checker for the discrete V step of PV-Tuning.  TEST INFRASTRUCTURE ONLY:
+ * it defines what the GPU library must compute, it is deliberately plain and
+ * slow, and it shares no code with the CUDA path.  Only the tests, the smoke
+ * check and the benchmark's CPU-baseline leg may call it.
+ *
+ * Every function follows one passage of the paper:
+ *   - group update norm and arg-top-tau choice: Algorithm 2 ("find tau
+ *     largest"), Section 3.4 ("largest update norm within each weight matrix"),
+ *     Algorithm 3 ("choose_subspace(update, tau)");
+ *   - target of the search: Eq. (8), y - (1/L) Z(grad phi(y)), in the scaled
+ *     space of the codebooks (Appendix J, "per-channel trainable scales");
+ *   - M = 1 search: Appendix C / Appendix J ("try every code in the codebook
+ *     and choose the one that minimises" the squared error);
+ *   - M >= 2 search: Appendix C / Appendix J (beam search, beam size 8, target =
+ *     gradient-updated dequantised weight), greedy residual form;
+ *   - untouched codes outside the subspace: Section 3.3 (x+_i = y_i for i not
+ *     in S^k);
+ *   - dequantisation: Algorithm 3 ("dequantize_weights").
+ *
+ * Arithmetic: the norm, the target and the dequantised weight are sequences of
+ * single IEEE binary32 operations (stated at each function) so that a GPU can
+ * reproduce them bit for bit; every distance is accumulated in binary64.
+ * Build with -O2 -ffp-contract=off: no operation may be fused except the
+ * explicit fmaf calls.
+ *
+ * Pins (tests marked "not gpu"): the paper's two printed assignment examples,
+ * brute-force enumeration of every code tuple on tiny inputs, a library
+ * nearest-centroid routine (the V step with phi = ||x - z||^2 is the K-means
+ * assignment step, Section 3.1), the expansion ||x-B||^2 = ||x||^2 - 2<x,B> +
+ * ||B||^2 (Appendix D), beam >= K equals exhaustive search, beam = 1 equals
+ * greedy residual quantisation, zero second codebook reduces to M = 1,
+ * monotonicity (Lemma 3.3), locality, fixed point, full-sort selection with
+ * crafted ties, closed-form dequantisation.  No end-to-end V-step result on a
+ * real layer is printed in the paper, so beyond these pins parity is unpinned.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define PVT_ORACLE_MAX_M 4
+#define PVT_ORACLE_MAX_BEAM 4096
+
+int pvt_oracle_num_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+void pvt_oracle_set_num_threads(int n) {
+#ifdef _OPENMP
+  if (n > 0) omp_set_num_threads(n);
+#else
+  (void)n;
+#endif
+}
+
+/* Squared norm of the update eta*g of every weight group (Algorithm 2; Section
+ * 3.4).  binary32: u_i = eta*g_i rounded once; acc = fmaf(u_i, u_i, acc) for i
+ * in index order starting from 0. */
+void pvt_oracle_group_norms(const float* g, int64_t rows, int64_t cols, int32_t dg, float eta,
+                            float* norms) {
+  const int64_t gpr = cols / dg;
+#pragma omp parallel for schedule(static)
+  for (int64_t j = 0; j < rows * gpr; ++j) {
+    const int64_t r = j / gpr, c = j % gpr;
+    const float* gj = g + r * cols + c * dg;
+    float acc = 0.0f;
+    for (int32_t i = 0; i < dg; ++i) {
+      const float u = eta * gj[i];
+      acc = fmaf(u, u, acc);
+    }
+    norms[j] = acc;
+  }
+}
+
+typedef struct {
+  float n;
+  uint32_t j;
+} norm_entry;
+
+static int by_norm_desc_then_index(const void* a, const void* b) {
+  const norm_entry* x = (const norm_entry*)a;
+  const norm_entry* y = (const norm_entry*)b;
+  if (x->n > y->n) return -1;
+  if (x->n < y->n) return 1;
+  if (x->j < y->j) return -1;
+  if (x->j > y->j) return 1;
+  return 0;
+}
+
+static int by_u32(const void* a, const void* b) {
+  const uint32_t x = *(const uint32_t*)a, y = *(const uint32_t*)b;
+  return (x > y) - (x < y);
+}
+
+/* arg top-k (Algorithm 2): order all groups by (norm descending, index
+ * ascending), keep the first k, return them in ascending index order.
+ * Returns 0, or -1 on a bad argument / non-finite norm. */
+int pvt_oracle_select(const float* norms, int64_t G, int64_t k, uint32_t* idx_out) {
+  if (k < 1 || k > G || G >= ((int64_t)1 << 32)) return -1;
+  norm_entry* e = (norm_entry*)malloc((size_t)G * sizeof(norm_entry));
+  if (!e) return -1;
+  for (int64_t j = 0; j < G; ++j) {
+    if (!isfinite(norms[j]) || norms[j] < 0.0f) {
+      free(e);
+      return -1;
+    }
+    e[j].n = norms[j];
+    e[j].j = (uint32_t)j;
+  }
+  qsort(e, (size_t)G, sizeof(norm_entry), by_norm_desc_then_index);
+  for (int64_t i = 0; i < k; ++i) idx_out[i] = e[i].j;
+  free(e);
+  qsort(idx_out, (size_t)k, sizeof(uint32_t), by_u32);
+  return 0;
+}
+
+/* Target of the search for the selected groups (Eq. 8, scaled space):
+ * t_i = (W_i - eta*g_i) / s_row, binary32: one fmaf(-eta, g_i, W_i), one
+ * division. */
+void pvt_oracle_targets(const float* W, const float* g, const float* scale, int64_t rows,
+                        int64_t cols, int32_t dg, float eta, const uint32_t* idx, int64_t k,
+                        float* t_out) {
+  (void)rows;
+  const int64_t gpr = cols / dg;
+#pragma omp parallel for schedule(static)
+  for (int64_t n = 0; n < k; ++n) {
+    const int64_t j = idx[n], r = j / gpr, c = j % gpr;
+    const float* Wj = W + r * cols + c * dg;
+    const float* gj = g + r * cols + c * dg;
+    for (int32_t i = 0; i < dg; ++i) t_out[n * dg + i] = fmaf(-eta, gj[i], Wj[i]) / scale[r];
+  }
+}
+
+/* ||r - c||^2 in binary64, terms added in index order. */
+static double sqdist(const double* r, const float* c, int32_t dg) {
+  double d = 0.0;
+  for (int32_t i = 0; i < dg; ++i) {
+    const double e = r[i] - (double)c[i];
+    d = d + e * e;
+  }
+  return d;
+}
+
+typedef struct {
+  double d;                       /* ||t - sum of chosen codewords||^2 */
+  int32_t code[PVT_ORACLE_MAX_M]; /* chosen codeword per codebook so far */
+} beam_entry;
+
+/* (distance, code tuple) lexicographic order over the first m codes */
+static int entry_less(const beam_entry* a, const beam_entry* b, int32_t m) {
+  if (a->d < b->d) return 1;
+  if (a->d > b->d) return 0;
+  for (int32_t i = 0; i < m; ++i) {
+    if (a->code[i] < b->code[i]) return 1;
+    if (a->code[i] > b->code[i]) return 0;
+  }
+  return 0;
+}
+
+static void residual_of(const float* t, const float* books, int32_t dg, int32_t K,
+                        const int32_t* code, int32_t m, double* r) {
+  for (int32_t i = 0; i < dg; ++i) r[i] = (double)t[i];
+  for (int32_t q = 0; q < m; ++q) {
+    const float* c = books + ((int64_t)q * K + code[q]) * dg;
+    for (int32_t i = 0; i < dg; ++i) r[i] = r[i] - (double)c[i];
+  }
+}
+
+/* M = 1 (Appendix C / Appendix J): every codeword of the codebook is tried;
+ * the result is the argmin of (||t - c||^2, code).  *d2 receives the smallest
+ * distance over the other codewords. */
+static void search_single(const float* t, int32_t dg, int32_t K, const float* book, int32_t* code,
+                          double* d1, double* d2) {
+  double r[64];
+  for (int32_t i = 0; i < dg; ++i) r[i] = (double)t[i];
+  int32_t arg = 0;
+  double best = sqdist(r, book, dg), second = INFINITY;
+  for (int32_t q = 1; q < K; ++q) {
+    const double d = sqdist(r, book + (int64_t)q * dg, dg);
+    if (d < best) { /* strict: equal distances keep the lower code */
+      second = best;
+      best = d;
+      arg = q;
+    } else if (d < second) {
+      second = d;
+    }
+  }
+  *code = arg;
+  *d1 = best;
+  *d2 = (K > 1) ? second : best;
+}
+
+/* M >= 2 (Appendix C / Appendix J: beam search, target = gradient-updated
+ * dequantised weight), greedy residual form.  Stage m extends each kept partial
+ * tuple by every codeword of codebook m and scores ||t - c^1 - ... - c^m||^2 with
+ * the residual carried in binary64.  After stages 1..M-1 the `beam` best partial
+ * tuples under (distance, tuple) are kept.  The final pool is every extension
+ * made at the last stage plus the previous tuple, so the result is never worse
+ * than the previous code (Lemma 3.3); result = argmin of (distance, tuple).
+ * Returns 0, -1 on allocation failure or an out-of-range previous code. */
+static int search_beam(const float* t, int32_t dg, int32_t M, int32_t K, const float* books,
+                       int32_t beam, const int32_t* prev, int32_t* code, double* d1, double* d2,
+                       double* gap_in, double* gap_out) {
+  double r[64];
+  int have_gap = 0;
+  int64_t nkept = 1; /* the single empty tuple */
+  beam_entry* kept = (beam_entry*)calloc(1, sizeof(beam_entry));
+  beam_entry* cand = NULL;
+  if (!kept) return -1;
+  for (int32_t m = 0; m < M; ++m) {
+    const int64_t ncand = nkept * K;
+    cand = (beam_entry*)malloc((size_t)ncand * sizeof(beam_entry));
+    if (!cand) {
+      free(kept);
+      return -1;
+    }
+    for (int64_t b = 0; b < nkept; ++b) {
+      residual_of(t, books, dg, K, kept[b].code, m, r);
+      for (int32_t q = 0; q < K; ++q) {
+        beam_entry* e = &cand[b * K + q];
+        *e = kept[b];
+        e->code[m] = q;
+        e->d = sqdist(r, books + ((int64_t)m * K + q) * dg, dg);
+      }
+    }
+    free(kept);
+    kept = NULL;
+    if (m == M - 1) break;
+    /* keep the `beam` best: selection by repeated minimum, one extra round to
+     * learn the first dropped tuple */
+    const int64_t nkeep = ncand < beam ? ncand : beam;
+    kept = (beam_entry*)malloc((size_t)(nkeep + 1) * sizeof(beam_entry));
+    if (!kept) {
+      free(cand);
+      return -1;
+    }
+    for (int64_t s = 0; s <= nkeep && s < ncand; ++s) {
+      int64_t arg = s;
+      for (int64_t c = s + 1; c < ncand; ++c)
+        if (entry_less(&cand[c], &cand[arg], m + 1)) arg = c;
+      const beam_entry tmp = cand[s];
+      cand[s] = cand[arg];
+      cand[arg] = tmp;
+      kept[s] = cand[s];
+    }
+    if (nkeep < ncand) {
+      const double din = kept[nkeep - 1].d, dout = kept[nkeep].d;
+      if (!have_gap || (dout - din) * (*gap_out) < (*gap_out - *gap_in) * dout) {
+        *gap_in = din;
+        *gap_out = dout;
+        have_gap = 1;
+      }
+    }
+    nkept = nkeep;
+    free(cand);
+    cand = NULL;
+  }
+
+  /* final pool */
+  const int64_t npool = nkept * K;
+  beam_entry best = cand[0], second = cand[0];
+  int have_second = 0;
+  for (int64_t c = 1; c < npool; ++c) {
+    if (entry_less(&cand[c], &best, M)) {
+      second = best;
+      have_second = 1;
+      best = cand[c];
+    } else if (!have_second || entry_less(&cand[c], &second, M)) {
+      second = cand[c];
+      have_second = 1;
+    }
+  }
+  beam_entry p;
+  memset(&p, 0, sizeof p);
+  int in_pool = 0, ok = 1;
+  for (int32_t q = 0; q < M; ++q) {
+    p.code[q] = prev[q];
+    if (prev[q] < 0 || prev[q] >= K) ok = 0;
+  }
+  if (ok) {
+    for (int64_t c = 0; c < npool && !in_pool; ++c) {
+      int same = 1;
+      for (int32_t q = 0; q < M; ++q) same = same && cand[c].code[q] == p.code[q];
+      in_pool = same;
+    }
+    if (!in_pool) {
+      residual_of(t, books, dg, K, p.code, M - 1, r);
+      p.d = sqdist(r, books + ((int64_t)(M - 1) * K + p.code[M - 1]) * dg, dg);
+      if (entry_less(&p, &best, M)) {
+        second = best;
+        have_second = 1;
+        best = p;
+      } else if (!have_second || entry_less(&p, &second, M)) {
+        second = p;
+        have_second = 1;
+      }
+    }
+  }
+  free(cand);
+  if (!ok) return -1;
+  for (int32_t q = 0; q < M; ++q) code[q] = best.code[q];
+  *d1 = best.d;
+  *d2 = have_second ? second.d : best.d;
+  if (!have_gap) {
+    *gap_in = best.d;
+    *gap_out = best.d;
+  }
+  return 0;
+}
+
+/* Nearest-codeword search for k targets t [k][dg].
+ * books: [M][K][dg] binary32 (fp16 codebooks widened exactly by the caller).
+ * prev, codes_out: [k][M].  d_best/d_second: smallest and second-smallest
+ * distance over the final pool (second: over pool members other than the
+ * winner).  bd_in/bd_out (may be NULL): distances of the last kept and the first
+ * dropped partial tuple at the beam stage where their gap is relatively
+ * smallest (both d_best when nothing is dropped).
+ * Returns 0, or -1 on bad arguments. */
+int pvt_oracle_encode(const float* t, int64_t k, int32_t dg, int32_t M, int32_t K,
+                      const float* books, int32_t beam, const int32_t* prev, int32_t* codes_out,
+                      double* d_best, double* d_second, double* bd_in, double* bd_out) {
+  if (M < 1 || M > PVT_ORACLE_MAX_M || K < 1 || dg < 1 || dg > 64) return -1;
+  if (M > 1 && (beam < 1 || beam > PVT_ORACLE_MAX_BEAM)) return -1;
+  int bad = 0;
+#pragma omp parallel for schedule(dynamic, 16)
+  for (int64_t n = 0; n < k; ++n) {
+    double gi = 0.0, go = 0.0;
+    if (M == 1) {
+      search_single(t + n * dg, dg, K, books, &codes_out[n], &d_best[n], &d_second[n]);
+      gi = go = d_best[n];
+    } else if (search_beam(t + n * dg, dg, M, K, books, beam, prev + n * M, codes_out + n * M,
+                           &d_best[n], &d_second[n], &gi, &go) != 0) {
+      bad = 1;
+    }
+    if (bd_in) bd_in[n] = gi;
+    if (bd_out) bd_out[n] = go;
+  }
+  return bad ? -1 : 0;
+}
+
+/* Squared error ||t - sum_m C_m[code_m]||^2 in binary64 for given code tuples
+ * (the same accumulation order as the search). */
+void pvt_oracle_tuple_error(const float* t, int64_t k, int32_t dg, int32_t M, int32_t K,
+                            const float* books, const int32_t* codes, double* d_out) {
+#pragma omp parallel for schedule(static)
+  for (int64_t n = 0; n < k; ++n) {
+    double r[64];
+    residual_of(t + n * dg, books, dg, K, codes + n * M, M - 1, r);
+    d_out[n] = sqdist(r, books + ((int64_t)(M - 1) * K + codes[n * M + M - 1]) * dg, dg);
+  }
+}
+
+/* W_hat = s_row * sum_m C_m[b_m] (Algorithm 3, dequantize_weights).  binary32:
+ * codewords added left to right, each addition rounded once, then one
+ * multiplication by the row scale. */
+void pvt_oracle_dequant(const int32_t* codes, const float* books, const float* scale, int64_t rows,
+                        int64_t cols, int32_t dg, int32_t M, int32_t K, float* W_hat) {
+  const int64_t gpr = cols / dg;
+#pragma omp parallel for schedule(static)
+  for (int64_t j = 0; j < rows * gpr; ++j) {
+    const int64_t r = j / gpr, c = j % gpr;
+    for (int32_t i = 0; i < dg; ++i) {
+      float v = books[((int64_t)0 * K + codes[j * M]) * dg + i];
+      for (int32_t q = 1; q < M; ++q) v = v + books[((int64_t)q * K + codes[j * M + q]) * dg + i];
+      W_hat[r * cols + c * dg + i] = scale[r] * v;
+    }
+  }
+}
