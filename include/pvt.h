@@ -1,0 +1,179 @@
+/*
+ * pvt.h -- C ABI of the B200 (sm_100a) library for the discrete "V step" of
+ * PV-Tuning on one vector-quantised linear layer.
+ *
+ * One training step of the method (Algorithm 3) dequantises the model, runs
+ * forward/backward passes to accumulate the dense gradient of every linear
+ * weight, updates the continuous parameters (P step) and then updates the
+ * discrete codes (V step):
+ *
+ *     update = W - eta * g                  (Eq. 8: y - (1/L_S) Z(grad phi(y)))
+ *     S      = choose_subspace(update, tau) (Algorithm 2: arg top-tau; Section
+ *                                            3.4: largest update norm per matrix)
+ *     codes[S] = find_nearest(update[S])    (Appendix C / Appendix J: try every
+ *                                            code, or beam search for additive
+ *                                            codebooks; codes outside S stay,
+ *                                            Section 3.3)
+ *
+ * and the next step starts with dequantize_weights (Algorithm 3, first line).
+ * This library is those three calls.
+ *
+ * Conventions
+ *   - A layer is `rows x cols`, row-major.  Weight groups are `group_dim` = 8
+ *     consecutive elements of a row (input dimension); group j = r * (cols/8) + c
+ *     covers W[r, 8c .. 8c+7].  G = rows * cols / 8 groups, G < 2^32.
+ *   - Every pointer is DEVICE memory owned by the caller (16-byte aligned where
+ *     stated).  The library allocates nothing and keeps no state between calls.
+ *   - Every call only enqueues work on `cuda_stream` (a cudaStream_t passed as
+ *     void*; NULL = the legacy default stream) and returns without synchronising,
+ *     except pvt_status.  Calls on one stream execute in order.
+ *   - Return value: PVT_OK (0) = enqueued; negative = rejected before anything
+ *     was enqueued (see the error codes).  No C++ exception crosses this ABI.
+ *   - Device-side problems never trap: the kernel records a PVT_DEV_* bit in the
+ *     status word at the start of the workspace, skips the offending item and
+ *     returns.  Read it with pvt_status.
+ */
+#ifndef PVT_H_
+#define PVT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* element types */
+#define PVT_F32 0
+#define PVT_F16 1
+#define PVT_U8 0
+#define PVT_U16 1
+
+/* host-side return codes */
+#define PVT_OK 0
+#define PVT_EINVAL (-1)       /* null / misaligned pointer, k = 0, k > G, cols % 8 != 0, G >= 2^32, bad eta */
+#define PVT_EUNSUPPORTED (-2) /* group_dim / M / K / dtype / beam combination this build has no kernel for */
+#define PVT_EWORKSPACE (-3)   /* ws_bytes smaller than pvt_workspace_bytes() */
+#define PVT_ECUDA (-4)        /* a CUDA runtime call or kernel launch failed; see pvt_last_cuda_error() */
+
+/* device-side status bits (pvt_status) */
+#define PVT_DEV_BAD_INDEX 1u    /* an entry of idx was >= G; that entry was skipped */
+#define PVT_DEV_BAD_CODE 2u     /* a stored code was >= K; treated as code 0 (dequant) or left out of the pool */
+#define PVT_DEV_WAIT_EXPIRED 4u /* a bounded wait on an on-chip barrier ran out; results of the call are invalid */
+#define PVT_DEV_INTERNAL 8u     /* an internal consistency check failed (selection count mismatch) */
+
+/*
+ * One quantised linear layer and the update direction of this step.
+ * Representation (Appendix J): M codebooks of K codewords of group_dim values
+ * each, one code per group and codebook, per-output-channel scale:
+ *     W_hat[r, 8c + i] = scale[r] * sum_m codebooks[m][codes[j][m]][i].
+ * Supported: group_dim 8; M = 1 with 2 <= K <= 65536 (codes U8 if K <= 256, else
+ * U16; U16 is accepted for any K); M = 2 with 2 <= K <= 256, codes U8, 1 <= beam
+ * <= 8.
+ */
+typedef struct pvt_layer {
+  int32_t rows, cols;     /* cols % group_dim == 0 */
+  int32_t group_dim;      /* 8 */
+  int32_t num_codebooks;  /* M */
+  int32_t codebook_size;  /* K */
+  int32_t codebook_dtype; /* PVT_F32 | PVT_F16 */
+  int32_t code_dtype;     /* PVT_U8 | PVT_U16 */
+  int32_t beam;           /* beam width of the M = 2 search; ignored for M = 1 */
+  float eta;              /* step size 1/L_S of Eq. 8; finite, >= 0 */
+  int32_t reserved_;      /* set to 0 */
+  const float* W;         /* [rows][cols] current dense weight y (16-byte aligned) */
+  const float* g;         /* [rows][cols] update direction: gradient or optimiser update (16-byte aligned) */
+  const float* scale;     /* [rows] finite, non-zero (not validated) */
+  const void* codebooks;  /* [M][K][group_dim] (16-byte aligned) */
+  void* codes;            /* [G][M]; read (previous codes) and overwritten in place by pvt_vstep_encode */
+} pvt_layer;
+
+/*
+ * Bytes of scratch that pvt_vstep_select / pvt_vstep_encode need for this layer
+ * and this k (the larger of the two needs).  Returns 0 if the layer or k is
+ * invalid.  The workspace must be 256-byte aligned; its first 256 bytes hold the
+ * status word and must be cleared once with pvt_workspace_init before first use.
+ */
+size_t pvt_workspace_bytes(const pvt_layer* layer, uint64_t k);
+
+/* Clears the status word of a fresh workspace (enqueued on the stream). */
+int pvt_workspace_init(void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Subspace choice (Algorithm 2, "arg top tau"; Section 3.4, "largest update norm
+ * within each weight matrix"; Algorithm 3, choose_subspace).
+ *   n_j = ||eta * g_j||^2 per group, in binary32: u_i = eta*g_i rounded once,
+ *   acc = fma(u_i, u_i, acc) for i = 0..7 from acc = 0.
+ *   idx_out[0..k) = the k groups with the largest n_j, ties at the threshold
+ *   resolved towards the lowest group index, written in ascending order.
+ * Reads layer->g, rows, cols, eta only.  idx_out: device, k uint32.
+ * k is a count (1 <= k <= G); a fraction tau maps to k = max(1, floor(tau*G)).
+ */
+int pvt_vstep_select(const pvt_layer* layer, uint64_t k, uint32_t* idx_out, void* ws, size_t ws_bytes,
+                     void* cuda_stream);
+
+/*
+ * Re-encode the k groups listed in idx (Eq. 8; Appendix C / Appendix J;
+ * Appendix D for the score ||c||^2 - 2 <t, c>).
+ *   target (binary32): t_i = fma(-eta, g_i, W_i) / scale[r].
+ *   M = 1: codes[j] = argmin over all K codewords of (||t - c||^2, code).
+ *   M = 2: greedy residual beam search: the `beam` codewords of codebook 1
+ *          nearest to t under (distance, code); each is extended by every
+ *          codeword of codebook 2; the pool is those beam*K pairs plus the
+ *          previous pair; codes[j] = argmin of (||t - c1 - c2||^2, code1, code2).
+ *   A fast binary32 score shortlists candidates; the decision among shortlisted
+ *   candidates is taken on binary64 distances sum_i (t_i - c_i)^2 accumulated in
+ *   index order, so ties break exactly as stated above.
+ *   Groups not in idx keep their codes bit for bit.
+ * idx: device, k uint32, each < G, no duplicates (duplicates race benignly: the
+ * same value is written twice).  err_out: device, k floats or NULL; receives the
+ * new squared error in the scaled space, rounded to binary32.
+ */
+int pvt_vstep_encode(const pvt_layer* layer, const uint32_t* idx, uint64_t k, float* err_out, void* ws,
+                     size_t ws_bytes, void* cuda_stream);
+
+/*
+ * dequantize_weights (Algorithm 3, first line): for every group
+ *   W_hat[r, 8c+i] = scale[r] * (C_1[b_1][i] (+ C_2[b_2][i]))   in binary32, the
+ *   sum rounded once, then the product rounded once; out_dtype PVT_F16 rounds that
+ *   binary32 value to nearest-even binary16.
+ * W_hat: device, rows x cols of out_dtype, 16-byte aligned.  `status` may be NULL
+ * or a device uint32 into which PVT_DEV_BAD_CODE is OR-ed.
+ */
+int pvt_dequant(const pvt_layer* layer, void* W_hat, int32_t out_dtype, uint32_t* status, void* cuda_stream);
+
+/*
+ * Synchronises the stream, returns the PVT_DEV_* bits accumulated in the
+ * workspace since the last pvt_status / pvt_workspace_init (>= 0) and clears them;
+ * or PVT_ECUDA.
+ */
+int pvt_status(void* ws, void* cuda_stream);
+
+/* Text for a host-side return code. */
+const char* pvt_strerror(int code);
+
+/* Text of the CUDA error behind the most recent PVT_ECUDA on this thread. */
+const char* pvt_last_cuda_error(void);
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int pvt_version(void);
+
+/*
+ * Benchmark instrumentation (no counterpart in the paper).  While enabled, every
+ * call brackets its kernels with CUDA events on the caller's stream;
+ * pvt_timing_read waits for the recorded events of one kernel class, returns
+ * their summed duration and count, and forgets them.
+ */
+#define PVT_KERNEL_SELECT 0      /* all kernels of pvt_vstep_select */
+#define PVT_KERNEL_ENCODE_MAIN 1 /* the search kernel of pvt_vstep_encode */
+#define PVT_KERNEL_ENCODE_AUX 2  /* codebook expansion before the M = 1 search */
+#define PVT_KERNEL_DEQUANT 3     /* the kernel of pvt_dequant */
+void pvt_timing_enable(int on);
+/* Kernels this process has launched through the library so far (memsets not counted). */
+unsigned long long pvt_launch_count(void);
+int pvt_timing_read(int kernel_id, float* total_ms, int* launches);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PVT_H_ */

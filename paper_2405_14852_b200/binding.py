@@ -1,0 +1,185 @@
+"""ctypes binding of libpvt.so: argument marshalling only.
+
+Every step of the V step (norms, selection, target formation, search, code
+write, dequantisation) runs in the CUDA kernels behind the C ABI declared in
+``include/pvt.h``; this module only turns torch tensors into pointers and sizes.
+There is no CPU fallback: if the library cannot be loaded, or a call is rejected,
+an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+from . import build as _build
+
+PVT_F32, PVT_F16 = 0, 1
+PVT_U8, PVT_U16 = 0, 1
+PVT_OK, PVT_EINVAL, PVT_EUNSUPPORTED, PVT_EWORKSPACE, PVT_ECUDA = 0, -1, -2, -3, -4
+PVT_DEV_BAD_INDEX, PVT_DEV_BAD_CODE, PVT_DEV_WAIT_EXPIRED, PVT_DEV_INTERNAL = 1, 2, 4, 8
+PVT_KERNEL_SELECT, PVT_KERNEL_ENCODE_MAIN, PVT_KERNEL_ENCODE_AUX, PVT_KERNEL_DEQUANT = 0, 1, 2, 3
+
+
+class pvt_layer(ctypes.Structure):
+    _fields_ = [
+        ("rows", ctypes.c_int32), ("cols", ctypes.c_int32), ("group_dim", ctypes.c_int32),
+        ("num_codebooks", ctypes.c_int32), ("codebook_size", ctypes.c_int32),
+        ("codebook_dtype", ctypes.c_int32), ("code_dtype", ctypes.c_int32), ("beam", ctypes.c_int32),
+        ("eta", ctypes.c_float), ("reserved_", ctypes.c_int32),
+        ("W", ctypes.c_void_p), ("g", ctypes.c_void_p), ("scale", ctypes.c_void_p),
+        ("codebooks", ctypes.c_void_p), ("codes", ctypes.c_void_p),
+    ]
+
+
+class PvtError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: {strerror(code)} (code {code})" + (f": {last_cuda_error()}" if code == PVT_ECUDA else ""))
+        self.code = code
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _build.LIB
+
+
+def lib():
+    """The loaded C library.  Builds it in-tree if nvcc is available and the
+    shared object is missing or stale; raises if it cannot be loaded."""
+    global _lib
+    if _lib is None:
+        path = library_path()
+        if _build.needs_build():
+            try:
+                _build.build()
+            except Exception as exc:  # no compiler on this machine: use the shipped object if there is one
+                if not os.path.exists(path):
+                    raise RuntimeError(f"libpvt.so is missing and could not be built: {exc}") from exc
+        L = ctypes.CDLL(path)
+        vp, u64, sz = ctypes.c_void_p, ctypes.c_uint64, ctypes.c_size_t
+        lp = ctypes.POINTER(pvt_layer)
+        L.pvt_workspace_bytes.restype = sz
+        L.pvt_workspace_bytes.argtypes = [lp, u64]
+        L.pvt_workspace_init.restype = ctypes.c_int
+        L.pvt_workspace_init.argtypes = [vp, sz, vp]
+        L.pvt_vstep_select.restype = ctypes.c_int
+        L.pvt_vstep_select.argtypes = [lp, u64, vp, vp, sz, vp]
+        L.pvt_vstep_encode.restype = ctypes.c_int
+        L.pvt_vstep_encode.argtypes = [lp, vp, u64, vp, vp, sz, vp]
+        L.pvt_dequant.restype = ctypes.c_int
+        L.pvt_dequant.argtypes = [lp, vp, ctypes.c_int32, vp, vp]
+        L.pvt_status.restype = ctypes.c_int
+        L.pvt_status.argtypes = [vp, vp]
+        L.pvt_strerror.restype = ctypes.c_char_p
+        L.pvt_strerror.argtypes = [ctypes.c_int]
+        L.pvt_last_cuda_error.restype = ctypes.c_char_p
+        L.pvt_version.restype = ctypes.c_int
+        L.pvt_timing_enable.restype = None
+        L.pvt_timing_enable.argtypes = [ctypes.c_int]
+        L.pvt_launch_count.restype = ctypes.c_ulonglong
+        L.pvt_timing_read.restype = ctypes.c_int
+        L.pvt_timing_read.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int)]
+        _lib = L
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return lib().pvt_strerror(code).decode()
+
+
+def last_cuda_error() -> str:
+    return lib().pvt_last_cuda_error().decode()
+
+
+def _check(code: int, what: str) -> None:
+    if code != PVT_OK:
+        raise PvtError(code, what)
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return s.cuda_stream
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def make_layer(rows: int, cols: int, W, g, scale, codebooks, codes, *, eta: float = 1.0, beam: int = 8,
+               group_dim: int = 8) -> pvt_layer:
+    """Describe a layer whose arrays are CUDA tensors (any of W, g, scale may be
+    None for calls that do not read them).  codebooks: [M, K, 8] float32/float16;
+    codes: [G, M] uint8/uint16."""
+    M, K = int(codebooks.shape[0]), int(codebooks.shape[1])
+    for t in (W, g, scale, codebooks, codes):
+        if t is not None and (not t.is_cuda or not t.is_contiguous()):
+            raise ValueError("layer tensors must be contiguous CUDA tensors")
+    cb_dtype = {torch.float32: PVT_F32, torch.float16: PVT_F16}[codebooks.dtype]
+    code_dtype = {torch.uint8: PVT_U8, torch.uint16: PVT_U16, torch.int16: PVT_U16}[codes.dtype]
+    return pvt_layer(rows, cols, group_dim, M, K, cb_dtype, code_dtype, beam, float(eta), 0,
+                     _ptr(W), _ptr(g), _ptr(scale), _ptr(codebooks), _ptr(codes))
+
+
+def pvt_workspace_bytes(layer: pvt_layer, k: int) -> int:
+    n = int(lib().pvt_workspace_bytes(ctypes.byref(layer), k))
+    if n == 0:
+        raise PvtError(PVT_EINVAL, "pvt_workspace_bytes")
+    return n
+
+
+def pvt_workspace_init(ws: torch.Tensor, stream=None) -> None:
+    _check(lib().pvt_workspace_init(ws.data_ptr(), ws.numel() * ws.element_size(), _stream_ptr(stream)),
+           "pvt_workspace_init")
+
+
+def new_workspace(layer: pvt_layer, k: int, device=None) -> torch.Tensor:
+    ws = torch.empty(pvt_workspace_bytes(layer, k), dtype=torch.uint8, device=device or "cuda")
+    pvt_workspace_init(ws)
+    return ws
+
+
+def pvt_vstep_select(layer: pvt_layer, k: int, idx_out: torch.Tensor, ws: torch.Tensor, stream=None) -> None:
+    _check(lib().pvt_vstep_select(ctypes.byref(layer), k, idx_out.data_ptr(), ws.data_ptr(),
+                                  ws.numel() * ws.element_size(), _stream_ptr(stream)), "pvt_vstep_select")
+
+
+def pvt_vstep_encode(layer: pvt_layer, idx: torch.Tensor, k: int, err_out: Optional[torch.Tensor],
+                     ws: torch.Tensor, stream=None) -> None:
+    _check(lib().pvt_vstep_encode(ctypes.byref(layer), idx.data_ptr(), k, _ptr(err_out), ws.data_ptr(),
+                                  ws.numel() * ws.element_size(), _stream_ptr(stream)), "pvt_vstep_encode")
+
+
+def pvt_dequant(layer: pvt_layer, W_hat: torch.Tensor, status: Optional[torch.Tensor] = None, stream=None) -> None:
+    out_dtype = {torch.float32: PVT_F32, torch.float16: PVT_F16}[W_hat.dtype]
+    _check(lib().pvt_dequant(ctypes.byref(layer), W_hat.data_ptr(), out_dtype, _ptr(status), _stream_ptr(stream)),
+           "pvt_dequant")
+
+
+def pvt_status(ws: torch.Tensor, stream=None) -> int:
+    rc = int(lib().pvt_status(ws.data_ptr(), _stream_ptr(stream)))
+    if rc < 0:
+        raise PvtError(rc, "pvt_status")
+    return rc
+
+
+def pvt_version() -> int:
+    return int(lib().pvt_version())
+
+
+def pvt_launch_count() -> int:
+    return int(lib().pvt_launch_count())
+
+
+def pvt_timing_enable(on: bool) -> None:
+    lib().pvt_timing_enable(1 if on else 0)
+
+
+def pvt_timing_read(kernel_id: int):
+    """(total milliseconds, launches) of one kernel class since the last read."""
+    ms, n = ctypes.c_float(0.0), ctypes.c_int(0)
+    _check(lib().pvt_timing_read(kernel_id, ctypes.byref(ms), ctypes.byref(n)), "pvt_timing_read")
+    return float(ms.value), int(n.value)

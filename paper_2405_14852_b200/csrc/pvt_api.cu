@@ -1,0 +1,236 @@
+// Host side of the C ABI: argument validation, workspace sizing, status word,
+// optional per-kernel timing.  Everything here runs on the host and only enqueues
+// work; the arithmetic of the V step lives in the kernels of the other files.
+#include <atomic>
+#include <mutex>
+#include <vector>
+
+#include "pvt_internal.h"
+
+namespace pvt {
+namespace {
+
+thread_local cudaError_t g_last_cuda = cudaSuccess;
+std::atomic<unsigned long long> g_launches{0};
+
+int fail_cuda(cudaError_t e) {
+  g_last_cuda = e;
+  return PVT_ECUDA;
+}
+
+int sm_count() {
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+      n <= 0) {
+    (void)cudaGetLastError();
+    return kSmCountFallback;
+  }
+  return n;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Shape / type checks shared by every entry point.  Returns PVT_OK and G, or the error.
+int check_layer(const pvt_layer* L, uint64_t* G_out) {
+  if (!L) return PVT_EINVAL;
+  if (L->rows <= 0 || L->cols <= 0) return PVT_EINVAL;
+  if (L->group_dim != kGroupDim) return L->group_dim > 0 ? PVT_EUNSUPPORTED : PVT_EINVAL;
+  if (L->cols % kGroupDim != 0) return PVT_EINVAL;
+  const uint64_t G = (uint64_t)L->rows * (uint64_t)(L->cols / kGroupDim);
+  if (G >= (1ull << 32)) return PVT_EINVAL;
+  if (!(L->eta >= 0.0f) || !(L->eta <= 3.0e38f)) return PVT_EINVAL;
+  *G_out = G;
+  return PVT_OK;
+}
+
+int check_quantiser(const pvt_layer* L) {
+  const int M = L->num_codebooks, K = L->codebook_size;
+  if (M < 1 || K < 1) return PVT_EINVAL;
+  if (L->codebook_dtype != PVT_F32 && L->codebook_dtype != PVT_F16) return PVT_EINVAL;
+  if (L->code_dtype != PVT_U8 && L->code_dtype != PVT_U16) return PVT_EINVAL;
+  if (M > 2 || K < 2) return PVT_EUNSUPPORTED;
+  if (M == 1 && K > 65536) return PVT_EUNSUPPORTED;
+  if (L->code_dtype == PVT_U8 && K > 256) return PVT_EINVAL;
+  if (M == 2 && K > 256) return PVT_EUNSUPPORTED;
+  return PVT_OK;
+}
+
+// ---- optional timing ----------------------------------------------------------
+struct Timing {
+  std::mutex mu;
+  bool enabled = false;
+  std::vector<std::pair<cudaEvent_t, cudaEvent_t>> spans[kKernCount];
+  cudaEvent_t open[kKernCount] = {};
+};
+Timing& timing() {
+  static Timing t;
+  return t;
+}
+
+}  // namespace
+
+void count_launches(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+
+void timing_begin(KernelId id, cudaStream_t stream) {
+  Timing& t = timing();
+  if (!t.enabled) return;
+  std::lock_guard<std::mutex> lock(t.mu);
+  cudaEvent_t a;
+  if (cudaEventCreate(&a) != cudaSuccess) return;
+  cudaEventRecord(a, stream);
+  t.open[id] = a;
+}
+
+void timing_end(KernelId id, cudaStream_t stream) {
+  Timing& t = timing();
+  if (!t.enabled) return;
+  std::lock_guard<std::mutex> lock(t.mu);
+  if (!t.open[id]) return;
+  cudaEvent_t b;
+  if (cudaEventCreate(&b) != cudaSuccess) return;
+  cudaEventRecord(b, stream);
+  t.spans[id].push_back({t.open[id], b});
+  t.open[id] = nullptr;
+}
+
+}  // namespace pvt
+
+using namespace pvt;
+
+extern "C" {
+
+size_t pvt_workspace_bytes(const pvt_layer* layer, uint64_t k) {
+  uint64_t G = 0;
+  if (check_layer(layer, &G) != PVT_OK || check_quantiser(layer) != PVT_OK) return 0;
+  if (k < 1 || k > G) return 0;
+  const int sms = sm_count();
+  size_t need = select_layout(G).bytes;
+  if (layer->num_codebooks == 1) {
+    const size_t e = encode_m1_layout((uint32_t)layer->codebook_size, k, sms, encode_m1_targets_per_thread(k, sms)).bytes;
+    need = e > need ? e : need;
+  } else {
+    const size_t e = encode_m2_workspace_bytes();
+    need = e > need ? e : need;
+  }
+  return need;
+}
+
+int pvt_workspace_init(void* ws, size_t ws_bytes, void* cuda_stream) {
+  if (!ws || ws_bytes < kWsHeaderBytes || (reinterpret_cast<uintptr_t>(ws) & (kWsAlign - 1))) return PVT_EINVAL;
+  const cudaError_t e = cudaMemsetAsync(ws, 0, kWsHeaderBytes, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? PVT_OK : fail_cuda(e);
+}
+
+int pvt_vstep_select(const pvt_layer* layer, uint64_t k, uint32_t* idx_out, void* ws, size_t ws_bytes,
+                     void* cuda_stream) {
+  uint64_t G = 0;
+  int rc = check_layer(layer, &G);
+  if (rc != PVT_OK) return rc;
+  if (k < 1 || k > G) return PVT_EINVAL;
+  if (!layer->g || !aligned16(layer->g) || !idx_out || !ws) return PVT_EINVAL;
+  if (reinterpret_cast<uintptr_t>(ws) & (kWsAlign - 1)) return PVT_EINVAL;
+  if (ws_bytes < select_layout(G).bytes) return PVT_EWORKSPACE;
+  const cudaError_t e = launch_select(*layer, G, k, idx_out, ws, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? PVT_OK : fail_cuda(e);
+}
+
+int pvt_vstep_encode(const pvt_layer* layer, const uint32_t* idx, uint64_t k, float* err_out, void* ws,
+                     size_t ws_bytes, void* cuda_stream) {
+  uint64_t G = 0;
+  int rc = check_layer(layer, &G);
+  if (rc != PVT_OK) return rc;
+  if ((rc = check_quantiser(layer)) != PVT_OK) return rc;
+  if (k < 1 || k > G) return PVT_EINVAL;
+  if (!layer->W || !layer->g || !layer->scale || !layer->codebooks || !layer->codes || !idx || !ws) return PVT_EINVAL;
+  if (!aligned16(layer->W) || !aligned16(layer->g) || !aligned16(layer->codebooks)) return PVT_EINVAL;
+  if (reinterpret_cast<uintptr_t>(ws) & (kWsAlign - 1)) return PVT_EINVAL;
+  const int sms = sm_count();
+  cudaError_t e;
+  if (layer->num_codebooks == 1) {
+    const EncodeM1Layout lay =
+        encode_m1_layout((uint32_t)layer->codebook_size, k, sms, encode_m1_targets_per_thread(k, sms));
+    if (ws_bytes < lay.bytes) return PVT_EWORKSPACE;
+    e = launch_encode_m1(*layer, G, idx, k, err_out, ws, sms, static_cast<cudaStream_t>(cuda_stream));
+  } else {
+    if (layer->code_dtype != PVT_U8) return PVT_EUNSUPPORTED;
+    if (layer->beam < 1 || layer->beam > 8) return PVT_EUNSUPPORTED;
+    if (ws_bytes < encode_m2_workspace_bytes()) return PVT_EWORKSPACE;
+    e = launch_encode_m2(*layer, G, idx, k, err_out, ws, sms, static_cast<cudaStream_t>(cuda_stream));
+  }
+  return e == cudaSuccess ? PVT_OK : fail_cuda(e);
+}
+
+int pvt_dequant(const pvt_layer* layer, void* W_hat, int32_t out_dtype, uint32_t* status, void* cuda_stream) {
+  uint64_t G = 0;
+  int rc = check_layer(layer, &G);
+  if (rc != PVT_OK) return rc;
+  if ((rc = check_quantiser(layer)) != PVT_OK) return rc;
+  if (out_dtype != PVT_F32 && out_dtype != PVT_F16) return PVT_EINVAL;
+  if (!layer->scale || !layer->codebooks || !layer->codes || !W_hat) return PVT_EINVAL;
+  if (!aligned16(layer->codebooks) || !aligned16(W_hat)) return PVT_EINVAL;
+  if (layer->num_codebooks == 2 && layer->code_dtype == PVT_U8 && (reinterpret_cast<uintptr_t>(layer->codes) & 1u))
+    return PVT_EINVAL;
+  const cudaError_t e = launch_dequant(*layer, G, W_hat, out_dtype, status, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? PVT_OK : fail_cuda(e);
+}
+
+int pvt_status(void* ws, void* cuda_stream) {
+  if (!ws) return PVT_EINVAL;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  uint32_t word = 0;
+  cudaError_t e = cudaMemcpyAsync(&word, ws, sizeof(word), cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e == cudaSuccess && word) e = cudaMemsetAsync(ws, 0, sizeof(word), s);
+  if (e != cudaSuccess) return fail_cuda(e);
+  return (int)(word & 0x7fffffffu);
+}
+
+const char* pvt_strerror(int code) {
+  switch (code) {
+    case PVT_OK: return "ok";
+    case PVT_EINVAL: return "invalid argument (null or misaligned pointer, k out of range, bad shape or eta)";
+    case PVT_EUNSUPPORTED: return "unsupported group_dim / codebook count / codebook size / dtype / beam";
+    case PVT_EWORKSPACE: return "workspace smaller than pvt_workspace_bytes()";
+    case PVT_ECUDA: return "CUDA runtime error (see pvt_last_cuda_error)";
+    default: return code > 0 ? "device status bits set" : "unknown error";
+  }
+}
+
+const char* pvt_last_cuda_error(void) { return cudaGetErrorString(g_last_cuda); }
+
+int pvt_version(void) { return 100; }
+
+unsigned long long pvt_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+void pvt_timing_enable(int on) {
+  Timing& t = timing();
+  std::lock_guard<std::mutex> lock(t.mu);
+  t.enabled = on != 0;
+}
+
+int pvt_timing_read(int kernel_id, float* total_ms, int* launches) {
+  if (kernel_id < 0 || kernel_id >= kKernCount || !total_ms || !launches) return PVT_EINVAL;
+  Timing& t = timing();
+  std::lock_guard<std::mutex> lock(t.mu);
+  float sum = 0.0f;
+  int n = 0;
+  for (auto& span : t.spans[kernel_id]) {
+    float ms = 0.0f;
+    cudaError_t e = cudaEventSynchronize(span.second);
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, span.first, span.second);
+    cudaEventDestroy(span.first);
+    cudaEventDestroy(span.second);
+    if (e != cudaSuccess) {
+      t.spans[kernel_id].clear();
+      return fail_cuda(e);
+    }
+    sum += ms;
+    ++n;
+  }
+  t.spans[kernel_id].clear();
+  *total_ms = sum;
+  *launches = n;
+  return PVT_OK;
+}
+
+}  // extern "C"

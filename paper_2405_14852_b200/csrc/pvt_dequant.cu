@@ -1,0 +1,153 @@
+// dequantize_weights (Algorithm 3, first line): W_hat = s_row * sum_m C_m[b_m] for
+// every weight group.  Streaming kernel: one group (8 weights) per thread, codes
+// read coalesced, codewords gathered from the L2-resident codebook (small
+// codebooks are first copied to shared memory), 32 B (fp32) or 16 B (fp16) written
+// per group with 128-bit stores.
+//
+// Arithmetic per element, binary32, each step rounded once: v = c1 (+ c2);
+// w = s * v; fp16 output = round-to-nearest-even of w.
+#include <cuda_fp16.h>
+
+#include "pvt_internal.h"
+
+namespace pvt {
+namespace {
+
+constexpr int kDqThreads = 256;
+constexpr int kDqSmemCodewords = 512;  // M*K up to this many codewords are staged in shared memory
+
+struct Vec8 {
+  float v[8];
+};
+
+template <bool CB_F16>
+__device__ __forceinline__ Vec8 load_codeword(const void* book, uint32_t code) {
+  Vec8 r;
+  if (CB_F16) {
+    const uint4 raw = *(reinterpret_cast<const uint4*>(book) + code);
+    const __half2* h = reinterpret_cast<const __half2*>(&raw);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float2 f = __half22float2(h[i]);
+      r.v[2 * i] = f.x;
+      r.v[2 * i + 1] = f.y;
+    }
+  } else {
+    const float4* p = reinterpret_cast<const float4*>(book) + 2 * (size_t)code;
+    const float4 a = p[0], b = p[1];
+    r.v[0] = a.x; r.v[1] = a.y; r.v[2] = a.z; r.v[3] = a.w;
+    r.v[4] = b.x; r.v[5] = b.y; r.v[6] = b.z; r.v[7] = b.w;
+  }
+  return r;
+}
+
+template <int M, bool CB_F16, bool CODE_U16, bool OUT_F16, bool SMEM_BOOK>
+__global__ void __launch_bounds__(kDqThreads) dequant_kernel(const void* __restrict__ codebooks,
+                                                              const void* __restrict__ codes,
+                                                              const float* __restrict__ scale, uint64_t G,
+                                                              uint32_t gpr, uint32_t K, void* __restrict__ W_hat,
+                                                              uint32_t* status) {
+  constexpr int kCwBytes = CB_F16 ? 16 : 32;
+  __shared__ __align__(16) unsigned char sh_book[SMEM_BOOK ? kDqSmemCodewords * kCwBytes : 16];
+  const void* book = codebooks;
+  if (SMEM_BOOK) {
+    const uint4* src = reinterpret_cast<const uint4*>(codebooks);
+    uint4* dst = reinterpret_cast<uint4*>(sh_book);
+    const int n16 = M * K * kCwBytes / 16;
+    for (int i = threadIdx.x; i < n16; i += kDqThreads) dst[i] = src[i];
+    __syncthreads();
+    book = sh_book;
+  }
+  const uint64_t j = (uint64_t)blockIdx.x * kDqThreads + threadIdx.x;
+  if (j >= G) return;
+  uint32_t b[M];
+  if (CODE_U16) {
+    const uint16_t* c = reinterpret_cast<const uint16_t*>(codes) + j * M;
+#pragma unroll
+    for (int m = 0; m < M; ++m) b[m] = c[m];
+  } else if (M == 2) {
+    const uint16_t both = reinterpret_cast<const uint16_t*>(codes)[j];  // two adjacent bytes
+    b[0] = both & 0xffu;
+    b[M - 1] = both >> 8;
+  } else {
+    b[0] = reinterpret_cast<const uint8_t*>(codes)[j];
+  }
+  bool bad = false;
+#pragma unroll
+  for (int m = 0; m < M; ++m) {
+    if (b[m] >= K) {
+      bad = true;
+      b[m] = 0;
+    }
+  }
+  if (bad && status) atomicOr(status, PVT_DEV_BAD_CODE);
+
+  Vec8 v = load_codeword<CB_F16>(book, b[0]);
+  if (M == 2) {
+    const Vec8 v2 = load_codeword<CB_F16>(book, K + b[M - 1]);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v.v[i] = __fadd_rn(v.v[i], v2.v[i]);
+  }
+  const float s = scale[j / gpr];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) v.v[i] = __fmul_rn(s, v.v[i]);
+
+  if (OUT_F16) {
+    __half2 h[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) h[i] = __floats2half2_rn(v.v[2 * i], v.v[2 * i + 1]);
+    __stcs(reinterpret_cast<uint4*>(W_hat) + j, *reinterpret_cast<const uint4*>(h));
+  } else {
+    float4* o = reinterpret_cast<float4*>(W_hat) + 2 * j;
+    __stcs(o, make_float4(v.v[0], v.v[1], v.v[2], v.v[3]));
+    __stcs(o + 1, make_float4(v.v[4], v.v[5], v.v[6], v.v[7]));
+  }
+}
+
+template <int M, bool CB_F16, bool CODE_U16, bool OUT_F16>
+cudaError_t launch_t(const pvt_layer& L, uint64_t G, void* W_hat, uint32_t* status, cudaStream_t stream) {
+  const unsigned blocks = (unsigned)((G + kDqThreads - 1) / kDqThreads);
+  const uint32_t gpr = (uint32_t)(L.cols / kGroupDim);
+  const uint32_t K = (uint32_t)L.codebook_size;
+  if ((uint32_t)M * K <= (uint32_t)kDqSmemCodewords)
+    dequant_kernel<M, CB_F16, CODE_U16, OUT_F16, true>
+        <<<blocks, kDqThreads, 0, stream>>>(L.codebooks, L.codes, L.scale, G, gpr, K, W_hat, status);
+  else
+    dequant_kernel<M, CB_F16, CODE_U16, OUT_F16, false>
+        <<<blocks, kDqThreads, 0, stream>>>(L.codebooks, L.codes, L.scale, G, gpr, K, W_hat, status);
+  return cudaGetLastError();
+}
+
+template <int M, bool CB_F16, bool CODE_U16>
+cudaError_t launch_o(const pvt_layer& L, uint64_t G, void* W_hat, int32_t out_dtype, uint32_t* status,
+                     cudaStream_t stream) {
+  return out_dtype == PVT_F16 ? launch_t<M, CB_F16, CODE_U16, true>(L, G, W_hat, status, stream)
+                              : launch_t<M, CB_F16, CODE_U16, false>(L, G, W_hat, status, stream);
+}
+
+template <int M, bool CB_F16>
+cudaError_t launch_c(const pvt_layer& L, uint64_t G, void* W_hat, int32_t out_dtype, uint32_t* status,
+                     cudaStream_t stream) {
+  return L.code_dtype == PVT_U16 ? launch_o<M, CB_F16, true>(L, G, W_hat, out_dtype, status, stream)
+                                 : launch_o<M, CB_F16, false>(L, G, W_hat, out_dtype, status, stream);
+}
+
+}  // namespace
+
+cudaError_t launch_dequant(const pvt_layer& L, uint64_t G, void* W_hat, int32_t out_dtype, uint32_t* status,
+                           cudaStream_t stream) {
+  timing_begin(kKernDequant, stream);
+  cudaError_t err;
+  const bool f16 = L.codebook_dtype == PVT_F16;
+  if (L.num_codebooks == 1)
+    err = f16 ? launch_c<1, true>(L, G, W_hat, out_dtype, status, stream)
+              : launch_c<1, false>(L, G, W_hat, out_dtype, status, stream);
+  else
+    err = f16 ? launch_c<2, true>(L, G, W_hat, out_dtype, status, stream)
+              : launch_c<2, false>(L, G, W_hat, out_dtype, status, stream);
+  count_launches(1);
+  timing_end(kKernDequant, stream);
+  return err;
+}
+
+}  // namespace pvt

@@ -1,0 +1,574 @@
+// Exhaustive nearest-codeword search of the V step for one codebook (Appendix C /
+// Appendix J: "try every code in the codebook"; Appendix D: the score
+// ||c||^2 - 2 <t, c>; Eq. 8 for the target t = (W - eta g) / s).
+//
+// Work decomposition: targets are cut into tiles of 256*TT groups, the codebook
+// into chunks of 256 codewords; the (tile, chunk) grid is flattened and split
+// evenly over one persistent CTA per SM, so a CTA works on a few segments
+// (tile, chunk range).  Per segment:
+//   1. every compute thread gathers TT targets (32 B of W and of g each), forms t
+//      in binary32 and keeps -t in registers, duplicated into f32x2 pairs;
+//   2. a producer warp streams the pre-expanded codebook (pairs of codewords
+//      interleaved, half squared norms appended) chunk by chunk into a 4-stage
+//      shared-memory ring with 1-D bulk tensor-memory-accelerator copies that
+//      complete on mbarriers;
+//   3. the compute warps read one codeword pair per iteration (broadcast loads)
+//      and evaluate score = ||c||^2/2 - <t, c> for both codewords and all TT
+//      targets with packed fma.rn.f32x2, folding the two scores into a running
+//      minimum with one three-input min: 8 FMAs and half a min per pair
+//      evaluation, no distance matrix, no index tracking in the hot loop;
+//   4. every 32 codewords the running minimum of that sub-chunk is compared with
+//      the best so far; sub-chunks within a rounding-error margin of the best are
+//      remembered (4 most recent per target);
+//   5. after the loop each warp revisits the remembered sub-chunks of its
+//      targets, recomputes the same binary32 score, and for every codeword within
+//      the margin of the minimum evaluates the binary64 distance sum (t_i-c_i)^2
+//      in index order; the result is the argmin of (distance, code).
+// The margin bounds twice the rounding error of the fast score, so the codeword
+// that is nearest in exact arithmetic is always among those rescored.
+// Segments that cover the whole codebook write the code directly; otherwise the
+// per-slice results go to the workspace and a small merge kernel finishes.
+#include <cuda_fp16.h>
+
+#include "pvt_internal.h"
+
+namespace pvt {
+
+EncodeM1Layout encode_m1_layout(uint32_t K, uint64_t k, int sm_count, int tt) {
+  EncodeM1Layout e;
+  e.n_chunks = (K + kChunkCodewords - 1) / kChunkCodewords;
+  e.tile = (uint32_t)(kEncThreads * tt);
+  e.n_tiles = (uint32_t)((k + e.tile - 1) / e.tile);
+  const uint64_t units = (uint64_t)e.n_tiles * e.n_chunks;
+  e.n_ctas = (uint32_t)(units < (uint64_t)sm_count ? units : (uint64_t)sm_count);
+  e.cbx_off = kWsHeaderBytes;
+  e.n2max_off = align_up(e.cbx_off + (size_t)e.n_chunks * kChunkBytes, kWsAlign);
+  e.partial_off = e.n2max_off + kWsAlign;
+  e.bytes = align_up(e.partial_off + (size_t)e.n_ctas * 2 * e.tile * sizeof(PartialResult), kWsAlign);
+  return e;
+}
+
+int encode_m1_targets_per_thread(uint64_t k, int sm_count) {
+  // 8 targets per thread amortise the shared-memory reads best, but tiles of 2048
+  // targets only pay off when there are many tiles per SM
+  return k >= (uint64_t)sm_count * 2048ull * 4ull ? 8 : 4;
+}
+
+namespace {
+
+constexpr float kPadHalfNorm = 3.0e38f;  // half norm of padding codewords: never near a minimum
+constexpr uint32_t kMaxSpins = 1u << 22;
+
+struct EncM1Params {
+  const float* W;
+  const float* g;
+  const float* scale;
+  const uint32_t* idx;
+  uint64_t k, G;
+  uint32_t gpr;
+  float eta;
+  const float* cbx;
+  const uint32_t* n2max_bits;
+  uint32_t n_chunks, K, n_tiles, n_ctas;
+  PartialResult* partial;
+  void* codes;
+  int code_u16;
+  float* err_out;
+  uint32_t* status;
+};
+
+// ---- codebook expansion ------------------------------------------------------
+// chunk block (kChunkBytes): 128 pairs * 16 floats, pair p holds
+// (c[2p][0], c[2p+1][0], c[2p][1], c[2p+1][1], ...), then 128 * 2 half norms.
+template <bool CB_F16>
+__global__ void expand_codebook_kernel(const void* __restrict__ book, uint32_t K, uint32_t n_chunks,
+                                       float* __restrict__ cbx, uint32_t* __restrict__ n2max_bits) {
+  const uint32_t kappa = blockIdx.x * blockDim.x + threadIdx.x;
+  float n2 = 0.0f;
+  if (kappa < n_chunks * kChunkCodewords) {
+    float c[8];
+    if (kappa < K) {
+      if (CB_F16) {
+        const uint4 raw = reinterpret_cast<const uint4*>(book)[kappa];
+        const __half2* h = reinterpret_cast<const __half2*>(&raw);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float2 f = __half22float2(h[i]);
+          c[2 * i] = f.x;
+          c[2 * i + 1] = f.y;
+        }
+      } else {
+        const float4* p = reinterpret_cast<const float4*>(book) + 2 * (size_t)kappa;
+        const float4 a = p[0], b = p[1];
+        c[0] = a.x; c[1] = a.y; c[2] = a.z; c[3] = a.w;
+        c[4] = b.x; c[5] = b.y; c[6] = b.z; c[7] = b.w;
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) n2 = __fmaf_rn(c[i], c[i], n2);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) c[i] = 0.0f;
+    }
+    const uint32_t chunk = kappa / kChunkCodewords, w = kappa % kChunkCodewords;
+    float* blk = cbx + (size_t)chunk * (kChunkBytes / 4);
+    const uint32_t pr = w >> 1, half = w & 1;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) blk[pr * 16 + 2 * i + half] = c[i];
+    blk[kChunkCodewords * 8 + pr * 2 + half] = kappa < K ? __fmul_rn(0.5f, n2) : kPadHalfNorm;
+  }
+  // max ||c||^2 over the codebook (non-negative floats order like their bit patterns)
+  uint32_t bits = __float_as_uint(n2);
+  bits = __reduce_max_sync(0xffffffffu, bits);
+  if ((threadIdx.x & 31) == 0 && bits) atomicMax(n2max_bits, bits);
+}
+
+// ---- PTX helpers ---------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// 1-D bulk copy global -> shared through the tensor memory accelerator; completes
+// `bytes` on the mbarrier.  Both addresses 16-byte aligned, bytes % 16 == 0.
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+// Bounded wait.  Gives up after kMaxSpins polls (or as soon as another thread gave
+// up), flags the CTA as aborted and reports through the status word.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          uint32_t* status) {
+  for (uint32_t spin = 0; spin < kMaxSpins; ++spin) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (spin > 32) __nanosleep(64);
+  }
+  *abort_flag = 1;
+  atomicOr(status, PVT_DEV_WAIT_EXPIRED);
+  return false;
+}
+
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ float min3(float a, float b, float c) {
+  float d;
+  asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  return (uint64_t)__float_as_uint(lo) | ((uint64_t)__float_as_uint(hi) << 32);
+}
+__device__ __forceinline__ void compute_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kEncThreads) : "memory"); }
+
+__device__ __forceinline__ uint64_t cta_unit_lo(uint64_t b, uint64_t units, uint64_t n_ctas) {
+  return b * units / n_ctas;  // units * n_ctas < 2^64 for every supported size
+}
+
+// ---- shared-memory layout of the search kernel -----------------------------------
+template <int TT>
+struct EncSmem {
+  static constexpr int TILE = kEncThreads * TT;
+  alignas(128) unsigned char stage[kEncStages][kChunkBytes];
+  alignas(8) uint64_t full_bar[kEncStages];
+  uint64_t empty_bar[kEncStages];
+  alignas(16) float t[TILE][8];       // targets of the tile (for the rescoring pass)
+  uint32_t group[TILE];               // group index of each target, 0xffffffff = none
+  float margin[TILE];
+  float best[TILE];                   // minimum fast score over the segment
+  float evicted_min[TILE];            // smallest sub-chunk minimum that fell out of the list
+  float list_min[kListLen][TILE];
+  uint16_t list_id[kListLen][TILE];
+  uint16_t list_cnt[TILE];
+  uint32_t abort_flag;
+};
+
+template <int TT>
+__global__ void __launch_bounds__(kEncThreads + 32, 1) encode_m1_kernel(const EncM1Params p) {
+  using Smem = EncSmem<TT>;
+  constexpr int TILE = Smem::TILE;
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  volatile uint32_t* abort_flag = &sm.abort_flag;
+
+  if (tid == 0) {
+    sm.abort_flag = 0;
+    for (int s = 0; s < kEncStages; ++s) {
+      mbar_init(smem_u32(&sm.full_bar[s]), 1);
+      mbar_init(smem_u32(&sm.empty_bar[s]), kEncThreads / 32);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  const uint64_t units = (uint64_t)p.n_tiles * p.n_chunks;
+  const uint64_t u_lo = cta_unit_lo(blockIdx.x, units, p.n_ctas);
+  const uint64_t u_hi = cta_unit_lo(blockIdx.x + 1, units, p.n_ctas);
+
+  if (warp == kEncThreads / 32) {
+    // ------------------------------------------------------------ producer warp
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool alive = true;
+      for (uint64_t u = u_lo; u < u_hi && alive;) {
+        const uint32_t c_lo = (uint32_t)(u % p.n_chunks);
+        const uint64_t left = u_hi - u;
+        const uint32_t c_hi = (uint32_t)((uint64_t)c_lo + left < p.n_chunks ? c_lo + left : p.n_chunks);
+        for (uint32_t c = c_lo; c < c_hi && alive; ++c, ++it) {
+          const uint32_t s = it % kEncStages;
+          if (it >= kEncStages)
+            alive = mbar_wait(smem_u32(&sm.empty_bar[s]), ((it / kEncStages) - 1) & 1, abort_flag, p.status);
+          if (!alive) break;
+          const uint32_t fb = smem_u32(&sm.full_bar[s]);
+          mbar_expect_tx(fb, kChunkBytes);
+          bulk_g2s(smem_u32(&sm.stage[s][0]), reinterpret_cast<const char*>(p.cbx) + (size_t)c * kChunkBytes,
+                   kChunkBytes, fb);
+        }
+        u += c_hi - c_lo;
+      }
+      if (!alive) {
+        // drain: let every copy that was issued land before the CTA may exit
+        for (uint32_t back = 1; back <= kEncStages && back <= it; ++back) {
+          const uint32_t j = it - back;
+          const uint32_t fb = smem_u32(&sm.full_bar[j % kEncStages]);
+          for (uint32_t spin = 0; spin < kMaxSpins; ++spin) {
+            if (mbar_try_wait(fb, (j / kEncStages) & 1)) break;
+            __nanosleep(64);
+          }
+        }
+      }
+    }
+    return;
+  }
+
+  // -------------------------------------------------------------- compute warps
+  const float n2max = __uint_as_float(*p.n2max_bits);
+  const float4* W4 = reinterpret_cast<const float4*>(p.W);
+  const float4* g4 = reinterpret_cast<const float4*>(p.g);
+  uint32_t it = 0;
+  bool first_segment = true;
+
+  for (uint64_t u = u_lo; u < u_hi;) {
+    const uint32_t tile = (uint32_t)(u / p.n_chunks);
+    const uint32_t c_lo = (uint32_t)(u % p.n_chunks);
+    const uint64_t left = u_hi - u;
+    const uint32_t c_hi = (uint32_t)((uint64_t)c_lo + left < p.n_chunks ? c_lo + left : p.n_chunks);
+    const bool full_cover = (c_lo == 0 && c_hi == p.n_chunks);
+
+    // 1. gather targets, form t (binary32: one fma, one division), set up tracking
+    uint64_t nt[TT][8];  // (-t_i, -t_i)
+    float thr[TT], best[TT], margin[TT];
+#pragma unroll
+    for (int tt = 0; tt < TT; ++tt) {
+      const int s = tt * kEncThreads + tid;
+      const uint64_t n = (uint64_t)tile * TILE + s;
+      uint32_t j = 0xffffffffu;
+      float t[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) t[i] = 0.0f;
+      if (n < p.k) {
+        j = p.idx[n];
+        if (j >= p.G) {
+          atomicOr(p.status, PVT_DEV_BAD_INDEX);
+          j = 0xffffffffu;
+        } else {
+          const float4 w0 = __ldg(W4 + 2 * (size_t)j), w1 = __ldg(W4 + 2 * (size_t)j + 1);
+          const float4 g0 = __ldg(g4 + 2 * (size_t)j), g1 = __ldg(g4 + 2 * (size_t)j + 1);
+          const float sc = __ldg(p.scale + j / p.gpr);
+          const float neg_eta = -p.eta;
+          t[0] = __fdiv_rn(__fmaf_rn(neg_eta, g0.x, w0.x), sc);
+          t[1] = __fdiv_rn(__fmaf_rn(neg_eta, g0.y, w0.y), sc);
+          t[2] = __fdiv_rn(__fmaf_rn(neg_eta, g0.z, w0.z), sc);
+          t[3] = __fdiv_rn(__fmaf_rn(neg_eta, g0.w, w0.w), sc);
+          t[4] = __fdiv_rn(__fmaf_rn(neg_eta, g1.x, w1.x), sc);
+          t[5] = __fdiv_rn(__fmaf_rn(neg_eta, g1.y, w1.y), sc);
+          t[6] = __fdiv_rn(__fmaf_rn(neg_eta, g1.z, w1.z), sc);
+          t[7] = __fdiv_rn(__fmaf_rn(neg_eta, g1.w, w1.w), sc);
+        }
+      }
+      float nt2 = 0.0f;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        nt2 = fmaf(t[i], t[i], nt2);
+        nt[tt][i] = pack2(-t[i], -t[i]);
+      }
+      // twice the rounding-error bound of the fast score, with a factor 2 to spare:
+      // |score_fl - score| <= 16.1 u (||c||^2/2 + ||t|| ||c||), u = 2^-24
+      margin[tt] = 3.8146973e-6f /* 2^-18 */ * (0.5f * n2max + sqrtf(nt2 * n2max)) + 1e-30f;
+      best[tt] = __int_as_float(0x7f800000);
+      thr[tt] = best[tt];
+      *reinterpret_cast<float4*>(&sm.t[s][0]) = make_float4(t[0], t[1], t[2], t[3]);
+      *reinterpret_cast<float4*>(&sm.t[s][4]) = make_float4(t[4], t[5], t[6], t[7]);
+      sm.group[s] = j;
+      sm.margin[s] = margin[tt];
+      sm.list_cnt[s] = 0;
+      sm.evicted_min[s] = __int_as_float(0x7f800000);
+    }
+
+    // 2.-4. stream the codebook chunks of this segment
+    for (uint32_t c = c_lo; c < c_hi; ++c, ++it) {
+      const uint32_t st = it % kEncStages;
+      mbar_wait(smem_u32(&sm.full_bar[st]), (it / kEncStages) & 1, abort_flag, p.status);
+      const unsigned char* stage = &sm.stage[st][0];
+#pragma unroll 1
+      for (int sub = 0; sub < kChunkCodewords / kSubCodewords; ++sub) {
+        float cmin[TT];
+#pragma unroll
+        for (int tt = 0; tt < TT; ++tt) cmin[tt] = __int_as_float(0x7f800000);
+        const ulonglong2* vals = reinterpret_cast<const ulonglong2*>(stage) + sub * (kSubCodewords / 2) * 4;
+        const uint64_t* norms =
+            reinterpret_cast<const uint64_t*>(stage + kChunkCodewords * 32) + sub * (kSubCodewords / 2);
+#pragma unroll 4
+        for (int pr = 0; pr < kSubCodewords / 2; ++pr) {
+          const ulonglong2 q0 = vals[4 * pr], q1 = vals[4 * pr + 1], q2 = vals[4 * pr + 2], q3 = vals[4 * pr + 3];
+          const uint64_t h = norms[pr];
+#pragma unroll
+          for (int tt = 0; tt < TT; ++tt) {
+            uint64_t acc = h;
+            acc = fma2(nt[tt][0], q0.x, acc);
+            acc = fma2(nt[tt][1], q0.y, acc);
+            acc = fma2(nt[tt][2], q1.x, acc);
+            acc = fma2(nt[tt][3], q1.y, acc);
+            acc = fma2(nt[tt][4], q2.x, acc);
+            acc = fma2(nt[tt][5], q2.y, acc);
+            acc = fma2(nt[tt][6], q3.x, acc);
+            acc = fma2(nt[tt][7], q3.y, acc);
+            cmin[tt] = min3(cmin[tt], __uint_as_float((uint32_t)acc), __uint_as_float((uint32_t)(acc >> 32)));
+          }
+        }
+        const uint32_t sub_id = c * (kChunkCodewords / kSubCodewords) + sub;
+#pragma unroll
+        for (int tt = 0; tt < TT; ++tt) {
+          if (cmin[tt] <= thr[tt]) {
+            const int s = tt * kEncThreads + tid;
+            const uint32_t cnt = sm.list_cnt[s];
+            const uint32_t slot = cnt & (kListLen - 1);
+            if (cnt >= kListLen) sm.evicted_min[s] = fminf(sm.evicted_min[s], sm.list_min[slot][s]);
+            sm.list_id[slot][s] = (uint16_t)sub_id;
+            sm.list_min[slot][s] = cmin[tt];
+            sm.list_cnt[s] = (uint16_t)(cnt + 1);
+            best[tt] = fminf(best[tt], cmin[tt]);
+            thr[tt] = best[tt] + margin[tt];
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&sm.empty_bar[st]));
+    }
+#pragma unroll
+    for (int tt = 0; tt < TT; ++tt) sm.best[tt * kEncThreads + tid] = best[tt];
+    compute_bar();
+
+    // 5. rescoring: one warp per target
+    const bool aborted = *abort_flag != 0;
+    const uint32_t slot_of_segment = first_segment ? 0u : 1u;
+    for (int s = warp; s < TILE && !aborted; s += kEncThreads / 32) {
+      const uint64_t n = (uint64_t)tile * TILE + s;
+      if (n >= p.k) break;
+      const uint32_t j = sm.group[s];
+      const float m = sm.best[s];
+      const float limit = m + sm.margin[s];
+      const uint32_t cnt = sm.list_cnt[s];
+      const bool overflow = cnt > kListLen && sm.evicted_min[s] <= limit;
+      const float4 ta = *reinterpret_cast<const float4*>(&sm.t[s][0]);
+      const float4 tb = *reinterpret_cast<const float4*>(&sm.t[s][4]);
+      const float t[8] = {ta.x, ta.y, ta.z, ta.w, tb.x, tb.y, tb.z, tb.w};
+      double best_d = __longlong_as_double(0x7ff0000000000000ll);
+      uint32_t best_code = 0xffffffffu;
+      const uint32_t subs_per_chunk = kChunkCodewords / kSubCodewords;
+      const uint32_t n_visit = overflow ? (c_hi - c_lo) * subs_per_chunk : min(cnt, (uint32_t)kListLen);
+      for (uint32_t v = 0; v < n_visit; ++v) {
+        uint32_t sub_id;
+        if (overflow) {
+          sub_id = c_lo * subs_per_chunk + v;
+        } else {
+          if (sm.list_min[v][s] > limit) continue;
+          sub_id = sm.list_id[v][s];
+        }
+        const uint32_t chunk = sub_id / subs_per_chunk;
+        const uint32_t w = (sub_id % subs_per_chunk) * kSubCodewords + lane;  // codeword within the chunk
+        const uint32_t kappa = chunk * kChunkCodewords + w;
+        const float* blk = p.cbx + (size_t)chunk * (kChunkBytes / 4);
+        const uint32_t pr = w >> 1, half = w & 1;
+        float cw[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) cw[i] = __ldg(blk + pr * 16 + 2 * i + half);
+        float f = __ldg(blk + kChunkCodewords * 8 + pr * 2 + half);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) f = __fmaf_rn(-t[i], cw[i], f);  // the same operations as the packed loop
+        const bool cand = (f <= limit) && (kappa < p.K);
+        uint32_t mask = __ballot_sync(0xffffffffu, cand);
+        if (mask) {
+          double d = 0.0;
+          if (cand) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const double e = __dsub_rn((double)t[i], (double)cw[i]);
+              d = __dadd_rn(d, __dmul_rn(e, e));
+            }
+          }
+          while (mask) {
+            const int src = __ffs(mask) - 1;
+            mask &= mask - 1;
+            const double dc = __shfl_sync(0xffffffffu, d, src);
+            const uint32_t kc = chunk * kChunkCodewords + (sub_id % subs_per_chunk) * kSubCodewords + src;
+            if (dc < best_d || (dc == best_d && kc < best_code)) {
+              best_d = dc;
+              best_code = kc;
+            }
+          }
+        }
+      }
+      if (lane == 0) {
+        const bool ok = j != 0xffffffffu && best_code < p.K;
+        if (full_cover) {
+          if (ok) {
+            if (p.code_u16)
+              reinterpret_cast<uint16_t*>(p.codes)[j] = (uint16_t)best_code;
+            else
+              reinterpret_cast<uint8_t*>(p.codes)[j] = (uint8_t)best_code;
+            if (p.err_out) p.err_out[n] = (float)best_d;
+          }
+        } else {
+          PartialResult r;
+          r.d = best_d;
+          r.code = best_code;
+          r.valid = ok ? 1u : 0u;
+          p.partial[((size_t)blockIdx.x * 2 + slot_of_segment) * TILE + s] = r;
+        }
+      }
+    }
+    compute_bar();
+    first_segment = false;
+    u += c_hi - c_lo;
+  }
+}
+
+// Merge the per-slice results of tiles whose codebook range was split over CTAs.
+template <int TT>
+__global__ void __launch_bounds__(256) encode_m1_merge_kernel(const EncM1Params p) {
+  constexpr int TILE = kEncThreads * TT;
+  const uint32_t tile = blockIdx.x;
+  const uint64_t units = (uint64_t)p.n_tiles * p.n_chunks;
+  const uint64_t t_lo = (uint64_t)tile * p.n_chunks, t_hi = t_lo + p.n_chunks - 1;
+  auto cta_of = [&](uint64_t u) {
+    uint64_t b = u * p.n_ctas / units;
+    while (b + 1 < p.n_ctas && cta_unit_lo(b + 1, units, p.n_ctas) <= u) ++b;
+    while (b > 0 && cta_unit_lo(b, units, p.n_ctas) > u) --b;
+    return (uint32_t)b;
+  };
+  const uint32_t b_first = cta_of(t_lo), b_last = cta_of(t_hi);
+  if (b_first == b_last) return;  // one CTA covered the whole codebook and wrote the result itself
+  for (int s = threadIdx.x; s < TILE; s += blockDim.x) {
+    const uint64_t n = (uint64_t)tile * TILE + s;
+    if (n >= p.k) break;
+    double best_d = __longlong_as_double(0x7ff0000000000000ll);
+    uint32_t best_code = 0xffffffffu;
+    bool ok = true;
+    for (uint32_t b = b_first; b <= b_last; ++b) {
+      const uint64_t lo = cta_unit_lo(b, units, p.n_ctas);
+      if (cta_unit_lo(b + 1, units, p.n_ctas) == lo) continue;  // CTA without work
+      const uint32_t slot = (lo / p.n_chunks == tile) ? 0u : 1u;
+      const PartialResult r = p.partial[((size_t)b * 2 + slot) * TILE + s];
+      ok = ok && r.valid;
+      if (r.d < best_d || (r.d == best_d && r.code < best_code)) {
+        best_d = r.d;
+        best_code = r.code;
+      }
+    }
+    if (ok && best_code < p.K) {
+      const uint32_t j = p.idx[n];
+      if (j < p.G) {
+        if (p.code_u16)
+          reinterpret_cast<uint16_t*>(p.codes)[j] = (uint16_t)best_code;
+        else
+          reinterpret_cast<uint8_t*>(p.codes)[j] = (uint8_t)best_code;
+        if (p.err_out) p.err_out[n] = (float)best_d;
+      }
+    }
+  }
+}
+
+template <int TT>
+cudaError_t launch_tt(const EncM1Params& p, cudaStream_t stream) {
+  const size_t smem = sizeof(EncSmem<TT>);
+  cudaError_t err = cudaFuncSetAttribute(encode_m1_kernel<TT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (err != cudaSuccess) return err;
+  timing_begin(kKernEncodeMain, stream);
+  encode_m1_kernel<TT><<<p.n_ctas, kEncThreads + 32, smem, stream>>>(p);
+  timing_end(kKernEncodeMain, stream);
+  if ((err = cudaGetLastError()) != cudaSuccess) return err;
+  count_launches(1);
+  if (p.n_ctas > 1) {
+    encode_m1_merge_kernel<TT><<<p.n_tiles, 256, 0, stream>>>(p);
+    count_launches(1);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_encode_m1(const pvt_layer& L, uint64_t G, const uint32_t* idx, uint64_t k, float* err_out,
+                             void* ws, int sm_count, cudaStream_t stream) {
+  const int tt = encode_m1_targets_per_thread(k, sm_count);
+  const EncodeM1Layout lay = encode_m1_layout((uint32_t)L.codebook_size, k, sm_count, tt);
+  char* base = static_cast<char*>(ws);
+  EncM1Params p;
+  p.W = L.W;
+  p.g = L.g;
+  p.scale = L.scale;
+  p.idx = idx;
+  p.k = k;
+  p.G = G;
+  p.gpr = (uint32_t)(L.cols / kGroupDim);
+  p.eta = L.eta;
+  p.cbx = reinterpret_cast<const float*>(base + lay.cbx_off);
+  p.n2max_bits = reinterpret_cast<const uint32_t*>(base + lay.n2max_off);
+  p.n_chunks = lay.n_chunks;
+  p.K = (uint32_t)L.codebook_size;
+  p.n_tiles = lay.n_tiles;
+  p.n_ctas = lay.n_ctas;
+  p.partial = reinterpret_cast<PartialResult*>(base + lay.partial_off);
+  p.codes = L.codes;
+  p.code_u16 = L.code_dtype == PVT_U16;
+  p.err_out = err_out;
+  p.status = reinterpret_cast<uint32_t*>(base);
+
+  cudaError_t err = cudaMemsetAsync(base + lay.n2max_off, 0, sizeof(uint32_t), stream);
+  if (err != cudaSuccess) return err;
+  timing_begin(kKernEncodeAux, stream);
+  const uint32_t n_cw = lay.n_chunks * kChunkCodewords;
+  if (L.codebook_dtype == PVT_F16)
+    expand_codebook_kernel<true><<<(n_cw + 255) / 256, 256, 0, stream>>>(
+        L.codebooks, p.K, lay.n_chunks, const_cast<float*>(p.cbx), const_cast<uint32_t*>(p.n2max_bits));
+  else
+    expand_codebook_kernel<false><<<(n_cw + 255) / 256, 256, 0, stream>>>(
+        L.codebooks, p.K, lay.n_chunks, const_cast<float*>(p.cbx), const_cast<uint32_t*>(p.n2max_bits));
+  count_launches(1);
+  timing_end(kKernEncodeAux, stream);
+  if ((err = cudaGetLastError()) != cudaSuccess) return err;
+  return tt == 8 ? launch_tt<8>(p, stream) : launch_tt<4>(p, stream);
+}
+
+}  // namespace pvt

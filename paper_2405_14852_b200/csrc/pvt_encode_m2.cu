@@ -1,0 +1,431 @@
+// Greedy residual beam search of the V step for two additive codebooks
+// (Appendix C: "find the best combination of codes via beam search"; Appendix J:
+// two 8-bit codebooks, group size 8, beam size 8, target = gradient-updated
+// dequantised weight; Eq. 8 for the target; Lemma 3.3 for keeping the previous
+// pair in the pool).
+//
+// One warp per target, persistent grid.  Lane l owns codewords l, l+32, ..., l+224
+// of both codebooks: its slice of codebook 2 stays in registers for the whole
+// kernel (packed as f32x2 pairs), codebook 1 is read from shared memory.
+//   stage 1: score1 = ||c1||^2/2 - <t, c1> for 256 codewords (8 per lane); the
+//            `beam` smallest are extracted with warp-wide integer minimum
+//            reductions on (score bits | code) keys.
+//   stage 2: for each beam entry r = t - c1 and
+//            score2 = ||r||^2/2 + ||c2||^2/2 - <r, c2> for 256 codewords; only the
+//            running minimum is kept.
+// Fast scores are binary32.  Every decision they cannot settle within twice their
+// rounding-error bound (membership of the beam, the final argmin) is taken on
+// binary64 distances accumulated in index order, so the result is the argmin of
+// (distance, code1, code2) over the pool exactly as defined.
+#include <cuda_fp16.h>
+
+#include "pvt_internal.h"
+
+namespace pvt {
+
+size_t encode_m2_workspace_bytes() { return kWsHeaderBytes; }
+
+namespace {
+
+constexpr int kM2Threads = 256;
+constexpr int kM2K = 256;  // codebooks are padded to this many codewords
+constexpr float kPadHalfNorm = 3.0e38f;
+constexpr float kInf = __builtin_huge_valf();
+
+struct EncM2Params {
+  const float* W;
+  const float* g;
+  const float* scale;
+  const uint32_t* idx;
+  uint64_t k, G;
+  uint32_t gpr;
+  float eta;
+  const void* books;
+  int cb_f16;
+  uint32_t K, beam;
+  uint16_t* codes;  // two adjacent bytes per group
+  float* err_out;
+  uint32_t* status;
+};
+
+struct M2Smem {
+  alignas(16) float c1[kM2K][8];
+  alignas(16) float c2[kM2K][8];
+  alignas(16) uint64_t p1[4][8][32];  // stage-1 operands: (c1[l+64q][i], c1[l+64q+32][i])
+  uint64_t h1[4][32];                 // (||c1||^2/2) pairs in the same order
+  float h2[kM2K];
+  float red[kM2Threads / 32][2];
+  float n1max, n2max;
+};
+
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ float min3(float a, float b, float c) {
+  float d;
+  asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  return (uint64_t)__float_as_uint(lo) | ((uint64_t)__float_as_uint(hi) << 32);
+}
+__device__ __forceinline__ float lo_of(uint64_t v) { return __uint_as_float((uint32_t)v); }
+__device__ __forceinline__ float hi_of(uint64_t v) { return __uint_as_float((uint32_t)(v >> 32)); }
+// order-preserving map binary32 -> u32
+__device__ __forceinline__ uint32_t ord(float f) {
+  const uint32_t b = __float_as_uint(f);
+  return b ^ ((b >> 31) ? 0xffffffffu : 0x80000000u);
+}
+__device__ __forceinline__ float unord(uint32_t o) {
+  return __uint_as_float(o ^ ((o >> 31) ? 0x80000000u : 0xffffffffu));
+}
+
+// ||t - c||^2 in binary64, the operations of the definition in index order
+__device__ __forceinline__ double exact1(const float* t, const float* c) {
+  double d = 0.0;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const double e = __dsub_rn((double)t[i], (double)c[i]);
+    d = __dadd_rn(d, __dmul_rn(e, e));
+  }
+  return d;
+}
+// ||(t - c1) - c2||^2 in binary64, residual carried in binary64
+__device__ __forceinline__ double exact2(const float* t, const float* c1, const float* c2) {
+  double d = 0.0;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const double r = __dsub_rn((double)t[i], (double)c1[i]);
+    const double e = __dsub_rn(r, (double)c2[i]);
+    d = __dadd_rn(d, __dmul_rn(e, e));
+  }
+  return d;
+}
+
+__device__ __forceinline__ float load_cb(const void* books, int f16, uint32_t m, uint32_t kappa, uint32_t K, int i) {
+  const size_t off = ((size_t)m * K + kappa) * 8 + i;
+  return f16 ? __half2float(reinterpret_cast<const __half*>(books)[off]) : reinterpret_cast<const float*>(books)[off];
+}
+
+__global__ void __launch_bounds__(kM2Threads, 1) encode_m2_kernel(const EncM2Params p) {
+  __shared__ M2Smem sm;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  // ---- stage the codebooks: one codeword per thread (K <= 256 = block size) ----
+  {
+    float c1[8], c2[8], n1 = 0.0f, n2 = 0.0f;
+    const bool real = (uint32_t)tid < p.K;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      c1[i] = real ? load_cb(p.books, p.cb_f16, 0, tid, p.K, i) : 0.0f;
+      c2[i] = real ? load_cb(p.books, p.cb_f16, 1, tid, p.K, i) : 0.0f;
+      n1 = __fmaf_rn(c1[i], c1[i], n1);
+      n2 = __fmaf_rn(c2[i], c2[i], n2);
+      sm.c1[tid][i] = c1[i];
+      sm.c2[tid][i] = c2[i];
+    }
+    const float h1 = real ? 0.5f * n1 : kPadHalfNorm, h2 = real ? 0.5f * n2 : kPadHalfNorm;
+    // codeword tid = l + 32*jj, jj = 2q + half
+    const int l = tid & 31, jj = tid >> 5, q = jj >> 1, half = jj & 1;
+    float* p1f = reinterpret_cast<float*>(&sm.p1[0][0][0]);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) p1f[(((q * 8 + i) * 32) + l) * 2 + half] = c1[i];
+    reinterpret_cast<float*>(&sm.h1[0][0])[(q * 32 + l) * 2 + half] = h1;
+    sm.h2[tid] = h2;
+    float m1 = n1, m2 = n2;
+#pragma unroll
+    for (int o = 16; o; o >>= 1) {
+      m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, o));
+      m2 = fmaxf(m2, __shfl_xor_sync(0xffffffffu, m2, o));
+    }
+    if (lane == 0) {
+      sm.red[warp][0] = m1;
+      sm.red[warp][1] = m2;
+    }
+    __syncthreads();
+    if (tid == 0) {
+      float a = 0.0f, b = 0.0f;
+      for (int w = 0; w < kM2Threads / 32; ++w) {
+        a = fmaxf(a, sm.red[w][0]);
+        b = fmaxf(b, sm.red[w][1]);
+      }
+      sm.n1max = a;
+      sm.n2max = b;
+    }
+    __syncthreads();
+  }
+  // this lane's slice of codebook 2, packed (c2[l+64q][i], c2[l+64q+32][i])
+  uint64_t c2p[4][8], h2p[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int ka = lane + 64 * q, kb = ka + 32;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) c2p[q][i] = pack2(sm.c2[ka][i], sm.c2[kb][i]);
+    h2p[q] = pack2(sm.h2[ka], sm.h2[kb]);
+  }
+  const float n1max = sm.n1max, n2max = sm.n2max;
+  const float s1max = sqrtf(n1max), s2max = sqrtf(n2max);
+  const uint32_t B = p.beam;  // already min(beam, K)
+
+  const float4* W4 = reinterpret_cast<const float4*>(p.W);
+  const float4* g4 = reinterpret_cast<const float4*>(p.g);
+  const uint64_t nwarps = (uint64_t)gridDim.x * (kM2Threads / 32);
+
+  for (uint64_t n = (uint64_t)blockIdx.x * (kM2Threads / 32) + warp; n < p.k; n += nwarps) {
+    const uint32_t j = __ldg(p.idx + n);
+    if (j >= p.G) {
+      if (lane == 0) atomicOr(p.status, PVT_DEV_BAD_INDEX);
+      continue;
+    }
+    // target, binary32: one fma, one division (every lane holds all 8 values)
+    float t[8];
+    {
+      const float4 w0 = __ldg(W4 + 2 * (size_t)j), w1 = __ldg(W4 + 2 * (size_t)j + 1);
+      const float4 g0 = __ldg(g4 + 2 * (size_t)j), g1 = __ldg(g4 + 2 * (size_t)j + 1);
+      const float sc = __ldg(p.scale + j / p.gpr), ne = -p.eta;
+      t[0] = __fdiv_rn(__fmaf_rn(ne, g0.x, w0.x), sc);
+      t[1] = __fdiv_rn(__fmaf_rn(ne, g0.y, w0.y), sc);
+      t[2] = __fdiv_rn(__fmaf_rn(ne, g0.z, w0.z), sc);
+      t[3] = __fdiv_rn(__fmaf_rn(ne, g0.w, w0.w), sc);
+      t[4] = __fdiv_rn(__fmaf_rn(ne, g1.x, w1.x), sc);
+      t[5] = __fdiv_rn(__fmaf_rn(ne, g1.y, w1.y), sc);
+      t[6] = __fdiv_rn(__fmaf_rn(ne, g1.z, w1.z), sc);
+      t[7] = __fdiv_rn(__fmaf_rn(ne, g1.w, w1.w), sc);
+    }
+    const uint32_t prev = p.codes[j];
+    float nt2 = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) nt2 = fmaf(t[i], t[i], nt2);
+    const float tnorm = sqrtf(nt2);
+    // twice the rounding-error bounds of the two fast scores (factor >= 2 to spare), u = 2^-24:
+    //   |score1_fl - score1| <= 16.1 u (||c1||^2/2 + ||t|| ||c1||)
+    //   |score2_fl - score2| <= 26 u (||t|| + max||c1|| + max||c2||)^2
+    const float margin1 = 3.8146973e-6f /* 2^-18 */ * (0.5f * n1max + tnorm * s1max) + 1e-30f;
+    const float sall = tnorm + s1max + s2max;
+    const float margin2 = 7.6293945e-6f /* 2^-17 */ * sall * sall + 1e-30f;
+
+    // ---- stage 1: 256 scores, 8 per lane
+    float f[8];
+    {
+      uint64_t acc[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) acc[q] = sm.h1[q][lane];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const uint64_t ntd = pack2(-t[i], -t[i]);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) acc[q] = fma2(ntd, sm.p1[q][i][lane], acc[q]);
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        f[2 * q] = lo_of(acc[q]);
+        f[2 * q + 1] = hi_of(acc[q]);
+      }
+    }
+    // extract the B smallest (score truncated to 24 bits | code): a first guess of the beam
+    uint32_t key[8];
+#pragma unroll
+    for (int jj = 0; jj < 8; ++jj) key[jj] = (ord(f[jj]) & 0xffffff00u) | (uint32_t)(lane + 32 * jj);
+    uint32_t beam_code[8];
+#pragma unroll
+    for (int b = 0; b < 8; ++b) {
+      beam_code[b] = 0;
+      if ((uint32_t)b < B) {
+        uint32_t lm = key[0];
+#pragma unroll
+        for (int jj = 1; jj < 8; ++jj) lm = min(lm, key[jj]);
+        const uint32_t m = __reduce_min_sync(0xffffffffu, lm);
+        beam_code[b] = m & 0xffu;
+#pragma unroll
+        for (int jj = 0; jj < 8; ++jj)
+          if (key[jj] == m) key[jj] = 0xffffffffu;
+      }
+    }
+    // is that guess provably the exact beam?  theta = largest score in the guess;
+    // every member of the exact beam scores <= theta + margin1; if exactly B
+    // codewords do, they are the guess and the exact beam at once.
+    {
+      float th = -kInf;
+      uint32_t cnt = 0;
+#pragma unroll
+      for (int jj = 0; jj < 8; ++jj)
+        if (key[jj] == 0xffffffffu) th = fmaxf(th, f[jj]);
+      const float theta = unord(__reduce_max_sync(0xffffffffu, ord(th)));
+      const float limit1 = theta + margin1;
+      uint32_t member = 0;
+#pragma unroll
+      for (int jj = 0; jj < 8; ++jj) {
+        const bool in = f[jj] <= limit1 && (uint32_t)(lane + 32 * jj) < p.K;
+        member |= in ? (1u << jj) : 0u;
+        cnt += in;
+      }
+      cnt = __reduce_add_sync(0xffffffffu, cnt);
+      if (cnt != B) {
+        // undecided: order the shortlisted codewords by (binary64 distance, code)
+        for (uint32_t b = 0; b < B; ++b) {
+          double ld = __longlong_as_double(0x7ff0000000000000ll);
+          uint32_t lk = 0xffffffffu;
+#pragma unroll
+          for (int jj = 0; jj < 8; ++jj) {
+            if (member & (1u << jj)) {
+              const uint32_t kap = lane + 32 * jj;
+              const double d = exact1(t, sm.c1[kap]);
+              if (d < ld || (d == ld && kap < lk)) {
+                ld = d;
+                lk = kap;
+              }
+            }
+          }
+          // warp-wide lexicographic minimum of (ld, lk); distances are >= 0 so their bits order like u64
+          const uint64_t bits = (uint64_t)__double_as_longlong(ld);
+          const uint32_t hi = (uint32_t)(bits >> 32), lo = (uint32_t)bits;
+          const uint32_t mhi = __reduce_min_sync(0xffffffffu, hi);
+          const uint32_t mlo = __reduce_min_sync(0xffffffffu, hi == mhi ? lo : 0xffffffffu);
+          const uint32_t mk = __reduce_min_sync(0xffffffffu, (hi == mhi && lo == mlo) ? lk : 0xffffffffu);
+          const uint32_t chosen = mk < kM2K ? mk : 0u;
+#pragma unroll
+          for (int bb = 0; bb < 8; ++bb)
+            if ((uint32_t)bb == b) beam_code[bb] = chosen;
+          if ((chosen & 31u) == (uint32_t)lane) member &= ~(1u << (chosen >> 5));
+        }
+      }
+    }
+
+    // ---- stage 2: every beam entry against codebook 2, running minimum only
+    float cm[8];
+#pragma unroll
+    for (int b = 0; b < 8; ++b) {
+      cm[b] = kInf;
+      if ((uint32_t)b < B) {
+        const float4 ca = *reinterpret_cast<const float4*>(&sm.c1[beam_code[b]][0]);
+        const float4 cb = *reinterpret_cast<const float4*>(&sm.c1[beam_code[b]][4]);
+        const float c1v[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
+        float r[8], rho = 0.0f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          r[i] = __fsub_rn(t[i], c1v[i]);
+          rho = __fmaf_rn(r[i], r[i], rho);
+        }
+        rho = __fmul_rn(0.5f, rho);
+        const uint64_t rho2 = pack2(rho, rho);
+        uint64_t acc[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) acc[q] = add2(h2p[q], rho2);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const uint64_t nrd = pack2(-r[i], -r[i]);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) acc[q] = fma2(nrd, c2p[q][i], acc[q]);
+        }
+        float m = min3(lo_of(acc[0]), hi_of(acc[0]), lo_of(acc[1]));
+        m = min3(m, hi_of(acc[1]), lo_of(acc[2]));
+        m = min3(m, hi_of(acc[2]), lo_of(acc[3]));
+        cm[b] = fminf(m, hi_of(acc[3]));
+      }
+    }
+    float lmin = cm[0];
+#pragma unroll
+    for (int b = 1; b < 8; ++b) lmin = fminf(lmin, cm[b]);
+    const float limit2 = unord(__reduce_min_sync(0xffffffffu, ord(lmin))) + margin2;
+
+    // ---- decision in binary64 among the pairs within the margin, plus the previous pair
+    double bd = __longlong_as_double(0x7ff0000000000000ll);
+    uint32_t bk = 0xffffffffu;  // code1 << 8 | code2: orders like (code1, code2)
+#pragma unroll
+    for (int b = 0; b < 8; ++b) {
+      if ((uint32_t)b < B && __any_sync(0xffffffffu, cm[b] <= limit2)) {
+        const uint32_t k1 = beam_code[b];
+        const float4 ca = *reinterpret_cast<const float4*>(&sm.c1[k1][0]);
+        const float4 cb = *reinterpret_cast<const float4*>(&sm.c1[k1][4]);
+        const float c1v[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
+        float r[8], rho = 0.0f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          r[i] = __fsub_rn(t[i], c1v[i]);
+          rho = __fmaf_rn(r[i], r[i], rho);
+        }
+        rho = __fmul_rn(0.5f, rho);
+#pragma unroll
+        for (int jj = 0; jj < 8; ++jj) {
+          const uint32_t k2 = lane + 32 * jj;
+          float s = __fadd_rn(sm.h2[k2], rho);  // the same operations as the packed evaluation
+#pragma unroll
+          for (int i = 0; i < 8; ++i) s = __fmaf_rn(-r[i], sm.c2[k2][i], s);
+          if (s <= limit2 && k2 < p.K) {
+            const double d = exact2(t, c1v, sm.c2[k2]);
+            const uint32_t kk = (k1 << 8) | k2;
+            if (d < bd || (d == bd && kk < bk)) {
+              bd = d;
+              bk = kk;
+            }
+          }
+        }
+      }
+    }
+    // previous pair (lane 0 carries it into the reduction)
+    if (lane == 0) {
+      const uint32_t q1 = prev & 0xffu, q2 = prev >> 8;
+      if (q1 < p.K && q2 < p.K) {
+        const double d = exact2(t, sm.c1[q1], sm.c2[q2]);
+        const uint32_t kk = (q1 << 8) | q2;
+        if (d < bd || (d == bd && kk < bk)) {
+          bd = d;
+          bk = kk;
+        }
+      } else {
+        atomicOr(p.status, PVT_DEV_BAD_CODE);
+      }
+    }
+    // warp-wide lexicographic minimum of (bd, bk)
+    {
+      const uint64_t bits = (uint64_t)__double_as_longlong(bd);
+      const uint32_t hi = (uint32_t)(bits >> 32), lo = (uint32_t)bits;
+      const uint32_t mhi = __reduce_min_sync(0xffffffffu, hi);
+      const uint32_t mlo = __reduce_min_sync(0xffffffffu, hi == mhi ? lo : 0xffffffffu);
+      const uint32_t mk = __reduce_min_sync(0xffffffffu, (hi == mhi && lo == mlo) ? bk : 0xffffffffu);
+      if (lane == 0 && mk != 0xffffffffu) {
+        p.codes[j] = (uint16_t)(((mk >> 8) & 0xffu) | ((mk & 0xffu) << 8));
+        if (p.err_out) p.err_out[n] = (float)__longlong_as_double((long long)(((uint64_t)mhi << 32) | mlo));
+      }
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_encode_m2(const pvt_layer& L, uint64_t G, const uint32_t* idx, uint64_t k, float* err_out,
+                             void* ws, int sm_count, cudaStream_t stream) {
+  EncM2Params p;
+  p.W = L.W;
+  p.g = L.g;
+  p.scale = L.scale;
+  p.idx = idx;
+  p.k = k;
+  p.G = G;
+  p.gpr = (uint32_t)(L.cols / kGroupDim);
+  p.eta = L.eta;
+  p.books = L.codebooks;
+  p.cb_f16 = L.codebook_dtype == PVT_F16;
+  p.K = (uint32_t)L.codebook_size;
+  p.beam = (uint32_t)L.beam < p.K ? (uint32_t)L.beam : p.K;
+  p.codes = reinterpret_cast<uint16_t*>(L.codes);
+  p.err_out = err_out;
+  p.status = reinterpret_cast<uint32_t*>(ws);
+  const uint64_t warps_per_cta = kM2Threads / 32;
+  uint64_t ctas = (k + warps_per_cta - 1) / warps_per_cta;
+  if (ctas > (uint64_t)sm_count) ctas = (uint64_t)sm_count;
+  timing_begin(kKernEncodeMain, stream);
+  encode_m2_kernel<<<(unsigned)ctas, kM2Threads, 0, stream>>>(p);
+  count_launches(1);
+  timing_end(kKernEncodeMain, stream);
+  return cudaGetLastError();
+}
+
+}  // namespace pvt

@@ -1,0 +1,96 @@
+// Internal declarations shared by the translation units of libpvt (host side
+// launchers, workspace layout, small device helpers).  Not part of the ABI.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "pvt.h"
+
+namespace pvt {
+
+constexpr int kGroupDim = 8;
+constexpr int kSmCountFallback = 148;
+
+// ---- workspace layout -------------------------------------------------------
+// [0, 256)            header: status word (u32 at 0), selection state, counters
+// [256, ...)          region shared by select and encode (they run one after the
+//                     other on a stream and never need each other's scratch)
+constexpr size_t kWsHeaderBytes = 256;
+constexpr size_t kWsAlign = 256;
+
+// selection -------------------------------------------------------------------
+constexpr int kSelTile = 4096;      // groups per block of the select kernels
+constexpr int kSelThreads = 256;    // 16 groups per thread
+constexpr int kSelBins0 = 2048;     // key bits [30:20]
+constexpr int kSelBins1 = 2048;     // key bits [19:9]
+constexpr int kSelBins2 = 512;      // key bits [8:0]
+
+struct SelectState {        // lives in the header at byte 64
+  uint32_t digit0, digit1;  // threshold digits found so far
+  uint32_t threshold;       // full threshold key once the last digit is known
+  uint32_t need_eq;         // how many groups with key == threshold are taken (lowest indices)
+  uint64_t k_left;          // groups still to be taken from the current bucket
+  uint32_t done[4];         // block-completion counters of the passes
+};
+constexpr size_t kSelStateOffset = 64;
+
+struct SelectLayout {
+  size_t hist_off;   // u32 [2048 + 2048 + 512]
+  size_t keys_off;   // u32 [G]
+  size_t tiles_off;  // u32 [2 * ntiles]: (greater, equal) counts, later exclusive offsets
+  size_t bytes;      // end of the region (from the workspace base)
+  uint32_t ntiles;
+};
+SelectLayout select_layout(uint64_t G);
+
+// encode, M = 1 ---------------------------------------------------------------
+constexpr int kEncThreads = 256;     // compute threads per CTA (8 warps) + 1 producer warp
+constexpr int kChunkCodewords = 256; // codewords per staged chunk (one bulk copy)
+constexpr int kSubCodewords = 32;    // tracking granularity of the running minimum
+constexpr int kChunkBytes = kChunkCodewords * (kGroupDim * 4 + 4);  // 9216: pairs interleaved + half norms
+constexpr int kEncStages = 4;
+constexpr int kListLen = 4;          // remembered near-minimum sub-chunks per target
+
+struct EncodeM1Layout {
+  size_t cbx_off;      // expanded codebook: n_chunks * kChunkBytes
+  size_t n2max_off;    // u32 bit pattern of max ||c||^2
+  size_t partial_off;  // per CTA: 2 segments * tile * 16 bytes
+  size_t bytes;
+  uint32_t n_chunks;
+  uint32_t tile;       // targets per tile (kEncThreads * TT)
+  uint32_t n_tiles;
+  uint32_t n_ctas;
+};
+EncodeM1Layout encode_m1_layout(uint32_t K, uint64_t k, int sm_count, int targets_per_thread);
+int encode_m1_targets_per_thread(uint64_t k, int sm_count);  // 4 or 8
+size_t encode_m2_workspace_bytes();
+
+struct PartialResult {  // one (target, codebook slice) result awaiting the merge
+  double d;
+  uint32_t code;
+  uint32_t valid;
+};
+
+// launchers (each returns a cudaError_t) --------------------------------------
+cudaError_t launch_select(const pvt_layer& L, uint64_t G, uint64_t k, uint32_t* idx_out, void* ws,
+                          cudaStream_t stream);
+cudaError_t launch_encode_m1(const pvt_layer& L, uint64_t G, const uint32_t* idx, uint64_t k, float* err_out,
+                             void* ws, int sm_count, cudaStream_t stream);
+cudaError_t launch_encode_m2(const pvt_layer& L, uint64_t G, const uint32_t* idx, uint64_t k, float* err_out,
+                             void* ws, int sm_count, cudaStream_t stream);
+cudaError_t launch_dequant(const pvt_layer& L, uint64_t G, void* W_hat, int32_t out_dtype, uint32_t* status,
+                           cudaStream_t stream);
+
+// optional per-kernel timing (benchmark instrumentation) ----------------------
+enum KernelId { kKernSelect = 0, kKernEncodeMain = 1, kKernEncodeAux = 2, kKernDequant = 3, kKernCount = 4 };
+void timing_begin(KernelId id, cudaStream_t stream);
+void timing_end(KernelId id, cudaStream_t stream);
+
+// number of kernels launched by this process through the library (a claim the benchmark reports)
+void count_launches(int n);
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace pvt

@@ -1,0 +1,91 @@
+"""The C ABI without a GPU: the library loads, exports every function that
+include/pvt.h declares, and rejects bad arguments before touching CUDA."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2405_14852_b200 import binding as B
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "pvt.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(pvt_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_function_is_exported():
+    names = declared_functions()
+    assert {"pvt_vstep_select", "pvt_vstep_encode", "pvt_dequant", "pvt_workspace_bytes", "pvt_status"} <= set(names)
+    L = ctypes.CDLL(B.library_path()) if os.path.exists(B.library_path()) else B.lib()
+    for n in names:
+        assert hasattr(L, n), f"{n} is declared in pvt.h but not exported"
+
+
+def test_version_and_error_text():
+    assert B.pvt_version() >= 100
+    for code in (0, -1, -2, -3, -4):
+        assert B.strerror(code)
+
+
+def _layer(**kw):
+    base = dict(rows=16, cols=64, group_dim=8, num_codebooks=1, codebook_size=256, codebook_dtype=B.PVT_F16,
+                code_dtype=B.PVT_U8, beam=8, eta=1.0, reserved_=0, W=0x1000, g=0x1000, scale=0x1000,
+                codebooks=0x1000, codes=0x1000)
+    base.update(kw)
+    return B.pvt_layer(**base)
+
+
+def test_workspace_bytes_depends_on_shape_not_on_a_device():
+    small = B.pvt_workspace_bytes(_layer(), 16)
+    big = B.pvt_workspace_bytes(_layer(rows=4096, cols=4096, codebook_size=65536, code_dtype=B.PVT_U16), 20971)
+    assert 0 < small < big
+    assert big >= 4 * 4096 * 512  # one key per group
+
+
+@pytest.mark.parametrize("kw,k,code", [
+    (dict(), 0, B.PVT_EINVAL),                      # k = 0
+    (dict(), 16 * 8 + 1, B.PVT_EINVAL),             # k > G
+    (dict(cols=60), 1, B.PVT_EINVAL),               # cols % 8
+    (dict(group_dim=16), 1, B.PVT_EUNSUPPORTED),
+    (dict(eta=-1.0), 1, B.PVT_EINVAL),
+    (dict(eta=float("nan")), 1, B.PVT_EINVAL),
+    (dict(g=None), 1, B.PVT_EINVAL),
+    (dict(g=0x1004), 1, B.PVT_EINVAL),              # misaligned
+])
+def test_select_rejects_bad_arguments_before_launch(kw, k, code):
+    L = _layer(**kw)
+    rc = B.lib().pvt_vstep_select(ctypes.byref(L), k, 0x2000, 0x4000, 1 << 30, None)
+    assert rc == code
+
+
+@pytest.mark.parametrize("kw,code", [
+    (dict(num_codebooks=3), B.PVT_EUNSUPPORTED),
+    (dict(codebook_size=1), B.PVT_EUNSUPPORTED),
+    (dict(codebook_size=70000, code_dtype=B.PVT_U16), B.PVT_EUNSUPPORTED),
+    (dict(codebook_size=512), B.PVT_EINVAL),        # 512 codewords do not fit U8 codes
+    (dict(num_codebooks=2, codebook_size=512, code_dtype=B.PVT_U16), B.PVT_EUNSUPPORTED),
+    (dict(num_codebooks=2, beam=9), B.PVT_EUNSUPPORTED),
+    (dict(codebook_dtype=7), B.PVT_EINVAL),
+    (dict(W=None), B.PVT_EINVAL),
+])
+def test_encode_rejects_bad_arguments_before_launch(kw, code):
+    L = _layer(**kw)
+    rc = B.lib().pvt_vstep_encode(ctypes.byref(L), 0x2000, 4, None, 0x4000, 1 << 30, None)
+    assert rc == code
+
+
+def test_too_small_workspace_is_reported():
+    L = _layer()
+    assert B.lib().pvt_vstep_select(ctypes.byref(L), 4, 0x2000, 0x4000, 256, None) == B.PVT_EWORKSPACE
+    assert B.lib().pvt_vstep_encode(ctypes.byref(L), 0x2000, 4, None, 0x4000, 256, None) == B.PVT_EWORKSPACE
+    assert B.lib().pvt_vstep_select(ctypes.byref(L), 4, 0x2000, 0x4010, 1 << 30, None) == B.PVT_EINVAL  # alignment
+
+
+def test_dequant_rejects_bad_arguments():
+    L = _layer()
+    assert B.lib().pvt_dequant(ctypes.byref(L), None, B.PVT_F32, None, None) == B.PVT_EINVAL
+    assert B.lib().pvt_dequant(ctypes.byref(L), 0x2000, 5, None, None) == B.PVT_EINVAL
