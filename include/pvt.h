@@ -55,6 +55,7 @@ extern "C" {
 #define PVT_EUNSUPPORTED (-2) /* group_dim / M / K / dtype / beam combination this build has no kernel for */
 #define PVT_EWORKSPACE (-3)   /* ws_bytes smaller than pvt_workspace_bytes() */
 #define PVT_ECUDA (-4)        /* a CUDA runtime call or kernel launch failed; see pvt_last_cuda_error() */
+#define PVT_ETOOLARGE (-5)    /* pvt_vstep_select_noalloc only: the layer exceeds the built-in scratch */
 
 /* device-side status bits (pvt_status) */
 #define PVT_DEV_BAD_INDEX 1u    /* an entry of idx was >= G; that entry was skipped */
@@ -111,6 +112,43 @@ int pvt_workspace_init(void* ws, size_t ws_bytes, void* cuda_stream);
  */
 int pvt_vstep_select(const pvt_layer* layer, uint64_t k, uint32_t* idx_out, void* ws, size_t ws_bytes,
                      void* cuda_stream);
+
+/*
+ * pvt_vstep_select for callers that cannot allocate device memory.  (No
+ * counterpart in the paper: this is a packaging variant of the call above and
+ * computes exactly the same idx_out.)
+ *
+ * Who needs it: code that has to pick the subspace at a point where no device
+ * allocation is possible -- a training process whose memory pool was handed out
+ * completely at start-up, a component living inside a host application that
+ * owns all device memory, or a thread that must not enter an allocator (a
+ * cudaMalloc would also synchronise the device).  Such callers cannot supply the
+ * ~4 bytes per group of workspace that pvt_vstep_select asks for.  Here the
+ * scratch is a fixed array inside the library image instead; the caller passes
+ * only the layer, k and the outputs.
+ *
+ * Limits and rules
+ *   - At most PVT_NOALLOC_MAX_GROUPS groups (2^21, e.g. one 4096 x 4096 layer);
+ *     a larger layer is rejected with PVT_ETOOLARGE before anything is enqueued.
+ *   - The array (about 8.03 MiB) is resident on every GPU that loads the library,
+ *     from load until the process exits, whether or not this call is ever used.
+ *   - The first call on each device looks up the array's device address (a
+ *     host-side runtime query; the device must be current).  Make that first
+ *     call outside any stream capture.
+ *   - Every call on a device uses the same array.  Calls whose kernels may
+ *     overlap on the GPU (different streams, different host threads) race on it
+ *     and give wrong results: issue them on one stream, or order them yourself.
+ *     What must start at zero is cleared at the start of every call; nothing
+ *     else of a previous call is relied upon.
+ *   - The call itself performs no allocation of any kind (no cudaMalloc /
+ *     cudaFree, no allocating library routine) and does not synchronise.
+ * status_out: NULL, or a device uint32 that receives the PVT_DEV_* bits of this
+ * call (written by a copy enqueued after the kernels).
+ * Other arguments and return codes as pvt_vstep_select.
+ */
+#define PVT_NOALLOC_MAX_GROUPS (1ull << 21)
+int pvt_vstep_select_noalloc(const pvt_layer* layer, uint64_t k, uint32_t* idx_out, uint32_t* status_out,
+                             void* cuda_stream);
 
 /*
  * Re-encode the k groups listed in idx (Eq. 8; Appendix C / Appendix J;

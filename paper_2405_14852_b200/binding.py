@@ -18,7 +18,8 @@ from . import build as _build
 
 PVT_F32, PVT_F16 = 0, 1
 PVT_U8, PVT_U16 = 0, 1
-PVT_OK, PVT_EINVAL, PVT_EUNSUPPORTED, PVT_EWORKSPACE, PVT_ECUDA = 0, -1, -2, -3, -4
+PVT_OK, PVT_EINVAL, PVT_EUNSUPPORTED, PVT_EWORKSPACE, PVT_ECUDA, PVT_ETOOLARGE = 0, -1, -2, -3, -4, -5
+PVT_NOALLOC_MAX_GROUPS = 1 << 21
 PVT_DEV_BAD_INDEX, PVT_DEV_BAD_CODE, PVT_DEV_WAIT_EXPIRED, PVT_DEV_INTERNAL = 1, 2, 4, 8
 PVT_KERNEL_SELECT, PVT_KERNEL_ENCODE_MAIN, PVT_KERNEL_ENCODE_AUX, PVT_KERNEL_DEQUANT = 0, 1, 2, 3
 
@@ -68,6 +69,8 @@ def lib():
         L.pvt_workspace_init.argtypes = [vp, sz, vp]
         L.pvt_vstep_select.restype = ctypes.c_int
         L.pvt_vstep_select.argtypes = [lp, u64, vp, vp, sz, vp]
+        L.pvt_vstep_select_noalloc.restype = ctypes.c_int
+        L.pvt_vstep_select_noalloc.argtypes = [lp, u64, vp, vp, vp]
         L.pvt_vstep_encode.restype = ctypes.c_int
         L.pvt_vstep_encode.argtypes = [lp, vp, u64, vp, vp, sz, vp]
         L.pvt_dequant.restype = ctypes.c_int
@@ -145,6 +148,17 @@ def new_workspace(layer: pvt_layer, k: int, device=None) -> torch.Tensor:
 def pvt_vstep_select(layer: pvt_layer, k: int, idx_out: torch.Tensor, ws: torch.Tensor, stream=None) -> None:
     _check(lib().pvt_vstep_select(ctypes.byref(layer), k, idx_out.data_ptr(), ws.data_ptr(),
                                   ws.numel() * ws.element_size(), _stream_ptr(stream)), "pvt_vstep_select")
+
+
+def pvt_vstep_select_noalloc(layer: pvt_layer, k: int, idx_out: torch.Tensor,
+                             status_out: Optional[torch.Tensor] = None, stream=None) -> None:
+    """pvt_vstep_select without a workspace argument: for callers that cannot
+    allocate device memory (frozen memory pool, host application owning the
+    device memory, allocator-free thread).  The scratch is a fixed array inside
+    the library, so the layer may have at most PVT_NOALLOC_MAX_GROUPS groups, and
+    calls that could overlap on the GPU must be ordered by the caller."""
+    _check(lib().pvt_vstep_select_noalloc(ctypes.byref(layer), k, idx_out.data_ptr(), _ptr(status_out),
+                                          _stream_ptr(stream)), "pvt_vstep_select_noalloc")
 
 
 def pvt_vstep_encode(layer: pvt_layer, idx: torch.Tensor, k: int, err_out: Optional[torch.Tensor],

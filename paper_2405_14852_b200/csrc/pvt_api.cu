@@ -69,6 +69,8 @@ Timing& timing() {
 
 }  // namespace
 
+void record_cuda_error(cudaError_t e) { g_last_cuda = e; }
+
 void count_launches(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
 
 void timing_begin(KernelId id, cudaStream_t stream) {
@@ -192,6 +194,7 @@ const char* pvt_strerror(int code) {
     case PVT_EUNSUPPORTED: return "unsupported group_dim / codebook count / codebook size / dtype / beam";
     case PVT_EWORKSPACE: return "workspace smaller than pvt_workspace_bytes()";
     case PVT_ECUDA: return "CUDA runtime error (see pvt_last_cuda_error)";
+    case PVT_ETOOLARGE: return "layer larger than the built-in scratch of pvt_vstep_select_noalloc (2^21 groups)";
     default: return code > 0 ? "device status bits set" : "unknown error";
   }
 }

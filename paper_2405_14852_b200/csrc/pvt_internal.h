@@ -88,6 +88,9 @@ enum KernelId { kKernSelect = 0, kKernEncodeMain = 1, kKernEncodeAux = 2, kKernD
 void timing_begin(KernelId id, cudaStream_t stream);
 void timing_end(KernelId id, cudaStream_t stream);
 
+// remembers the CUDA error behind a PVT_ECUDA return for pvt_last_cuda_error (per host thread)
+void record_cuda_error(cudaError_t e);
+
 // number of kernels launched by this process through the library (a claim the benchmark reports)
 void count_launches(int n);
 
