@@ -180,7 +180,7 @@ def run_ours(args):
         sampler.start()
         time.sleep(0.3)
     B.pvt_timing_enable(True)
-    for kid in range(4):
+    for kid in range(5):
         B.pvt_timing_read(kid)
     launches0 = B.pvt_launch_count()
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
@@ -194,7 +194,7 @@ def run_ours(args):
     barrier()
     launches = B.pvt_launch_count() - launches0
     total_ms = sum(a.elapsed_time(b) for a, b in ev)
-    kern = {kid: B.pvt_timing_read(kid) for kid in range(4)}
+    kern = {kid: B.pvt_timing_read(kid) for kid in range(5)}
     B.pvt_timing_enable(False)
     st = B.pvt_status(ws)
     if st != 0:
@@ -247,6 +247,8 @@ def run_ours(args):
         stages["encode_search"] = {"ms": enc_avg_ms, "pairs": pairs,
                                    "pairs_per_s": pairs / (enc_avg_ms * 1e-3)}
         stages["encode_codebook_prep"] = {"ms": aux_ms / max(aux_n, 1)}
+        rs_ms, rs_n = kern[B.PVT_KERNEL_ENCODE_RESCORE]
+        stages["encode_rescore"] = {"ms": rs_ms / max(rs_n, 1)}
         stages["dequant"] = {"ms": dq_ms / max(dq_n, 1), "algorithmic_bytes": dq_bytes,
                              "gbs": dq_bytes / (dq_ms / max(dq_n, 1) * 1e-3) / 1e9 if dq_n else None}
         if hbm:

@@ -206,6 +206,7 @@ int pvt_version(void);
 #define PVT_KERNEL_ENCODE_MAIN 1 /* the search kernel of pvt_vstep_encode */
 #define PVT_KERNEL_ENCODE_AUX 2  /* codebook expansion before the M = 1 search */
 #define PVT_KERNEL_DEQUANT 3     /* the kernel of pvt_dequant */
+#define PVT_KERNEL_ENCODE_RESCORE 4 /* exact rescoring and code write after the M = 1 search */
 void pvt_timing_enable(int on);
 /* Kernels this process has launched through the library so far (memsets not counted). */
 unsigned long long pvt_launch_count(void);

@@ -22,6 +22,7 @@ PVT_OK, PVT_EINVAL, PVT_EUNSUPPORTED, PVT_EWORKSPACE, PVT_ECUDA, PVT_ETOOLARGE =
 PVT_NOALLOC_MAX_GROUPS = 1 << 21
 PVT_DEV_BAD_INDEX, PVT_DEV_BAD_CODE, PVT_DEV_WAIT_EXPIRED, PVT_DEV_INTERNAL = 1, 2, 4, 8
 PVT_KERNEL_SELECT, PVT_KERNEL_ENCODE_MAIN, PVT_KERNEL_ENCODE_AUX, PVT_KERNEL_DEQUANT = 0, 1, 2, 3
+PVT_KERNEL_ENCODE_RESCORE = 4
 
 
 class pvt_layer(ctypes.Structure):

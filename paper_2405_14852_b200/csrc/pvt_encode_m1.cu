@@ -2,10 +2,11 @@
 // Appendix J: "try every code in the codebook"; Appendix D: the score
 // ||c||^2 - 2 <t, c>; Eq. 8 for the target t = (W - eta g) / s).
 //
-// Work decomposition: targets are cut into tiles of 256*TT groups, the codebook
-// into chunks of 256 codewords; the (tile, chunk) grid is flattened and split
-// evenly over one persistent CTA per SM, so a CTA works on a few segments
-// (tile, chunk range).  Per segment:
+// Two kernels.
+//
+// Search.  Targets are cut into tiles of 256*TT groups, the codebook into slices
+// of whole 256-codeword chunks; the (tile, slice) units are dealt round-robin to
+// one persistent CTA per SM.  Per unit:
 //   1. every compute thread gathers TT targets (32 B of W and of g each), forms t
 //      in binary32 and keeps -t in registers, duplicated into f32x2 pairs;
 //   2. a producer warp streams the pre-expanded codebook (pairs of codewords
@@ -20,14 +21,15 @@
 //   4. every 32 codewords the running minimum of that sub-chunk is compared with
 //      the best so far; sub-chunks within a rounding-error margin of the best are
 //      remembered (4 most recent per target);
-//   5. after the loop each warp revisits the remembered sub-chunks of its
-//      targets, recomputes the same binary32 score, and for every codeword within
-//      the margin of the minimum evaluates the binary64 distance sum (t_i-c_i)^2
-//      in index order; the result is the argmin of (distance, code).
+//   5. at the end of the unit each thread writes, per target, the remembered
+//      sub-chunks that are still within the margin of the slice minimum, and folds
+//      the slice minimum into a per-target global minimum (atomic).
+// Rescoring.  One warp per target: every remembered sub-chunk of every slice whose
+// minimum lies within the margin of the global minimum is revisited, the binary64
+// distance sum (t_i-c_i)^2 (index order) of each of its codewords is evaluated
+// from the caller's codebook, and the argmin of (distance, code) is written.
 // The margin bounds twice the rounding error of the fast score, so the codeword
 // that is nearest in exact arithmetic is always among those rescored.
-// Segments that cover the whole codebook write the code directly; otherwise the
-// per-slice results go to the workspace and a small merge kernel finishes.
 #include <cuda_fp16.h>
 
 #include "pvt_internal.h"
@@ -39,12 +41,28 @@ EncodeM1Layout encode_m1_layout(uint32_t K, uint64_t k, int sm_count, int tt) {
   e.n_chunks = (K + kChunkCodewords - 1) / kChunkCodewords;
   e.tile = (uint32_t)(kEncThreads * tt);
   e.n_tiles = (uint32_t)((k + e.tile - 1) / e.tile);
-  const uint64_t units = (uint64_t)e.n_tiles * e.n_chunks;
+  // slices: the fewest that keep the last round of units over the SMs nearly full
+  uint32_t best_s = 1;
+  double best_eff = 0.0;
+  const uint32_t s_max = e.n_chunks < (uint32_t)kMaxSlices ? e.n_chunks : (uint32_t)kMaxSlices;
+  for (uint32_t s = 1; s <= s_max; ++s) {
+    const uint64_t units = (uint64_t)e.n_tiles * s;
+    const uint64_t rounds = (units + sm_count - 1) / sm_count;
+    const double eff = (double)units / (double)(rounds * sm_count);
+    if (eff > best_eff + 0.03) {
+      best_eff = eff;
+      best_s = s;
+    }
+  }
+  e.n_slices = best_s;
+  const uint64_t units = (uint64_t)e.n_tiles * e.n_slices;
   e.n_ctas = (uint32_t)(units < (uint64_t)sm_count ? units : (uint64_t)sm_count);
   e.cbx_off = kWsHeaderBytes;
   e.n2max_off = align_up(e.cbx_off + (size_t)e.n_chunks * kChunkBytes, kWsAlign);
-  e.partial_off = e.n2max_off + kWsAlign;
-  e.bytes = align_up(e.partial_off + (size_t)e.n_ctas * 2 * e.tile * sizeof(PartialResult), kWsAlign);
+  e.gbest_off = e.n2max_off + kWsAlign;
+  e.margin_off = align_up(e.gbest_off + sizeof(uint32_t) * k, kWsAlign);
+  e.rec_off = align_up(e.margin_off + sizeof(float) * k, kWsAlign);
+  e.bytes = align_up(e.rec_off + (size_t)e.n_tiles * e.n_slices * e.tile * sizeof(CandRecord), kWsAlign);
   return e;
 }
 
@@ -69,13 +87,43 @@ struct EncM1Params {
   float eta;
   const float* cbx;
   const uint32_t* n2max_bits;
-  uint32_t n_chunks, K, n_tiles, n_ctas;
-  PartialResult* partial;
+  uint32_t n_chunks, K, n_tiles, n_slices, tile;
+  uint32_t* gbest;
+  float* margin;
+  CandRecord* rec;
+  const void* book;  // the caller's codebook [K][8]
   void* codes;
   int code_u16;
   float* err_out;
   uint32_t* status;
 };
+
+// order-preserving map binary32 -> u32 (and back)
+__device__ __forceinline__ uint32_t ord(float f) {
+  const uint32_t b = __float_as_uint(f);
+  return b ^ ((b >> 31) ? 0xffffffffu : 0x80000000u);
+}
+__device__ __forceinline__ float unord(uint32_t o) {
+  return __uint_as_float(o ^ ((o >> 31) ? 0x80000000u : 0xffffffffu));
+}
+
+// t = (W - eta g) / s of group j in binary32: one fma, one division per element
+__device__ __forceinline__ void form_target(const EncM1Params& p, uint32_t j, float* t) {
+  const float4* W4 = reinterpret_cast<const float4*>(p.W);
+  const float4* g4 = reinterpret_cast<const float4*>(p.g);
+  const float4 w0 = __ldg(W4 + 2 * (size_t)j), w1 = __ldg(W4 + 2 * (size_t)j + 1);
+  const float4 g0 = __ldg(g4 + 2 * (size_t)j), g1 = __ldg(g4 + 2 * (size_t)j + 1);
+  const float sc = __ldg(p.scale + j / p.gpr);
+  const float neg_eta = -p.eta;
+  t[0] = __fdiv_rn(__fmaf_rn(neg_eta, g0.x, w0.x), sc);
+  t[1] = __fdiv_rn(__fmaf_rn(neg_eta, g0.y, w0.y), sc);
+  t[2] = __fdiv_rn(__fmaf_rn(neg_eta, g0.z, w0.z), sc);
+  t[3] = __fdiv_rn(__fmaf_rn(neg_eta, g0.w, w0.w), sc);
+  t[4] = __fdiv_rn(__fmaf_rn(neg_eta, g1.x, w1.x), sc);
+  t[5] = __fdiv_rn(__fmaf_rn(neg_eta, g1.y, w1.y), sc);
+  t[6] = __fdiv_rn(__fmaf_rn(neg_eta, g1.z, w1.z), sc);
+  t[7] = __fdiv_rn(__fmaf_rn(neg_eta, g1.w, w1.w), sc);
+}
 
 // ---- codebook expansion ------------------------------------------------------
 // chunk block (kChunkBytes): 128 pairs * 16 floats, pair p holds
@@ -179,12 +227,6 @@ __device__ __forceinline__ float min3(float a, float b, float c) {
 __device__ __forceinline__ uint64_t pack2(float lo, float hi) {
   return (uint64_t)__float_as_uint(lo) | ((uint64_t)__float_as_uint(hi) << 32);
 }
-__device__ __forceinline__ void compute_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kEncThreads) : "memory"); }
-
-__device__ __forceinline__ uint64_t cta_unit_lo(uint64_t b, uint64_t units, uint64_t n_ctas) {
-  return b * units / n_ctas;  // units * n_ctas < 2^64 for every supported size
-}
-
 // ---- shared-memory layout of the search kernel -----------------------------------
 template <int TT>
 struct EncSmem {
@@ -192,10 +234,6 @@ struct EncSmem {
   alignas(128) unsigned char stage[kEncStages][kChunkBytes];
   alignas(8) uint64_t full_bar[kEncStages];
   uint64_t empty_bar[kEncStages];
-  alignas(16) float t[TILE][8];       // targets of the tile (for the rescoring pass)
-  uint32_t group[TILE];               // group index of each target, 0xffffffff = none
-  float margin[TILE];
-  float best[TILE];                   // minimum fast score over the segment
   float evicted_min[TILE];            // smallest sub-chunk minimum that fell out of the list
   float list_min[kListLen][TILE];
   uint16_t list_id[kListLen][TILE];
@@ -222,19 +260,17 @@ __global__ void __launch_bounds__(kEncThreads + 32, 1) encode_m1_kernel(const En
   }
   __syncthreads();
 
-  const uint64_t units = (uint64_t)p.n_tiles * p.n_chunks;
-  const uint64_t u_lo = cta_unit_lo(blockIdx.x, units, p.n_ctas);
-  const uint64_t u_hi = cta_unit_lo(blockIdx.x + 1, units, p.n_ctas);
+  const uint64_t units = (uint64_t)p.n_tiles * p.n_slices;
 
   if (warp == kEncThreads / 32) {
     // ------------------------------------------------------------ producer warp
     if (lane == 0) {
       uint32_t it = 0;
       bool alive = true;
-      for (uint64_t u = u_lo; u < u_hi && alive;) {
-        const uint32_t c_lo = (uint32_t)(u % p.n_chunks);
-        const uint64_t left = u_hi - u;
-        const uint32_t c_hi = (uint32_t)((uint64_t)c_lo + left < p.n_chunks ? c_lo + left : p.n_chunks);
+      for (uint64_t u = blockIdx.x; u < units && alive; u += gridDim.x) {
+        const uint32_t sl = (uint32_t)(u % p.n_slices);
+        const uint32_t c_lo = (uint32_t)((uint64_t)sl * p.n_chunks / p.n_slices);
+        const uint32_t c_hi = (uint32_t)((uint64_t)(sl + 1) * p.n_chunks / p.n_slices);
         for (uint32_t c = c_lo; c < c_hi && alive; ++c, ++it) {
           const uint32_t s = it % kEncStages;
           if (it >= kEncStages)
@@ -245,7 +281,6 @@ __global__ void __launch_bounds__(kEncThreads + 32, 1) encode_m1_kernel(const En
           bulk_g2s(smem_u32(&sm.stage[s][0]), reinterpret_cast<const char*>(p.cbx) + (size_t)c * kChunkBytes,
                    kChunkBytes, fb);
         }
-        u += c_hi - c_lo;
       }
       if (!alive) {
         // drain: let every copy that was issued land before the CTA may exit
@@ -264,48 +299,27 @@ __global__ void __launch_bounds__(kEncThreads + 32, 1) encode_m1_kernel(const En
 
   // -------------------------------------------------------------- compute warps
   const float n2max = __uint_as_float(*p.n2max_bits);
-  const float4* W4 = reinterpret_cast<const float4*>(p.W);
-  const float4* g4 = reinterpret_cast<const float4*>(p.g);
   uint32_t it = 0;
-  bool first_segment = true;
 
-  for (uint64_t u = u_lo; u < u_hi;) {
-    const uint32_t tile = (uint32_t)(u / p.n_chunks);
-    const uint32_t c_lo = (uint32_t)(u % p.n_chunks);
-    const uint64_t left = u_hi - u;
-    const uint32_t c_hi = (uint32_t)((uint64_t)c_lo + left < p.n_chunks ? c_lo + left : p.n_chunks);
-    const bool full_cover = (c_lo == 0 && c_hi == p.n_chunks);
+  for (uint64_t u = blockIdx.x; u < units; u += gridDim.x) {
+    const uint32_t tile = (uint32_t)(u / p.n_slices);
+    const uint32_t sl = (uint32_t)(u % p.n_slices);
+    const uint32_t c_lo = (uint32_t)((uint64_t)sl * p.n_chunks / p.n_slices);
+    const uint32_t c_hi = (uint32_t)((uint64_t)(sl + 1) * p.n_chunks / p.n_slices);
 
-    // 1. gather targets, form t (binary32: one fma, one division), set up tracking
+    // 1. gather targets, form t, set up tracking
     uint64_t nt[TT][8];  // (-t_i, -t_i)
     float thr[TT], best[TT], margin[TT];
 #pragma unroll
     for (int tt = 0; tt < TT; ++tt) {
       const int s = tt * kEncThreads + tid;
       const uint64_t n = (uint64_t)tile * TILE + s;
-      uint32_t j = 0xffffffffu;
       float t[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) t[i] = 0.0f;
       if (n < p.k) {
-        j = p.idx[n];
-        if (j >= p.G) {
-          atomicOr(p.status, PVT_DEV_BAD_INDEX);
-          j = 0xffffffffu;
-        } else {
-          const float4 w0 = __ldg(W4 + 2 * (size_t)j), w1 = __ldg(W4 + 2 * (size_t)j + 1);
-          const float4 g0 = __ldg(g4 + 2 * (size_t)j), g1 = __ldg(g4 + 2 * (size_t)j + 1);
-          const float sc = __ldg(p.scale + j / p.gpr);
-          const float neg_eta = -p.eta;
-          t[0] = __fdiv_rn(__fmaf_rn(neg_eta, g0.x, w0.x), sc);
-          t[1] = __fdiv_rn(__fmaf_rn(neg_eta, g0.y, w0.y), sc);
-          t[2] = __fdiv_rn(__fmaf_rn(neg_eta, g0.z, w0.z), sc);
-          t[3] = __fdiv_rn(__fmaf_rn(neg_eta, g0.w, w0.w), sc);
-          t[4] = __fdiv_rn(__fmaf_rn(neg_eta, g1.x, w1.x), sc);
-          t[5] = __fdiv_rn(__fmaf_rn(neg_eta, g1.y, w1.y), sc);
-          t[6] = __fdiv_rn(__fmaf_rn(neg_eta, g1.z, w1.z), sc);
-          t[7] = __fdiv_rn(__fmaf_rn(neg_eta, g1.w, w1.w), sc);
-        }
+        const uint32_t j = p.idx[n];
+        if (j < p.G) form_target(p, j, t);  // an index out of range is reported by the rescoring kernel
       }
       float nt2 = 0.0f;
 #pragma unroll
@@ -318,15 +332,11 @@ __global__ void __launch_bounds__(kEncThreads + 32, 1) encode_m1_kernel(const En
       margin[tt] = 3.8146973e-6f /* 2^-18 */ * (0.5f * n2max + sqrtf(nt2 * n2max)) + 1e-30f;
       best[tt] = __int_as_float(0x7f800000);
       thr[tt] = best[tt];
-      *reinterpret_cast<float4*>(&sm.t[s][0]) = make_float4(t[0], t[1], t[2], t[3]);
-      *reinterpret_cast<float4*>(&sm.t[s][4]) = make_float4(t[4], t[5], t[6], t[7]);
-      sm.group[s] = j;
-      sm.margin[s] = margin[tt];
       sm.list_cnt[s] = 0;
       sm.evicted_min[s] = __int_as_float(0x7f800000);
     }
 
-    // 2.-4. stream the codebook chunks of this segment
+    // 2.-4. stream the codebook chunks of this slice
     for (uint32_t c = c_lo; c < c_hi; ++c, ++it) {
       const uint32_t st = it % kEncStages;
       mbar_wait(smem_u32(&sm.full_bar[st]), (it / kEncStages) & 1, abort_flag, p.status);
@@ -376,154 +386,136 @@ __global__ void __launch_bounds__(kEncThreads + 32, 1) encode_m1_kernel(const En
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&sm.empty_bar[st]));
     }
-#pragma unroll
-    for (int tt = 0; tt < TT; ++tt) sm.best[tt * kEncThreads + tid] = best[tt];
-    compute_bar();
 
-    // 5. rescoring: one warp per target
-    const bool aborted = *abort_flag != 0;
-    const uint32_t slot_of_segment = first_segment ? 0u : 1u;
-    for (int s = warp; s < TILE && !aborted; s += kEncThreads / 32) {
-      const uint64_t n = (uint64_t)tile * TILE + s;
-      if (n >= p.k) break;
-      const uint32_t j = sm.group[s];
-      const float m = sm.best[s];
-      const float limit = m + sm.margin[s];
-      const uint32_t cnt = sm.list_cnt[s];
-      const bool overflow = cnt > kListLen && sm.evicted_min[s] <= limit;
-      const float4 ta = *reinterpret_cast<const float4*>(&sm.t[s][0]);
-      const float4 tb = *reinterpret_cast<const float4*>(&sm.t[s][4]);
-      const float t[8] = {ta.x, ta.y, ta.z, ta.w, tb.x, tb.y, tb.z, tb.w};
-      double best_d = __longlong_as_double(0x7ff0000000000000ll);
-      uint32_t best_code = 0xffffffffu;
-      const uint32_t subs_per_chunk = kChunkCodewords / kSubCodewords;
-      const uint32_t n_visit = overflow ? (c_hi - c_lo) * subs_per_chunk : min(cnt, (uint32_t)kListLen);
-      for (uint32_t v = 0; v < n_visit; ++v) {
-        uint32_t sub_id;
-        if (overflow) {
-          sub_id = c_lo * subs_per_chunk + v;
-        } else {
-          if (sm.list_min[v][s] > limit) continue;
-          sub_id = sm.list_id[v][s];
-        }
-        const uint32_t chunk = sub_id / subs_per_chunk;
-        const uint32_t w = (sub_id % subs_per_chunk) * kSubCodewords + lane;  // codeword within the chunk
-        const uint32_t kappa = chunk * kChunkCodewords + w;
-        const float* blk = p.cbx + (size_t)chunk * (kChunkBytes / 4);
-        const uint32_t pr = w >> 1, half = w & 1;
-        float cw[8];
+    // 5. leave the candidates of this (tile, slice) for the rescoring kernel
+    if (*abort_flag == 0) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) cw[i] = __ldg(blk + pr * 16 + 2 * i + half);
-        float f = __ldg(blk + kChunkCodewords * 8 + pr * 2 + half);
+      for (int tt = 0; tt < TT; ++tt) {
+        const int s = tt * kEncThreads + tid;
+        const uint64_t n = (uint64_t)tile * TILE + s;
+        if (n >= p.k) continue;
+        const float limit = best[tt] + margin[tt];
+        const uint32_t cnt = sm.list_cnt[s];
+        CandRecord r;
+        r.best = best[tt];
+        r.pad = 0;
+        uint32_t m = 0;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) f = __fmaf_rn(-t[i], cw[i], f);  // the same operations as the packed loop
-        const bool cand = (f <= limit) && (kappa < p.K);
-        uint32_t mask = __ballot_sync(0xffffffffu, cand);
-        if (mask) {
-          double d = 0.0;
-          if (cand) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              const double e = __dsub_rn((double)t[i], (double)cw[i]);
-              d = __dadd_rn(d, __dmul_rn(e, e));
-            }
-          }
-          while (mask) {
-            const int src = __ffs(mask) - 1;
-            mask &= mask - 1;
-            const double dc = __shfl_sync(0xffffffffu, d, src);
-            const uint32_t kc = chunk * kChunkCodewords + (sub_id % subs_per_chunk) * kSubCodewords + src;
-            if (dc < best_d || (dc == best_d && kc < best_code)) {
-              best_d = dc;
-              best_code = kc;
-            }
-          }
+        for (int v = 0; v < kListLen; ++v) {
+          r.sub[v] = 0;
+          if ((uint32_t)v < cnt && sm.list_min[v][s] <= limit) r.sub[m++] = sm.list_id[v][s];
         }
-      }
-      if (lane == 0) {
-        const bool ok = j != 0xffffffffu && best_code < p.K;
-        if (full_cover) {
-          if (ok) {
-            if (p.code_u16)
-              reinterpret_cast<uint16_t*>(p.codes)[j] = (uint16_t)best_code;
-            else
-              reinterpret_cast<uint8_t*>(p.codes)[j] = (uint8_t)best_code;
-            if (p.err_out) p.err_out[n] = (float)best_d;
-          }
-        } else {
-          PartialResult r;
-          r.d = best_d;
-          r.code = best_code;
-          r.valid = ok ? 1u : 0u;
-          p.partial[((size_t)blockIdx.x * 2 + slot_of_segment) * TILE + s] = r;
-        }
+        r.cnt = (cnt > (uint32_t)kListLen && sm.evicted_min[s] <= limit) ? kCandOverflow : (uint16_t)m;
+        *reinterpret_cast<uint4*>(&p.rec[((size_t)tile * p.n_slices + sl) * TILE + s]) =
+            *reinterpret_cast<const uint4*>(&r);
+        atomicMin(&p.gbest[n], ord(best[tt]));
+        if (sl == 0) p.margin[n] = margin[tt];
       }
     }
-    compute_bar();
-    first_segment = false;
-    u += c_hi - c_lo;
   }
 }
 
-// Merge the per-slice results of tiles whose codebook range was split over CTAs.
-template <int TT>
-__global__ void __launch_bounds__(256) encode_m1_merge_kernel(const EncM1Params p) {
-  constexpr int TILE = kEncThreads * TT;
-  const uint32_t tile = blockIdx.x;
-  const uint64_t units = (uint64_t)p.n_tiles * p.n_chunks;
-  const uint64_t t_lo = (uint64_t)tile * p.n_chunks, t_hi = t_lo + p.n_chunks - 1;
-  auto cta_of = [&](uint64_t u) {
-    uint64_t b = u * p.n_ctas / units;
-    while (b + 1 < p.n_ctas && cta_unit_lo(b + 1, units, p.n_ctas) <= u) ++b;
-    while (b > 0 && cta_unit_lo(b, units, p.n_ctas) > u) --b;
-    return (uint32_t)b;
+// ---- rescoring --------------------------------------------------------------------
+template <bool CB_F16>
+__device__ __forceinline__ void load_codeword(const void* book, uint32_t kappa, float* c) {
+  if (CB_F16) {
+    const uint4 raw = __ldg(reinterpret_cast<const uint4*>(book) + kappa);
+    const __half2* h = reinterpret_cast<const __half2*>(&raw);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float2 f = __half22float2(h[i]);
+      c[2 * i] = f.x;
+      c[2 * i + 1] = f.y;
+    }
+  } else {
+    const float4* q = reinterpret_cast<const float4*>(book) + 2 * (size_t)kappa;
+    const float4 a = __ldg(q), b = __ldg(q + 1);
+    c[0] = a.x; c[1] = a.y; c[2] = a.z; c[3] = a.w;
+    c[4] = b.x; c[5] = b.y; c[6] = b.z; c[7] = b.w;
+  }
+}
+
+// One warp per target.  `sub_cw` = codewords per sub-chunk of the search kernel
+// that wrote the records (a multiple of 32).
+template <bool CB_F16>
+__global__ void __launch_bounds__(256) rescore_m1_kernel(const EncM1Params p, uint32_t sub_cw) {
+  const int lane = threadIdx.x & 31;
+  const uint64_t n = (uint64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (n >= p.k) return;
+  const uint32_t j = __ldg(p.idx + n);
+  if (j >= p.G) {
+    if (lane == 0) atomicOr(p.status, PVT_DEV_BAD_INDEX);
+    return;
+  }
+  float t[8];
+  form_target(p, j, t);
+  const float limit = unord(p.gbest[n]) + p.margin[n];
+  const uint32_t tile = (uint32_t)(n / p.tile), s = (uint32_t)(n % p.tile);
+  const uint32_t subs_per_chunk = kChunkCodewords / sub_cw;
+  double best_d = __longlong_as_double(0x7ff0000000000000ll);
+  uint32_t best_code = 0xffffffffu;
+
+  auto visit = [&](uint32_t sub) {
+    for (uint32_t w = lane; w < sub_cw; w += 32) {
+      const uint32_t kappa = sub * sub_cw + w;
+      if (kappa < p.K) {
+        float c[8];
+        load_codeword<CB_F16>(p.book, kappa, c);
+        double d = 0.0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const double e = __dsub_rn((double)t[i], (double)c[i]);
+          d = __dadd_rn(d, __dmul_rn(e, e));
+        }
+        if (d < best_d || (d == best_d && kappa < best_code)) {
+          best_d = d;
+          best_code = kappa;
+        }
+      }
+    }
   };
-  const uint32_t b_first = cta_of(t_lo), b_last = cta_of(t_hi);
-  if (b_first == b_last) return;  // one CTA covered the whole codebook and wrote the result itself
-  for (int s = threadIdx.x; s < TILE; s += blockDim.x) {
-    const uint64_t n = (uint64_t)tile * TILE + s;
-    if (n >= p.k) break;
-    double best_d = __longlong_as_double(0x7ff0000000000000ll);
-    uint32_t best_code = 0xffffffffu;
-    bool ok = true;
-    for (uint32_t b = b_first; b <= b_last; ++b) {
-      const uint64_t lo = cta_unit_lo(b, units, p.n_ctas);
-      if (cta_unit_lo(b + 1, units, p.n_ctas) == lo) continue;  // CTA without work
-      const uint32_t slot = (lo / p.n_chunks == tile) ? 0u : 1u;
-      const PartialResult r = p.partial[((size_t)b * 2 + slot) * TILE + s];
-      ok = ok && r.valid;
-      if (r.d < best_d || (r.d == best_d && r.code < best_code)) {
-        best_d = r.d;
-        best_code = r.code;
-      }
+
+  for (uint32_t sl = 0; sl < p.n_slices; ++sl) {
+    const uint4 raw = __ldg(reinterpret_cast<const uint4*>(&p.rec[((size_t)tile * p.n_slices + sl) * p.tile + s]));
+    const CandRecord r = *reinterpret_cast<const CandRecord*>(&raw);
+    if (!(r.best <= limit)) continue;
+    if (r.cnt == kCandOverflow) {
+      const uint32_t c_lo = (uint32_t)((uint64_t)sl * p.n_chunks / p.n_slices);
+      const uint32_t c_hi = (uint32_t)((uint64_t)(sl + 1) * p.n_chunks / p.n_slices);
+      for (uint32_t sub = c_lo * subs_per_chunk; sub < c_hi * subs_per_chunk; ++sub) visit(sub);
+    } else {
+      const uint32_t cnt = r.cnt < (uint16_t)kListLen ? r.cnt : (uint32_t)kListLen;
+      for (uint32_t e = 0; e < cnt; ++e) visit(r.sub[e]);
     }
-    if (ok && best_code < p.K) {
-      const uint32_t j = p.idx[n];
-      if (j < p.G) {
-        if (p.code_u16)
-          reinterpret_cast<uint16_t*>(p.codes)[j] = (uint16_t)best_code;
-        else
-          reinterpret_cast<uint8_t*>(p.codes)[j] = (uint8_t)best_code;
-        if (p.err_out) p.err_out[n] = (float)best_d;
-      }
+  }
+  // warp-wide lexicographic minimum of (distance, code); distances are >= 0 so their bits order like u64
+  const uint64_t bits = (uint64_t)__double_as_longlong(best_d);
+  const uint32_t hi = (uint32_t)(bits >> 32), lo = (uint32_t)bits;
+  const uint32_t mhi = __reduce_min_sync(0xffffffffu, hi);
+  const uint32_t mlo = __reduce_min_sync(0xffffffffu, hi == mhi ? lo : 0xffffffffu);
+  const uint32_t mk = __reduce_min_sync(0xffffffffu, (hi == mhi && lo == mlo) ? best_code : 0xffffffffu);
+  if (lane == 0) {
+    if (mk < p.K) {
+      if (p.code_u16)
+        reinterpret_cast<uint16_t*>(p.codes)[j] = (uint16_t)mk;
+      else
+        reinterpret_cast<uint8_t*>(p.codes)[j] = (uint8_t)mk;
+      if (p.err_out) p.err_out[n] = (float)__longlong_as_double((long long)(((uint64_t)mhi << 32) | mlo));
+    } else {
+      atomicOr(p.status, PVT_DEV_INTERNAL);  // no candidate survived: the search did not complete
     }
   }
 }
 
 template <int TT>
-cudaError_t launch_tt(const EncM1Params& p, cudaStream_t stream) {
+cudaError_t launch_tt(const EncM1Params& p, uint32_t n_ctas, cudaStream_t stream) {
   const size_t smem = sizeof(EncSmem<TT>);
   cudaError_t err = cudaFuncSetAttribute(encode_m1_kernel<TT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (err != cudaSuccess) return err;
   timing_begin(kKernEncodeMain, stream);
-  encode_m1_kernel<TT><<<p.n_ctas, kEncThreads + 32, smem, stream>>>(p);
+  encode_m1_kernel<TT><<<n_ctas, kEncThreads + 32, smem, stream>>>(p);
   timing_end(kKernEncodeMain, stream);
-  if ((err = cudaGetLastError()) != cudaSuccess) return err;
   count_launches(1);
-  if (p.n_ctas > 1) {
-    encode_m1_merge_kernel<TT><<<p.n_tiles, 256, 0, stream>>>(p);
-    count_launches(1);
-  }
   return cudaGetLastError();
 }
 
@@ -548,8 +540,12 @@ cudaError_t launch_encode_m1(const pvt_layer& L, uint64_t G, const uint32_t* idx
   p.n_chunks = lay.n_chunks;
   p.K = (uint32_t)L.codebook_size;
   p.n_tiles = lay.n_tiles;
-  p.n_ctas = lay.n_ctas;
-  p.partial = reinterpret_cast<PartialResult*>(base + lay.partial_off);
+  p.n_slices = lay.n_slices;
+  p.tile = lay.tile;
+  p.gbest = reinterpret_cast<uint32_t*>(base + lay.gbest_off);
+  p.margin = reinterpret_cast<float*>(base + lay.margin_off);
+  p.rec = reinterpret_cast<CandRecord*>(base + lay.rec_off);
+  p.book = L.codebooks;
   p.codes = L.codes;
   p.code_u16 = L.code_dtype == PVT_U16;
   p.err_out = err_out;
@@ -557,9 +553,11 @@ cudaError_t launch_encode_m1(const pvt_layer& L, uint64_t G, const uint32_t* idx
 
   cudaError_t err = cudaMemsetAsync(base + lay.n2max_off, 0, sizeof(uint32_t), stream);
   if (err != cudaSuccess) return err;
+  if ((err = cudaMemsetAsync(p.gbest, 0xff, sizeof(uint32_t) * k, stream)) != cudaSuccess) return err;
   timing_begin(kKernEncodeAux, stream);
   const uint32_t n_cw = lay.n_chunks * kChunkCodewords;
-  if (L.codebook_dtype == PVT_F16)
+  const bool f16 = L.codebook_dtype == PVT_F16;
+  if (f16)
     expand_codebook_kernel<true><<<(n_cw + 255) / 256, 256, 0, stream>>>(
         L.codebooks, p.K, lay.n_chunks, const_cast<float*>(p.cbx), const_cast<uint32_t*>(p.n2max_bits));
   else
@@ -568,7 +566,17 @@ cudaError_t launch_encode_m1(const pvt_layer& L, uint64_t G, const uint32_t* idx
   count_launches(1);
   timing_end(kKernEncodeAux, stream);
   if ((err = cudaGetLastError()) != cudaSuccess) return err;
-  return tt == 8 ? launch_tt<8>(p, stream) : launch_tt<4>(p, stream);
+  err = tt == 8 ? launch_tt<8>(p, lay.n_ctas, stream) : launch_tt<4>(p, lay.n_ctas, stream);
+  if (err != cudaSuccess) return err;
+  timing_begin(kKernEncodeRescore, stream);
+  const unsigned blocks = (unsigned)((k + 7) / 8);
+  if (f16)
+    rescore_m1_kernel<true><<<blocks, 256, 0, stream>>>(p, kSubCodewords);
+  else
+    rescore_m1_kernel<false><<<blocks, 256, 0, stream>>>(p, kSubCodewords);
+  count_launches(1);
+  timing_end(kKernEncodeRescore, stream);
+  return cudaGetLastError();
 }
 
 }  // namespace pvt

@@ -46,32 +46,41 @@ struct SelectLayout {
 SelectLayout select_layout(uint64_t G);
 
 // encode, M = 1 ---------------------------------------------------------------
+// The search kernel leaves, per (target, codebook slice), the sub-chunks of the
+// codebook that may hold the nearest codeword; the rescoring kernel evaluates the
+// exact distances of those codewords and writes the code.
 constexpr int kEncThreads = 256;     // compute threads per CTA (8 warps) + 1 producer warp
 constexpr int kChunkCodewords = 256; // codewords per staged chunk (one bulk copy)
 constexpr int kSubCodewords = 32;    // tracking granularity of the running minimum
 constexpr int kChunkBytes = kChunkCodewords * (kGroupDim * 4 + 4);  // 9216: pairs interleaved + half norms
 constexpr int kEncStages = 4;
-constexpr int kListLen = 4;          // remembered near-minimum sub-chunks per target
+constexpr int kListLen = 4;          // remembered near-minimum sub-chunks per (target, slice)
+constexpr int kMaxSlices = 16;
+constexpr uint16_t kCandOverflow = 0xffffu;
+
+struct CandRecord {        // 16 bytes, one per (target, codebook slice)
+  float best;              // smallest fast score of the slice
+  uint16_t sub[kListLen];  // sub-chunk ids whose minimum lies within the margin of `best`
+  uint16_t cnt;            // valid entries of sub[]; kCandOverflow: rescan the whole slice
+  uint16_t pad;
+};
 
 struct EncodeM1Layout {
   size_t cbx_off;      // expanded codebook: n_chunks * kChunkBytes
   size_t n2max_off;    // u32 bit pattern of max ||c||^2
-  size_t partial_off;  // per CTA: 2 segments * tile * 16 bytes
+  size_t gbest_off;    // u32 [k]: order-preserving image of the smallest fast score over all slices
+  size_t margin_off;   // f32 [k]: rounding-error margin of the fast score of each target
+  size_t rec_off;      // CandRecord [n_tiles][n_slices][tile]
   size_t bytes;
   uint32_t n_chunks;
   uint32_t tile;       // targets per tile (kEncThreads * TT)
   uint32_t n_tiles;
+  uint32_t n_slices;   // codebook slices per tile (whole chunks each)
   uint32_t n_ctas;
 };
 EncodeM1Layout encode_m1_layout(uint32_t K, uint64_t k, int sm_count, int targets_per_thread);
 int encode_m1_targets_per_thread(uint64_t k, int sm_count);  // 4 or 8
 size_t encode_m2_workspace_bytes();
-
-struct PartialResult {  // one (target, codebook slice) result awaiting the merge
-  double d;
-  uint32_t code;
-  uint32_t valid;
-};
 
 // launchers (each returns a cudaError_t) --------------------------------------
 cudaError_t launch_select(const pvt_layer& L, uint64_t G, uint64_t k, uint32_t* idx_out, void* ws,
@@ -84,7 +93,9 @@ cudaError_t launch_dequant(const pvt_layer& L, uint64_t G, void* W_hat, int32_t 
                            cudaStream_t stream);
 
 // optional per-kernel timing (benchmark instrumentation) ----------------------
-enum KernelId { kKernSelect = 0, kKernEncodeMain = 1, kKernEncodeAux = 2, kKernDequant = 3, kKernCount = 4 };
+enum KernelId {
+  kKernSelect = 0, kKernEncodeMain = 1, kKernEncodeAux = 2, kKernDequant = 3, kKernEncodeRescore = 4, kKernCount = 5
+};
 void timing_begin(KernelId id, cudaStream_t stream);
 void timing_end(KernelId id, cudaStream_t stream);
 
