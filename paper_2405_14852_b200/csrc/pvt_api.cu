@@ -108,7 +108,10 @@ size_t pvt_workspace_bytes(const pvt_layer* layer, uint64_t k) {
   const int sms = sm_count();
   size_t need = select_layout(G).bytes;
   if (layer->num_codebooks == 1) {
-    const size_t e = encode_m1_layout((uint32_t)layer->codebook_size, k, sms, encode_m1_targets_per_thread(k, sms)).bytes;
+    const size_t e =
+        encode_m1_use_tc(*layer, k)
+            ? encode_m1_tc_layout((uint32_t)layer->codebook_size, k, sms).bytes
+            : encode_m1_layout((uint32_t)layer->codebook_size, k, sms, encode_m1_targets_per_thread(k, sms)).bytes;
     need = e > need ? e : need;
   } else {
     const size_t e = encode_m2_workspace_bytes();
@@ -148,7 +151,10 @@ int pvt_vstep_encode(const pvt_layer* layer, const uint32_t* idx, uint64_t k, fl
   if (reinterpret_cast<uintptr_t>(ws) & (kWsAlign - 1)) return PVT_EINVAL;
   const int sms = sm_count();
   cudaError_t e;
-  if (layer->num_codebooks == 1) {
+  if (layer->num_codebooks == 1 && encode_m1_use_tc(*layer, k)) {
+    if (ws_bytes < encode_m1_tc_layout((uint32_t)layer->codebook_size, k, sms).bytes) return PVT_EWORKSPACE;
+    e = launch_encode_m1_tc(*layer, G, idx, k, err_out, ws, sms, static_cast<cudaStream_t>(cuda_stream));
+  } else if (layer->num_codebooks == 1) {
     const EncodeM1Layout lay =
         encode_m1_layout((uint32_t)layer->codebook_size, k, sms, encode_m1_targets_per_thread(k, sms));
     if (ws_bytes < lay.bytes) return PVT_EWORKSPACE;
@@ -172,7 +178,7 @@ int pvt_dequant(const pvt_layer* layer, void* W_hat, int32_t out_dtype, uint32_t
   if (!aligned16(layer->codebooks) || !aligned16(W_hat)) return PVT_EINVAL;
   if (layer->num_codebooks == 2 && layer->code_dtype == PVT_U8 && (reinterpret_cast<uintptr_t>(layer->codes) & 1u))
     return PVT_EINVAL;
-  const cudaError_t e = launch_dequant(*layer, G, W_hat, out_dtype, status, static_cast<cudaStream_t>(cuda_stream));
+  const cudaError_t e = launch_dequant(*layer, G, W_hat, out_dtype, status, sm_count(), static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? PVT_OK : fail_cuda(e);
 }
 

@@ -1,5 +1,5 @@
 // dequantize_weights (Algorithm 3, first line): W_hat = s_row * sum_m C_m[b_m] for
-// every weight group.  Streaming kernel: one group (8 weights) per thread, codes
+// every weight group.  Streaming kernel, persistent grid: four groups (8 weights each) in flight per thread, codes
 // read coalesced, codewords gathered from the L2-resident codebook (small
 // codebooks are first copied to shared memory), 32 B (fp32) or 16 B (fp16) written
 // per group with 128-bit stores.
@@ -14,6 +14,7 @@ namespace pvt {
 namespace {
 
 constexpr int kDqThreads = 256;
+constexpr int kDqUnroll = 4;          // groups in flight per thread
 constexpr int kDqSmemCodewords = 512;  // M*K up to this many codewords are staged in shared memory
 
 struct Vec8 {
@@ -58,58 +59,92 @@ __global__ void __launch_bounds__(kDqThreads) dequant_kernel(const void* __restr
     __syncthreads();
     book = sh_book;
   }
-  const uint64_t j = (uint64_t)blockIdx.x * kDqThreads + threadIdx.x;
-  if (j >= G) return;
-  uint32_t b[M];
-  if (CODE_U16) {
-    const uint16_t* c = reinterpret_cast<const uint16_t*>(codes) + j * M;
+  // kDqUnroll groups per thread and iteration, a block apart, all their loads issued
+  // before the first use: the code -> codeword -> store chain of one group is two
+  // dependent memory round trips, so several groups must be in flight per thread
+  const uint64_t stride = (uint64_t)gridDim.x * (kDqThreads * kDqUnroll);
+  for (uint64_t base = (uint64_t)blockIdx.x * (kDqThreads * kDqUnroll); base < G; base += stride) {
+    uint32_t b[kDqUnroll][M];
+    bool bad = false;
 #pragma unroll
-    for (int m = 0; m < M; ++m) b[m] = c[m];
-  } else if (M == 2) {
-    const uint16_t both = reinterpret_cast<const uint16_t*>(codes)[j];  // two adjacent bytes
-    b[0] = both & 0xffu;
-    b[M - 1] = both >> 8;
-  } else {
-    b[0] = reinterpret_cast<const uint8_t*>(codes)[j];
-  }
-  bool bad = false;
+    for (int u = 0; u < kDqUnroll; ++u) {
+      const uint64_t j = base + (uint64_t)u * kDqThreads + threadIdx.x;
 #pragma unroll
-  for (int m = 0; m < M; ++m) {
-    if (b[m] >= K) {
-      bad = true;
-      b[m] = 0;
+      for (int m = 0; m < M; ++m) b[u][m] = 0;
+      if (j < G) {
+        if (CODE_U16) {
+          const uint16_t* c = reinterpret_cast<const uint16_t*>(codes) + j * M;
+#pragma unroll
+          for (int m = 0; m < M; ++m) b[u][m] = __ldcs(c + m);
+        } else if (M == 2) {
+          const uint16_t both = __ldcs(reinterpret_cast<const uint16_t*>(codes) + j);  // two adjacent bytes
+          b[u][0] = both & 0xffu;
+          b[u][M - 1] = both >> 8;
+        } else {
+          b[u][0] = __ldcs(reinterpret_cast<const uint8_t*>(codes) + j);
+        }
+#pragma unroll
+        for (int m = 0; m < M; ++m) {
+          if (b[u][m] >= K) {
+            bad = true;
+            b[u][m] = 0;
+          }
+        }
+      }
     }
-  }
-  if (bad && status) atomicOr(status, PVT_DEV_BAD_CODE);
-
-  Vec8 v = load_codeword<CB_F16>(book, b[0]);
-  if (M == 2) {
-    const Vec8 v2 = load_codeword<CB_F16>(book, K + b[M - 1]);
+    if (bad && status) atomicOr(status, PVT_DEV_BAD_CODE);
+    Vec8 v[kDqUnroll];
+    float s[kDqUnroll];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) v.v[i] = __fadd_rn(v.v[i], v2.v[i]);
-  }
-  const float s = scale[j / gpr];
+    for (int u = 0; u < kDqUnroll; ++u) {
+      const uint64_t j = base + (uint64_t)u * kDqThreads + threadIdx.x;
+      v[u] = load_codeword<CB_F16>(book, b[u][0]);
+      if (M == 2) {
+        const Vec8 v2 = load_codeword<CB_F16>(book, K + b[u][M - 1]);
 #pragma unroll
-  for (int i = 0; i < 8; ++i) v.v[i] = __fmul_rn(s, v.v[i]);
-
-  if (OUT_F16) {
-    __half2 h[4];
+        for (int i = 0; i < 8; ++i) v[u].v[i] = __fadd_rn(v[u].v[i], v2.v[i]);
+      }
+      s[u] = j < G ? __ldg(scale + j / gpr) : 0.0f;
+    }
 #pragma unroll
-    for (int i = 0; i < 4; ++i) h[i] = __floats2half2_rn(v.v[2 * i], v.v[2 * i + 1]);
-    __stcs(reinterpret_cast<uint4*>(W_hat) + j, *reinterpret_cast<const uint4*>(h));
-  } else {
-    float4* o = reinterpret_cast<float4*>(W_hat) + 2 * j;
-    __stcs(o, make_float4(v.v[0], v.v[1], v.v[2], v.v[3]));
-    __stcs(o + 1, make_float4(v.v[4], v.v[5], v.v[6], v.v[7]));
+    for (int u = 0; u < kDqUnroll; ++u) {
+      const uint64_t j = base + (uint64_t)u * kDqThreads + threadIdx.x;
+      if (j >= G) continue;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[u].v[i] = __fmul_rn(s[u], v[u].v[i]);
+      if (OUT_F16) {
+        __half2 h[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) h[i] = __floats2half2_rn(v[u].v[2 * i], v[u].v[2 * i + 1]);
+        __stcs(reinterpret_cast<uint4*>(W_hat) + j, *reinterpret_cast<const uint4*>(h));
+      } else {
+        float4* o = reinterpret_cast<float4*>(W_hat) + 2 * j;
+        __stcs(o, make_float4(v[u].v[0], v[u].v[1], v[u].v[2], v[u].v[3]));
+        __stcs(o + 1, make_float4(v[u].v[4], v[u].v[5], v[u].v[6], v[u].v[7]));
+      }
+    }
   }
 }
 
 template <int M, bool CB_F16, bool CODE_U16, bool OUT_F16>
-cudaError_t launch_t(const pvt_layer& L, uint64_t G, void* W_hat, uint32_t* status, cudaStream_t stream) {
-  const unsigned blocks = (unsigned)((G + kDqThreads - 1) / kDqThreads);
+cudaError_t launch_t(const pvt_layer& L, uint64_t G, void* W_hat, uint32_t* status, int sm_count,
+                     cudaStream_t stream) {
+  const bool smem_book = (uint32_t)M * (uint32_t)L.codebook_size <= (uint32_t)kDqSmemCodewords;
+  // persistent grid: as many blocks as are resident at once
+  int per_sm = 0;
+  cudaError_t oe = smem_book ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+                                   &per_sm, dequant_kernel<M, CB_F16, CODE_U16, OUT_F16, true>, kDqThreads, 0)
+                             : cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+                                   &per_sm, dequant_kernel<M, CB_F16, CODE_U16, OUT_F16, false>, kDqThreads, 0);
+  if (oe != cudaSuccess) return oe;
+  if (per_sm < 1) per_sm = 1;
+  const uint64_t per_block = (uint64_t)kDqThreads * kDqUnroll;
+  const uint64_t want = (G + per_block - 1) / per_block;
+  const uint64_t cap = (uint64_t)sm_count * (uint64_t)per_sm;
+  const unsigned blocks = (unsigned)(want < cap ? want : cap);
   const uint32_t gpr = (uint32_t)(L.cols / kGroupDim);
   const uint32_t K = (uint32_t)L.codebook_size;
-  if ((uint32_t)M * K <= (uint32_t)kDqSmemCodewords)
+  if (smem_book)
     dequant_kernel<M, CB_F16, CODE_U16, OUT_F16, true>
         <<<blocks, kDqThreads, 0, stream>>>(L.codebooks, L.codes, L.scale, G, gpr, K, W_hat, status);
   else
@@ -120,31 +155,31 @@ cudaError_t launch_t(const pvt_layer& L, uint64_t G, void* W_hat, uint32_t* stat
 
 template <int M, bool CB_F16, bool CODE_U16>
 cudaError_t launch_o(const pvt_layer& L, uint64_t G, void* W_hat, int32_t out_dtype, uint32_t* status,
-                     cudaStream_t stream) {
-  return out_dtype == PVT_F16 ? launch_t<M, CB_F16, CODE_U16, true>(L, G, W_hat, status, stream)
-                              : launch_t<M, CB_F16, CODE_U16, false>(L, G, W_hat, status, stream);
+                     int sm_count, cudaStream_t stream) {
+  return out_dtype == PVT_F16 ? launch_t<M, CB_F16, CODE_U16, true>(L, G, W_hat, status, sm_count, stream)
+                              : launch_t<M, CB_F16, CODE_U16, false>(L, G, W_hat, status, sm_count, stream);
 }
 
 template <int M, bool CB_F16>
 cudaError_t launch_c(const pvt_layer& L, uint64_t G, void* W_hat, int32_t out_dtype, uint32_t* status,
-                     cudaStream_t stream) {
-  return L.code_dtype == PVT_U16 ? launch_o<M, CB_F16, true>(L, G, W_hat, out_dtype, status, stream)
-                                 : launch_o<M, CB_F16, false>(L, G, W_hat, out_dtype, status, stream);
+                     int sm_count, cudaStream_t stream) {
+  return L.code_dtype == PVT_U16 ? launch_o<M, CB_F16, true>(L, G, W_hat, out_dtype, status, sm_count, stream)
+                                 : launch_o<M, CB_F16, false>(L, G, W_hat, out_dtype, status, sm_count, stream);
 }
 
 }  // namespace
 
 cudaError_t launch_dequant(const pvt_layer& L, uint64_t G, void* W_hat, int32_t out_dtype, uint32_t* status,
-                           cudaStream_t stream) {
+                           int sm_count, cudaStream_t stream) {
   timing_begin(kKernDequant, stream);
   cudaError_t err;
   const bool f16 = L.codebook_dtype == PVT_F16;
   if (L.num_codebooks == 1)
-    err = f16 ? launch_c<1, true>(L, G, W_hat, out_dtype, status, stream)
-              : launch_c<1, false>(L, G, W_hat, out_dtype, status, stream);
+    err = f16 ? launch_c<1, true>(L, G, W_hat, out_dtype, status, sm_count, stream)
+              : launch_c<1, false>(L, G, W_hat, out_dtype, status, sm_count, stream);
   else
-    err = f16 ? launch_c<2, true>(L, G, W_hat, out_dtype, status, stream)
-              : launch_c<2, false>(L, G, W_hat, out_dtype, status, stream);
+    err = f16 ? launch_c<2, true>(L, G, W_hat, out_dtype, status, sm_count, stream)
+              : launch_c<2, false>(L, G, W_hat, out_dtype, status, sm_count, stream);
   count_launches(1);
   timing_end(kKernDequant, stream);
   return err;

@@ -32,7 +32,7 @@
 // that is nearest in exact arithmetic is always among those rescored.
 #include <cuda_fp16.h>
 
-#include "pvt_internal.h"
+#include "pvt_encode_m1.cuh"
 
 namespace pvt {
 
@@ -72,58 +72,11 @@ int encode_m1_targets_per_thread(uint64_t k, int sm_count) {
   return k >= (uint64_t)sm_count * 2048ull * 4ull ? 8 : 4;
 }
 
+using namespace m1;
+
 namespace {
 
 constexpr float kPadHalfNorm = 3.0e38f;  // half norm of padding codewords: never near a minimum
-constexpr uint32_t kMaxSpins = 1u << 22;
-
-struct EncM1Params {
-  const float* W;
-  const float* g;
-  const float* scale;
-  const uint32_t* idx;
-  uint64_t k, G;
-  uint32_t gpr;
-  float eta;
-  const float* cbx;
-  const uint32_t* n2max_bits;
-  uint32_t n_chunks, K, n_tiles, n_slices, tile;
-  uint32_t* gbest;
-  float* margin;
-  CandRecord* rec;
-  const void* book;  // the caller's codebook [K][8]
-  void* codes;
-  int code_u16;
-  float* err_out;
-  uint32_t* status;
-};
-
-// order-preserving map binary32 -> u32 (and back)
-__device__ __forceinline__ uint32_t ord(float f) {
-  const uint32_t b = __float_as_uint(f);
-  return b ^ ((b >> 31) ? 0xffffffffu : 0x80000000u);
-}
-__device__ __forceinline__ float unord(uint32_t o) {
-  return __uint_as_float(o ^ ((o >> 31) ? 0x80000000u : 0xffffffffu));
-}
-
-// t = (W - eta g) / s of group j in binary32: one fma, one division per element
-__device__ __forceinline__ void form_target(const EncM1Params& p, uint32_t j, float* t) {
-  const float4* W4 = reinterpret_cast<const float4*>(p.W);
-  const float4* g4 = reinterpret_cast<const float4*>(p.g);
-  const float4 w0 = __ldg(W4 + 2 * (size_t)j), w1 = __ldg(W4 + 2 * (size_t)j + 1);
-  const float4 g0 = __ldg(g4 + 2 * (size_t)j), g1 = __ldg(g4 + 2 * (size_t)j + 1);
-  const float sc = __ldg(p.scale + j / p.gpr);
-  const float neg_eta = -p.eta;
-  t[0] = __fdiv_rn(__fmaf_rn(neg_eta, g0.x, w0.x), sc);
-  t[1] = __fdiv_rn(__fmaf_rn(neg_eta, g0.y, w0.y), sc);
-  t[2] = __fdiv_rn(__fmaf_rn(neg_eta, g0.z, w0.z), sc);
-  t[3] = __fdiv_rn(__fmaf_rn(neg_eta, g0.w, w0.w), sc);
-  t[4] = __fdiv_rn(__fmaf_rn(neg_eta, g1.x, w1.x), sc);
-  t[5] = __fdiv_rn(__fmaf_rn(neg_eta, g1.y, w1.y), sc);
-  t[6] = __fdiv_rn(__fmaf_rn(neg_eta, g1.z, w1.z), sc);
-  t[7] = __fdiv_rn(__fmaf_rn(neg_eta, g1.w, w1.w), sc);
-}
 
 // ---- codebook expansion ------------------------------------------------------
 // chunk block (kChunkBytes): 128 pairs * 16 floats, pair p holds
@@ -168,50 +121,6 @@ __global__ void expand_codebook_kernel(const void* __restrict__ book, uint32_t K
   uint32_t bits = __float_as_uint(n2);
   bits = __reduce_max_sync(0xffffffffu, bits);
   if ((threadIdx.x & 31) == 0 && bits) atomicMax(n2max_bits, bits);
-}
-
-// ---- PTX helpers ---------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// 1-D bulk copy global -> shared through the tensor memory accelerator; completes
-// `bytes` on the mbarrier.  Both addresses 16-byte aligned, bytes % 16 == 0.
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-               "l"(src), "r"(bytes), "r"(bar)
-               : "memory");
-}
-// Bounded wait.  Gives up after kMaxSpins polls (or as soon as another thread gave
-// up), flags the CTA as aborted and reports through the status word.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                          uint32_t* status) {
-  for (uint32_t spin = 0; spin < kMaxSpins; ++spin) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (spin > 32) __nanosleep(64);
-  }
-  *abort_flag = 1;
-  atomicOr(status, PVT_DEV_WAIT_EXPIRED);
-  return false;
 }
 
 __device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
@@ -269,8 +178,8 @@ __global__ void __launch_bounds__(kEncThreads + 32, 1) encode_m1_kernel(const En
       bool alive = true;
       for (uint64_t u = blockIdx.x; u < units && alive; u += gridDim.x) {
         const uint32_t sl = (uint32_t)(u % p.n_slices);
-        const uint32_t c_lo = (uint32_t)((uint64_t)sl * p.n_chunks / p.n_slices);
-        const uint32_t c_hi = (uint32_t)((uint64_t)(sl + 1) * p.n_chunks / p.n_slices);
+        uint32_t c_lo, c_hi;
+        slice_units(p, sl, &c_lo, &c_hi);
         for (uint32_t c = c_lo; c < c_hi && alive; ++c, ++it) {
           const uint32_t s = it % kEncStages;
           if (it >= kEncStages)
@@ -304,8 +213,8 @@ __global__ void __launch_bounds__(kEncThreads + 32, 1) encode_m1_kernel(const En
   for (uint64_t u = blockIdx.x; u < units; u += gridDim.x) {
     const uint32_t tile = (uint32_t)(u / p.n_slices);
     const uint32_t sl = (uint32_t)(u % p.n_slices);
-    const uint32_t c_lo = (uint32_t)((uint64_t)sl * p.n_chunks / p.n_slices);
-    const uint32_t c_hi = (uint32_t)((uint64_t)(sl + 1) * p.n_chunks / p.n_slices);
+    uint32_t c_lo, c_hi;
+    slice_units(p, sl, &c_lo, &c_hi);
 
     // 1. gather targets, form t, set up tracking
     uint64_t nt[TT][8];  // (-t_i, -t_i)
@@ -435,10 +344,10 @@ __device__ __forceinline__ void load_codeword(const void* book, uint32_t kappa, 
   }
 }
 
-// One warp per target.  `sub_cw` = codewords per sub-chunk of the search kernel
-// that wrote the records (a multiple of 32).
+// One warp per target.
 template <bool CB_F16>
-__global__ void __launch_bounds__(256) rescore_m1_kernel(const EncM1Params p, uint32_t sub_cw) {
+__global__ void __launch_bounds__(256) rescore_m1_kernel(const EncM1Params p) {
+  const uint32_t sub_cw = p.sub_cw;
   const int lane = threadIdx.x & 31;
   const uint64_t n = (uint64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (n >= p.k) return;
@@ -451,7 +360,7 @@ __global__ void __launch_bounds__(256) rescore_m1_kernel(const EncM1Params p, ui
   form_target(p, j, t);
   const float limit = unord(p.gbest[n]) + p.margin[n];
   const uint32_t tile = (uint32_t)(n / p.tile), s = (uint32_t)(n % p.tile);
-  const uint32_t subs_per_chunk = kChunkCodewords / sub_cw;
+  const uint32_t subs_per_unit = p.unit_cw / sub_cw;
   double best_d = __longlong_as_double(0x7ff0000000000000ll);
   uint32_t best_code = 0xffffffffu;
 
@@ -480,12 +389,32 @@ __global__ void __launch_bounds__(256) rescore_m1_kernel(const EncM1Params p, ui
     const CandRecord r = *reinterpret_cast<const CandRecord*>(&raw);
     if (!(r.best <= limit)) continue;
     if (r.cnt == kCandOverflow) {
-      const uint32_t c_lo = (uint32_t)((uint64_t)sl * p.n_chunks / p.n_slices);
-      const uint32_t c_hi = (uint32_t)((uint64_t)(sl + 1) * p.n_chunks / p.n_slices);
-      for (uint32_t sub = c_lo * subs_per_chunk; sub < c_hi * subs_per_chunk; ++sub) visit(sub);
+      uint32_t u_lo, u_hi;
+      slice_units(p, sl, &u_lo, &u_hi);
+      for (uint32_t sub = u_lo * subs_per_unit; sub < u_hi * subs_per_unit; ++sub) visit(sub);
     } else {
       const uint32_t cnt = r.cnt < (uint16_t)kListLen ? r.cnt : (uint32_t)kListLen;
       for (uint32_t e = 0; e < cnt; ++e) visit(r.sub[e]);
+    }
+  }
+  if (p.exc_count) {  // codewords whose fast score is not trustworthy: always evaluated
+    const uint32_t n_exc = __ldg(p.exc_count);
+    for (uint32_t e = lane; e < n_exc && e < p.K; e += 32) {
+      const uint32_t kappa = __ldg(p.exc_list + e);
+      if (kappa < p.K) {
+        float c[8];
+        load_codeword<CB_F16>(p.book, kappa, c);
+        double d = 0.0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const double df = __dsub_rn((double)t[i], (double)c[i]);
+          d = __dadd_rn(d, __dmul_rn(df, df));
+        }
+        if (d < best_d || (d == best_d && kappa < best_code)) {
+          best_d = d;
+          best_code = kappa;
+        }
+      }
     }
   }
   // warp-wide lexicographic minimum of (distance, code); distances are >= 0 so their bits order like u64
@@ -537,7 +466,11 @@ cudaError_t launch_encode_m1(const pvt_layer& L, uint64_t G, const uint32_t* idx
   p.eta = L.eta;
   p.cbx = reinterpret_cast<const float*>(base + lay.cbx_off);
   p.n2max_bits = reinterpret_cast<const uint32_t*>(base + lay.n2max_off);
-  p.n_chunks = lay.n_chunks;
+  p.n_units = lay.n_chunks;
+  p.unit_cw = kChunkCodewords;
+  p.sub_cw = kSubCodewords;
+  p.exc_count = nullptr;
+  p.exc_list = nullptr;
   p.K = (uint32_t)L.codebook_size;
   p.n_tiles = lay.n_tiles;
   p.n_slices = lay.n_slices;
@@ -568,12 +501,16 @@ cudaError_t launch_encode_m1(const pvt_layer& L, uint64_t G, const uint32_t* idx
   if ((err = cudaGetLastError()) != cudaSuccess) return err;
   err = tt == 8 ? launch_tt<8>(p, lay.n_ctas, stream) : launch_tt<4>(p, lay.n_ctas, stream);
   if (err != cudaSuccess) return err;
+  return launch_rescore_m1(p, f16, stream);
+}
+
+cudaError_t launch_rescore_m1(const EncM1Params& p, bool codebook_f16, cudaStream_t stream) {
   timing_begin(kKernEncodeRescore, stream);
-  const unsigned blocks = (unsigned)((k + 7) / 8);
-  if (f16)
-    rescore_m1_kernel<true><<<blocks, 256, 0, stream>>>(p, kSubCodewords);
+  const unsigned blocks = (unsigned)((p.k + 7) / 8);
+  if (codebook_f16)
+    rescore_m1_kernel<true><<<blocks, 256, 0, stream>>>(p);
   else
-    rescore_m1_kernel<false><<<blocks, 256, 0, stream>>>(p, kSubCodewords);
+    rescore_m1_kernel<false><<<blocks, 256, 0, stream>>>(p);
   count_launches(1);
   timing_end(kKernEncodeRescore, stream);
   return cudaGetLastError();

@@ -1,0 +1,558 @@
+// Exhaustive nearest-codeword search of the V step for one fp16 codebook on the
+// tensor cores (Appendix C / Appendix J: "try every code in the codebook";
+// Appendix D: the score ||c||^2 - 2 <t, c>; Eq. 8 for the target).
+//
+// The score matrix S[n][kappa] = 2^e_n (<t_n, c_kappa> - ||c_kappa||^2 / 2) is a
+// dense contraction of depth 8 (+ the norm term): it is evaluated tile by tile
+// with tcgen05.mma (fp16 operands, fp32 accumulators in tensor memory) and never
+// leaves the SM -- the epilogue reads each accumulator row once and keeps only
+// its running maximum and the 64-codeword sub-chunks that come within an error
+// margin of it.  The exact decision (binary64 distances, argmin of (distance,
+// code)) is taken afterwards by the rescoring kernel on those sub-chunks, so the
+// fp16 rounding of the operands only has to be bounded, not small.
+//
+// Operands (K = 32 halves per row = four 16-byte K chunks, no swizzle, K-major
+// "interleaved" core-matrix layout: 8 rows x 16 bytes per core matrix, K chunks
+// 128 bytes apart, 8-row groups 512 bytes apart; one MMA instruction consumes two
+// K chunks, so a step is two instructions per A block, the second accumulating):
+//   A row n     = [ hi_0 .. hi_7 | lo_0 .. lo_7 | 2^e x 8 | 0 x 8 ]
+//                 hi_i = fp16(2^e t_i), lo_i = fp16(2^e t_i - hi_i)
+//   B row kappa = [ c_0 .. c_7   | c_0 .. c_7   | -h_hi, -h_lo, -h_lo2, 0 x 5 | 0 x 8 ]
+//                 h = ||c||^2/2 = h_hi + h_lo + h_lo2
+// Splitting t into two halves keeps 22 of its 24 significant bits, so the fast
+// score is about as accurate as a binary32 evaluation and very few sub-chunks
+// come within the margin.  The codebook image is written once per call by a small
+// kernel in exactly the shared-memory byte order, so every 128-codeword step
+// arrives with one 1-D bulk copy (8 KB); the A rows are written by the threads
+// that own the targets.  e_n is chosen per target so that max_i |2^e t_i| lies in
+// [1/2, 1).
+//
+// CTA = 256 targets (two 128-row A blocks) x a slice of the codebook, one CTA per
+// SM, persistent over (tile, slice) units.  Warps 0-7: own one target per thread,
+// build A, run the epilogue (warp w reads tensor-memory lanes 32 (w % 4) .. of the
+// accumulator of A block w / 4).  Warp 8: bulk-copy producer.  Warp 9: allocates
+// tensor memory and issues the MMAs (one thread).  Tensor memory: 2 buffers x 2
+// accumulators x 128 columns = 512 columns, so the MMAs of step i+1 overlap the
+// epilogue of step i.
+//
+// Codewords whose half squared norm exceeds the fp16 range get a sentinel row
+// that can never win and are listed as "exceptions": the rescoring kernel always
+// evaluates them exactly.  Targets outside the range the scaling can serve
+// (non-finite, or max |t_i| >= 256) are rescored against the whole codebook.
+#include "pvt_encode_m1.cuh"
+
+namespace pvt {
+
+using namespace m1;
+
+namespace {
+
+constexpr int kTcTile = 256;            // targets per CTA tile
+constexpr int kTcStepCw = 128;          // codewords per MMA step (the N of one instruction)
+constexpr int kTcRowBytes = 64;         // 32 halves
+constexpr int kTcStepBytes = kTcStepCw * kTcRowBytes;  // 8192
+constexpr int kTcGroupBytes = 8 * kTcRowBytes;         // one 8-row group: 4 core matrices of 128 bytes
+constexpr int kTcSubCw = 64;            // tracking granularity of the running maximum
+constexpr int kTcStages = 12;           // bulk-copy ring
+constexpr int kTcEpiThreads = 256;
+constexpr int kTcThreads = kTcEpiThreads + 64;
+constexpr uint32_t kTmemCols = 512;
+constexpr float kMaxHalfNorm = 60000.0f;  // largest ||c||^2/2 the image represents
+constexpr float kNegInf = -__builtin_huge_valf();
+
+}  // namespace
+
+bool encode_m1_use_tc(const pvt_layer& L, uint64_t k) {
+  (void)k;
+  return L.num_codebooks == 1 && L.codebook_dtype == PVT_F16 && L.codebook_size >= 1024;
+}
+
+EncodeM1TcLayout encode_m1_tc_layout(uint32_t K, uint64_t k, int sm_count) {
+  EncodeM1TcLayout e;
+  e.n_steps = (K + kTcStepCw - 1) / kTcStepCw;
+  e.n_tiles = (uint32_t)((k + kTcTile - 1) / kTcTile);
+  uint32_t best_s = 1;
+  double best_eff = 0.0;
+  // a slice should keep at least 16 steps so that building A stays a small part of a unit
+  uint32_t s_max = e.n_steps / 16;
+  if (s_max < 1) s_max = 1;
+  if (s_max > (uint32_t)kMaxSlices) s_max = (uint32_t)kMaxSlices;
+  for (uint32_t s = 1; s <= s_max; ++s) {
+    const uint64_t units = (uint64_t)e.n_tiles * s;
+    const uint64_t rounds = (units + sm_count - 1) / sm_count;
+    const double eff = (double)units / (double)(rounds * sm_count);
+    if (eff > best_eff + 0.03) {
+      best_eff = eff;
+      best_s = s;
+    }
+  }
+  e.n_slices = best_s;
+  const uint64_t units = (uint64_t)e.n_tiles * e.n_slices;
+  e.n_ctas = (uint32_t)(units < (uint64_t)sm_count ? units : (uint64_t)sm_count);
+  e.bimg_off = kWsHeaderBytes;
+  e.stats_off = align_up(e.bimg_off + (size_t)e.n_steps * kTcStepBytes, kWsAlign);
+  e.exc_off = e.stats_off + kWsAlign;
+  e.gbest_off = align_up(e.exc_off + sizeof(uint32_t) * K, kWsAlign);
+  e.margin_off = align_up(e.gbest_off + sizeof(uint32_t) * k, kWsAlign);
+  e.rec_off = align_up(e.margin_off + sizeof(float) * k, kWsAlign);
+  e.bytes = align_up(e.rec_off + (size_t)e.n_tiles * e.n_slices * kTcTile * sizeof(CandRecord), kWsAlign);
+  return e;
+}
+
+namespace {
+
+// stats block in the workspace: [0] bit pattern of max ||c||^2 over representable codewords, [1] exception count
+struct TcStats {
+  uint32_t n2max_bits;
+  uint32_t exc_count;
+};
+
+// ---- codebook image ------------------------------------------------------------
+__global__ void __launch_bounds__(256) tc_prep_kernel(const uint4* __restrict__ book, uint32_t K, uint32_t n_steps,
+                                                       unsigned char* __restrict__ bimg, TcStats* stats,
+                                                       uint32_t* __restrict__ exc_list) {
+  const uint32_t kappa = blockIdx.x * blockDim.x + threadIdx.x;
+  uint32_t n2bits = 0;
+  if (kappa < n_steps * kTcStepCw) {
+    const bool real = kappa < K;
+    uint4 raw = make_uint4(0, 0, 0, 0);
+    float n2 = 0.0f;
+    if (real) {
+      raw = __ldg(book + kappa);
+      const __half2* h = reinterpret_cast<const __half2*>(&raw);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float2 f = __half22float2(h[i]);
+        n2 = __fmaf_rn(f.x, f.x, n2);
+        n2 = __fmaf_rn(f.y, f.y, n2);
+      }
+    }
+    const float hn = 0.5f * n2;
+    const bool rep = real && (hn <= kMaxHalfNorm);  // false for NaN / Inf as well
+    if (real && !rep) {
+      const uint32_t pos = atomicAdd(&stats->exc_count, 1u);
+      if (pos < K) exc_list[pos] = kappa;
+    }
+    uint4 k0, k1;
+    if (rep) {
+      const __half h_hi = __float2half_rn(hn);
+      const float r1 = hn - __half2float(h_hi);
+      const __half h_lo = __float2half_rn(r1);
+      const float r2 = r1 - __half2float(h_lo);
+      const __half h_lo2 = __float2half_rn(r2);
+      const __half2 a = __halves2half2(__hneg(h_hi), __hneg(h_lo));
+      const __half2 b = __halves2half2(__hneg(h_lo2), __float2half_rn(0.0f));
+      k0 = raw;
+      k1 = make_uint4(*reinterpret_cast<const uint32_t*>(&a), *reinterpret_cast<const uint32_t*>(&b), 0u, 0u);
+      n2bits = __float_as_uint(n2);
+    } else {
+      // padding and exceptions: zero codeword with the most negative norm terms, never a maximum
+      k0 = make_uint4(0, 0, 0, 0);
+      k1 = make_uint4(0xfbfffbffu, 0xfbfffbffu, 0xfbfffbffu, 0xfbfffbffu);  // -65504 x 8
+    }
+    const uint32_t step = kappa / kTcStepCw, r = kappa % kTcStepCw;
+    unsigned char* row = bimg + (size_t)step * kTcStepBytes + (r >> 3) * kTcGroupBytes + (r & 7) * 16;
+    *reinterpret_cast<uint4*>(row) = k0;        // pairs with hi
+    *reinterpret_cast<uint4*>(row + 128) = k0;  // pairs with lo
+    *reinterpret_cast<uint4*>(row + 256) = k1;  // norm terms
+    *reinterpret_cast<uint4*>(row + 384) = make_uint4(0, 0, 0, 0);
+  }
+  n2bits = __reduce_max_sync(0xffffffffu, n2bits);
+  if ((threadIdx.x & 31) == 0 && n2bits) atomicMax(&stats->n2max_bits, n2bits);
+}
+
+// ---- tcgen05 wrappers -----------------------------------------------------------
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]^T, fp16 x fp16 -> fp32, M = 128, N = 128, K = 16;
+// accumulate == 0 overwrites D
+__device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                         uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// arrive on the mbarrier once all MMAs issued so far by this thread have completed
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// shared-memory operand descriptor: K-major, no swizzle, K chunks 128 B apart, 8-row groups kTcGroupBytes apart
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr) {
+  return (uint64_t)((saddr & 0x3ffffu) >> 4) | ((uint64_t)(128u >> 4) << 16) |
+         ((uint64_t)((uint32_t)kTcGroupBytes >> 4) << 32) | (1ull << 46);
+}
+// instruction descriptor: D fp32, A and B fp16, both K-major, N = 128, M = 128
+constexpr uint64_t kDescTwoChunks = 256u >> 4;  // start-address field advance for two K chunks
+constexpr uint32_t kIdesc = (1u << 4) | ((uint32_t)(kTcStepCw >> 3) << 17) | ((128u >> 4) << 24);
+
+// 32 lanes x 64 consecutive columns of 32-bit accumulators -> 64 registers per thread
+__device__ __forceinline__ void tmem_ld64(uint32_t taddr, uint32_t* v) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x64.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, "
+      "%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, "
+      "%48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31]), "=r"(v[32]),
+        "=r"(v[33]), "=r"(v[34]), "=r"(v[35]), "=r"(v[36]), "=r"(v[37]), "=r"(v[38]), "=r"(v[39]), "=r"(v[40]),
+        "=r"(v[41]), "=r"(v[42]), "=r"(v[43]), "=r"(v[44]), "=r"(v[45]), "=r"(v[46]), "=r"(v[47]), "=r"(v[48]),
+        "=r"(v[49]), "=r"(v[50]), "=r"(v[51]), "=r"(v[52]), "=r"(v[53]), "=r"(v[54]), "=r"(v[55]), "=r"(v[56]),
+        "=r"(v[57]), "=r"(v[58]), "=r"(v[59]), "=r"(v[60]), "=r"(v[61]), "=r"(v[62]), "=r"(v[63])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ float max64(const uint32_t* v) {
+  float m0 = max3(__uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]));
+  float m1 = max3(__uint_as_float(v[3]), __uint_as_float(v[4]), __uint_as_float(v[5]));
+  float m2 = max3(__uint_as_float(v[6]), __uint_as_float(v[7]), __uint_as_float(v[8]));
+  float m3 = max3(__uint_as_float(v[9]), __uint_as_float(v[10]), __uint_as_float(v[11]));
+#pragma unroll
+  for (int i = 12; i < 60; i += 8) {
+    m0 = max3(m0, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+    m1 = max3(m1, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+    m2 = max3(m2, __uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
+    m3 = max3(m3, __uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
+  }
+  m0 = max3(m0, __uint_as_float(v[60]), __uint_as_float(v[61]));
+  m1 = max3(m1, __uint_as_float(v[62]), __uint_as_float(v[63]));
+  return fmaxf(max3(m0, m1, m2), m3);
+}
+
+// ---- shared memory -----------------------------------------------------------------
+struct TcSmem {
+  alignas(128) unsigned char a[2][kTcStepBytes];  // two A blocks of 128 targets
+  alignas(128) unsigned char b[kTcStages][kTcStepBytes];
+  alignas(8) uint64_t full_bar[kTcStages];
+  uint64_t empty_bar[kTcStages];
+  uint64_t tmem_full[2];
+  uint64_t tmem_empty[2];
+  uint64_t a_ready;
+  uint64_t drain_bar;
+  float evicted_max[kTcTile];           // largest sub-chunk maximum that fell out of the list
+  float list_max[kListLen][kTcTile];
+  uint16_t list_id[kListLen][kTcTile];
+  uint16_t list_cnt[kTcTile];
+  uint32_t tmem_base;
+  uint32_t abort_flag;
+};
+
+__global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1Params p,
+                                                                      const unsigned char* __restrict__ bimg,
+                                                                      const TcStats* __restrict__ stats) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  TcSmem& sm = *reinterpret_cast<TcSmem*>(smem_raw);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  volatile uint32_t* abort_flag = &sm.abort_flag;
+
+  if (tid == 0) {
+    sm.abort_flag = 0;
+    for (int s = 0; s < kTcStages; ++s) {
+      mbar_init(smem_u32(&sm.full_bar[s]), 1);
+      mbar_init(smem_u32(&sm.empty_bar[s]), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&sm.tmem_full[b]), 1);
+      mbar_init(smem_u32(&sm.tmem_empty[b]), kTcEpiThreads / 32);
+    }
+    mbar_init(smem_u32(&sm.a_ready), kTcEpiThreads);
+    mbar_init(smem_u32(&sm.drain_bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 9) {
+    tmem_alloc(smem_u32(&sm.tmem_base), kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&sm.tmem_base);
+
+  const uint64_t units = (uint64_t)p.n_tiles * p.n_slices;
+
+  if (warp == 8) {
+    // ------------------------------------------------------------ bulk-copy producer
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool alive = true;
+      for (uint64_t u = blockIdx.x; u < units && alive; u += gridDim.x) {
+        uint32_t s_lo, s_hi;
+        slice_units(p, (uint32_t)(u % p.n_slices), &s_lo, &s_hi);
+        for (uint32_t st = s_lo; st < s_hi && alive; ++st, ++it) {
+          const uint32_t s = it % kTcStages;
+          if (it >= kTcStages)
+            alive = mbar_wait(smem_u32(&sm.empty_bar[s]), ((it / kTcStages) - 1) & 1, abort_flag, p.status);
+          if (!alive) break;
+          const uint32_t fb = smem_u32(&sm.full_bar[s]);
+          mbar_expect_tx(fb, kTcStepBytes);
+          bulk_g2s(smem_u32(&sm.b[s][0]), bimg + (size_t)st * kTcStepBytes, kTcStepBytes, fb);
+        }
+      }
+      if (!alive) {
+        // let every copy that was issued land before the CTA may exit
+        for (uint32_t back = 1; back <= kTcStages && back <= it; ++back) {
+          const uint32_t j = it - back;
+          const uint32_t fb = smem_u32(&sm.full_bar[j % kTcStages]);
+          for (uint32_t spin = 0; spin < kMaxSpins; ++spin) {
+            if (mbar_try_wait(fb, (j / kTcStages) & 1)) break;
+            __nanosleep(64);
+          }
+        }
+      }
+    }
+  } else if (warp == 9) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint64_t a_desc0 = smem_desc(smem_u32(&sm.a[0][0]));
+      const uint64_t a_desc1 = smem_desc(smem_u32(&sm.a[1][0]));
+      uint32_t it = 0, unit_i = 0;
+      bool alive = true;
+      for (uint64_t u = blockIdx.x; u < units && alive; u += gridDim.x, ++unit_i) {
+        uint32_t s_lo, s_hi;
+        slice_units(p, (uint32_t)(u % p.n_slices), &s_lo, &s_hi);
+        alive = mbar_wait(smem_u32(&sm.a_ready), unit_i & 1, abort_flag, p.status);
+        tc_fence_after();
+        for (uint32_t st = s_lo; st < s_hi && alive; ++st, ++it) {
+          const uint32_t s = it % kTcStages, buf = it & 1;
+          alive = mbar_wait(smem_u32(&sm.full_bar[s]), (it / kTcStages) & 1, abort_flag, p.status);
+          if (alive) alive = mbar_wait(smem_u32(&sm.tmem_empty[buf]), ((it >> 1) & 1) ^ 1, abort_flag, p.status);
+          if (!alive) break;
+          tc_fence_after();
+          const uint64_t b_desc = smem_desc(smem_u32(&sm.b[s][0]));
+          // K chunks 0-1 (hi, lo against c), then chunks 2-3 (the norm terms) on top
+          umma_f16(tmem_base + buf * 256, a_desc0, b_desc, kIdesc, 0);
+          umma_f16(tmem_base + buf * 256, a_desc0 + kDescTwoChunks, b_desc + kDescTwoChunks, kIdesc, 1);
+          umma_f16(tmem_base + buf * 256 + 128, a_desc1, b_desc, kIdesc, 0);
+          umma_f16(tmem_base + buf * 256 + 128, a_desc1 + kDescTwoChunks, b_desc + kDescTwoChunks, kIdesc, 1);
+          umma_commit(smem_u32(&sm.empty_bar[s]));   // the stage is free once both MMAs have read it
+          umma_commit(smem_u32(&sm.tmem_full[buf])); // the accumulators are ready
+        }
+      }
+      if (!alive) {
+        // wait (bounded) for whatever was issued before tensor memory is released
+        umma_commit(smem_u32(&sm.drain_bar));
+        for (uint32_t spin = 0; spin < kMaxSpins; ++spin) {
+          if (mbar_try_wait(smem_u32(&sm.drain_bar), 0)) break;
+          __nanosleep(64);
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ target owners / epilogue
+    const float n2max = __uint_as_float(stats->n2max_bits);
+    const float cnmax = sqrtf(n2max), hmax = 0.5f * n2max;
+    const uint32_t rb = (uint32_t)tid >> 7, r = (uint32_t)tid & 127u;
+    unsigned char* a_row = &sm.a[rb][(r >> 3) * kTcGroupBytes + (r & 7) * 16];
+    const uint32_t lane_base = ((uint32_t)(warp & 3) * 32u) << 16;
+    uint32_t it = 0;
+    bool alive = true;
+
+    for (uint64_t u = blockIdx.x; u < units && alive; u += gridDim.x) {
+      const uint32_t tile = (uint32_t)(u / p.n_slices), sl = (uint32_t)(u % p.n_slices);
+      uint32_t s_lo, s_hi;
+      slice_units(p, sl, &s_lo, &s_hi);
+      const uint64_t n = (uint64_t)tile * kTcTile + tid;
+
+      // the target of this thread, its scaling, its A row
+      float t[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) t[i] = 0.0f;
+      bool have = false;
+      if (n < p.k) {
+        const uint32_t j = p.idx[n];
+        if (j < p.G) {  // an index out of range is reported by the rescoring kernel
+          form_target(p, j, t);
+          have = true;
+        }
+      }
+      float m = 0.0f, nt2 = 0.0f;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        m = fmaxf(m, fabsf(t[i]));
+        nt2 = fmaf(t[i], t[i], nt2);
+      }
+      bool in_range = (m < 256.0f) && (nt2 == nt2);  // also false for Inf / NaN
+      int e = 0;
+      if (in_range && m > 0.0f) {
+        e = -ilogbf(m) - 1;
+        e = e > 15 ? 15 : e;
+      }
+      const float sc = in_range ? scalbnf(1.0f, e) : 0.0f;
+      {
+        __half2 hi[4], lo[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float x = in_range ? t[2 * i] * sc : 0.0f, y = in_range ? t[2 * i + 1] * sc : 0.0f;  // exact products
+          hi[i] = __floats2half2_rn(x, y);
+          const float2 back = __half22float2(hi[i]);
+          lo[i] = __floats2half2_rn(x - back.x, y - back.y);  // exact differences, rounded once
+        }
+        const __half2 s2 = __floats2half2_rn(sc, sc);
+        const uint32_t sb = *reinterpret_cast<const uint32_t*>(&s2);
+        *reinterpret_cast<uint4*>(a_row) = *reinterpret_cast<const uint4*>(hi);
+        *reinterpret_cast<uint4*>(a_row + 128) = *reinterpret_cast<const uint4*>(lo);
+        *reinterpret_cast<uint4*>(a_row + 256) = make_uint4(sb, sb, sb, sb);
+        *reinterpret_cast<uint4*>(a_row + 384) = make_uint4(0, 0, 0, 0);
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the MMA
+      mbar_arrive(smem_u32(&sm.a_ready));
+
+      // twice the error bound of the fast score, in its own (scaled) units, with a factor 2 to spare.
+      // |hi + lo - 2^e t_i| <= 2^-22 |2^e t_i| (2^-25 where lo is subnormal); the norm split is exact to
+      // 2^-33 h; products of halves are exact in fp32; the accumulation of at most 32 terms in fp32, rounded
+      // or truncated, stays below 2^-19 of the sum of magnitudes 2^e (||t|| ||c|| + h)
+      const float margin = sc * 1.52587890625e-5f /* 2^-16 */ * (sqrtf(nt2) * cnmax + hmax) +
+                           4.76837158203125e-7f /* 2^-21 */ * cnmax + 1e-30f;
+      float best = kNegInf, thr = kNegInf;
+      sm.list_cnt[tid] = 0;
+      sm.evicted_max[tid] = kNegInf;
+
+      for (uint32_t st = s_lo; st < s_hi; ++st, ++it) {
+        const uint32_t buf = it & 1;
+        // warp-uniform outcome: the tensor-memory loads below need the whole warp
+        alive = __all_sync(0xffffffffu, mbar_wait(smem_u32(&sm.tmem_full[buf]), (it >> 1) & 1, abort_flag, p.status));
+        if (!alive) break;
+        tc_fence_after();
+        const uint32_t taddr = tmem_base + lane_base + buf * 256 + rb * 128;
+        uint32_t v[64], w[64];
+        tmem_ld64(taddr, v);
+        tmem_ld64(taddr + 64, w);
+        tmem_ld_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&sm.tmem_empty[buf]));
+        const float m0 = max64(v), m1 = max64(w);
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          const float mx = half ? m1 : m0;
+          if (mx >= thr) {
+            const uint32_t cnt = sm.list_cnt[tid];
+            const uint32_t slot = cnt & (kListLen - 1);
+            if (cnt >= kListLen) sm.evicted_max[tid] = fmaxf(sm.evicted_max[tid], sm.list_max[slot][tid]);
+            sm.list_id[slot][tid] = (uint16_t)(st * 2 + half);
+            sm.list_max[slot][tid] = mx;
+            sm.list_cnt[tid] = (uint16_t)(cnt + 1);
+            best = fmaxf(best, mx);
+            thr = best - margin;
+          }
+        }
+      }
+
+      // leave the candidates of this (tile, slice) for the rescoring kernel (minimum convention: -S)
+      if (alive && have) {
+        CandRecord rec;
+        rec.pad = 0;
+        uint32_t cnt_out = 0;
+#pragma unroll
+        for (int q = 0; q < kListLen; ++q) rec.sub[q] = 0;
+        if (in_range) {
+          const float limit = best - margin;
+          const uint32_t cnt = sm.list_cnt[tid];
+#pragma unroll
+          for (int q = 0; q < kListLen; ++q)
+            if ((uint32_t)q < cnt && sm.list_max[q][tid] >= limit) rec.sub[cnt_out++] = sm.list_id[q][tid];
+          rec.best = -best;
+          rec.cnt = (cnt > (uint32_t)kListLen && sm.evicted_max[tid] >= limit) ? kCandOverflow : (uint16_t)cnt_out;
+        } else {
+          rec.best = kNegInf;  // passes every limit: the whole slice is rescored exactly
+          rec.cnt = kCandOverflow;
+        }
+        *reinterpret_cast<uint4*>(&p.rec[((size_t)tile * p.n_slices + sl) * kTcTile + tid]) =
+            *reinterpret_cast<const uint4*>(&rec);
+        atomicMin(&p.gbest[n], ord(rec.best));
+        if (sl == 0) p.margin[n] = in_range ? margin : 0.0f;
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 9) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_encode_m1_tc(const pvt_layer& L, uint64_t G, const uint32_t* idx, uint64_t k, float* err_out,
+                                void* ws, int sm_count, cudaStream_t stream) {
+  const EncodeM1TcLayout lay = encode_m1_tc_layout((uint32_t)L.codebook_size, k, sm_count);
+  char* base = static_cast<char*>(ws);
+  TcStats* stats = reinterpret_cast<TcStats*>(base + lay.stats_off);
+  EncM1Params p;
+  p.W = L.W;
+  p.g = L.g;
+  p.scale = L.scale;
+  p.idx = idx;
+  p.k = k;
+  p.G = G;
+  p.gpr = (uint32_t)(L.cols / kGroupDim);
+  p.eta = L.eta;
+  p.cbx = nullptr;
+  p.n2max_bits = &stats->n2max_bits;
+  p.K = (uint32_t)L.codebook_size;
+  p.n_tiles = lay.n_tiles;
+  p.n_slices = lay.n_slices;
+  p.tile = kTcTile;
+  p.n_units = lay.n_steps;
+  p.unit_cw = kTcStepCw;
+  p.sub_cw = kTcSubCw;
+  p.exc_count = &stats->exc_count;
+  p.exc_list = reinterpret_cast<const uint32_t*>(base + lay.exc_off);
+  p.gbest = reinterpret_cast<uint32_t*>(base + lay.gbest_off);
+  p.margin = reinterpret_cast<float*>(base + lay.margin_off);
+  p.rec = reinterpret_cast<CandRecord*>(base + lay.rec_off);
+  p.book = L.codebooks;
+  p.codes = L.codes;
+  p.code_u16 = L.code_dtype == PVT_U16;
+  p.err_out = err_out;
+  p.status = reinterpret_cast<uint32_t*>(base);
+
+  cudaError_t err = cudaMemsetAsync(stats, 0, sizeof(TcStats), stream);
+  if (err != cudaSuccess) return err;
+  if ((err = cudaMemsetAsync(p.gbest, 0xff, sizeof(uint32_t) * k, stream)) != cudaSuccess) return err;
+  timing_begin(kKernEncodeAux, stream);
+  const uint32_t n_cw = lay.n_steps * kTcStepCw;
+  tc_prep_kernel<<<(n_cw + 255) / 256, 256, 0, stream>>>(reinterpret_cast<const uint4*>(L.codebooks), p.K, lay.n_steps,
+                                                         reinterpret_cast<unsigned char*>(base + lay.bimg_off), stats,
+                                                         reinterpret_cast<uint32_t*>(base + lay.exc_off));
+  count_launches(1);
+  timing_end(kKernEncodeAux, stream);
+  if ((err = cudaGetLastError()) != cudaSuccess) return err;
+
+  const size_t smem = sizeof(TcSmem);
+  if ((err = cudaFuncSetAttribute(encode_m1_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) !=
+      cudaSuccess)
+    return err;
+  timing_begin(kKernEncodeMain, stream);
+  encode_m1_tc_kernel<<<lay.n_ctas, kTcThreads, smem, stream>>>(
+      p, reinterpret_cast<const unsigned char*>(base + lay.bimg_off), stats);
+  timing_end(kKernEncodeMain, stream);
+  count_launches(1);
+  if ((err = cudaGetLastError()) != cudaSuccess) return err;
+  return launch_rescore_m1(p, true, stream);
+}
+
+}  // namespace pvt

@@ -82,15 +82,32 @@ EncodeM1Layout encode_m1_layout(uint32_t K, uint64_t k, int sm_count, int target
 int encode_m1_targets_per_thread(uint64_t k, int sm_count);  // 4 or 8
 size_t encode_m2_workspace_bytes();
 
+// encode, M = 1 on the tensor cores (fp16 codebooks of at least 1024 codewords)
+struct EncodeM1TcLayout {
+  size_t bimg_off;    // codebook image in operand order: n_steps * 4096 bytes
+  size_t stats_off;   // max ||c||^2 (bit pattern), exception count
+  size_t exc_off;     // u32 [K]: codewords the image cannot represent
+  size_t gbest_off, margin_off, rec_off;
+  size_t bytes;
+  uint32_t n_steps;   // 128-codeword steps
+  uint32_t n_tiles;   // tiles of 256 targets
+  uint32_t n_slices;
+  uint32_t n_ctas;
+};
+bool encode_m1_use_tc(const pvt_layer& L, uint64_t k);
+EncodeM1TcLayout encode_m1_tc_layout(uint32_t K, uint64_t k, int sm_count);
+
 // launchers (each returns a cudaError_t) --------------------------------------
 cudaError_t launch_select(const pvt_layer& L, uint64_t G, uint64_t k, uint32_t* idx_out, void* ws,
                           cudaStream_t stream);
 cudaError_t launch_encode_m1(const pvt_layer& L, uint64_t G, const uint32_t* idx, uint64_t k, float* err_out,
                              void* ws, int sm_count, cudaStream_t stream);
+cudaError_t launch_encode_m1_tc(const pvt_layer& L, uint64_t G, const uint32_t* idx, uint64_t k, float* err_out,
+                                void* ws, int sm_count, cudaStream_t stream);
 cudaError_t launch_encode_m2(const pvt_layer& L, uint64_t G, const uint32_t* idx, uint64_t k, float* err_out,
                              void* ws, int sm_count, cudaStream_t stream);
 cudaError_t launch_dequant(const pvt_layer& L, uint64_t G, void* W_hat, int32_t out_dtype, uint32_t* status,
-                           cudaStream_t stream);
+                           int sm_count, cudaStream_t stream);
 
 // optional per-kernel timing (benchmark instrumentation) ----------------------
 enum KernelId {
