@@ -126,6 +126,8 @@ def run_ours(args):
 
     cfg, which, tau = workloads()[args.workload]
     name, rows, cols, M, K, f16, rowmax, _ = synth.CONFIGS[cfg][which]
+    B.pvt_set_m1_search({"auto": B.PVT_M1_AUTO, "fp32": B.PVT_M1_FP32, "tensor": B.PVT_M1_TENSOR}[args.search])
+    tensor_engine = M == 1 and f16 and (args.search == "tensor" or (args.search == "auto" and K >= 1024))
 
     def gpu_nearest(X, C):  # only the recipe of a second codebook needs it: the library's own search
         return _nearest_on_gpu(X, C)
@@ -152,7 +154,13 @@ def run_ours(args):
     h_codes_out = torch.empty_like(h["codes"]).pin_memory()
     desc = B.make_layer(rows, cols, d["W"], d["g"], d["scale"], d["codebooks"], d["codes"], eta=L.eta, beam=L.beam)
     ws = B.new_workspace(desc, k, device=dev)
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)  # twice the L2
+    flush = torch.empty(64 << 20, dtype=torch.int32, device=dev)  # 256 MiB, twice the L2
+
+    def flush_l2():
+        # write, then read: the write evicts every line of the step's arrays, the read leaves the L2 full of
+        # clean lines, so that no write-back of the flush buffer is charged to the step that follows
+        flush.fill_(1)
+        flush.sum()
 
     def step():
         B.pvt_vstep_select(desc, k, idx, ws)
@@ -187,7 +195,7 @@ def run_ours(args):
     barrier()
     for a, b in ev:
         d["codes"].copy_(codes0)  # same previous codes every step (untimed)
-        flush.fill_(1)            # evict W, g and the codebook from L2 (untimed)
+        flush_l2()                # evict W, g and the codebook from L2 (untimed)
         a.record()
         step()
         b.record()
@@ -255,6 +263,28 @@ def run_ours(args):
             for s in ("select", "dequant"):
                 if stages[s]["gbs"]:
                     stages[s]["frac_of_measured_hbm"] = stages[s]["gbs"] / hbm
+        if tensor_engine:
+            # dense contraction on the tensor cores: algorithmic flops against the measured fp16/bf16 peak
+            tpeak = peaks.get("bf16_tflops")
+            roofline = {"kernel": "encode search (M=1, tcgen05)", "bound": "tensor", "achieved": achieved,
+                        "peak": tpeak, "unit": "TFLOP/s", "frac": achieved / tpeak,
+                        "peak_is": ("measured bf16 matmul (fp16 operands run at the same rate)"
+                                    if not peaks.get("fallback") else "fallback of the profiling recipe"),
+                        "flop_per_pair": FLOP_PER_PAIR, "avg_launch_ms": enc_avg_ms, "launches": enc_n,
+                        "executed_tflops": achieved * 4.0,  # operands are padded from depth 8 to depth 32
+                        "frac_of_fp32_alu_roofline": achieved / alu_peak,
+                        "frac_of_epilogue_bound": (pairs / (enc_avg_ms * 1e-3)) /
+                                                  (props.multi_processor_count * 128 * sm_max_mhz * 1e6),
+                        "epilogue_bound_is": "one accumulator read per pair: 128 lanes per SM per clock",
+                        "traffic": None}
+        else:
+            roofline = {"kernel": "encode search (M=1, fp32 pipe)" if M == 1 else "encode beam search (M=2)",
+                        "bound": "alu", "achieved": achieved, "peak": alu_peak, "unit": "TFLOP/s",
+                        "frac": achieved / alu_peak,
+                        "peak_is": f"{props.multi_processor_count} SMs x 128 FP32 lanes x 2 flop x "
+                                   f"{sm_max_mhz:.0f} MHz (derived; no measured FP32 peak)",
+                        "flop_per_pair": FLOP_PER_PAIR, "avg_launch_ms": enc_avg_ms, "launches": enc_n,
+                        "traffic": None}
         line = {
             "metric": METRIC, "value": world * k / (ms_per_step * 1e-3), "unit": UNIT,
             "pairs_per_s": world * pairs / (ms_per_step * 1e-3),
@@ -264,21 +294,16 @@ def run_ours(args):
             "config": {"workload": args.workload, "rows": rows, "cols": cols, "group_dim": 8, "groups": G,
                        "num_codebooks": M, "codebook_size": K, "codebook_dtype": "f16" if f16 else "f32",
                        "tau": tau, "k": k, "pairs_per_group": pairs_per_group,
+                       "search_engine": ("tensor" if tensor_engine else "fp32") if M == 1 else "beam",
                        "dequant_dtype": "f16" if args.dequant_fp16 else "f32",
-                       "l2": "flushed before every timed step (256 MiB write)",
+                       "l2": "flushed before every timed step (256 MiB written, then read)",
                        "parallelism": f"independent layers x{world}"},
             "e2e": {"value": world * k / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "what": "pinned host W, g, scale, codebook, codes -> device; select+encode+dequant; "
                             "idx and codes -> pinned host"},
             "gpu_launches": int(launches),
-            "roofline": {"kernel": "encode search (M=1)" if M == 1 else "encode beam search (M=2)",
-                         "bound": "alu", "achieved": achieved, "peak": alu_peak, "unit": "TFLOP/s",
-                         "frac": achieved / alu_peak,
-                         "peak_is": f"{props.multi_processor_count} SMs x 128 FP32 lanes x 2 flop x "
-                                    f"{sm_max_mhz:.0f} MHz (derived; no measured FP32 peak)",
-                         "flop_per_pair": FLOP_PER_PAIR, "avg_launch_ms": enc_avg_ms, "launches": enc_n,
-                         "traffic": None},
+            "roofline": roofline,
             "stages": stages,
             "clocks": clocks,
         }
@@ -422,6 +447,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--search", default="auto", choices=["auto", "fp32", "tensor"],
+                    help="engine of the single-codebook search")
     ap.add_argument("--dequant-fp16", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)

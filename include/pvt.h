@@ -197,6 +197,19 @@ const char* pvt_last_cuda_error(void);
 int pvt_version(void);
 
 /*
+ * Engine of the single-codebook search (no counterpart in the paper; both engines
+ * compute the same codes).  PVT_M1_AUTO, the default: tensor cores (tcgen05) for
+ * fp16 codebooks of at least 1024 codewords, the FP32 pipe otherwise.
+ * PVT_M1_FP32: always the FP32 pipe.  PVT_M1_TENSOR: tensor cores for every fp16
+ * codebook.  Process-wide; it also changes what pvt_workspace_bytes returns, so
+ * set it before sizing workspaces.  Other values are ignored.
+ */
+#define PVT_M1_AUTO 0
+#define PVT_M1_FP32 1
+#define PVT_M1_TENSOR 2
+void pvt_set_m1_search(int mode);
+
+/*
  * Benchmark instrumentation (no counterpart in the paper).  While enabled, every
  * call brackets its kernels with CUDA events on the caller's stream;
  * pvt_timing_read waits for the recorded events of one kernel class, returns

@@ -23,6 +23,7 @@ PVT_NOALLOC_MAX_GROUPS = 1 << 21
 PVT_DEV_BAD_INDEX, PVT_DEV_BAD_CODE, PVT_DEV_WAIT_EXPIRED, PVT_DEV_INTERNAL = 1, 2, 4, 8
 PVT_KERNEL_SELECT, PVT_KERNEL_ENCODE_MAIN, PVT_KERNEL_ENCODE_AUX, PVT_KERNEL_DEQUANT = 0, 1, 2, 3
 PVT_KERNEL_ENCODE_RESCORE = 4
+PVT_M1_AUTO, PVT_M1_FP32, PVT_M1_TENSOR = 0, 1, 2
 
 
 class pvt_layer(ctypes.Structure):
@@ -82,6 +83,8 @@ def lib():
         L.pvt_strerror.argtypes = [ctypes.c_int]
         L.pvt_last_cuda_error.restype = ctypes.c_char_p
         L.pvt_version.restype = ctypes.c_int
+        L.pvt_set_m1_search.restype = None
+        L.pvt_set_m1_search.argtypes = [ctypes.c_int]
         L.pvt_timing_enable.restype = None
         L.pvt_timing_enable.argtypes = [ctypes.c_int]
         L.pvt_launch_count.restype = ctypes.c_ulonglong
@@ -183,6 +186,11 @@ def pvt_status(ws: torch.Tensor, stream=None) -> int:
 
 def pvt_version() -> int:
     return int(lib().pvt_version())
+
+
+def pvt_set_m1_search(mode: int) -> None:
+    """Engine of the single-codebook search: PVT_M1_AUTO, PVT_M1_FP32 or PVT_M1_TENSOR."""
+    lib().pvt_set_m1_search(mode)
 
 
 def pvt_launch_count() -> int:

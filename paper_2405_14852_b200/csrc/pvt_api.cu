@@ -209,6 +209,10 @@ const char* pvt_last_cuda_error(void) { return cudaGetErrorString(g_last_cuda); 
 
 int pvt_version(void) { return 100; }
 
+void pvt_set_m1_search(int mode) {
+  if (mode == PVT_M1_AUTO || mode == PVT_M1_FP32 || mode == PVT_M1_TENSOR) set_m1_search(mode);
+}
+
 unsigned long long pvt_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 void pvt_timing_enable(int on) {

@@ -39,6 +39,8 @@
 // that can never win and are listed as "exceptions": the rescoring kernel always
 // evaluates them exactly.  Targets outside the range the scaling can serve
 // (non-finite, or max |t_i| >= 256) are rescored against the whole codebook.
+#include <atomic>
+
 #include "pvt_encode_m1.cuh"
 
 namespace pvt {
@@ -62,9 +64,19 @@ constexpr float kNegInf = -__builtin_huge_valf();
 
 }  // namespace
 
+namespace {
+std::atomic<int> g_m1_search{PVT_M1_AUTO};
+}
+
+void set_m1_search(int mode) { g_m1_search.store(mode, std::memory_order_relaxed); }
+
 bool encode_m1_use_tc(const pvt_layer& L, uint64_t k) {
   (void)k;
-  return L.num_codebooks == 1 && L.codebook_dtype == PVT_F16 && L.codebook_size >= 1024;
+  if (L.num_codebooks != 1 || L.codebook_dtype != PVT_F16) return false;  // the operand image is fp16
+  const int mode = g_m1_search.load(std::memory_order_relaxed);
+  if (mode == PVT_M1_FP32) return false;
+  if (mode == PVT_M1_TENSOR) return true;
+  return L.codebook_size >= 1024;  // below that the FP32 pipe with its larger target tiles is as fast
 }
 
 EncodeM1TcLayout encode_m1_tc_layout(uint32_t K, uint64_t k, int sm_count) {

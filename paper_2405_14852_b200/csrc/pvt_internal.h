@@ -95,6 +95,7 @@ struct EncodeM1TcLayout {
   uint32_t n_ctas;
 };
 bool encode_m1_use_tc(const pvt_layer& L, uint64_t k);
+void set_m1_search(int mode);
 EncodeM1TcLayout encode_m1_tc_layout(uint32_t K, uint64_t k, int sm_count);
 
 // launchers (each returns a cudaError_t) --------------------------------------

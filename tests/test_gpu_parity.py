@@ -1,6 +1,8 @@
 """Parity of the CUDA library (through the C ABI) with the CPU checker on the
 same seeded inputs: selection bit-exact, codes bit-exact outside the 1e-6 gap
 band (error within 1e-6 relative inside it), dequantised weights bit-exact."""
+import contextlib
+
 import numpy as np
 import pytest
 import torch
@@ -15,6 +17,16 @@ pytestmark = pytest.mark.gpu
 
 REL = 1e-6  # relative gap / error tolerance of the acceptance rule
 DEQ_ABS = 1e-6  # absolute tolerance on dequantised fp32 weights (bit-exact expected)
+
+
+@contextlib.contextmanager
+def search_engine(name):
+    """Run the single-codebook search on one engine (fp32 pipe / tensor cores)."""
+    B.pvt_set_m1_search({"fp32": B.PVT_M1_FP32, "tensor": B.PVT_M1_TENSOR, "auto": B.PVT_M1_AUTO}[name])
+    try:
+        yield
+    finally:
+        B.pvt_set_m1_search(B.PVT_M1_AUTO)
 
 
 def oracle_nearest(X, C):
@@ -182,12 +194,38 @@ def test_config_1_all_groups():
     (4096, True, 256, 512, 3000),
     (65536, True, 1024, 1024, 2500),  # full 16-bit codebook, codebook split over many CTAs
 ])
-def test_single_codebook_search(K, f16, rows, cols, k):
+@pytest.mark.parametrize("engine", ["fp32", "tensor"])
+def test_single_codebook_search(K, f16, rows, cols, k, engine):
     L = synth.make_layer(rows, cols, cfg=60, codebook_size=K, codebook_fp16=f16)
     rng = np.random.default_rng(61)
     idx = np.sort(rng.choice(L.num_groups, size=k, replace=False)).astype(np.uint32)
-    exact, band = check_encode(L, idx)
+    with search_engine(engine):
+        exact, band = check_encode(L, idx)
     assert exact >= k - max(4, k // 500)
+
+
+@pytest.mark.parametrize("engine", ["fp32", "tensor"])
+def test_single_codebook_search_codewords_and_targets_at_extreme_scales(engine):
+    """Codewords whose squared norm leaves the half-precision range, targets that
+    sit next to them, targets far outside the codebook's range and vanishing
+    targets: every one of them must still get its exact nearest codeword."""
+    L = synth.make_layer(96, 256, cfg=75, codebook_size=3000, codebook_fp16=True, row_max_scale=False)
+    cb = L.codebooks[0]
+    cb[5] = np.array([250, 250, 0, 0, 0, 0, 0, 0], np.float16)       # ||c||^2 / 2 = 62500
+    cb[2999] = np.array([-200, 0, 0, 180, 0, 0, 150, 0], np.float16)  # 47450 (representable) 
+    cb[77] = np.array([30000, -30000, 0, 0, 0, 0, 0, 1], np.float16)  # far beyond
+    G = L.num_groups
+    Wg = L.W.reshape(G, 8)
+    Wg[0:40] = cb[5].astype(np.float32) + np.random.default_rng(76).normal(0, 1.0, (40, 8)).astype(np.float32)
+    Wg[40:80] = cb[2999].astype(np.float32) * np.float32(0.98)
+    Wg[80:120] = cb[77].astype(np.float32) * np.float32(1.01)          # |t| far above 256
+    Wg[120:160] *= np.float32(1e4)                                     # |t| ~ 200 .. 800: partly out of range
+    Wg[160:200] *= np.float32(1e-9)                                    # vanishing targets
+    L.g[:] = 0
+    idx = np.arange(400, dtype=np.uint32)
+    with search_engine(engine):
+        exact, band = check_encode(L, idx)
+    assert exact >= 396
 
 
 def test_single_codebook_unsorted_indices_and_scaled_step():
