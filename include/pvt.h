@@ -123,14 +123,14 @@ int pvt_vstep_select(const pvt_layer* layer, uint64_t k, uint32_t* idx_out, void
  * completely at start-up, a component living inside a host application that
  * owns all device memory, or a thread that must not enter an allocator (a
  * cudaMalloc would also synchronise the device).  Such callers cannot supply the
- * ~4 bytes per group of workspace that pvt_vstep_select asks for.  Here the
+ * ~5 bytes per group of workspace that pvt_vstep_select asks for.  Here the
  * scratch is a fixed array inside the library image instead; the caller passes
  * only the layer, k and the outputs.
  *
  * Limits and rules
  *   - At most PVT_NOALLOC_MAX_GROUPS groups (2^21, e.g. one 4096 x 4096 layer);
  *     a larger layer is rejected with PVT_ETOOLARGE before anything is enqueued.
- *   - The array (about 8.03 MiB) is resident on every GPU that loads the library,
+ *   - The array (about 10.03 MiB) is resident on every GPU that loads the library,
  *     from load until the process exits, whether or not this call is ever used.
  *   - The first call on each device looks up the array's device address (a
  *     host-side runtime query; the device must be current).  Make that first

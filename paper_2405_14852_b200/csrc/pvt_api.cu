@@ -71,6 +71,8 @@ Timing& timing() {
 
 void record_cuda_error(cudaError_t e) { g_last_cuda = e; }
 
+int device_sm_count() { return sm_count(); }
+
 void count_launches(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
 
 void timing_begin(KernelId id, cudaStream_t stream) {
@@ -135,7 +137,7 @@ int pvt_vstep_select(const pvt_layer* layer, uint64_t k, uint32_t* idx_out, void
   if (!layer->g || !aligned16(layer->g) || !idx_out || !ws) return PVT_EINVAL;
   if (reinterpret_cast<uintptr_t>(ws) & (kWsAlign - 1)) return PVT_EINVAL;
   if (ws_bytes < select_layout(G).bytes) return PVT_EWORKSPACE;
-  const cudaError_t e = launch_select(*layer, G, k, idx_out, ws, static_cast<cudaStream_t>(cuda_stream));
+  const cudaError_t e = launch_select(*layer, G, k, idx_out, ws, sm_count(), static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? PVT_OK : fail_cuda(e);
 }
 

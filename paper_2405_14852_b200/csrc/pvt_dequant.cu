@@ -1,8 +1,8 @@
 // dequantize_weights (Algorithm 3, first line): W_hat = s_row * sum_m C_m[b_m] for
-// every weight group.  Streaming kernel, persistent grid: four groups (8 weights each) in flight per thread, codes
-// read coalesced, codewords gathered from the L2-resident codebook (small
-// codebooks are first copied to shared memory), 32 B (fp32) or 16 B (fp16) written
-// per group with 128-bit stores.
+// every weight group.  Streaming kernel, persistent grid: two threads per group (four
+// weights each), four half-groups in flight per thread, codes read coalesced,
+// codewords gathered from the L2-resident codebook (small codebooks are first copied
+// to shared memory), every store instruction of a warp covers whole 32-byte sectors.
 //
 // Arithmetic per element, binary32, each step rounded once: v = c1 (+ c2);
 // w = s * v; fp16 output = round-to-nearest-even of w.
@@ -14,34 +14,24 @@ namespace pvt {
 namespace {
 
 constexpr int kDqThreads = 256;
-constexpr int kDqUnroll = 4;          // groups in flight per thread
+constexpr int kDqUnroll = 4;          // half-groups in flight per thread
 constexpr int kDqSmemCodewords = 512;  // M*K up to this many codewords are staged in shared memory
 
-struct Vec8 {
-  float v[8];
-};
-
+// elements 4*half .. 4*half+3 of one codeword, widened to binary32
 template <bool CB_F16>
-__device__ __forceinline__ Vec8 load_codeword(const void* book, uint32_t code) {
-  Vec8 r;
+__device__ __forceinline__ float4 load_half_codeword(const void* book, uint32_t code, uint32_t half) {
   if (CB_F16) {
-    const uint4 raw = *(reinterpret_cast<const uint4*>(book) + code);
-    const __half2* h = reinterpret_cast<const __half2*>(&raw);
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const float2 f = __half22float2(h[i]);
-      r.v[2 * i] = f.x;
-      r.v[2 * i + 1] = f.y;
-    }
+    const uint2 raw = *(reinterpret_cast<const uint2*>(book) + 2 * (size_t)code + half);
+    const float2 lo = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
+    const float2 hi = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
+    return make_float4(lo.x, lo.y, hi.x, hi.y);
   } else {
-    const float4* p = reinterpret_cast<const float4*>(book) + 2 * (size_t)code;
-    const float4 a = p[0], b = p[1];
-    r.v[0] = a.x; r.v[1] = a.y; r.v[2] = a.z; r.v[3] = a.w;
-    r.v[4] = b.x; r.v[5] = b.y; r.v[6] = b.z; r.v[7] = b.w;
+    return *(reinterpret_cast<const float4*>(book) + 2 * (size_t)code + half);
   }
-  return r;
 }
 
+// Two threads per group, four elements each: a warp then writes 512 (fp32) or 256 (fp16)
+// contiguous bytes per store instruction, i.e. whole 32-byte sectors.
 template <int M, bool CB_F16, bool CODE_U16, bool OUT_F16, bool SMEM_BOOK>
 __global__ void __launch_bounds__(kDqThreads) dequant_kernel(const void* __restrict__ codebooks,
                                                               const void* __restrict__ codes,
@@ -59,29 +49,31 @@ __global__ void __launch_bounds__(kDqThreads) dequant_kernel(const void* __restr
     __syncthreads();
     book = sh_book;
   }
-  // kDqUnroll groups per thread and iteration, a block apart, all their loads issued
+  // kDqUnroll half-groups per thread and iteration, a block apart, all their loads issued
   // before the first use: the code -> codeword -> store chain of one group is two
-  // dependent memory round trips, so several groups must be in flight per thread
+  // dependent memory round trips, so several must be in flight per thread
+  const uint64_t H = 2 * G;
   const uint64_t stride = (uint64_t)gridDim.x * (kDqThreads * kDqUnroll);
-  for (uint64_t base = (uint64_t)blockIdx.x * (kDqThreads * kDqUnroll); base < G; base += stride) {
+  for (uint64_t base = (uint64_t)blockIdx.x * (kDqThreads * kDqUnroll); base < H; base += stride) {
     uint32_t b[kDqUnroll][M];
     bool bad = false;
 #pragma unroll
     for (int u = 0; u < kDqUnroll; ++u) {
-      const uint64_t j = base + (uint64_t)u * kDqThreads + threadIdx.x;
+      const uint64_t h = base + (uint64_t)u * kDqThreads + threadIdx.x;
+      const uint32_t j = (uint32_t)(h >> 1);
 #pragma unroll
       for (int m = 0; m < M; ++m) b[u][m] = 0;
-      if (j < G) {
+      if (h < H) {
         if (CODE_U16) {
-          const uint16_t* c = reinterpret_cast<const uint16_t*>(codes) + j * M;
+          const uint16_t* c = reinterpret_cast<const uint16_t*>(codes) + (size_t)j * M;
 #pragma unroll
-          for (int m = 0; m < M; ++m) b[u][m] = __ldcs(c + m);
+          for (int m = 0; m < M; ++m) b[u][m] = __ldg(c + m);
         } else if (M == 2) {
-          const uint16_t both = __ldcs(reinterpret_cast<const uint16_t*>(codes) + j);  // two adjacent bytes
+          const uint16_t both = __ldg(reinterpret_cast<const uint16_t*>(codes) + j);  // two adjacent bytes
           b[u][0] = both & 0xffu;
           b[u][M - 1] = both >> 8;
         } else {
-          b[u][0] = __ldcs(reinterpret_cast<const uint8_t*>(codes) + j);
+          b[u][0] = __ldg(reinterpret_cast<const uint8_t*>(codes) + j);
         }
 #pragma unroll
         for (int m = 0; m < M; ++m) {
@@ -93,34 +85,34 @@ __global__ void __launch_bounds__(kDqThreads) dequant_kernel(const void* __restr
       }
     }
     if (bad && status) atomicOr(status, PVT_DEV_BAD_CODE);
-    Vec8 v[kDqUnroll];
+    float4 v[kDqUnroll];
     float s[kDqUnroll];
 #pragma unroll
     for (int u = 0; u < kDqUnroll; ++u) {
-      const uint64_t j = base + (uint64_t)u * kDqThreads + threadIdx.x;
-      v[u] = load_codeword<CB_F16>(book, b[u][0]);
+      const uint64_t h = base + (uint64_t)u * kDqThreads + threadIdx.x;
+      const uint32_t j = (uint32_t)(h >> 1), half = (uint32_t)h & 1u;
+      v[u] = load_half_codeword<CB_F16>(book, b[u][0], half);
       if (M == 2) {
-        const Vec8 v2 = load_codeword<CB_F16>(book, K + b[u][M - 1]);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) v[u].v[i] = __fadd_rn(v[u].v[i], v2.v[i]);
+        const float4 v2 = load_half_codeword<CB_F16>(book, K + b[u][M - 1], half);
+        v[u].x = __fadd_rn(v[u].x, v2.x);
+        v[u].y = __fadd_rn(v[u].y, v2.y);
+        v[u].z = __fadd_rn(v[u].z, v2.z);
+        v[u].w = __fadd_rn(v[u].w, v2.w);
       }
-      s[u] = j < G ? __ldg(scale + j / gpr) : 0.0f;
+      s[u] = h < H ? __ldg(scale + j / gpr) : 0.0f;  // G < 2^32: a 32-bit division
     }
 #pragma unroll
     for (int u = 0; u < kDqUnroll; ++u) {
-      const uint64_t j = base + (uint64_t)u * kDqThreads + threadIdx.x;
-      if (j >= G) continue;
-#pragma unroll
-      for (int i = 0; i < 8; ++i) v[u].v[i] = __fmul_rn(s[u], v[u].v[i]);
+      const uint64_t h = base + (uint64_t)u * kDqThreads + threadIdx.x;
+      if (h >= H) continue;
+      const float4 w = make_float4(__fmul_rn(s[u], v[u].x), __fmul_rn(s[u], v[u].y), __fmul_rn(s[u], v[u].z),
+                                   __fmul_rn(s[u], v[u].w));
       if (OUT_F16) {
-        __half2 h[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) h[i] = __floats2half2_rn(v[u].v[2 * i], v[u].v[2 * i + 1]);
-        __stcs(reinterpret_cast<uint4*>(W_hat) + j, *reinterpret_cast<const uint4*>(h));
+        const __half2 lo = __floats2half2_rn(w.x, w.y), hi = __floats2half2_rn(w.z, w.w);
+        __stcs(reinterpret_cast<uint2*>(W_hat) + h,
+               make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi)));
       } else {
-        float4* o = reinterpret_cast<float4*>(W_hat) + 2 * j;
-        __stcs(o, make_float4(v[u].v[0], v[u].v[1], v[u].v[2], v[u].v[3]));
-        __stcs(o + 1, make_float4(v[u].v[4], v[u].v[5], v[u].v[6], v[u].v[7]));
+        __stcs(reinterpret_cast<float4*>(W_hat) + h, w);
       }
     }
   }
@@ -139,7 +131,7 @@ cudaError_t launch_t(const pvt_layer& L, uint64_t G, void* W_hat, uint32_t* stat
   if (oe != cudaSuccess) return oe;
   if (per_sm < 1) per_sm = 1;
   const uint64_t per_block = (uint64_t)kDqThreads * kDqUnroll;
-  const uint64_t want = (G + per_block - 1) / per_block;
+  const uint64_t want = (2 * G + per_block - 1) / per_block;
   const uint64_t cap = (uint64_t)sm_count * (uint64_t)per_sm;
   const unsigned blocks = (unsigned)(want < cap ? want : cap);
   const uint32_t gpr = (uint32_t)(L.cols / kGroupDim);

@@ -120,7 +120,7 @@ __global__ void expand_codebook_kernel(const void* __restrict__ book, uint32_t K
   // max ||c||^2 over the codebook (non-negative floats order like their bit patterns)
   uint32_t bits = __float_as_uint(n2);
   bits = __reduce_max_sync(0xffffffffu, bits);
-  if ((threadIdx.x & 31) == 0 && bits) atomicMax(n2max_bits, bits);
+  if ((threadIdx.x & 31) == 0 && bits > __ldcg(n2max_bits)) atomicMax(n2max_bits, bits);
 }
 
 __device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
@@ -344,22 +344,26 @@ __device__ __forceinline__ void load_codeword(const void* book, uint32_t kappa, 
   }
 }
 
-// One warp per target.
+// One warp per target.  Memory round trips are kept to three: (index, global minimum,
+// margin, one record per lane) -> (W, g, scale) -> codewords.
 template <bool CB_F16>
 __global__ void __launch_bounds__(256) rescore_m1_kernel(const EncM1Params p) {
   const uint32_t sub_cw = p.sub_cw;
   const int lane = threadIdx.x & 31;
   const uint64_t n = (uint64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (n >= p.k) return;
+  const uint32_t tile = (uint32_t)(n / p.tile), s = (uint32_t)(n % p.tile);
   const uint32_t j = __ldg(p.idx + n);
+  const float limit = unord(p.gbest[n]) + p.margin[n];
+  uint4 raw = make_uint4(0x7f800000u, 0, 0, 0);  // best = +inf: never within the limit
+  if ((uint32_t)lane < p.n_slices)
+    raw = __ldg(reinterpret_cast<const uint4*>(&p.rec[((size_t)tile * p.n_slices + lane) * p.tile + s]));
   if (j >= p.G) {
     if (lane == 0) atomicOr(p.status, PVT_DEV_BAD_INDEX);
     return;
   }
   float t[8];
   form_target(p, j, t);
-  const float limit = unord(p.gbest[n]) + p.margin[n];
-  const uint32_t tile = (uint32_t)(n / p.tile), s = (uint32_t)(n % p.tile);
   const uint32_t subs_per_unit = p.unit_cw / sub_cw;
   double best_d = __longlong_as_double(0x7ff0000000000000ll);
   uint32_t best_code = 0xffffffffu;
@@ -384,17 +388,22 @@ __global__ void __launch_bounds__(256) rescore_m1_kernel(const EncM1Params p) {
     }
   };
 
-  for (uint32_t sl = 0; sl < p.n_slices; ++sl) {
-    const uint4 raw = __ldg(reinterpret_cast<const uint4*>(&p.rec[((size_t)tile * p.n_slices + sl) * p.tile + s]));
-    const CandRecord r = *reinterpret_cast<const CandRecord*>(&raw);
-    if (!(r.best <= limit)) continue;
-    if (r.cnt == kCandOverflow) {
+  // slices whose minimum lies within the margin of the global minimum (kMaxSlices <= 32: one record per lane)
+  uint32_t live = __ballot_sync(0xffffffffu, __uint_as_float(raw.x) <= limit);
+  while (live) {
+    const int sl = __ffs(live) - 1;
+    live &= live - 1;
+    const uint32_t s01 = __shfl_sync(0xffffffffu, raw.y, sl), s23 = __shfl_sync(0xffffffffu, raw.z, sl);
+    const uint32_t cnt = __shfl_sync(0xffffffffu, raw.w, sl) & 0xffffu;
+    if (cnt == kCandOverflow) {
       uint32_t u_lo, u_hi;
-      slice_units(p, sl, &u_lo, &u_hi);
+      slice_units(p, (uint32_t)sl, &u_lo, &u_hi);
       for (uint32_t sub = u_lo * subs_per_unit; sub < u_hi * subs_per_unit; ++sub) visit(sub);
     } else {
-      const uint32_t cnt = r.cnt < (uint16_t)kListLen ? r.cnt : (uint32_t)kListLen;
-      for (uint32_t e = 0; e < cnt; ++e) visit(r.sub[e]);
+      if (cnt > 0) visit(s01 & 0xffffu);
+      if (cnt > 1) visit(s01 >> 16);
+      if (cnt > 2) visit(s23 & 0xffffu);
+      if (cnt > 3) visit(s23 >> 16);
     }
   }
   if (p.exc_count) {  // codewords whose fast score is not trustworthy: always evaluated

@@ -170,7 +170,7 @@ __global__ void __launch_bounds__(256) tc_prep_kernel(const uint4* __restrict__ 
     *reinterpret_cast<uint4*>(row + 384) = make_uint4(0, 0, 0, 0);
   }
   n2bits = __reduce_max_sync(0xffffffffu, n2bits);
-  if ((threadIdx.x & 31) == 0 && n2bits) atomicMax(&stats->n2max_bits, n2bits);
+  if ((threadIdx.x & 31) == 0 && n2bits > __ldcg(&stats->n2max_bits)) atomicMax(&stats->n2max_bits, n2bits);
 }
 
 // ---- tcgen05 wrappers -----------------------------------------------------------

@@ -33,6 +33,7 @@ struct SelectState {        // lives in the header at byte 64
   uint32_t need_eq;         // how many groups with key == threshold are taken (lowest indices)
   uint64_t k_left;          // groups still to be taken from the current bucket
   uint32_t done[4];         // block-completion counters of the passes
+  uint32_t cand_count;      // keys found inside the threshold bucket of the first digit
 };
 constexpr size_t kSelStateOffset = 64;
 
@@ -40,6 +41,8 @@ struct SelectLayout {
   size_t hist_off;   // u32 [2048 + 2048 + 512]
   size_t keys_off;   // u32 [G]
   size_t tiles_off;  // u32 [2 * ntiles]: (greater, equal) counts, later exclusive offsets
+  size_t cand_off;   // u32 [cand_cap]: keys of the threshold bucket, any order
+  uint32_t cand_cap;
   size_t bytes;      // end of the region (from the workspace base)
   uint32_t ntiles;
 };
@@ -99,7 +102,7 @@ void set_m1_search(int mode);
 EncodeM1TcLayout encode_m1_tc_layout(uint32_t K, uint64_t k, int sm_count);
 
 // launchers (each returns a cudaError_t) --------------------------------------
-cudaError_t launch_select(const pvt_layer& L, uint64_t G, uint64_t k, uint32_t* idx_out, void* ws,
+cudaError_t launch_select(const pvt_layer& L, uint64_t G, uint64_t k, uint32_t* idx_out, void* ws, int sm_count,
                           cudaStream_t stream);
 cudaError_t launch_encode_m1(const pvt_layer& L, uint64_t G, const uint32_t* idx, uint64_t k, float* err_out,
                              void* ws, int sm_count, cudaStream_t stream);
@@ -119,6 +122,9 @@ void timing_end(KernelId id, cudaStream_t stream);
 
 // remembers the CUDA error behind a PVT_ECUDA return for pvt_last_cuda_error (per host thread)
 void record_cuda_error(cudaError_t e);
+
+// multiprocessors of the current device
+int device_sm_count();
 
 // number of kernels launched by this process through the library (a claim the benchmark reports)
 void count_launches(int n);

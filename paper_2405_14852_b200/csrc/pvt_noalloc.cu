@@ -21,9 +21,11 @@ namespace {
 
 // Largest layer the built-in scratch serves: 2^21 groups of 8 weights, e.g. a
 // 4096 x 4096 matrix.  Layout needs: 256 B header + 18 KiB histograms + 4 B per
-// group + 8 B per tile of 4096 groups, each part rounded up to 256 B.
+// group (keys) + 8 B per tile of 4096 groups + 1 B per group (candidate list of a
+// quarter of the groups), each part rounded up to 256 B.
 constexpr uint64_t kNoAllocMaxGroups = 1ull << 21;
-constexpr size_t kNoAllocScratchBytes = 256 + 18432 + 4 * kNoAllocMaxGroups + 8 * (kNoAllocMaxGroups / kSelTile) + 1024;
+constexpr size_t kNoAllocScratchBytes =
+    256 + 18432 + 4 * kNoAllocMaxGroups + 8 * (kNoAllocMaxGroups / kSelTile) + kNoAllocMaxGroups + 1280;
 
 // File-scope device array.  In host code this name is only a handle for the
 // runtime's symbol table, not a device address: the address is looked up with
@@ -76,7 +78,7 @@ extern "C" int pvt_vstep_select_noalloc(const pvt_layer* layer, uint64_t k, uint
   // the array keeps whatever the previous call left: the status word must start at zero
   // (launch_select clears the selection state and the histograms itself)
   if (e == cudaSuccess) e = cudaMemsetAsync(ws, 0, sizeof(uint32_t), stream);
-  if (e == cudaSuccess) e = launch_select(*layer, G, k, idx_out, ws, stream);
+  if (e == cudaSuccess) e = launch_select(*layer, G, k, idx_out, ws, device_sm_count(), stream);
   if (e == cudaSuccess && status_out)
     e = cudaMemcpyAsync(status_out, ws, sizeof(uint32_t), cudaMemcpyDeviceToDevice, stream);
   if (e != cudaSuccess) {

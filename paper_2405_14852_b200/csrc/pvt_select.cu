@@ -4,10 +4,12 @@
 // threshold resolved towards the lowest group index, result in ascending order.
 //
 // Passes (all on one stream, no host round trip, no inter-block waiting):
-//   1. norm_hist:   read g once (32 B per group), write the key of every group,
-//                   histogram key bits [30:20]
-//   2. hist_mid:    histogram bits [19:9] of the keys inside the threshold bucket
-//   3. hist_low:    histogram bits [8:0] of the keys that match both digits
+//   1. norm_hist:   persistent grid; read g once (32 B per group), write the key of
+//                   every group, histogram key bits [30:20]
+//   2. refine_mid:  read the keys; those inside the threshold bucket are
+//                   histogrammed on bits [19:9] and copied to a compact candidate
+//                   list (usually a few per cent of the groups)
+//   3. refine_low:  histogram bits [8:0] of the candidates that match both digits
 //   4. tile_count:  per tile of 4096 groups: how many keys > threshold, == threshold
 //   5. scatter:     ordered compaction: position = (#greater before) +
 //                   min(#equal before, number of ties to take)
@@ -20,29 +22,24 @@ namespace pvt {
 SelectLayout select_layout(uint64_t G) {
   SelectLayout s;
   s.ntiles = (uint32_t)((G + kSelTile - 1) / kSelTile);
+  // candidates: a quarter of the groups is far more than a threshold bucket of real gradients holds; when
+  // it is not enough (many equal norms) the low pass reads the keys instead
+  uint64_t cap = G / 4;
+  if (cap < 65536) cap = 65536;
+  if (cap > G) cap = G;
+  s.cand_cap = (uint32_t)cap;
   s.hist_off = kWsHeaderBytes;
   s.keys_off = align_up(s.hist_off + sizeof(uint32_t) * (kSelBins0 + kSelBins1 + kSelBins2), kWsAlign);
   s.tiles_off = align_up(s.keys_off + sizeof(uint32_t) * G, kWsAlign);
-  s.bytes = align_up(s.tiles_off + sizeof(uint32_t) * 2 * (size_t)s.ntiles, kWsAlign);
+  s.cand_off = align_up(s.tiles_off + sizeof(uint32_t) * 2 * (size_t)s.ntiles, kWsAlign);
+  s.bytes = align_up(s.cand_off + sizeof(uint32_t) * (size_t)s.cand_cap, kWsAlign);
   return s;
 }
 
 namespace {
 
-// n_j = ||eta * g_j||^2 in binary32: u = eta*g_i rounded once, acc = fma(u, u, acc)
+// Keys: n_j = ||eta * g_j||^2 in binary32: u = eta*g_i rounded once, acc = fma(u, u, acc)
 // in index order from 0.  Non-negative, so the bit pattern orders like the value.
-__device__ __forceinline__ uint32_t group_key(const float4 a, const float4 b, float eta) {
-  float acc = 0.0f, u;
-  u = __fmul_rn(eta, a.x); acc = __fmaf_rn(u, u, acc);
-  u = __fmul_rn(eta, a.y); acc = __fmaf_rn(u, u, acc);
-  u = __fmul_rn(eta, a.z); acc = __fmaf_rn(u, u, acc);
-  u = __fmul_rn(eta, a.w); acc = __fmaf_rn(u, u, acc);
-  u = __fmul_rn(eta, b.x); acc = __fmaf_rn(u, u, acc);
-  u = __fmul_rn(eta, b.y); acc = __fmaf_rn(u, u, acc);
-  u = __fmul_rn(eta, b.z); acc = __fmaf_rn(u, u, acc);
-  u = __fmul_rn(eta, b.w); acc = __fmaf_rn(u, u, acc);
-  return __float_as_uint(acc);
-}
 
 // Block-wide: true in every thread of the block that took the last ticket.
 __device__ __forceinline__ bool last_block_done(uint32_t* counter) {
@@ -102,14 +99,13 @@ __device__ void find_digit(const uint32_t* hist, uint64_t k_left, uint32_t* digi
   }
 }
 
-__device__ __forceinline__ void hist_add_matched(uint32_t* sh_hist, uint32_t bin, bool valid) {
-  // one shared-memory atomic per distinct bin of the warp: synthetic gradients put
-  // most keys of a warp into a handful of bins
-  const uint32_t b = valid ? bin : 0xffffffffu;
-  const uint32_t peers = __match_any_sync(0xffffffffu, b);
-  if (valid && (threadIdx.x & 31) == (uint32_t)(__ffs(peers) - 1)) atomicAdd(&sh_hist[bin], (uint32_t)__popc(peers));
-}
+constexpr int kNormPer = 4;                              // 16-byte loads per thread and iteration of the norm pass
+constexpr int kNormTile = kSelThreads * kNormPer / 2;    // 512 groups: two threads per group
 
+// Two adjacent lanes share a group: the even lane holds elements 0..3, the odd lane 4..7,
+// so a warp reads 512 contiguous bytes per load instruction.  The sum is a single chain
+// in index order: the even lane runs its four steps from 0, hands the partial sum to the
+// odd lane, which runs the remaining four.
 __global__ void __launch_bounds__(kSelThreads) norm_hist_kernel(const float* __restrict__ g, uint64_t G, float eta,
                                                                  uint64_t k, uint32_t* __restrict__ keys,
                                                                  uint32_t* __restrict__ hist0, SelectState* st) {
@@ -117,20 +113,37 @@ __global__ void __launch_bounds__(kSelThreads) norm_hist_kernel(const float* __r
   __shared__ uint64_t sh_scan[kSelThreads / 32];
   for (int b = threadIdx.x; b < kSelBins0; b += kSelThreads) sh_hist[b] = 0;
   __syncthreads();
-  const uint64_t j0 = (uint64_t)blockIdx.x * kSelTile;
   const float4* g4 = reinterpret_cast<const float4*>(g);
-  constexpr int PER = kSelTile / kSelThreads;
-#pragma unroll 4
-  for (int i = 0; i < PER; ++i) {
-    const uint64_t j = j0 + (uint64_t)i * kSelThreads + threadIdx.x;
-    const bool valid = j < G;
-    uint32_t key = 0;
-    if (valid) {
-      const float4 a = __ldcs(g4 + 2 * j), b = __ldcs(g4 + 2 * j + 1);
-      key = group_key(a, b, eta);
-      keys[j] = key;
+  const uint64_t F = 2 * G;  // 16-byte pieces
+  const uint32_t n_tiles = (uint32_t)((G + kNormTile - 1) / kNormTile);
+  const bool odd = threadIdx.x & 1;
+  for (uint32_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+    const uint64_t f0 = (uint64_t)tile * (2 * kNormTile) + threadIdx.x;
+    float4 a[kNormPer];
+#pragma unroll
+    for (int i = 0; i < kNormPer; ++i) {  // all loads of the iteration first
+      const uint64_t f = f0 + (uint64_t)i * kSelThreads;
+      a[i] = f < F ? __ldcs(g4 + f) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
-    hist_add_matched(sh_hist, key >> 20, valid);
+#pragma unroll
+    for (int i = 0; i < kNormPer; ++i) {
+      const uint64_t f = f0 + (uint64_t)i * kSelThreads;
+      float u, lo = 0.0f;
+      u = __fmul_rn(eta, a[i].x); lo = __fmaf_rn(u, u, lo);
+      u = __fmul_rn(eta, a[i].y); lo = __fmaf_rn(u, u, lo);
+      u = __fmul_rn(eta, a[i].z); lo = __fmaf_rn(u, u, lo);
+      u = __fmul_rn(eta, a[i].w); lo = __fmaf_rn(u, u, lo);
+      float acc = __shfl_up_sync(0xffffffffu, lo, 1);  // odd lanes: the sum over elements 0..3 of their group
+      u = __fmul_rn(eta, a[i].x); acc = __fmaf_rn(u, u, acc);
+      u = __fmul_rn(eta, a[i].y); acc = __fmaf_rn(u, u, acc);
+      u = __fmul_rn(eta, a[i].z); acc = __fmaf_rn(u, u, acc);
+      u = __fmul_rn(eta, a[i].w); acc = __fmaf_rn(u, u, acc);
+      if (odd && f < F) {
+        const uint32_t key = __float_as_uint(acc);
+        keys[f >> 1] = key;
+        atomicAdd(&sh_hist[key >> 20], 1u);
+      }
+    }
   }
   __syncthreads();
   for (int b = threadIdx.x; b < kSelBins0; b += kSelThreads)
@@ -138,48 +151,116 @@ __global__ void __launch_bounds__(kSelThreads) norm_hist_kernel(const float* __r
   if (last_block_done(&st->done[0])) find_digit<kSelBins0>(hist0, k, &st->digit0, &st->k_left, sh_scan);
 }
 
-// PASS 1: bins = key bits [19:9] of keys whose bits [30:20] equal digit0.
-// PASS 2: bins = key bits [8:0] of keys whose bits [30:9] equal (digit0, digit1).
-template <int PASS>
-__global__ void __launch_bounds__(kSelThreads) hist_refine_kernel(const uint32_t* __restrict__ keys, uint64_t G,
-                                                                   uint32_t* __restrict__ hist, SelectState* st) {
-  constexpr int NBINS = PASS == 1 ? kSelBins1 : kSelBins2;
-  __shared__ uint32_t sh_hist[NBINS];
+// Keys whose bits [30:20] equal digit0: histogram of bits [19:9], and a compact copy
+// (order irrelevant) for the last refinement.  Bucket members are first collected in
+// shared memory; a block reserves room in the global list with one atomic per flush.
+constexpr int kMidStage = 2048;  // bucket members a block collects before it flushes
+
+__global__ void __launch_bounds__(kSelThreads) refine_mid_kernel(const uint32_t* __restrict__ keys, uint64_t G,
+                                                                  uint32_t* __restrict__ hist1,
+                                                                  uint32_t* __restrict__ cand, uint32_t cand_cap,
+                                                                  SelectState* st) {
+  __shared__ uint32_t sh_hist[kSelBins1];
   __shared__ uint64_t sh_scan[kSelThreads / 32];
-  for (int b = threadIdx.x; b < NBINS; b += kSelThreads) sh_hist[b] = 0;
+  __shared__ uint32_t sh_stage[kMidStage + 8 * kSelThreads];  // room for one more iteration after the check
+  __shared__ uint32_t sh_n, sh_base;
+  for (int b = threadIdx.x; b < kSelBins1; b += kSelThreads) sh_hist[b] = 0;
+  if (threadIdx.x == 0) sh_n = 0;
   __syncthreads();
-  const uint32_t prefix = PASS == 1 ? st->digit0 : ((st->digit0 << 11) | st->digit1);
-  const uint64_t j0 = (uint64_t)blockIdx.x * kSelTile;
-  constexpr int PER = kSelTile / kSelThreads;
-#pragma unroll 4
-  for (int i = 0; i < PER; ++i) {
-    const uint64_t j = j0 + (uint64_t)i * kSelThreads + threadIdx.x;
-    if (j < G) {
-      const uint32_t key = keys[j];
-      if (PASS == 1) {
-        if ((key >> 20) == prefix) atomicAdd(&sh_hist[(key >> 9) & 0x7ffu], 1u);
-      } else {
-        if ((key >> 9) == prefix) atomicAdd(&sh_hist[key & 0x1ffu], 1u);
+  const uint32_t prefix = st->digit0;
+  const uint64_t n_quads = (G + 3) / 4;
+  const uint64_t stride = (uint64_t)gridDim.x * kSelThreads;
+
+  auto flush = [&]() {  // called by the whole block
+    __syncthreads();
+    const uint32_t n = sh_n;
+    if (threadIdx.x == 0 && n) sh_base = atomicAdd(&st->cand_count, n);
+    __syncthreads();
+    const uint32_t base = sh_base;
+    for (uint32_t i = threadIdx.x; i < n; i += kSelThreads)
+      if (base + i < cand_cap) cand[base + i] = sh_stage[i];
+    __syncthreads();
+    if (threadIdx.x == 0) sh_n = 0;
+    __syncthreads();
+  };
+
+  for (uint64_t q0 = (uint64_t)blockIdx.x * kSelThreads; q0 < n_quads; q0 += 2 * stride) {
+    // two independent 16-byte loads per thread and iteration
+    uint32_t key[8];
+    uint32_t have[2] = {0, 0};
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const uint64_t q = q0 + (uint64_t)h * stride + threadIdx.x;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) key[4 * h + i] = 0;
+      if (q < n_quads) {
+        if (4 * q + 4 <= G) {
+          const uint4 v = *reinterpret_cast<const uint4*>(keys + 4 * q);
+          key[4 * h] = v.x; key[4 * h + 1] = v.y; key[4 * h + 2] = v.z; key[4 * h + 3] = v.w;
+          have[h] = 4;
+        } else {
+          have[h] = (uint32_t)(G - 4 * q);
+          for (uint32_t i = 0; i < have[h]; ++i) key[4 * h + i] = keys[4 * q + i];
+        }
       }
     }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        if ((uint32_t)i < have[h] && (key[4 * h + i] >> 20) == prefix) {
+          atomicAdd(&sh_hist[(key[4 * h + i] >> 9) & 0x7ffu], 1u);
+          sh_stage[atomicAdd(&sh_n, 1u)] = key[4 * h + i];
+        }
+      }
+    }
+    __syncthreads();
+    const uint32_t collected = sh_n;  // the same value in every thread
+    __syncthreads();                  // nobody adds to it again before everybody has read it
+    if (collected >= (uint32_t)kMidStage) flush();
   }
-  __syncthreads();
-  for (int b = threadIdx.x; b < NBINS; b += kSelThreads)
-    if (sh_hist[b]) atomicAdd(&hist[b], sh_hist[b]);
-  if (last_block_done(&st->done[PASS])) {
+  flush();
+  for (int b = threadIdx.x; b < kSelBins1; b += kSelThreads)
+    if (sh_hist[b]) atomicAdd(&hist1[b], sh_hist[b]);
+  if (last_block_done(&st->done[1])) {
     const uint64_t k_left = st->k_left;
     __syncthreads();
-    if (PASS == 1) {
-      find_digit<NBINS>(hist, k_left, &st->digit1, &st->k_left, sh_scan);
-    } else {
-      __shared__ uint32_t d2;
-      __shared__ uint64_t kn;
-      find_digit<NBINS>(hist, k_left, &d2, &kn, sh_scan);
-      __syncthreads();
-      if (threadIdx.x == 0) {
-        st->threshold = (st->digit0 << 20) | (st->digit1 << 9) | d2;
-        st->need_eq = (uint32_t)kn;
-      }
+    find_digit<kSelBins1>(hist1, k_left, &st->digit1, &st->k_left, sh_scan);
+  }
+}
+
+// Bits [8:0] of the candidates that match (digit0, digit1); reads the candidate list, or
+// all keys if the list did not hold every bucket member.
+__global__ void __launch_bounds__(kSelThreads) refine_low_kernel(const uint32_t* __restrict__ keys, uint64_t G,
+                                                                  const uint32_t* __restrict__ cand,
+                                                                  uint32_t cand_cap, uint32_t* __restrict__ hist2,
+                                                                  SelectState* st) {
+  __shared__ uint32_t sh_hist[kSelBins2];
+  __shared__ uint64_t sh_scan[kSelThreads / 32];
+  for (int b = threadIdx.x; b < kSelBins2; b += kSelThreads) sh_hist[b] = 0;
+  __syncthreads();
+  const uint32_t prefix = (st->digit0 << 11) | st->digit1;
+  const uint32_t n_cand = st->cand_count;
+  const bool listed = n_cand <= cand_cap;
+  const uint32_t* src = listed ? cand : keys;
+  const uint64_t n = listed ? (uint64_t)n_cand : G;
+  for (uint64_t i = (uint64_t)blockIdx.x * kSelThreads + threadIdx.x; i < n; i += (uint64_t)gridDim.x * kSelThreads) {
+    const uint32_t key = src[i];
+    if ((key >> 9) == prefix) atomicAdd(&sh_hist[key & 0x1ffu], 1u);
+  }
+  __syncthreads();
+  for (int b = threadIdx.x; b < kSelBins2; b += kSelThreads)
+    if (sh_hist[b]) atomicAdd(&hist2[b], sh_hist[b]);
+  if (last_block_done(&st->done[2])) {
+    const uint64_t k_left = st->k_left;
+    __shared__ uint32_t d2;
+    __shared__ uint64_t kn;
+    __syncthreads();
+    find_digit<kSelBins2>(hist2, k_left, &d2, &kn, sh_scan);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      st->threshold = (st->digit0 << 20) | (st->digit1 << 9) | d2;
+      st->need_eq = (uint32_t)kn;
     }
   }
 }
@@ -193,12 +274,20 @@ __global__ void __launch_bounds__(kSelThreads) tile_count_kernel(const uint32_t*
   __syncthreads();
   const uint32_t T = st->threshold;
   const uint64_t j0 = (uint64_t)blockIdx.x * kSelTile;
-  constexpr int PER = kSelTile / kSelThreads;
+  constexpr int QUADS = kSelTile / (4 * kSelThreads);  // 16-byte loads per thread, all issued before use
   uint32_t gt = 0, eq = 0;
-#pragma unroll 4
-  for (int i = 0; i < PER; ++i) {
-    const uint64_t j = j0 + (uint64_t)i * kSelThreads + threadIdx.x;
-    if (j < G) {
+  if (j0 + kSelTile <= G) {
+    uint4 v[QUADS];
+#pragma unroll
+    for (int i = 0; i < QUADS; ++i)
+      v[i] = *reinterpret_cast<const uint4*>(keys + j0 + 4 * ((uint64_t)i * kSelThreads + threadIdx.x));
+#pragma unroll
+    for (int i = 0; i < QUADS; ++i) {
+      gt += (v[i].x > T) + (v[i].y > T) + (v[i].z > T) + (v[i].w > T);
+      eq += (v[i].x == T) + (v[i].y == T) + (v[i].z == T) + (v[i].w == T);
+    }
+  } else {
+    for (uint64_t j = j0 + threadIdx.x; j < G; j += kSelThreads) {
       const uint32_t key = keys[j];
       gt += key > T;
       eq += key == T;
@@ -296,7 +385,7 @@ __global__ void iota_kernel(uint32_t* idx_out, uint64_t k) {
 
 }  // namespace
 
-cudaError_t launch_select(const pvt_layer& L, uint64_t G, uint64_t k, uint32_t* idx_out, void* ws,
+cudaError_t launch_select(const pvt_layer& L, uint64_t G, uint64_t k, uint32_t* idx_out, void* ws, int sm_count,
                           cudaStream_t stream) {
   timing_begin(kKernSelect, stream);
   cudaError_t err = cudaSuccess;
@@ -316,13 +405,30 @@ cudaError_t launch_select(const pvt_layer& L, uint64_t G, uint64_t k, uint32_t* 
   uint32_t* hist2 = hist1 + kSelBins1;
   uint32_t* keys = reinterpret_cast<uint32_t*>(base + lay.keys_off);
   uint32_t* tiles = reinterpret_cast<uint32_t*>(base + lay.tiles_off);
-  if ((err = cudaMemsetAsync(st, 0, sizeof(SelectState), stream)) != cudaSuccess) return err;
-  if ((err = cudaMemsetAsync(hist0, 0, sizeof(uint32_t) * (kSelBins0 + kSelBins1 + kSelBins2), stream)) !=
+  // selection state (header, from byte 64) and the three histograms are adjacent: one clear
+  static_assert(kSelStateOffset + sizeof(SelectState) <= kWsHeaderBytes, "selection state must fit the header");
+  if ((err = cudaMemsetAsync(st, 0, (kWsHeaderBytes - kSelStateOffset) +
+                                        sizeof(uint32_t) * (kSelBins0 + kSelBins1 + kSelBins2), stream)) !=
       cudaSuccess)
     return err;
-  norm_hist_kernel<<<lay.ntiles, kSelThreads, 0, stream>>>(L.g, G, L.eta, k, keys, hist0, st);
-  hist_refine_kernel<1><<<lay.ntiles, kSelThreads, 0, stream>>>(keys, G, hist1, st);
-  hist_refine_kernel<2><<<lay.ntiles, kSelThreads, 0, stream>>>(keys, G, hist2, st);
+  uint32_t* cand = reinterpret_cast<uint32_t*>(base + lay.cand_off);
+  // persistent grids: exactly the blocks that are resident at once
+  int norm_per_sm = 0, mid_per_sm = 0;
+  if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&norm_per_sm, norm_hist_kernel, kSelThreads, 0)) !=
+          cudaSuccess ||
+      (err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&mid_per_sm, refine_mid_kernel, kSelThreads, 0)) !=
+          cudaSuccess)
+    return err;
+  const uint64_t norm_tiles = (G + kNormTile - 1) / kNormTile;
+  const uint64_t norm_res = (uint64_t)sm_count * (uint64_t)(norm_per_sm > 0 ? norm_per_sm : 1);
+  const unsigned norm_grid = (unsigned)(norm_tiles < norm_res ? norm_tiles : norm_res);
+  const uint64_t quad_blocks = ((G + 3) / 4 + 2 * kSelThreads - 1) / (2 * kSelThreads);
+  const uint64_t mid_res = (uint64_t)sm_count * (uint64_t)(mid_per_sm > 0 ? mid_per_sm : 1);
+  const unsigned mid_grid = (unsigned)(quad_blocks < mid_res ? quad_blocks : mid_res);
+  norm_hist_kernel<<<norm_grid, kSelThreads, 0, stream>>>(L.g, G, L.eta, k, keys, hist0, st);
+  refine_mid_kernel<<<mid_grid, kSelThreads, 0, stream>>>(keys, G, hist1, cand, lay.cand_cap, st);
+  const unsigned low_grid = (unsigned)(lay.cand_cap / 8192 < (uint32_t)sm_count ? lay.cand_cap / 8192 + 1 : sm_count);
+  refine_low_kernel<<<low_grid, kSelThreads, 0, stream>>>(keys, G, cand, lay.cand_cap, hist2, st);
   tile_count_kernel<<<lay.ntiles, kSelThreads, 0, stream>>>(keys, G, tiles, lay.ntiles, k, st, status);
   scatter_kernel<<<lay.ntiles, kSelThreads, 0, stream>>>(keys, G, tiles, st, k, idx_out);
   err = cudaGetLastError();
