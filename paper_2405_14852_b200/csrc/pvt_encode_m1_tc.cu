@@ -30,10 +30,11 @@
 // CTA = 256 targets (two 128-row A blocks) x a slice of the codebook, one CTA per
 // SM, persistent over (tile, slice) units.  Warps 0-7: own one target per thread,
 // build A, run the epilogue (warp w reads tensor-memory lanes 32 (w % 4) .. of the
-// accumulator of A block w / 4).  Warp 8: bulk-copy producer.  Warp 9: allocates
-// tensor memory and issues the MMAs (one thread).  Tensor memory: 2 buffers x 2
-// accumulators x 128 columns = 512 columns, so the MMAs of step i+1 overlap the
-// epilogue of step i.
+// accumulator of A block w / 4).  Warp 8: bulk-copy producer.  Warps 9 and 10: one
+// thread each issues the MMAs of one A block (issuing is the scarce resource: about
+// 60 cycles per instruction and per commit), warp 9 also allocates tensor memory.
+// Tensor memory: 2 buffers x 2 accumulators x 128 columns = 512 columns, so the MMAs
+// of step i+1 overlap the epilogue of step i.
 //
 // Codewords whose half squared norm exceeds the fp16 range get a sentinel row
 // that can never win and are listed as "exceptions": the rescoring kernel always
@@ -57,7 +58,7 @@ constexpr int kTcGroupBytes = 8 * kTcRowBytes;         // one 8-row group: 4 cor
 constexpr int kTcSubCw = 64;            // tracking granularity of the running maximum
 constexpr int kTcStages = 12;           // bulk-copy ring
 constexpr int kTcEpiThreads = 256;
-constexpr int kTcThreads = kTcEpiThreads + 64;
+constexpr int kTcThreads = kTcEpiThreads + 96;  // + producer warp + one MMA warp per A block
 constexpr uint32_t kTmemCols = 512;
 constexpr float kMaxHalfNorm = 60000.0f;  // largest ||c||^2/2 the image represents
 constexpr float kNegInf = -__builtin_huge_valf();
@@ -228,7 +229,22 @@ __device__ __forceinline__ void tmem_ld64(uint32_t taddr, uint32_t* v) {
       : "r"(taddr)
       : "memory");
 }
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// Wait for the outstanding tensor-memory loads.  The registers are passed through the
+// statement so that no use of them can be scheduled ahead of the wait.
+__device__ __forceinline__ void tmem_ld_wait(uint32_t* v) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]),
+                 "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15]),
+                 "+r"(v[16]), "+r"(v[17]), "+r"(v[18]), "+r"(v[19]), "+r"(v[20]), "+r"(v[21]), "+r"(v[22]),
+                 "+r"(v[23]), "+r"(v[24]), "+r"(v[25]), "+r"(v[26]), "+r"(v[27]), "+r"(v[28]), "+r"(v[29]),
+                 "+r"(v[30]), "+r"(v[31]), "+r"(v[32]), "+r"(v[33]), "+r"(v[34]), "+r"(v[35]), "+r"(v[36]),
+                 "+r"(v[37]), "+r"(v[38]), "+r"(v[39]), "+r"(v[40]), "+r"(v[41]), "+r"(v[42]), "+r"(v[43]),
+                 "+r"(v[44]), "+r"(v[45]), "+r"(v[46]), "+r"(v[47]), "+r"(v[48]), "+r"(v[49]), "+r"(v[50]),
+                 "+r"(v[51]), "+r"(v[52]), "+r"(v[53]), "+r"(v[54]), "+r"(v[55]), "+r"(v[56]), "+r"(v[57]),
+                 "+r"(v[58]), "+r"(v[59]), "+r"(v[60]), "+r"(v[61]), "+r"(v[62]), "+r"(v[63])
+               :
+               : "memory");
+}
 
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float d;
@@ -258,10 +274,10 @@ struct TcSmem {
   alignas(128) unsigned char b[kTcStages][kTcStepBytes];
   alignas(8) uint64_t full_bar[kTcStages];
   uint64_t empty_bar[kTcStages];
-  uint64_t tmem_full[2];
-  uint64_t tmem_empty[2];
+  uint64_t tmem_full[2][2];   // per buffer and A block
+  uint64_t tmem_empty[2][2];
   uint64_t a_ready;
-  uint64_t drain_bar;
+  uint64_t drain_bar[2];
   float evicted_max[kTcTile];           // largest sub-chunk maximum that fell out of the list
   float list_max[kListLen][kTcTile];
   uint16_t list_id[kListLen][kTcTile];
@@ -282,14 +298,17 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
     sm.abort_flag = 0;
     for (int s = 0; s < kTcStages; ++s) {
       mbar_init(smem_u32(&sm.full_bar[s]), 1);
-      mbar_init(smem_u32(&sm.empty_bar[s]), 1);
+      mbar_init(smem_u32(&sm.empty_bar[s]), 2);  // one commit per MMA warp
     }
     for (int b = 0; b < 2; ++b) {
-      mbar_init(smem_u32(&sm.tmem_full[b]), 1);
-      mbar_init(smem_u32(&sm.tmem_empty[b]), kTcEpiThreads / 32);
+      for (int q = 0; q < 2; ++q) {
+        mbar_init(smem_u32(&sm.tmem_full[b][q]), 1);
+        mbar_init(smem_u32(&sm.tmem_empty[b][q]), kTcEpiThreads / 64);  // the four warps of the block
+      }
     }
     mbar_init(smem_u32(&sm.a_ready), kTcEpiThreads);
-    mbar_init(smem_u32(&sm.drain_bar), 1);
+    mbar_init(smem_u32(&sm.drain_bar[0]), 1);
+    mbar_init(smem_u32(&sm.drain_bar[1]), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 9) {
@@ -333,11 +352,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
         }
       }
     }
-  } else if (warp == 9) {
-    // ------------------------------------------------------------ MMA issuer
+  } else if (warp >= 9) {
+    // ------------------------------------------------------------ MMA issuers: warp 9 -> A block 0, warp 10 -> A block 1
     if (lane == 0) {
-      const uint64_t a_desc0 = smem_desc(smem_u32(&sm.a[0][0]));
-      const uint64_t a_desc1 = smem_desc(smem_u32(&sm.a[1][0]));
+      const uint32_t q = (uint32_t)warp - 9u;
+      const uint64_t a_desc = smem_desc(smem_u32(&sm.a[q][0]));
       uint32_t it = 0, unit_i = 0;
       bool alive = true;
       for (uint64_t u = blockIdx.x; u < units && alive; u += gridDim.x, ++unit_i) {
@@ -348,24 +367,23 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
         for (uint32_t st = s_lo; st < s_hi && alive; ++st, ++it) {
           const uint32_t s = it % kTcStages, buf = it & 1;
           alive = mbar_wait(smem_u32(&sm.full_bar[s]), (it / kTcStages) & 1, abort_flag, p.status);
-          if (alive) alive = mbar_wait(smem_u32(&sm.tmem_empty[buf]), ((it >> 1) & 1) ^ 1, abort_flag, p.status);
+          if (alive) alive = mbar_wait(smem_u32(&sm.tmem_empty[buf][q]), ((it >> 1) & 1) ^ 1, abort_flag, p.status);
           if (!alive) break;
           tc_fence_after();
           const uint64_t b_desc = smem_desc(smem_u32(&sm.b[s][0]));
           // K chunks 0-1 (hi, lo against c), then chunks 2-3 (the norm terms) on top
-          umma_f16(tmem_base + buf * 256, a_desc0, b_desc, kIdesc, 0);
-          umma_f16(tmem_base + buf * 256, a_desc0 + kDescTwoChunks, b_desc + kDescTwoChunks, kIdesc, 1);
-          umma_f16(tmem_base + buf * 256 + 128, a_desc1, b_desc, kIdesc, 0);
-          umma_f16(tmem_base + buf * 256 + 128, a_desc1 + kDescTwoChunks, b_desc + kDescTwoChunks, kIdesc, 1);
-          umma_commit(smem_u32(&sm.empty_bar[s]));   // the stage is free once both MMAs have read it
-          umma_commit(smem_u32(&sm.tmem_full[buf])); // the accumulators are ready
+          const uint32_t d = tmem_base + buf * 256 + q * 128;
+          umma_f16(d, a_desc, b_desc, kIdesc, 0);
+          umma_f16(d, a_desc + kDescTwoChunks, b_desc + kDescTwoChunks, kIdesc, 1);
+          umma_commit(smem_u32(&sm.tmem_full[buf][q]));  // the accumulator is ready
+          umma_commit(smem_u32(&sm.empty_bar[s]));       // this warp no longer reads the stage
         }
       }
       if (!alive) {
         // wait (bounded) for whatever was issued before tensor memory is released
-        umma_commit(smem_u32(&sm.drain_bar));
+        umma_commit(smem_u32(&sm.drain_bar[q]));
         for (uint32_t spin = 0; spin < kMaxSpins; ++spin) {
-          if (mbar_try_wait(smem_u32(&sm.drain_bar), 0)) break;
+          if (mbar_try_wait(smem_u32(&sm.drain_bar[q]), 0)) break;
           __nanosleep(64);
         }
       }
@@ -440,35 +458,56 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
       sm.list_cnt[tid] = 0;
       sm.evicted_max[tid] = kNegInf;
 
+      // Software-pipelined epilogue.  The 128 columns of a step are read as two halves into
+      // two register sets; the first half of step i+1 is requested (if its MMAs are done)
+      // before the maximum of the second half of step i is computed, and a buffer goes back
+      // to the MMA warp as soon as both halves are in registers.
+      uint32_t v[64], w[64];
+      bool pending = false;  // the first half of step `st` is already in flight
+      auto note = [&](float mx, uint32_t sub) {
+        if (mx >= thr) {
+          const uint32_t cnt = sm.list_cnt[tid];
+          const uint32_t slot = cnt & (kListLen - 1);
+          if (cnt >= kListLen) sm.evicted_max[tid] = fmaxf(sm.evicted_max[tid], sm.list_max[slot][tid]);
+          sm.list_id[slot][tid] = (uint16_t)sub;
+          sm.list_max[slot][tid] = mx;
+          sm.list_cnt[tid] = (uint16_t)(cnt + 1);
+          best = fmaxf(best, mx);
+          thr = best - margin;
+        }
+      };
       for (uint32_t st = s_lo; st < s_hi; ++st, ++it) {
         const uint32_t buf = it & 1;
-        // warp-uniform outcome: the tensor-memory loads below need the whole warp
-        alive = __all_sync(0xffffffffu, mbar_wait(smem_u32(&sm.tmem_full[buf]), (it >> 1) & 1, abort_flag, p.status));
-        if (!alive) break;
-        tc_fence_after();
         const uint32_t taddr = tmem_base + lane_base + buf * 256 + rb * 128;
-        uint32_t v[64], w[64];
-        tmem_ld64(taddr, v);
+        if (!pending) {
+          // one lane polls (256 threads polling one barrier slow every barrier operation of the CTA
+          // down); the warp-wide exchange orders the other lanes after its observation
+          bool ok = true;
+          if (lane == 0) ok = mbar_wait(smem_u32(&sm.tmem_full[buf][rb]), (it >> 1) & 1, abort_flag, p.status);
+          alive = __shfl_sync(0xffffffffu, ok, 0);
+          if (!alive) break;
+          tc_fence_after();
+          tmem_ld64(taddr, v);
+        }
+        tmem_ld_wait(v);
         tmem_ld64(taddr + 64, w);
-        tmem_ld_wait();
+        note(max64(v), 2 * st);
+        tmem_ld_wait(w);
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&sm.tmem_empty[buf]));
-        const float m0 = max64(v), m1 = max64(w);
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          const float mx = half ? m1 : m0;
-          if (mx >= thr) {
-            const uint32_t cnt = sm.list_cnt[tid];
-            const uint32_t slot = cnt & (kListLen - 1);
-            if (cnt >= kListLen) sm.evicted_max[tid] = fmaxf(sm.evicted_max[tid], sm.list_max[slot][tid]);
-            sm.list_id[slot][tid] = (uint16_t)(st * 2 + half);
-            sm.list_max[slot][tid] = mx;
-            sm.list_cnt[tid] = (uint16_t)(cnt + 1);
-            best = fmaxf(best, mx);
-            thr = best - margin;
+        if (lane == 0) mbar_arrive(smem_u32(&sm.tmem_empty[buf][rb]));
+        pending = false;
+        if (st + 1 < s_hi) {
+          const uint32_t nbuf = (it + 1) & 1;
+          bool ready = false;
+          if (lane == 0) ready = mbar_try_wait(smem_u32(&sm.tmem_full[nbuf][rb]), ((it + 1) >> 1) & 1);
+          if (__shfl_sync(0xffffffffu, ready, 0)) {
+            tc_fence_after();
+            tmem_ld64(tmem_base + lane_base + nbuf * 256 + rb * 128, v);
+            pending = true;
           }
         }
+        note(max64(w), 2 * st + 1);
       }
 
       // leave the candidates of this (tile, slice) for the rescoring kernel (minimum convention: -S)
