@@ -30,10 +30,9 @@
 // CTA = 256 targets (two 128-row A blocks) x a slice of the codebook, one CTA per
 // SM, persistent over (tile, slice) units.  Warps 0-7: own one target per thread,
 // build A, run the epilogue (warp w reads tensor-memory lanes 32 (w % 4) .. of the
-// accumulator of A block w / 4).  Warp 8: bulk-copy producer (stages of four steps).
-// Warps 9 and 10: one thread each issues the MMAs of every other step (issuing and
-// above all waiting on barriers is slow for a lone thread), warp 9 also allocates
-// tensor memory.
+// accumulator of A block w / 4).  Warp 8: bulk-copy producer.  Warps 9 and 10: one
+// thread each issues the MMAs of one A block (issuing is the scarce resource: about
+// 60 cycles per instruction and per commit), warp 9 also allocates tensor memory.
 // Tensor memory: 2 buffers x 2 accumulators x 128 columns = 512 columns, so the MMAs
 // of step i+1 overlap the epilogue of step i.
 //
@@ -57,10 +56,9 @@ constexpr int kTcRowBytes = 64;         // 32 halves
 constexpr int kTcStepBytes = kTcStepCw * kTcRowBytes;  // 8192
 constexpr int kTcGroupBytes = 8 * kTcRowBytes;         // one 8-row group: 4 core matrices of 128 bytes
 constexpr int kTcSubCw = 64;            // tracking granularity of the running maximum
-constexpr int kTcGroupSteps = 4;        // steps per codebook stage: one barrier hand-over serves four steps
-constexpr int kTcStages = 3;            // codebook stages (32 KB each)
+constexpr int kTcStages = 12;           // bulk-copy ring
 constexpr int kTcEpiThreads = 256;
-constexpr int kTcThreads = kTcEpiThreads + 96;  // + producer warp + one MMA warp per accumulator buffer
+constexpr int kTcThreads = kTcEpiThreads + 96;  // + producer warp + one MMA warp per A block
 constexpr uint32_t kTmemCols = 512;
 constexpr float kMaxHalfNorm = 60000.0f;  // largest ||c||^2/2 the image represents
 constexpr float kNegInf = -__builtin_huge_valf();
@@ -273,11 +271,11 @@ __device__ __forceinline__ float max64(const uint32_t* v) {
 // ---- shared memory -----------------------------------------------------------------
 struct TcSmem {
   alignas(128) unsigned char a[2][kTcStepBytes];  // two A blocks of 128 targets
-  alignas(128) unsigned char b[kTcStages][kTcGroupSteps][kTcStepBytes];
+  alignas(128) unsigned char b[kTcStages][kTcStepBytes];
   alignas(8) uint64_t full_bar[kTcStages];
   uint64_t empty_bar[kTcStages];
-  uint64_t tmem_full[2];   // per accumulator buffer (both A blocks)
-  uint64_t tmem_empty[2];
+  uint64_t tmem_full[2][2];   // per buffer and A block
+  uint64_t tmem_empty[2][2];
   uint64_t a_ready;
   uint64_t drain_bar[2];
   float evicted_max[kTcTile];           // largest sub-chunk maximum that fell out of the list
@@ -300,11 +298,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
     sm.abort_flag = 0;
     for (int s = 0; s < kTcStages; ++s) {
       mbar_init(smem_u32(&sm.full_bar[s]), 1);
-      mbar_init(smem_u32(&sm.empty_bar[s]), 1);  // released by the epilogue (warp 0)
+      mbar_init(smem_u32(&sm.empty_bar[s]), 2);  // one commit per MMA warp
     }
     for (int b = 0; b < 2; ++b) {
-      mbar_init(smem_u32(&sm.tmem_full[b]), 1);
-      mbar_init(smem_u32(&sm.tmem_empty[b]), kTcEpiThreads / 32);
+      for (int q = 0; q < 2; ++q) {
+        mbar_init(smem_u32(&sm.tmem_full[b][q]), 1);
+        mbar_init(smem_u32(&sm.tmem_empty[b][q]), kTcEpiThreads / 64);  // the four warps of the block
+      }
     }
     mbar_init(smem_u32(&sm.a_ready), kTcEpiThreads);
     mbar_init(smem_u32(&sm.drain_bar[0]), 1);
@@ -325,36 +325,25 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
   if (warp == 8) {
     // ------------------------------------------------------------ bulk-copy producer
     if (lane == 0) {
-      // total number of steps of this CTA (needed for the byte count of the last, partial group)
-      uint32_t total = 0;
-      for (uint64_t u = blockIdx.x; u < units; u += gridDim.x) {
-        uint32_t s_lo, s_hi;
-        slice_units(p, (uint32_t)(u % p.n_slices), &s_lo, &s_hi);
-        total += s_hi - s_lo;
-      }
       uint32_t it = 0;
       bool alive = true;
       for (uint64_t u = blockIdx.x; u < units && alive; u += gridDim.x) {
         uint32_t s_lo, s_hi;
         slice_units(p, (uint32_t)(u % p.n_slices), &s_lo, &s_hi);
         for (uint32_t st = s_lo; st < s_hi && alive; ++st, ++it) {
-          const uint32_t grp = it / kTcGroupSteps, sub = it % kTcGroupSteps, s = grp % kTcStages;
+          const uint32_t s = it % kTcStages;
+          if (it >= kTcStages)
+            alive = mbar_wait(smem_u32(&sm.empty_bar[s]), ((it / kTcStages) - 1) & 1, abort_flag, p.status);
+          if (!alive) break;
           const uint32_t fb = smem_u32(&sm.full_bar[s]);
-          if (sub == 0) {
-            if (grp >= (uint32_t)kTcStages)
-              alive = mbar_wait(smem_u32(&sm.empty_bar[s]), ((grp / kTcStages) - 1) & 1, abort_flag, p.status);
-            if (!alive) break;
-            const uint32_t left = total - it;
-            mbar_expect_tx(fb, (left < (uint32_t)kTcGroupSteps ? left : (uint32_t)kTcGroupSteps) * kTcStepBytes);
-          }
-          bulk_g2s(smem_u32(&sm.b[s][sub][0]), bimg + (size_t)st * kTcStepBytes, kTcStepBytes, fb);
+          mbar_expect_tx(fb, kTcStepBytes);
+          bulk_g2s(smem_u32(&sm.b[s][0]), bimg + (size_t)st * kTcStepBytes, kTcStepBytes, fb);
         }
       }
       if (!alive) {
         // let every copy that was issued land before the CTA may exit
-        const uint32_t groups = (it + kTcGroupSteps - 1) / kTcGroupSteps;
-        for (uint32_t back = 1; back <= (uint32_t)kTcStages && back <= groups; ++back) {
-          const uint32_t j = groups - back;
+        for (uint32_t back = 1; back <= kTcStages && back <= it; ++back) {
+          const uint32_t j = it - back;
           const uint32_t fb = smem_u32(&sm.full_bar[j % kTcStages]);
           for (uint32_t spin = 0; spin < kMaxSpins; ++spin) {
             if (mbar_try_wait(fb, (j / kTcStages) & 1)) break;
@@ -364,50 +353,37 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
       }
     }
   } else if (warp >= 9) {
-    // ------------------------------------------------------------ MMA issuers: warp 9 -> even steps (buffer 0), warp 10 -> odd
-    // A wait on an mbarrier costs a lone thread about 200 cycles even when the phase is already over, an MMA or
-    // a commit about 60: per step one wait for the accumulators, a quarter of a wait for the codebook stage,
-    // four MMAs (both A blocks) and one commit; two threads share the steps.
+    // ------------------------------------------------------------ MMA issuers: warp 9 -> A block 0, warp 10 -> A block 1
     if (lane == 0) {
-      const uint32_t mine = (uint32_t)warp - 9u;
-      const uint64_t a_desc0 = smem_desc(smem_u32(&sm.a[0][0]));
-      const uint64_t a_desc1 = smem_desc(smem_u32(&sm.a[1][0]));
-      const uint32_t d0 = tmem_base + mine * 256, d1 = d0 + 128;
-      const uint32_t full_tmem = smem_u32(&sm.tmem_full[mine]), empty_tmem = smem_u32(&sm.tmem_empty[mine]);
-      uint32_t it = 0, unit_i = 0, waited_group = 0xffffffffu;
+      const uint32_t q = (uint32_t)warp - 9u;
+      const uint64_t a_desc = smem_desc(smem_u32(&sm.a[q][0]));
+      uint32_t it = 0, unit_i = 0;
       bool alive = true;
       for (uint64_t u = blockIdx.x; u < units && alive; u += gridDim.x, ++unit_i) {
         uint32_t s_lo, s_hi;
         slice_units(p, (uint32_t)(u % p.n_slices), &s_lo, &s_hi);
         alive = mbar_wait(smem_u32(&sm.a_ready), unit_i & 1, abort_flag, p.status);
         tc_fence_after();
-        const uint32_t it_end = it + (s_hi - s_lo);
-        if ((it & 1u) != mine) ++it;
-        for (; it < it_end && alive; it += 2) {
-          const uint32_t grp = it / kTcGroupSteps, sub = it % kTcGroupSteps, s = grp % kTcStages;
-          if (grp != waited_group) {
-            alive = mbar_wait(smem_u32(&sm.full_bar[s]), (grp / kTcStages) & 1, abort_flag, p.status);
-            waited_group = grp;
-          }
-          if (alive) alive = mbar_wait(empty_tmem, ((it >> 1) & 1) ^ 1, abort_flag, p.status);
+        for (uint32_t st = s_lo; st < s_hi && alive; ++st, ++it) {
+          const uint32_t s = it % kTcStages, buf = it & 1;
+          alive = mbar_wait(smem_u32(&sm.full_bar[s]), (it / kTcStages) & 1, abort_flag, p.status);
+          if (alive) alive = mbar_wait(smem_u32(&sm.tmem_empty[buf][q]), ((it >> 1) & 1) ^ 1, abort_flag, p.status);
           if (!alive) break;
           tc_fence_after();
-          const uint64_t b_desc = smem_desc(smem_u32(&sm.b[s][sub][0]));
+          const uint64_t b_desc = smem_desc(smem_u32(&sm.b[s][0]));
           // K chunks 0-1 (hi, lo against c), then chunks 2-3 (the norm terms) on top
-          umma_f16(d0, a_desc0, b_desc, kIdesc, 0);
-          umma_f16(d0, a_desc0 + kDescTwoChunks, b_desc + kDescTwoChunks, kIdesc, 1);
-          umma_f16(d1, a_desc1, b_desc, kIdesc, 0);
-          umma_f16(d1, a_desc1 + kDescTwoChunks, b_desc + kDescTwoChunks, kIdesc, 1);
-          umma_commit(full_tmem);  // the accumulators of this step are ready; the epilogue also learns from it
-                                   // that the step's share of the codebook stage has been read
+          const uint32_t d = tmem_base + buf * 256 + q * 128;
+          umma_f16(d, a_desc, b_desc, kIdesc, 0);
+          umma_f16(d, a_desc + kDescTwoChunks, b_desc + kDescTwoChunks, kIdesc, 1);
+          umma_commit(smem_u32(&sm.tmem_full[buf][q]));  // the accumulator is ready
+          umma_commit(smem_u32(&sm.empty_bar[s]));       // this warp no longer reads the stage
         }
-        it = it_end;
       }
       if (!alive) {
         // wait (bounded) for whatever was issued before tensor memory is released
-        umma_commit(smem_u32(&sm.drain_bar[mine]));
+        umma_commit(smem_u32(&sm.drain_bar[q]));
         for (uint32_t spin = 0; spin < kMaxSpins; ++spin) {
-          if (mbar_try_wait(smem_u32(&sm.drain_bar[mine]), 0)) break;
+          if (mbar_try_wait(smem_u32(&sm.drain_bar[q]), 0)) break;
           __nanosleep(64);
         }
       }
@@ -486,12 +462,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
       // two register sets; the first half of step i+1 is requested (if its MMAs are done)
       // before the maximum of the second half of step i is computed, and a buffer goes back
       // to the MMA warp as soon as both halves are in registers.
-      // Warp 0 hands a codebook stage back to the producer once it has seen the MMAs of the stage's last step
-      // complete (it sees every step's completion in order, and a step's commit covers both A blocks).
-      auto release_stage = [&](uint32_t step_seen) {
-        if (tid == 0 && (step_seen % kTcGroupSteps) == (uint32_t)kTcGroupSteps - 1)
-          mbar_arrive(smem_u32(&sm.empty_bar[(step_seen / kTcGroupSteps) % kTcStages]));
-      };
       uint32_t v[64], w[64];
       bool pending = false;  // the first half of step `st` is already in flight
       auto note = [&](float mx, uint32_t sub) {
@@ -513,10 +483,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
           // one lane polls (256 threads polling one barrier slow every barrier operation of the CTA
           // down); the warp-wide exchange orders the other lanes after its observation
           bool ok = true;
-          if (lane == 0) ok = mbar_wait(smem_u32(&sm.tmem_full[buf]), (it >> 1) & 1, abort_flag, p.status);
+          if (lane == 0) ok = mbar_wait(smem_u32(&sm.tmem_full[buf][rb]), (it >> 1) & 1, abort_flag, p.status);
           alive = __shfl_sync(0xffffffffu, ok, 0);
           if (!alive) break;
-          release_stage(it);
           tc_fence_after();
           tmem_ld64(taddr, v);
         }
@@ -526,14 +495,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
         tmem_ld_wait(w);
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&sm.tmem_empty[buf]));
+        if (lane == 0) mbar_arrive(smem_u32(&sm.tmem_empty[buf][rb]));
         pending = false;
         if (st + 1 < s_hi) {
           const uint32_t nbuf = (it + 1) & 1;
           bool ready = false;
-          if (lane == 0) ready = mbar_try_wait(smem_u32(&sm.tmem_full[nbuf]), ((it + 1) >> 1) & 1);
+          if (lane == 0) ready = mbar_try_wait(smem_u32(&sm.tmem_full[nbuf][rb]), ((it + 1) >> 1) & 1);
           if (__shfl_sync(0xffffffffu, ready, 0)) {
-            release_stage(it + 1);
             tc_fence_after();
             tmem_ld64(tmem_base + lane_base + nbuf * 256 + rb * 128, v);
             pending = true;
