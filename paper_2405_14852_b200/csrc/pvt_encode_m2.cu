@@ -4,15 +4,21 @@
 // dequantised weight; Eq. 8 for the target; Lemma 3.3 for keeping the previous
 // pair in the pool).
 //
-// One warp per target, persistent grid.  Lane l owns codewords l, l+32, ..., l+224
-// of both codebooks: its slice of codebook 2 stays in registers for the whole
-// kernel (packed as f32x2 pairs), codebook 1 is read from shared memory.
-//   stage 1: score1 = ||c1||^2/2 - <t, c1> for 256 codewords (8 per lane); the
-//            `beam` smallest are extracted with warp-wide integer minimum
-//            reductions on (score bits | code) keys.
-//   stage 2: for each beam entry r = t - c1 and
-//            score2 = ||r||^2/2 + ||c2||^2/2 - <r, c2> for 256 codewords; only the
-//            running minimum is kept.
+// A warp handles four targets at a time; both codebooks live in shared memory;
+// two CTAs (16 warps) share an SM.
+//   stage 1 (per target, the whole warp): lane l owns codewords l, l+32, ..., l+224
+//            of codebook 1: score1 = ||c1||^2/2 - <t, c1> for 256 codewords (8 per
+//            lane, packed f32x2); the `beam` smallest are extracted with warp-wide
+//            integer minimum reductions on (score bits | code) keys.
+//   stage 2 (four targets x eight beam entries = 32 lanes): every lane takes one
+//            (target, beam entry), forms its residual r = t - c1 and streams all of
+//            codebook 2 from shared memory (broadcast loads of codeword pairs):
+//            score2 = ||r||^2/2 + ||c2||^2/2 - <r, c2>, 8 packed FMAs per pair of
+//            codewords, one three-input min; only the minimum of each 32-codeword
+//            sub-chunk is kept.
+//   decision: the eight lanes of a target agree on the smallest score; sub-chunks
+//            within the rounding-error margin of it are revisited and the
+//            codewords within the margin get their binary64 distance.
 // Fast scores are binary32.  Every decision they cannot settle within twice their
 // rounding-error bound (membership of the beam, the final argmin) is taken on
 // binary64 distances accumulated in index order, so the result is the argmin of
@@ -48,12 +54,18 @@ struct EncM2Params {
   uint32_t* status;
 };
 
+constexpr int kM2Group = 4;  // targets per warp iteration: 4 targets x 8 beam entries = 32 lanes
+
 struct M2Smem {
   alignas(16) float c1[kM2K][8];
   alignas(16) float c2[kM2K][8];
   alignas(16) uint64_t p1[4][8][32];  // stage-1 operands: (c1[l+64q][i], c1[l+64q+32][i])
   uint64_t h1[4][32];                 // (||c1||^2/2) pairs in the same order
+  alignas(16) float x2[kM2K / 2][16]; // stage-2 operands: pair p holds (c2[2p][0], c2[2p+1][0], c2[2p][1], ...)
+  alignas(8) float hx2[kM2K / 2][2];  // (||c2||^2/2) of the pair
   float h2[kM2K];
+  alignas(16) float wt[kM2Threads / 32][kM2Group][8];     // the targets of a warp's group
+  alignas(16) uint32_t wk[kM2Threads / 32][kM2Group][8];  // their beam entries (codes of codebook 1)
   float red[kM2Threads / 32][2];
   float n1max, n2max;
 };
@@ -114,7 +126,7 @@ __device__ __forceinline__ float load_cb(const void* books, int f16, uint32_t m,
   return f16 ? __half2float(reinterpret_cast<const __half*>(books)[off]) : reinterpret_cast<const float*>(books)[off];
 }
 
-__global__ void __launch_bounds__(kM2Threads, 1) encode_m2_kernel(const EncM2Params p) {
+__global__ void __launch_bounds__(kM2Threads, 2) encode_m2_kernel(const EncM2Params p) {
   __shared__ M2Smem sm;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
@@ -136,8 +148,12 @@ __global__ void __launch_bounds__(kM2Threads, 1) encode_m2_kernel(const EncM2Par
     const int l = tid & 31, jj = tid >> 5, q = jj >> 1, half = jj & 1;
     float* p1f = reinterpret_cast<float*>(&sm.p1[0][0][0]);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) p1f[(((q * 8 + i) * 32) + l) * 2 + half] = c1[i];
+    for (int i = 0; i < 8; ++i) {
+      p1f[(((q * 8 + i) * 32) + l) * 2 + half] = c1[i];
+      sm.x2[tid >> 1][2 * i + (tid & 1)] = c2[i];
+    }
     reinterpret_cast<float*>(&sm.h1[0][0])[(q * 32 + l) * 2 + half] = h1;
+    sm.hx2[tid >> 1][tid & 1] = h2;
     sm.h2[tid] = h2;
     float m1 = n1, m2 = n2;
 #pragma unroll
@@ -161,15 +177,6 @@ __global__ void __launch_bounds__(kM2Threads, 1) encode_m2_kernel(const EncM2Par
     }
     __syncthreads();
   }
-  // this lane's slice of codebook 2, packed (c2[l+64q][i], c2[l+64q+32][i])
-  uint64_t c2p[4][8], h2p[4];
-#pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    const int ka = lane + 64 * q, kb = ka + 32;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) c2p[q][i] = pack2(sm.c2[ka][i], sm.c2[kb][i]);
-    h2p[q] = pack2(sm.h2[ka], sm.h2[kb]);
-  }
   const float n1max = sm.n1max, n2max = sm.n2max;
   const float s1max = sqrtf(n1max), s2max = sqrtf(n2max);
   const uint32_t B = p.beam;  // already min(beam, K)
@@ -177,201 +184,265 @@ __global__ void __launch_bounds__(kM2Threads, 1) encode_m2_kernel(const EncM2Par
   const float4* W4 = reinterpret_cast<const float4*>(p.W);
   const float4* g4 = reinterpret_cast<const float4*>(p.g);
   const uint64_t nwarps = (uint64_t)gridDim.x * (kM2Threads / 32);
+  const uint64_t n_groups = (p.k + kM2Group - 1) / kM2Group;
+  const uint32_t my_q = (uint32_t)lane >> 3, my_b = (uint32_t)lane & 7u;
 
-  for (uint64_t n = (uint64_t)blockIdx.x * (kM2Threads / 32) + warp; n < p.k; n += nwarps) {
-    const uint32_t j = __ldg(p.idx + n);
-    if (j >= p.G) {
-      if (lane == 0) atomicOr(p.status, PVT_DEV_BAD_INDEX);
-      continue;
-    }
-    // target, binary32: one fma, one division (every lane holds all 8 values)
-    float t[8];
-    {
-      const float4 w0 = __ldg(W4 + 2 * (size_t)j), w1 = __ldg(W4 + 2 * (size_t)j + 1);
-      const float4 g0 = __ldg(g4 + 2 * (size_t)j), g1 = __ldg(g4 + 2 * (size_t)j + 1);
-      const float sc = __ldg(p.scale + j / p.gpr), ne = -p.eta;
-      t[0] = __fdiv_rn(__fmaf_rn(ne, g0.x, w0.x), sc);
-      t[1] = __fdiv_rn(__fmaf_rn(ne, g0.y, w0.y), sc);
-      t[2] = __fdiv_rn(__fmaf_rn(ne, g0.z, w0.z), sc);
-      t[3] = __fdiv_rn(__fmaf_rn(ne, g0.w, w0.w), sc);
-      t[4] = __fdiv_rn(__fmaf_rn(ne, g1.x, w1.x), sc);
-      t[5] = __fdiv_rn(__fmaf_rn(ne, g1.y, w1.y), sc);
-      t[6] = __fdiv_rn(__fmaf_rn(ne, g1.z, w1.z), sc);
-      t[7] = __fdiv_rn(__fmaf_rn(ne, g1.w, w1.w), sc);
-    }
-    const uint32_t prev = p.codes[j];
-    float nt2 = 0.0f;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) nt2 = fmaf(t[i], t[i], nt2);
-    const float tnorm = sqrtf(nt2);
-    // twice the rounding-error bounds of the two fast scores (factor >= 2 to spare), u = 2^-24:
-    //   |score1_fl - score1| <= 16.1 u (||c1||^2/2 + ||t|| ||c1||)
-    //   |score2_fl - score2| <= 26 u (||t|| + max||c1|| + max||c2||)^2
-    const float margin1 = 3.8146973e-6f /* 2^-18 */ * (0.5f * n1max + tnorm * s1max) + 1e-30f;
-    const float sall = tnorm + s1max + s2max;
-    const float margin2 = 7.6293945e-6f /* 2^-17 */ * sall * sall + 1e-30f;
+  for (uint64_t gi = (uint64_t)blockIdx.x * (kM2Threads / 32) + warp; gi < n_groups; gi += nwarps) {
+    // what this lane needs of its own target (target my_q of the group)
+    uint32_t my_j = 0xffffffffu, my_prev = 0;
+    float my_margin2 = 0.0f;
 
-    // ---- stage 1: 256 scores, 8 per lane
-    float f[8];
-    {
-      uint64_t acc[4];
-#pragma unroll
-      for (int q = 0; q < 4; ++q) acc[q] = sm.h1[q][lane];
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const uint64_t ntd = pack2(-t[i], -t[i]);
-#pragma unroll
-        for (int q = 0; q < 4; ++q) acc[q] = fma2(ntd, sm.p1[q][i][lane], acc[q]);
+    // ---- stage 1, one target after the other, the whole warp on each
+#pragma unroll 1
+    for (uint32_t q = 0; q < (uint32_t)kM2Group; ++q) {
+      const uint64_t n = gi * kM2Group + q;
+      if (n >= p.k) break;
+      const uint32_t j = __ldg(p.idx + n);
+      if (j >= p.G) {
+        if (lane == 0) atomicOr(p.status, PVT_DEV_BAD_INDEX);
+        continue;
       }
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        f[2 * q] = lo_of(acc[q]);
-        f[2 * q + 1] = hi_of(acc[q]);
+      // target, binary32: one fma, one division (every lane holds all 8 values)
+      float t[8];
+      {
+        const float4 w0 = __ldg(W4 + 2 * (size_t)j), w1 = __ldg(W4 + 2 * (size_t)j + 1);
+        const float4 g0 = __ldg(g4 + 2 * (size_t)j), g1 = __ldg(g4 + 2 * (size_t)j + 1);
+        const float sc = __ldg(p.scale + j / p.gpr), ne = -p.eta;
+        t[0] = __fdiv_rn(__fmaf_rn(ne, g0.x, w0.x), sc);
+        t[1] = __fdiv_rn(__fmaf_rn(ne, g0.y, w0.y), sc);
+        t[2] = __fdiv_rn(__fmaf_rn(ne, g0.z, w0.z), sc);
+        t[3] = __fdiv_rn(__fmaf_rn(ne, g0.w, w0.w), sc);
+        t[4] = __fdiv_rn(__fmaf_rn(ne, g1.x, w1.x), sc);
+        t[5] = __fdiv_rn(__fmaf_rn(ne, g1.y, w1.y), sc);
+        t[6] = __fdiv_rn(__fmaf_rn(ne, g1.z, w1.z), sc);
+        t[7] = __fdiv_rn(__fmaf_rn(ne, g1.w, w1.w), sc);
       }
-    }
-    // extract the B smallest (score truncated to 24 bits | code): a first guess of the beam
-    uint32_t key[8];
+      const uint32_t prev = p.codes[j];
+      float nt2 = 0.0f;
 #pragma unroll
-    for (int jj = 0; jj < 8; ++jj) key[jj] = (ord(f[jj]) & 0xffffff00u) | (uint32_t)(lane + 32 * jj);
-    uint32_t beam_code[8];
-#pragma unroll
-    for (int b = 0; b < 8; ++b) {
-      beam_code[b] = 0;
-      if ((uint32_t)b < B) {
-        uint32_t lm = key[0];
-#pragma unroll
-        for (int jj = 1; jj < 8; ++jj) lm = min(lm, key[jj]);
-        const uint32_t m = __reduce_min_sync(0xffffffffu, lm);
-        beam_code[b] = m & 0xffu;
-#pragma unroll
-        for (int jj = 0; jj < 8; ++jj)
-          if (key[jj] == m) key[jj] = 0xffffffffu;
-      }
-    }
-    // is that guess provably the exact beam?  theta = largest score in the guess;
-    // every member of the exact beam scores <= theta + margin1; if exactly B
-    // codewords do, they are the guess and the exact beam at once.
-    {
-      float th = -kInf;
-      uint32_t cnt = 0;
-#pragma unroll
-      for (int jj = 0; jj < 8; ++jj)
-        if (key[jj] == 0xffffffffu) th = fmaxf(th, f[jj]);
-      const float theta = unord(__reduce_max_sync(0xffffffffu, ord(th)));
-      const float limit1 = theta + margin1;
-      uint32_t member = 0;
-#pragma unroll
-      for (int jj = 0; jj < 8; ++jj) {
-        const bool in = f[jj] <= limit1 && (uint32_t)(lane + 32 * jj) < p.K;
-        member |= in ? (1u << jj) : 0u;
-        cnt += in;
-      }
-      cnt = __reduce_add_sync(0xffffffffu, cnt);
-      if (cnt != B) {
-        // undecided: order the shortlisted codewords by (binary64 distance, code)
-        for (uint32_t b = 0; b < B; ++b) {
-          double ld = __longlong_as_double(0x7ff0000000000000ll);
-          uint32_t lk = 0xffffffffu;
-#pragma unroll
-          for (int jj = 0; jj < 8; ++jj) {
-            if (member & (1u << jj)) {
-              const uint32_t kap = lane + 32 * jj;
-              const double d = exact1(t, sm.c1[kap]);
-              if (d < ld || (d == ld && kap < lk)) {
-                ld = d;
-                lk = kap;
-              }
-            }
-          }
-          // warp-wide lexicographic minimum of (ld, lk); distances are >= 0 so their bits order like u64
-          const uint64_t bits = (uint64_t)__double_as_longlong(ld);
-          const uint32_t hi = (uint32_t)(bits >> 32), lo = (uint32_t)bits;
-          const uint32_t mhi = __reduce_min_sync(0xffffffffu, hi);
-          const uint32_t mlo = __reduce_min_sync(0xffffffffu, hi == mhi ? lo : 0xffffffffu);
-          const uint32_t mk = __reduce_min_sync(0xffffffffu, (hi == mhi && lo == mlo) ? lk : 0xffffffffu);
-          const uint32_t chosen = mk < kM2K ? mk : 0u;
-#pragma unroll
-          for (int bb = 0; bb < 8; ++bb)
-            if ((uint32_t)bb == b) beam_code[bb] = chosen;
-          if ((chosen & 31u) == (uint32_t)lane) member &= ~(1u << (chosen >> 5));
-        }
-      }
-    }
+      for (int i = 0; i < 8; ++i) nt2 = fmaf(t[i], t[i], nt2);
+      const float tnorm = sqrtf(nt2);
+      // twice the rounding-error bounds of the two fast scores (factor >= 2 to spare), u = 2^-24:
+      //   |score1_fl - score1| <= 16.1 u (||c1||^2/2 + ||t|| ||c1||)
+      //   |score2_fl - score2| <= 26 u (||t|| + max||c1|| + max||c2||)^2
+      const float margin1 = 3.8146973e-6f /* 2^-18 */ * (0.5f * n1max + tnorm * s1max) + 1e-30f;
+      const float sall = tnorm + s1max + s2max;
+      const float margin2 = 7.6293945e-6f /* 2^-17 */ * sall * sall + 1e-30f;
 
-    // ---- stage 2: every beam entry against codebook 2, running minimum only
-    float cm[8];
-#pragma unroll
-    for (int b = 0; b < 8; ++b) {
-      cm[b] = kInf;
-      if ((uint32_t)b < B) {
-        const float4 ca = *reinterpret_cast<const float4*>(&sm.c1[beam_code[b]][0]);
-        const float4 cb = *reinterpret_cast<const float4*>(&sm.c1[beam_code[b]][4]);
-        const float c1v[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
-        float r[8], rho = 0.0f;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          r[i] = __fsub_rn(t[i], c1v[i]);
-          rho = __fmaf_rn(r[i], r[i], rho);
-        }
-        rho = __fmul_rn(0.5f, rho);
-        const uint64_t rho2 = pack2(rho, rho);
+      // 256 scores, 8 per lane
+      float f[8];
+      {
         uint64_t acc[4];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) acc[q] = add2(h2p[q], rho2);
+        for (int qq = 0; qq < 4; ++qq) acc[qq] = sm.h1[qq][lane];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-          const uint64_t nrd = pack2(-r[i], -r[i]);
+          const uint64_t ntd = pack2(-t[i], -t[i]);
 #pragma unroll
-          for (int q = 0; q < 4; ++q) acc[q] = fma2(nrd, c2p[q][i], acc[q]);
+          for (int qq = 0; qq < 4; ++qq) acc[qq] = fma2(ntd, sm.p1[qq][i][lane], acc[qq]);
         }
-        float m = min3(lo_of(acc[0]), hi_of(acc[0]), lo_of(acc[1]));
-        m = min3(m, hi_of(acc[1]), lo_of(acc[2]));
-        m = min3(m, hi_of(acc[2]), lo_of(acc[3]));
-        cm[b] = fminf(m, hi_of(acc[3]));
+#pragma unroll
+        for (int qq = 0; qq < 4; ++qq) {
+          f[2 * qq] = lo_of(acc[qq]);
+          f[2 * qq + 1] = hi_of(acc[qq]);
+        }
+      }
+      // extract the B smallest (score truncated to 24 bits | code): a first guess of the beam
+      uint32_t key[8];
+#pragma unroll
+      for (int jj = 0; jj < 8; ++jj) key[jj] = (ord(f[jj]) & 0xffffff00u) | (uint32_t)(lane + 32 * jj);
+      uint32_t beam_code[8];
+#pragma unroll
+      for (int b = 0; b < 8; ++b) {
+        beam_code[b] = 0;
+        if ((uint32_t)b < B) {
+          uint32_t lm = key[0];
+#pragma unroll
+          for (int jj = 1; jj < 8; ++jj) lm = min(lm, key[jj]);
+          const uint32_t m = __reduce_min_sync(0xffffffffu, lm);
+          beam_code[b] = m & 0xffu;
+#pragma unroll
+          for (int jj = 0; jj < 8; ++jj)
+            if (key[jj] == m) key[jj] = 0xffffffffu;
+        }
+      }
+      // is that guess provably the exact beam?  theta = largest score in the guess;
+      // every member of the exact beam scores <= theta + margin1; if exactly B
+      // codewords do, they are the guess and the exact beam at once.
+      {
+        float th = -kInf;
+        uint32_t cnt = 0;
+#pragma unroll
+        for (int jj = 0; jj < 8; ++jj)
+          if (key[jj] == 0xffffffffu) th = fmaxf(th, f[jj]);
+        const float theta = unord(__reduce_max_sync(0xffffffffu, ord(th)));
+        const float limit1 = theta + margin1;
+        uint32_t member = 0;
+#pragma unroll
+        for (int jj = 0; jj < 8; ++jj) {
+          const bool in = f[jj] <= limit1 && (uint32_t)(lane + 32 * jj) < p.K;
+          member |= in ? (1u << jj) : 0u;
+          cnt += in;
+        }
+        cnt = __reduce_add_sync(0xffffffffu, cnt);
+        if (cnt != B) {
+          // undecided: order the shortlisted codewords by (binary64 distance, code)
+          for (uint32_t b = 0; b < B; ++b) {
+            double ld = __longlong_as_double(0x7ff0000000000000ll);
+            uint32_t lk = 0xffffffffu;
+#pragma unroll
+            for (int jj = 0; jj < 8; ++jj) {
+              if (member & (1u << jj)) {
+                const uint32_t kap = lane + 32 * jj;
+                const double d = exact1(t, sm.c1[kap]);
+                if (d < ld || (d == ld && kap < lk)) {
+                  ld = d;
+                  lk = kap;
+                }
+              }
+            }
+            // warp-wide lexicographic minimum of (ld, lk); distances are >= 0 so their bits order like u64
+            const uint64_t bits = (uint64_t)__double_as_longlong(ld);
+            const uint32_t hi = (uint32_t)(bits >> 32), lo = (uint32_t)bits;
+            const uint32_t mhi = __reduce_min_sync(0xffffffffu, hi);
+            const uint32_t mlo = __reduce_min_sync(0xffffffffu, hi == mhi ? lo : 0xffffffffu);
+            const uint32_t mk = __reduce_min_sync(0xffffffffu, (hi == mhi && lo == mlo) ? lk : 0xffffffffu);
+            const uint32_t chosen = mk < kM2K ? mk : 0u;
+#pragma unroll
+            for (int bb = 0; bb < 8; ++bb)
+              if ((uint32_t)bb == b) beam_code[bb] = chosen;
+            if ((chosen & 31u) == (uint32_t)lane) member &= ~(1u << (chosen >> 5));
+          }
+        }
+      }
+      // hand the target and its beam to the lanes of stage 2
+      if (lane == 0) {
+        *reinterpret_cast<float4*>(&sm.wt[warp][q][0]) = make_float4(t[0], t[1], t[2], t[3]);
+        *reinterpret_cast<float4*>(&sm.wt[warp][q][4]) = make_float4(t[4], t[5], t[6], t[7]);
+        *reinterpret_cast<uint4*>(&sm.wk[warp][q][0]) = make_uint4(beam_code[0], beam_code[1], beam_code[2], beam_code[3]);
+        *reinterpret_cast<uint4*>(&sm.wk[warp][q][4]) = make_uint4(beam_code[4], beam_code[5], beam_code[6], beam_code[7]);
+      }
+      if (my_q == q) {
+        my_j = j;
+        my_prev = prev;
+        my_margin2 = margin2;
       }
     }
-    float lmin = cm[0];
-#pragma unroll
-    for (int b = 1; b < 8; ++b) lmin = fminf(lmin, cm[b]);
-    const float limit2 = unord(__reduce_min_sync(0xffffffffu, ord(lmin))) + margin2;
+    __syncwarp();
 
-    // ---- decision in binary64 among the pairs within the margin, plus the previous pair
+    // ---- stage 2: lane = (target my_q, beam entry my_b) against all of codebook 2
+    const bool active = my_j != 0xffffffffu && my_b < B;
+    float t[8], c1v[8], r[8];
+    uint32_t k1 = 0;
+    {
+      const float4 ta = *reinterpret_cast<const float4*>(&sm.wt[warp][my_q][0]);
+      const float4 tb = *reinterpret_cast<const float4*>(&sm.wt[warp][my_q][4]);
+      t[0] = ta.x; t[1] = ta.y; t[2] = ta.z; t[3] = ta.w; t[4] = tb.x; t[5] = tb.y; t[6] = tb.z; t[7] = tb.w;
+      k1 = active ? sm.wk[warp][my_q][my_b] : 0u;
+      const float4 ca = *reinterpret_cast<const float4*>(&sm.c1[k1][0]);
+      const float4 cb = *reinterpret_cast<const float4*>(&sm.c1[k1][4]);
+      c1v[0] = ca.x; c1v[1] = ca.y; c1v[2] = ca.z; c1v[3] = ca.w; c1v[4] = cb.x; c1v[5] = cb.y; c1v[6] = cb.z; c1v[7] = cb.w;
+    }
+    float rho = 0.0f;
+    uint64_t nrd[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      r[i] = active ? __fsub_rn(t[i], c1v[i]) : 0.0f;
+      rho = __fmaf_rn(r[i], r[i], rho);
+      nrd[i] = pack2(-r[i], -r[i]);
+    }
+    rho = __fmul_rn(0.5f, rho);
+    const uint64_t rho2 = pack2(rho, rho);
+    float sub_min[8];
+#pragma unroll
+    for (int sub = 0; sub < 8; ++sub) {
+      float cmin = kInf;
+      const ulonglong2* vals = reinterpret_cast<const ulonglong2*>(&sm.x2[0][0]) + sub * 16 * 4;
+      const uint64_t* norms = reinterpret_cast<const uint64_t*>(&sm.hx2[0][0]) + sub * 16;
+#pragma unroll 4
+      for (int pr = 0; pr < 16; ++pr) {
+        const ulonglong2 q0 = vals[4 * pr], q1 = vals[4 * pr + 1], q2 = vals[4 * pr + 2], q3 = vals[4 * pr + 3];
+        uint64_t acc = add2(norms[pr], rho2);
+        acc = fma2(nrd[0], q0.x, acc);
+        acc = fma2(nrd[1], q0.y, acc);
+        acc = fma2(nrd[2], q1.x, acc);
+        acc = fma2(nrd[3], q1.y, acc);
+        acc = fma2(nrd[4], q2.x, acc);
+        acc = fma2(nrd[5], q2.y, acc);
+        acc = fma2(nrd[6], q3.x, acc);
+        acc = fma2(nrd[7], q3.y, acc);
+        cmin = min3(cmin, lo_of(acc), hi_of(acc));
+      }
+      sub_min[sub] = active ? cmin : kInf;
+    }
+    float gmin = sub_min[0];
+#pragma unroll
+    for (int sub = 1; sub < 8; ++sub) gmin = fminf(gmin, sub_min[sub]);
+#pragma unroll
+    for (int o = 1; o < 8; o <<= 1) gmin = fminf(gmin, __shfl_xor_sync(0xffffffffu, gmin, o));
+    const float limit2 = gmin + my_margin2;
+
+    // ---- decision in binary64 among the pairs within the margin, plus the previous pair.
+    // A sub-chunk within the margin is revisited by the whole warp, one codeword per lane, on behalf of the
+    // lane (target, beam entry) that found it; that lane keeps the best (distance, code pair).
     double bd = __longlong_as_double(0x7ff0000000000000ll);
     uint32_t bk = 0xffffffffu;  // code1 << 8 | code2: orders like (code1, code2)
 #pragma unroll
-    for (int b = 0; b < 8; ++b) {
-      if ((uint32_t)b < B && __any_sync(0xffffffffu, cm[b] <= limit2)) {
-        const uint32_t k1 = beam_code[b];
-        const float4 ca = *reinterpret_cast<const float4*>(&sm.c1[k1][0]);
-        const float4 cb = *reinterpret_cast<const float4*>(&sm.c1[k1][4]);
-        const float c1v[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
-        float r[8], rho = 0.0f;
+    for (int sub = 0; sub < 8; ++sub) {
+      uint32_t hits = __ballot_sync(0xffffffffu, sub_min[sub] <= limit2);  // false for inactive lanes
+      while (hits) {
+        const int src = __ffs(hits) - 1;
+        hits &= hits - 1;
+        const uint32_t sq = (uint32_t)src >> 3;
+        const uint32_t sk1 = __shfl_sync(0xffffffffu, k1, src);
+        const float slimit = __shfl_sync(0xffffffffu, limit2, src);
+        // the owner's target, codeword of codebook 1, residual and its half norm: the same operations
+        float st[8], sc1[8], sr[8], srho = 0.0f;
+        {
+          const float4 ta = *reinterpret_cast<const float4*>(&sm.wt[warp][sq][0]);
+          const float4 tb = *reinterpret_cast<const float4*>(&sm.wt[warp][sq][4]);
+          const float4 ca = *reinterpret_cast<const float4*>(&sm.c1[sk1][0]);
+          const float4 cb = *reinterpret_cast<const float4*>(&sm.c1[sk1][4]);
+          st[0] = ta.x; st[1] = ta.y; st[2] = ta.z; st[3] = ta.w; st[4] = tb.x; st[5] = tb.y; st[6] = tb.z; st[7] = tb.w;
+          sc1[0] = ca.x; sc1[1] = ca.y; sc1[2] = ca.z; sc1[3] = ca.w;
+          sc1[4] = cb.x; sc1[5] = cb.y; sc1[6] = cb.z; sc1[7] = cb.w;
+        }
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-          r[i] = __fsub_rn(t[i], c1v[i]);
-          rho = __fmaf_rn(r[i], r[i], rho);
+          sr[i] = __fsub_rn(st[i], sc1[i]);
+          srho = __fmaf_rn(sr[i], sr[i], srho);
         }
-        rho = __fmul_rn(0.5f, rho);
+        srho = __fmul_rn(0.5f, srho);
+        const uint32_t k2 = sub * 32 + lane;
+        float s2 = __fadd_rn(sm.h2[k2], srho);  // the same operations as the packed evaluation
 #pragma unroll
-        for (int jj = 0; jj < 8; ++jj) {
-          const uint32_t k2 = lane + 32 * jj;
-          float s = __fadd_rn(sm.h2[k2], rho);  // the same operations as the packed evaluation
-#pragma unroll
-          for (int i = 0; i < 8; ++i) s = __fmaf_rn(-r[i], sm.c2[k2][i], s);
-          if (s <= limit2 && k2 < p.K) {
-            const double d = exact2(t, c1v, sm.c2[k2]);
-            const uint32_t kk = (k1 << 8) | k2;
-            if (d < bd || (d == bd && kk < bk)) {
-              bd = d;
-              bk = kk;
+        for (int i = 0; i < 8; ++i) s2 = __fmaf_rn(-sr[i], sm.c2[k2][i], s2);
+        const bool cand = s2 <= slimit && k2 < p.K;
+        if (__any_sync(0xffffffffu, cand)) {
+          double d = __longlong_as_double(0x7ff0000000000000ll);
+          uint32_t kk = 0xffffffffu;
+          if (cand) {
+            d = exact2(st, sc1, sm.c2[k2]);
+            kk = (sk1 << 8) | k2;
+          }
+          // warp-wide lexicographic minimum of (d, kk); distances are >= 0 so their bits order like u64
+          const uint64_t bits = (uint64_t)__double_as_longlong(d);
+          const uint32_t hi = (uint32_t)(bits >> 32), lo = (uint32_t)bits;
+          const uint32_t mhi = __reduce_min_sync(0xffffffffu, hi);
+          const uint32_t mlo = __reduce_min_sync(0xffffffffu, hi == mhi ? lo : 0xffffffffu);
+          const uint32_t mk = __reduce_min_sync(0xffffffffu, (hi == mhi && lo == mlo) ? kk : 0xffffffffu);
+          if (lane == src) {
+            const double md = __longlong_as_double((long long)(((uint64_t)mhi << 32) | mlo));
+            if (md < bd || (md == bd && mk < bk)) {
+              bd = md;
+              bk = mk;
             }
           }
         }
       }
     }
-    // previous pair (lane 0 carries it into the reduction)
-    if (lane == 0) {
-      const uint32_t q1 = prev & 0xffu, q2 = prev >> 8;
+    if (my_b == 0 && my_j != 0xffffffffu) {  // the previous pair joins the pool
+      const uint32_t q1 = my_prev & 0xffu, q2 = my_prev >> 8;
       if (q1 < p.K && q2 < p.K) {
         const double d = exact2(t, sm.c1[q1], sm.c2[q2]);
         const uint32_t kk = (q1 << 8) | q2;
@@ -383,18 +454,24 @@ __global__ void __launch_bounds__(kM2Threads, 1) encode_m2_kernel(const EncM2Par
         atomicOr(p.status, PVT_DEV_BAD_CODE);
       }
     }
-    // warp-wide lexicographic minimum of (bd, bk)
-    {
+    // lexicographic minimum of (bd, bk) over the eight lanes of the target
+#pragma unroll
+    for (int o = 1; o < 8; o <<= 1) {
       const uint64_t bits = (uint64_t)__double_as_longlong(bd);
-      const uint32_t hi = (uint32_t)(bits >> 32), lo = (uint32_t)bits;
-      const uint32_t mhi = __reduce_min_sync(0xffffffffu, hi);
-      const uint32_t mlo = __reduce_min_sync(0xffffffffu, hi == mhi ? lo : 0xffffffffu);
-      const uint32_t mk = __reduce_min_sync(0xffffffffu, (hi == mhi && lo == mlo) ? bk : 0xffffffffu);
-      if (lane == 0 && mk != 0xffffffffu) {
-        p.codes[j] = (uint16_t)(((mk >> 8) & 0xffu) | ((mk & 0xffu) << 8));
-        if (p.err_out) p.err_out[n] = (float)__longlong_as_double((long long)(((uint64_t)mhi << 32) | mlo));
+      const uint32_t ohi = __shfl_xor_sync(0xffffffffu, (uint32_t)(bits >> 32), o);
+      const uint32_t olo = __shfl_xor_sync(0xffffffffu, (uint32_t)bits, o);
+      const uint32_t ok = __shfl_xor_sync(0xffffffffu, bk, o);
+      const double od = __longlong_as_double((long long)(((uint64_t)ohi << 32) | olo));
+      if (od < bd || (od == bd && ok < bk)) {
+        bd = od;
+        bk = ok;
       }
     }
+    if (my_b == 0 && my_j != 0xffffffffu && bk != 0xffffffffu) {
+      p.codes[my_j] = (uint16_t)(((bk >> 8) & 0xffu) | ((bk & 0xffu) << 8));
+      if (p.err_out) p.err_out[gi * kM2Group + my_q] = (float)bd;
+    }
+    __syncwarp();  // the group's scratch is rewritten by the next iteration
   }
 }
 
@@ -419,8 +496,9 @@ cudaError_t launch_encode_m2(const pvt_layer& L, uint64_t G, const uint32_t* idx
   p.err_out = err_out;
   p.status = reinterpret_cast<uint32_t*>(ws);
   const uint64_t warps_per_cta = kM2Threads / 32;
-  uint64_t ctas = (k + warps_per_cta - 1) / warps_per_cta;
-  if (ctas > (uint64_t)sm_count) ctas = (uint64_t)sm_count;
+  const uint64_t groups = (k + kM2Group - 1) / kM2Group;
+  uint64_t ctas = (groups + warps_per_cta - 1) / warps_per_cta;
+  if (ctas > 2 * (uint64_t)sm_count) ctas = 2 * (uint64_t)sm_count;  // two CTAs (16 warps) per SM
   timing_begin(kKernEncodeMain, stream);
   encode_m2_kernel<<<(unsigned)ctas, kM2Threads, 0, stream>>>(p);
   count_launches(1);
