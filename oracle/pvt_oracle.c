@@ -374,3 +374,57 @@ void pvt_oracle_dequant(const int32_t* codes, const float* books, const float* s
     }
   }
 }
+
+/* ---- P step, the part that shares its inputs with the V step ---------------------------------------------
+ * Algorithm 3, P-step lines: grad_codebooks = backprop(grad_phi); codebooks = adam(grad_codebooks)
+ * (Section 3.4: adaptive learning rates for the P step; Appendix J: beta1 = 0.9, beta2 = 0.95; codebooks and
+ * per-channel scales are the trainable continuous parameters of the representation).
+ *
+ * backprop is the chain rule through dequantize_weights, W_hat[r, dg*c + i] = s_r * v_{j,i},
+ * v_j = sum_m C_m[b_{j,m}] (the binary32 sum that dequantisation forms):
+ *     grad_codebooks[m][kappa][i] = sum over groups j with b_{j,m} = kappa of  s_{r(j)} * g[j][i]
+ *     grad_scale[r]               = sum over groups j of row r and over i of   g[j][i] * v_{j,i}
+ * Each product of two binary32 numbers is exact in binary64; the sums run in group order in binary64.
+ * Pins: automatic differentiation of the same forward map in a library, central finite differences of a
+ * quadratic phi, linearity in g, and the case of a single shared code (the gradient is the plain sum).
+ */
+void pvt_oracle_pstep_grad(const float* g, const float* scale, const int32_t* codes, const float* books,
+                           int64_t rows, int64_t cols, int32_t dg, int32_t M, int32_t K, double* grad_books,
+                           double* grad_scale) {
+  const int64_t gpr = cols / dg;
+  memset(grad_books, 0, sizeof(double) * (size_t)M * K * dg);
+  memset(grad_scale, 0, sizeof(double) * (size_t)rows);
+  for (int64_t j = 0; j < rows * gpr; ++j) {
+    const int64_t r = j / gpr, c = j % gpr;
+    const float* gj = g + r * cols + c * dg;
+    for (int32_t i = 0; i < dg; ++i) {
+      float v = books[((int64_t)0 * K + codes[j * M]) * dg + i];
+      for (int32_t q = 1; q < M; ++q) v = v + books[((int64_t)q * K + codes[j * M + q]) * dg + i];
+      grad_scale[r] += (double)gj[i] * (double)v;
+      for (int32_t q = 0; q < M; ++q)
+        grad_books[((int64_t)q * K + codes[j * M + q]) * dg + i] += (double)scale[r] * (double)gj[i];
+    }
+  }
+}
+
+/* One Adam update of n binary32 parameters (Kingma & Ba; Algorithm 3 "adam(grad_codebooks)").  The
+ * gradient arrives in binary64 and is rounded once to binary32; then, all in binary32, each operation
+ * rounded once, in this order:
+ *     m = fmaf(beta1, m, (1 - beta1) * gr)          v = fmaf(beta2, v, ((1 - beta2) * gr) * gr)
+ *     p = p - (lr * (m / bias1)) / (sqrtf(v / bias2) + eps)
+ * bias1 = 1 - beta1^t and bias2 = 1 - beta2^t are passed in (binary32) by the caller.
+ * Pins: a library Adam, and the closed form of the first step, lr * gr / (|gr| + eps). */
+void pvt_oracle_adam(float* param, const double* grad, float* exp_avg, float* exp_avg_sq, int64_t n, float lr,
+                     float beta1, float beta2, float eps, float bias1, float bias2) {
+  const float omb1 = 1.0f - beta1, omb2 = 1.0f - beta2;
+  for (int64_t i = 0; i < n; ++i) {
+    const float gr = (float)grad[i];
+    const float m = fmaf(beta1, exp_avg[i], omb1 * gr);
+    const float v = fmaf(beta2, exp_avg_sq[i], (omb2 * gr) * gr);
+    exp_avg[i] = m;
+    exp_avg_sq[i] = v;
+    const float num = lr * (m / bias1);
+    const float den = sqrtf(v / bias2) + eps;
+    param[i] = param[i] - num / den;
+  }
+}

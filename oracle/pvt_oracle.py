@@ -177,3 +177,41 @@ def vstep(W, g, scale, codebooks, codes, eta: float, k: int, beam: int = 8, idx=
     new_codes = codes2.copy()
     new_codes[idx.astype(np.int64)] = enc.codes.astype(codes.dtype)
     return VStepResult(idx, t, enc, new_codes.reshape(codes.shape))
+
+
+def pstep_grad(g, scale, codes, codebooks, rows: int, cols: int):
+    """Chain rule of dequantize_weights: (grad_codebooks fp64 [M, K, dg], grad_scale fp64 [rows])."""
+    g = _f32(g)
+    books = _f32(codebooks)
+    M, K, dg = books.shape
+    G = rows * (cols // dg)
+    codes = np.ascontiguousarray(np.asarray(codes).reshape(G, M), dtype=np.int32)
+    if codes.min() < 0 or codes.max() >= K:
+        raise ValueError("code out of range")
+    scale = _f32(scale)
+    gb = np.zeros((M, K, dg))
+    gs = np.zeros(rows)
+    lib().pvt_oracle_pstep_grad(_p(g, ctypes.c_float), _p(scale, ctypes.c_float), _p(codes, ctypes.c_int32),
+                                _p(books, ctypes.c_float), ctypes.c_int64(rows), ctypes.c_int64(cols),
+                                ctypes.c_int32(dg), ctypes.c_int32(M), ctypes.c_int32(K),
+                                _p(gb, ctypes.c_double), _p(gs, ctypes.c_double))
+    return gb, gs
+
+
+def adam(param, grad, exp_avg, exp_avg_sq, step: int, lr: float, beta1: float = 0.9, beta2: float = 0.95,
+         eps: float = 1e-8):
+    """One Adam update in place on fp32 arrays; returns (bias1, bias2) as used."""
+    assert param.dtype == np.float32 and exp_avg.dtype == np.float32 and exp_avg_sq.dtype == np.float32
+    grad = np.ascontiguousarray(grad, dtype=np.float64)
+    bias1, bias2 = adam_bias(step, beta1, beta2)
+    lib().pvt_oracle_adam(_p(param, ctypes.c_float), _p(grad, ctypes.c_double), _p(exp_avg, ctypes.c_float),
+                          _p(exp_avg_sq, ctypes.c_float), ctypes.c_int64(param.size), ctypes.c_float(lr),
+                          ctypes.c_float(beta1), ctypes.c_float(beta2), ctypes.c_float(eps),
+                          ctypes.c_float(bias1), ctypes.c_float(bias2))
+    return bias1, bias2
+
+
+def adam_bias(step: int, beta1: float, beta2: float):
+    """Bias corrections 1 - beta^t of step t >= 1: powers of the binary32 betas in binary64, rounded to binary32."""
+    b1, b2 = float(np.float32(beta1)), float(np.float32(beta2))
+    return float(np.float32(1.0 - b1 ** step)), float(np.float32(1.0 - b2 ** step))

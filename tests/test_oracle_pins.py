@@ -388,3 +388,95 @@ def test_config_1_all_groups_reencoded_matches_brute_force():
     d = ((t[:, None] - L.codebooks[0][None].astype(np.float64)) ** 2).sum(-1)
     decisive = (res.enc.d_second - res.enc.d_best) > 1e-6 * res.enc.d_second
     assert np.array_equal(d.argmin(1)[decisive], res.enc.codes[decisive, 0])
+
+
+# ------------------------------------------------------------------ P step: backprop to codebooks / scales, Adam
+
+
+def _pstep_case(seed, rows=12, cols=40, K=9, M=2):
+    rng = np.random.default_rng(seed)
+    g = rng.normal(size=(rows, cols)).astype(np.float32)
+    s = rng.uniform(0.5, 2.0, rows).astype(np.float32)
+    books = rng.normal(size=(M, K, 8)).astype(np.float32)
+    codes = rng.integers(0, K, (rows * cols // 8, M))
+    return g, s, books, codes, rows, cols
+
+
+def test_pstep_grad_equals_library_autodiff_of_dequantisation():
+    """Algorithm 3: grad_codebooks = backprop(grad_phi).  Differentiate <g, W_hat(codebooks, scales)> with a
+    library's reverse mode and compare (for M = 1 the forward map has no rounding, so the match is to fp64
+    accuracy; for M = 2 the checker differentiates through the binary32 sum of the two codewords)."""
+    import torch
+    for M, tol_s in ((1, 1e-12), (2, 1e-5)):
+        g, s, books, codes, rows, cols = _pstep_case(3 + M, M=M)
+        gb, gs = oracle.pstep_grad(g, s, codes, books, rows, cols)
+        Bk = torch.tensor(books, dtype=torch.float64, requires_grad=True)
+        S = torch.tensor(s, dtype=torch.float64, requires_grad=True)
+        c = torch.tensor(codes)
+        v = sum(Bk[m][c[:, m]] for m in range(M)).reshape(rows, cols // 8, 8)
+        W = (S[:, None, None] * v).reshape(rows, cols)
+        (W * torch.tensor(g, dtype=torch.float64)).sum().backward()
+        assert np.abs(gb - Bk.grad.numpy()).max() <= 1e-12 * np.abs(gb).max()
+        assert np.abs(gs - S.grad.numpy()).max() <= tol_s * np.abs(gs).max()
+
+
+def test_pstep_grad_matches_finite_differences_of_a_quadratic():
+    """phi(W_hat) = 1/2 ||W_hat - Z||^2 has gradient W_hat - Z; perturb single codebook entries and scales."""
+    g0, s, books, codes, rows, cols = _pstep_case(11, M=1)
+    Z = g0  # any matrix
+    def phi(bk, sc):
+        W = oracle.dequant(codes, bk, sc, rows, cols).astype(np.float64)
+        return 0.5 * ((W - Z) ** 2).sum()
+    W0 = oracle.dequant(codes, books, s, rows, cols)
+    g = (W0.astype(np.float64) - Z).astype(np.float32)
+    gb, gs = oracle.pstep_grad(g, s, codes, books, rows, cols)
+    h = 1e-2  # phi is quadratic: the central difference is exact up to rounding
+    for (kap, i) in ((0, 0), (3, 5), (8, 7)):
+        bp, bm = books.copy(), books.copy()
+        bp[0, kap, i] += h
+        bm[0, kap, i] -= h
+        fd = (phi(bp, s) - phi(bm, s)) / (float(bp[0, kap, i]) - float(bm[0, kap, i]))
+        assert abs(fd - gb[0, kap, i]) <= 2e-3 * max(1.0, abs(fd))
+    for r in (0, 7):
+        sp, sm = s.copy(), s.copy()
+        sp[r] += h
+        sm[r] -= h
+        fd = (phi(books, sp) - phi(books, sm)) / (float(sp[r]) - float(sm[r]))
+        assert abs(fd - gs[r]) <= 2e-3 * max(1.0, abs(fd))
+
+
+def test_pstep_grad_linearity_and_single_code():
+    g, s, books, codes, rows, cols = _pstep_case(13, M=2)
+    gb1, gs1 = oracle.pstep_grad(g, s, codes, books, rows, cols)
+    gb2, gs2 = oracle.pstep_grad(2 * g, s, codes, books, rows, cols)  # doubling is exact in binary32
+    assert np.array_equal(gb2, 2 * gb1) and np.array_equal(gs2, 2 * gs1)
+    # every group uses code (4, 4): the gradient of that codeword is the scaled column-group sum, all others zero
+    codes[:] = 4
+    gb, _ = oracle.pstep_grad(g, s, codes, books, rows, cols)
+    want = (s[:, None].astype(np.float64) * g.astype(np.float64)).reshape(rows, cols // 8, 8).sum(axis=(0, 1))
+    assert np.allclose(gb[0, 4], want, rtol=1e-13, atol=1e-13) and np.allclose(gb[1, 4], want, rtol=1e-13, atol=1e-13)
+    gb[:, 4] = 0
+    assert not gb.any()
+
+
+def test_adam_first_step_closed_form_and_library():
+    """First step from zero moments: update = lr * g / (|g| + eps) whatever the betas; further steps against
+    a library Adam (Appendix J: beta1 = 0.9, beta2 = 0.95)."""
+    import torch
+    rng = np.random.default_rng(17)
+    n = 1000
+    p0 = rng.normal(size=n).astype(np.float32)
+    grads = [rng.normal(size=n) * 10.0 ** rng.integers(-3, 2, n) for _ in range(4)]
+    p, m, v = p0.copy(), np.zeros(n, np.float32), np.zeros(n, np.float32)
+    oracle.adam(p, grads[0], m, v, 1, 3e-4)
+    g32 = grads[0].astype(np.float32).astype(np.float64)
+    want = p0 - 3e-4 * g32 / (np.abs(g32) + 1e-8)
+    assert np.allclose(p, want, rtol=0, atol=2e-7 * np.abs(p0).max() + 1e-9)
+    tp = torch.tensor(p0, dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.Adam([tp], lr=3e-4, betas=(0.9, 0.95), eps=1e-8)
+    p, m, v = p0.copy(), np.zeros(n, np.float32), np.zeros(n, np.float32)
+    for t, gr in enumerate(grads, 1):
+        oracle.adam(p, gr, m, v, t, 3e-4)
+        tp.grad = torch.tensor(gr.astype(np.float32).astype(np.float64))
+        opt.step()
+    assert np.allclose(p, tp.detach().numpy(), rtol=0, atol=4e-7 * np.abs(p0).max() + 1e-8)
