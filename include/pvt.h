@@ -181,6 +181,36 @@ int pvt_vstep_encode(const pvt_layer* layer, const uint32_t* idx, uint64_t k, fl
 int pvt_dequant(const pvt_layer* layer, void* W_hat, int32_t out_dtype, uint32_t* status, void* cuda_stream);
 
 /*
+ * P step, the half that shares its inputs with the V step (Algorithm 3, P-step lines:
+ * grad_codebooks = backprop(grad_phi)).  Chain rule through dequantize_weights,
+ * W_hat[r, 8c+i] = scale[r] * v[j][i], v[j] = sum_m C_m[codes[j][m]] (the binary32 sum
+ * pvt_dequant forms):
+ *   grad_codebooks[m][kappa][i] = sum over groups j with codes[j][m] == kappa of scale[r(j)] * g[j][i]
+ *   grad_scale[r]               = sum over the groups j of row r and over i of g[j][i] * v[j][i]
+ * Products are exact in binary64; sums are accumulated in binary64 by atomic adds, so
+ * results vary from run to run in the order of binary64 roundings only.
+ * Reads layer->g, scale, codes, codebooks, shape.  grad_codebooks: device, M*K*8 doubles;
+ * grad_scale: device, rows doubles, or NULL.  Both are overwritten.  `status` may be NULL
+ * or a device uint32 into which PVT_DEV_BAD_CODE is OR-ed (such groups contribute nothing).
+ */
+int pvt_pstep_grad(const pvt_layer* layer, double* grad_codebooks, double* grad_scale, uint32_t* status,
+                   void* cuda_stream);
+
+/*
+ * One Adam update of n binary32 parameters (Algorithm 3: codebooks = adam(grad_codebooks);
+ * Section 3.4; Appendix J: beta1 = 0.9, beta2 = 0.95).  The binary64 gradient is rounded
+ * once to binary32 (gr); then, in binary32, every operation rounded once:
+ *   m = fma(beta1, m, (1 - beta1) * gr)        v = fma(beta2, v, ((1 - beta2) * gr) * gr)
+ *   p = p - (lr * (m / bias1)) / (sqrt(v / bias2) + eps)
+ * with bias1 = 1 - beta1^t, bias2 = 1 - beta2^t of step t >= 1 supplied by the caller.
+ * param, exp_avg, exp_avg_sq: device, n floats, updated in place.  param_f16: NULL, or
+ * device n halves that receive the updated parameters rounded to nearest-even (the
+ * fp16 codebook the V step reads).  grad: device, n doubles.
+ */
+int pvt_adam_update(float* param, void* param_f16, const double* grad, float* exp_avg, float* exp_avg_sq, uint64_t n,
+                    float lr, float beta1, float beta2, float eps, float bias1, float bias2, void* cuda_stream);
+
+/*
  * Synchronises the stream, returns the PVT_DEV_* bits accumulated in the
  * workspace since the last pvt_status / pvt_workspace_init (>= 0) and clears them;
  * or PVT_ECUDA.
@@ -220,6 +250,8 @@ void pvt_set_m1_search(int mode);
 #define PVT_KERNEL_ENCODE_AUX 2  /* codebook expansion before the M = 1 search */
 #define PVT_KERNEL_DEQUANT 3     /* the kernel of pvt_dequant */
 #define PVT_KERNEL_ENCODE_RESCORE 4 /* exact rescoring and code write after the M = 1 search */
+#define PVT_KERNEL_PSTEP_GRAD 5  /* the kernel of pvt_pstep_grad */
+#define PVT_KERNEL_ADAM 6        /* the kernel of pvt_adam_update */
 void pvt_timing_enable(int on);
 /* Kernels this process has launched through the library so far (memsets not counted). */
 unsigned long long pvt_launch_count(void);

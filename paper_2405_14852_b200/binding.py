@@ -23,6 +23,7 @@ PVT_NOALLOC_MAX_GROUPS = 1 << 21
 PVT_DEV_BAD_INDEX, PVT_DEV_BAD_CODE, PVT_DEV_WAIT_EXPIRED, PVT_DEV_INTERNAL = 1, 2, 4, 8
 PVT_KERNEL_SELECT, PVT_KERNEL_ENCODE_MAIN, PVT_KERNEL_ENCODE_AUX, PVT_KERNEL_DEQUANT = 0, 1, 2, 3
 PVT_KERNEL_ENCODE_RESCORE = 4
+PVT_KERNEL_PSTEP_GRAD, PVT_KERNEL_ADAM = 5, 6
 PVT_M1_AUTO, PVT_M1_FP32, PVT_M1_TENSOR = 0, 1, 2
 
 
@@ -77,6 +78,11 @@ def lib():
         L.pvt_vstep_encode.argtypes = [lp, vp, u64, vp, vp, sz, vp]
         L.pvt_dequant.restype = ctypes.c_int
         L.pvt_dequant.argtypes = [lp, vp, ctypes.c_int32, vp, vp]
+        L.pvt_pstep_grad.restype = ctypes.c_int
+        L.pvt_pstep_grad.argtypes = [lp, vp, vp, vp, vp]
+        L.pvt_adam_update.restype = ctypes.c_int
+        fl = ctypes.c_float
+        L.pvt_adam_update.argtypes = [vp, vp, vp, vp, vp, u64, fl, fl, fl, fl, fl, fl, vp]
         L.pvt_status.restype = ctypes.c_int
         L.pvt_status.argtypes = [vp, vp]
         L.pvt_strerror.restype = ctypes.c_char_p
@@ -175,6 +181,33 @@ def pvt_dequant(layer: pvt_layer, W_hat: torch.Tensor, status: Optional[torch.Te
     out_dtype = {torch.float32: PVT_F32, torch.float16: PVT_F16}[W_hat.dtype]
     _check(lib().pvt_dequant(ctypes.byref(layer), W_hat.data_ptr(), out_dtype, _ptr(status), _stream_ptr(stream)),
            "pvt_dequant")
+
+
+def pvt_pstep_grad(layer: pvt_layer, grad_codebooks: torch.Tensor, grad_scale: Optional[torch.Tensor] = None,
+                   status: Optional[torch.Tensor] = None, stream=None) -> None:
+    """grad_codebooks [M, K, 8] float64, grad_scale [rows] float64 or None (both overwritten)."""
+    assert grad_codebooks.dtype == torch.float64 and (grad_scale is None or grad_scale.dtype == torch.float64)
+    _check(lib().pvt_pstep_grad(ctypes.byref(layer), grad_codebooks.data_ptr(), _ptr(grad_scale), _ptr(status),
+                                _stream_ptr(stream)), "pvt_pstep_grad")
+
+
+def adam_bias(step: int, beta1: float, beta2: float):
+    """Bias corrections 1 - beta^t of step t >= 1 as the binary32 numbers pvt_adam_update takes."""
+    f32 = lambda x: ctypes.c_float(x).value
+    return f32(1.0 - f32(beta1) ** step), f32(1.0 - f32(beta2) ** step)
+
+
+def pvt_adam_update(param: torch.Tensor, grad: torch.Tensor, exp_avg: torch.Tensor, exp_avg_sq: torch.Tensor,
+                    step: int, lr: float, beta1: float = 0.9, beta2: float = 0.95, eps: float = 1e-8,
+                    param_f16: Optional[torch.Tensor] = None, stream=None) -> None:
+    """One Adam update in place (param, exp_avg, exp_avg_sq float32; grad float64; optional float16 copy)."""
+    assert param.dtype == torch.float32 and grad.dtype == torch.float64
+    assert exp_avg.dtype == torch.float32 and exp_avg_sq.dtype == torch.float32
+    assert param_f16 is None or param_f16.dtype == torch.float16
+    bias1, bias2 = adam_bias(step, beta1, beta2)
+    _check(lib().pvt_adam_update(param.data_ptr(), _ptr(param_f16), grad.data_ptr(), exp_avg.data_ptr(),
+                                 exp_avg_sq.data_ptr(), param.numel(), lr, beta1, beta2, eps, bias1, bias2,
+                                 _stream_ptr(stream)), "pvt_adam_update")
 
 
 def pvt_status(ws: torch.Tensor, stream=None) -> int:

@@ -184,6 +184,34 @@ int pvt_dequant(const pvt_layer* layer, void* W_hat, int32_t out_dtype, uint32_t
   return e == cudaSuccess ? PVT_OK : fail_cuda(e);
 }
 
+int pvt_pstep_grad(const pvt_layer* layer, double* grad_codebooks, double* grad_scale, uint32_t* status,
+                   void* cuda_stream) {
+  uint64_t G = 0;
+  int rc = check_layer(layer, &G);
+  if (rc != PVT_OK) return rc;
+  if ((rc = check_quantiser(layer)) != PVT_OK) return rc;
+  if (!layer->g || !layer->scale || !layer->codebooks || !layer->codes || !grad_codebooks) return PVT_EINVAL;
+  if (!aligned16(layer->g) || !aligned16(layer->codebooks)) return PVT_EINVAL;
+  if ((reinterpret_cast<uintptr_t>(grad_codebooks) & 7u) || (reinterpret_cast<uintptr_t>(grad_scale) & 7u))
+    return PVT_EINVAL;
+  if (layer->num_codebooks == 2 && layer->code_dtype == PVT_U8 && (reinterpret_cast<uintptr_t>(layer->codes) & 1u))
+    return PVT_EINVAL;
+  const cudaError_t e = launch_pstep_grad(*layer, G, grad_codebooks, grad_scale, status, sm_count(),
+                                          static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? PVT_OK : fail_cuda(e);
+}
+
+int pvt_adam_update(float* param, void* param_f16, const double* grad, float* exp_avg, float* exp_avg_sq, uint64_t n,
+                    float lr, float beta1, float beta2, float eps, float bias1, float bias2, void* cuda_stream) {
+  if (!param || !grad || !exp_avg || !exp_avg_sq || n == 0) return PVT_EINVAL;
+  if (!(lr >= 0.0f) || !(beta1 >= 0.0f && beta1 < 1.0f) || !(beta2 >= 0.0f && beta2 < 1.0f) || !(eps >= 0.0f))
+    return PVT_EINVAL;
+  if (!(bias1 > 0.0f && bias1 <= 1.0f) || !(bias2 > 0.0f && bias2 <= 1.0f)) return PVT_EINVAL;
+  const cudaError_t e = launch_adam(param, param_f16, grad, exp_avg, exp_avg_sq, n, lr, beta1, beta2, eps, bias1, bias2,
+                                    sm_count(), static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? PVT_OK : fail_cuda(e);
+}
+
 int pvt_status(void* ws, void* cuda_stream) {
   if (!ws) return PVT_EINVAL;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);

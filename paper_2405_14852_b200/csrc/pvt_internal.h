@@ -113,9 +113,16 @@ cudaError_t launch_encode_m2(const pvt_layer& L, uint64_t G, const uint32_t* idx
 cudaError_t launch_dequant(const pvt_layer& L, uint64_t G, void* W_hat, int32_t out_dtype, uint32_t* status,
                            int sm_count, cudaStream_t stream);
 
+cudaError_t launch_pstep_grad(const pvt_layer& L, uint64_t G, double* grad_books, double* grad_scale, uint32_t* status,
+                              int sm_count, cudaStream_t stream);
+cudaError_t launch_adam(float* param, void* param_f16, const double* grad, float* exp_avg, float* exp_avg_sq,
+                        uint64_t n, float lr, float beta1, float beta2, float eps, float bias1, float bias2,
+                        int sm_count, cudaStream_t stream);
+
 // optional per-kernel timing (benchmark instrumentation) ----------------------
 enum KernelId {
-  kKernSelect = 0, kKernEncodeMain = 1, kKernEncodeAux = 2, kKernDequant = 3, kKernEncodeRescore = 4, kKernCount = 5
+  kKernSelect = 0, kKernEncodeMain = 1, kKernEncodeAux = 2, kKernDequant = 3, kKernEncodeRescore = 4,
+  kKernPstepGrad = 5, kKernAdam = 6, kKernCount = 7
 };
 void timing_begin(KernelId id, cudaStream_t stream);
 void timing_end(KernelId id, cudaStream_t stream);
