@@ -428,3 +428,25 @@ void pvt_oracle_adam(float* param, const double* grad, float* exp_avg, float* ex
     param[i] = param[i] - num / den;
   }
 }
+
+/* Update direction of the V step as the paper runs it (Section 3.4: grad phi(y) in Eq. 8 is replaced by a single
+ * Adam update; Algorithm 3, V-step line "update = adam(grad_phi) ..."; the subspace is then chosen by the
+ * magnitude of this update).  Moments as in Adam; the direction is the bias-corrected ratio, all in binary32,
+ * every operation rounded once:
+ *     m = fmaf(beta1, m, (1 - beta1) * g)        v = fmaf(beta2, v, ((1 - beta2) * g) * g)
+ *     u = (m / bias1) / (sqrtf(v / bias2) + eps)
+ * The V step then runs on (W, u, eta = learning rate of the codes).
+ * Pins: the first step's closed form g / (|g| + eps), and a library Adam with learning rate 1 started at 0,
+ * whose parameter is minus the accumulated directions. */
+void pvt_oracle_adam_direction(const float* grad, float* exp_avg, float* exp_avg_sq, float* dir, int64_t n,
+                               float beta1, float beta2, float eps, float bias1, float bias2) {
+  const float omb1 = 1.0f - beta1, omb2 = 1.0f - beta2;
+  for (int64_t i = 0; i < n; ++i) {
+    const float gr = grad[i];
+    const float m = fmaf(beta1, exp_avg[i], omb1 * gr);
+    const float v = fmaf(beta2, exp_avg_sq[i], (omb2 * gr) * gr);
+    exp_avg[i] = m;
+    exp_avg_sq[i] = v;
+    dir[i] = (m / bias1) / (sqrtf(v / bias2) + eps);
+  }
+}

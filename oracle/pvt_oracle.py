@@ -215,3 +215,17 @@ def adam_bias(step: int, beta1: float, beta2: float):
     """Bias corrections 1 - beta^t of step t >= 1: powers of the binary32 betas in binary64, rounded to binary32."""
     b1, b2 = float(np.float32(beta1)), float(np.float32(beta2))
     return float(np.float32(1.0 - b1 ** step)), float(np.float32(1.0 - b2 ** step))
+
+
+def adam_direction(grad, exp_avg, exp_avg_sq, step: int, beta1: float = 0.9, beta2: float = 0.95,
+                   eps: float = 1e-8) -> np.ndarray:
+    """Adam-normalised update direction (fp32), moments updated in place."""
+    grad = _f32(grad)
+    assert exp_avg.dtype == np.float32 and exp_avg_sq.dtype == np.float32
+    out = np.empty(grad.shape, dtype=np.float32)
+    bias1, bias2 = adam_bias(step, beta1, beta2)
+    lib().pvt_oracle_adam_direction(_p(grad, ctypes.c_float), _p(exp_avg, ctypes.c_float),
+                                    _p(exp_avg_sq, ctypes.c_float), _p(out, ctypes.c_float),
+                                    ctypes.c_int64(grad.size), ctypes.c_float(beta1), ctypes.c_float(beta2),
+                                    ctypes.c_float(eps), ctypes.c_float(bias1), ctypes.c_float(bias2))
+    return out

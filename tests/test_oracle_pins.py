@@ -480,3 +480,25 @@ def test_adam_first_step_closed_form_and_library():
         tp.grad = torch.tensor(gr.astype(np.float32).astype(np.float64))
         opt.step()
     assert np.allclose(p, tp.detach().numpy(), rtol=0, atol=4e-7 * np.abs(p0).max() + 1e-8)
+
+
+def test_adam_direction_first_step_and_library():
+    """Section 3.4: the V step's gradient is replaced by one Adam update.  First step: g / (|g| + eps); over
+    several steps a library Adam with learning rate 1 started at zero accumulates minus the directions."""
+    import torch
+    rng = np.random.default_rng(19)
+    n = 500
+    grads = [(rng.normal(size=n) * 10.0 ** rng.integers(-3, 2, n)).astype(np.float32) for _ in range(4)]
+    m, v = np.zeros(n, np.float32), np.zeros(n, np.float32)
+    u = oracle.adam_direction(grads[0], m, v, 1)
+    g64 = grads[0].astype(np.float64)
+    assert np.allclose(u, g64 / (np.abs(g64) + 1e-8), rtol=3e-7, atol=0)
+    tp = torch.zeros(n, dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.Adam([tp], lr=1.0, betas=(0.9, 0.95), eps=1e-8)
+    m, v = np.zeros(n, np.float32), np.zeros(n, np.float32)
+    acc = np.zeros(n)
+    for t, gr in enumerate(grads, 1):
+        acc += oracle.adam_direction(gr, m, v, t).astype(np.float64)
+        tp.grad = torch.tensor(gr.astype(np.float64))
+        opt.step()
+    assert np.allclose(-acc, tp.detach().numpy(), rtol=2e-6, atol=1e-7)
