@@ -501,4 +501,5 @@ def test_adam_direction_first_step_and_library():
         acc += oracle.adam_direction(gr, m, v, t).astype(np.float64)
         tp.grad = torch.tensor(gr.astype(np.float64))
         opt.step()
-    assert np.allclose(-acc, tp.detach().numpy(), rtol=2e-6, atol=1e-7)
+    # directions are O(1) and each carries a few binary32 roundings; their sum may cancel, so the bound is absolute
+    assert np.allclose(-acc, tp.detach().numpy(), rtol=0, atol=2e-6)
