@@ -211,6 +211,21 @@ int pvt_adam_update(float* param, void* param_f16, const double* grad, float* ex
                     float lr, float beta1, float beta2, float eps, float bias1, float bias2, void* cuda_stream);
 
 /*
+ * Update direction of the V step as the paper runs it (Section 3.4: grad phi(y) of Eq. 8 is
+ * replaced by a single Adam update, and the subspace is chosen by the magnitude of that
+ * update; Algorithm 3, V-step line "update = adam(grad_phi) ...").  Per weight, binary32,
+ * every operation rounded once:
+ *   m = fma(beta1, m, (1 - beta1) * g)        v = fma(beta2, v, ((1 - beta2) * g) * g)
+ *   dir = (m / bias1) / (sqrt(v / bias2) + eps)
+ * The V step then runs with layer->g = dir and layer->eta = the learning rate of the codes.
+ * grad, exp_avg, exp_avg_sq, dir: device, n floats, 16-byte aligned, n % 4 == 0 (n = rows *
+ * cols of a layer); exp_avg and exp_avg_sq are updated in place; dir may alias grad.
+ * bias1 = 1 - beta1^t, bias2 = 1 - beta2^t of step t >= 1.
+ */
+int pvt_adam_direction(const float* grad, float* exp_avg, float* exp_avg_sq, float* dir, uint64_t n, float beta1,
+                       float beta2, float eps, float bias1, float bias2, void* cuda_stream);
+
+/*
  * Synchronises the stream, returns the PVT_DEV_* bits accumulated in the
  * workspace since the last pvt_status / pvt_workspace_init (>= 0) and clears them;
  * or PVT_ECUDA.

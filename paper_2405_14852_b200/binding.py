@@ -83,6 +83,8 @@ def lib():
         L.pvt_adam_update.restype = ctypes.c_int
         fl = ctypes.c_float
         L.pvt_adam_update.argtypes = [vp, vp, vp, vp, vp, u64, fl, fl, fl, fl, fl, fl, vp]
+        L.pvt_adam_direction.restype = ctypes.c_int
+        L.pvt_adam_direction.argtypes = [vp, vp, vp, vp, u64, fl, fl, fl, fl, fl, vp]
         L.pvt_status.restype = ctypes.c_int
         L.pvt_status.argtypes = [vp, vp]
         L.pvt_strerror.restype = ctypes.c_char_p
@@ -208,6 +210,17 @@ def pvt_adam_update(param: torch.Tensor, grad: torch.Tensor, exp_avg: torch.Tens
     _check(lib().pvt_adam_update(param.data_ptr(), _ptr(param_f16), grad.data_ptr(), exp_avg.data_ptr(),
                                  exp_avg_sq.data_ptr(), param.numel(), lr, beta1, beta2, eps, bias1, bias2,
                                  _stream_ptr(stream)), "pvt_adam_update")
+
+
+def pvt_adam_direction(grad: torch.Tensor, exp_avg: torch.Tensor, exp_avg_sq: torch.Tensor, out: torch.Tensor,
+                       step: int, beta1: float = 0.9, beta2: float = 0.95, eps: float = 1e-8, stream=None) -> None:
+    """Adam-normalised update direction of the V step (all float32; moments updated in place)."""
+    for t in (grad, exp_avg, exp_avg_sq, out):
+        assert t.dtype == torch.float32 and t.is_contiguous()
+    bias1, bias2 = adam_bias(step, beta1, beta2)
+    _check(lib().pvt_adam_direction(grad.data_ptr(), exp_avg.data_ptr(), exp_avg_sq.data_ptr(), out.data_ptr(),
+                                    grad.numel(), beta1, beta2, eps, bias1, bias2, _stream_ptr(stream)),
+           "pvt_adam_direction")
 
 
 def pvt_status(ws: torch.Tensor, stream=None) -> int:

@@ -212,6 +212,17 @@ int pvt_adam_update(float* param, void* param_f16, const double* grad, float* ex
   return e == cudaSuccess ? PVT_OK : fail_cuda(e);
 }
 
+int pvt_adam_direction(const float* grad, float* exp_avg, float* exp_avg_sq, float* dir, uint64_t n, float beta1,
+                       float beta2, float eps, float bias1, float bias2, void* cuda_stream) {
+  if (!grad || !exp_avg || !exp_avg_sq || !dir || n == 0 || n % 4 != 0) return PVT_EINVAL;
+  if (!aligned16(grad) || !aligned16(exp_avg) || !aligned16(exp_avg_sq) || !aligned16(dir)) return PVT_EINVAL;
+  if (!(beta1 >= 0.0f && beta1 < 1.0f) || !(beta2 >= 0.0f && beta2 < 1.0f) || !(eps >= 0.0f)) return PVT_EINVAL;
+  if (!(bias1 > 0.0f && bias1 <= 1.0f) || !(bias2 > 0.0f && bias2 <= 1.0f)) return PVT_EINVAL;
+  const cudaError_t e = launch_adam_direction(grad, exp_avg, exp_avg_sq, dir, n, beta1, beta2, eps, bias1, bias2,
+                                              sm_count(), static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? PVT_OK : fail_cuda(e);
+}
+
 int pvt_status(void* ws, void* cuda_stream) {
   if (!ws) return PVT_EINVAL;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);

@@ -119,6 +119,10 @@ cudaError_t launch_adam(float* param, void* param_f16, const double* grad, float
                         uint64_t n, float lr, float beta1, float beta2, float eps, float bias1, float bias2,
                         int sm_count, cudaStream_t stream);
 
+cudaError_t launch_adam_direction(const float* grad, float* exp_avg, float* exp_avg_sq, float* dir, uint64_t n,
+                                  float beta1, float beta2, float eps, float bias1, float bias2, int sm_count,
+                                  cudaStream_t stream);
+
 // optional per-kernel timing (benchmark instrumentation) ----------------------
 enum KernelId {
   kKernSelect = 0, kKernEncodeMain = 1, kKernEncodeAux = 2, kKernDequant = 3, kKernEncodeRescore = 4,

@@ -178,7 +178,45 @@ __global__ void __launch_bounds__(256) adam_kernel(float* __restrict__ param, __
   }
 }
 
+// Adam-normalised update direction of the V step (Section 3.4): moments as in Adam, u = (m / bias1) /
+// (sqrt(v / bias2) + eps), binary32, each operation rounded once.  Four elements per thread (128-bit accesses).
+__global__ void __launch_bounds__(256) adam_direction_kernel(const float4* __restrict__ grad, float4* __restrict__ exp_avg,
+                                                              float4* __restrict__ exp_avg_sq, float4* __restrict__ dir,
+                                                              uint64_t n4, float beta1, float beta2, float eps,
+                                                              float bias1, float bias2) {
+  const float omb1 = __fsub_rn(1.0f, beta1), omb2 = __fsub_rn(1.0f, beta2);
+  auto one = [&](float gr, float& m, float& v) {
+    m = __fmaf_rn(beta1, m, __fmul_rn(omb1, gr));
+    v = __fmaf_rn(beta2, v, __fmul_rn(__fmul_rn(omb2, gr), gr));
+    return __fdiv_rn(__fdiv_rn(m, bias1), __fadd_rn(__fsqrt_rn(__fdiv_rn(v, bias2)), eps));
+  };
+  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (uint64_t)gridDim.x * blockDim.x) {
+    const float4 g = __ldcs(grad + i);
+    float4 m = exp_avg[i], v = exp_avg_sq[i], u;
+    u.x = one(g.x, m.x, v.x);
+    u.y = one(g.y, m.y, v.y);
+    u.z = one(g.z, m.z, v.z);
+    u.w = one(g.w, m.w, v.w);
+    exp_avg[i] = m;
+    exp_avg_sq[i] = v;
+    dir[i] = u;
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_adam_direction(const float* grad, float* exp_avg, float* exp_avg_sq, float* dir, uint64_t n,
+                                  float beta1, float beta2, float eps, float bias1, float bias2, int sm_count,
+                                  cudaStream_t stream) {
+  timing_begin(kKernAdam, stream);
+  const uint64_t n4 = n / 4, want = (n4 + 255) / 256, cap = (uint64_t)sm_count * 8;
+  adam_direction_kernel<<<(unsigned)(want < cap ? want : cap), 256, 0, stream>>>(
+      reinterpret_cast<const float4*>(grad), reinterpret_cast<float4*>(exp_avg), reinterpret_cast<float4*>(exp_avg_sq),
+      reinterpret_cast<float4*>(dir), n4, beta1, beta2, eps, bias1, bias2);
+  count_launches(1);
+  timing_end(kKernAdam, stream);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_pstep_grad(const pvt_layer& L, uint64_t G, double* grad_books, double* grad_scale, uint32_t* status,
                               int sm_count, cudaStream_t stream) {

@@ -114,3 +114,37 @@ def test_p_step_then_v_step_round_trip():
     import helpers
     got_codes = dev.codes.cpu().numpy().reshape(-1, 1)
     helpers.check_codes_against_oracle(ref.t, got_books, got_codes[ref.idx.astype(np.int64)], ref.enc, 1e-6)
+
+
+def test_adam_direction_bit_exact_and_v_step_on_it():
+    """Section 3.4: the V step runs on the Adam-normalised update.  The direction kernel is bit-exact against
+    the checker; a V step with g := direction and eta := the learning rate of the codes matches the checker's
+    V step on the same direction."""
+    L = synth.make_layer(256, 512, cfg=122, codebook_size=2048, codebook_fp16=True)
+    n = L.g.size
+    m, v = np.zeros(n, np.float32), np.zeros(n, np.float32)
+    dm, dv = torch.zeros(n, device="cuda"), torch.zeros(n, device="cuda")
+    dgrad = torch.from_numpy(L.g.reshape(-1).copy()).cuda()
+    ddir = torch.empty(n, device="cuda")
+    rng = np.random.default_rng(123)
+    for step in (1, 2, 3):
+        grad = (L.g.reshape(-1) * rng.uniform(0.5, 1.5, n)).astype(np.float32)
+        want = oracle.adam_direction(grad, m, v, step)
+        dgrad.copy_(torch.from_numpy(grad))
+        B.pvt_adam_direction(dgrad, dm, dv, ddir, step)
+        torch.cuda.synchronize()
+        assert ddir.cpu().numpy().tobytes() == want.tobytes()
+        assert dm.cpu().numpy().tobytes() == m.tobytes() and dv.cpu().numpy().tobytes() == v.tobytes()
+    # V step on the direction with the codes' learning rate (Appendix J: 3e-3)
+    L.g = want.reshape(L.g.shape)
+    L.eta = 3e-3
+    k = synth.subspace_size("0.01", L.num_groups)
+    ref = oracle.vstep(L.W, L.g, L.scale, L.codebooks, L.codes, L.eta, k, L.beam)
+    dev = VStepLayer.from_host(L)
+    idx, _ = dev.step(k)
+    torch.cuda.synchronize()
+    assert dev.status() == 0
+    assert np.array_equal(idx.cpu().numpy().astype(np.uint32), ref.idx)
+    import helpers
+    got = dev.codes.cpu().numpy().reshape(-1, 1)
+    helpers.check_codes_against_oracle(ref.t, L.codebooks, got[ref.idx.astype(np.int64)], ref.enc, 1e-6)
