@@ -30,11 +30,14 @@
 // CTA = 256 targets (two 128-row A blocks) x a slice of the codebook, one CTA per
 // SM, persistent over (tile, slice) units.  Warps 0-7: own one target per thread,
 // build A, run the epilogue (warp w reads tensor-memory lanes 32 (w % 4) .. of the
-// accumulator of A block w / 4).  Warp 8: bulk-copy producer.  Warps 9 and 10: one
-// thread each issues the MMAs of one A block (issuing is the scarce resource: about
-// 60 cycles per instruction and per commit), warp 9 also allocates tensor memory.
-// Tensor memory: 2 buffers x 2 accumulators x 128 columns = 512 columns, so the MMAs
-// of step i+1 overlap the epilogue of step i.
+// accumulator of A block w / 4).  Warp 8: bulk-copy producer (stages of four steps).
+// Warps 9 and 10: one thread each issues the MMAs of one A block, warp 9 also
+// allocates tensor memory.  Tensor memory: 2 buffers x 2 accumulators x 128 columns =
+// 512 columns, so the MMAs of step i+1 overlap the epilogue of step i.  The pace is set
+// by the hand-over ring of an accumulator buffer (issue -> execute -> completion seen ->
+// read out -> release seen) and tensor memory holds only two such buffers; a lone
+// thread pays about 150 cycles per mbarrier wait and 50 per MMA or commit, so the
+// issuing threads do as little as possible per step.
 //
 // Codewords whose half squared norm exceeds the fp16 range get a sentinel row
 // that can never win and are listed as "exceptions": the rescoring kernel always
@@ -56,7 +59,8 @@ constexpr int kTcRowBytes = 64;         // 32 halves
 constexpr int kTcStepBytes = kTcStepCw * kTcRowBytes;  // 8192
 constexpr int kTcGroupBytes = 8 * kTcRowBytes;         // one 8-row group: 4 core matrices of 128 bytes
 constexpr int kTcSubCw = 64;            // tracking granularity of the running maximum
-constexpr int kTcStages = 12;           // bulk-copy ring
+constexpr int kTcGroupSteps = 4;        // steps per codebook stage: the MMA threads wait for the codebook once per four steps
+constexpr int kTcStages = 3;            // codebook stages (32 KB each)
 constexpr int kTcEpiThreads = 256;
 constexpr int kTcThreads = kTcEpiThreads + 96;  // + producer warp + one MMA warp per A block
 constexpr uint32_t kTmemCols = 512;
@@ -271,17 +275,15 @@ __device__ __forceinline__ float max64(const uint32_t* v) {
 // ---- shared memory -----------------------------------------------------------------
 struct TcSmem {
   alignas(128) unsigned char a[2][kTcStepBytes];  // two A blocks of 128 targets
-  alignas(128) unsigned char b[kTcStages][kTcStepBytes];
+  alignas(128) unsigned char b[kTcStages][kTcGroupSteps][kTcStepBytes];
   alignas(8) uint64_t full_bar[kTcStages];
   uint64_t empty_bar[kTcStages];
   uint64_t tmem_full[2][2];   // per buffer and A block
   uint64_t tmem_empty[2][2];
   uint64_t a_ready;
   uint64_t drain_bar[2];
-  float evicted_max[kTcTile];           // largest sub-chunk maximum that fell out of the list
   float list_max[kListLen][kTcTile];
   uint16_t list_id[kListLen][kTcTile];
-  uint16_t list_cnt[kTcTile];
   uint32_t tmem_base;
   uint32_t abort_flag;
 };
@@ -298,7 +300,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
     sm.abort_flag = 0;
     for (int s = 0; s < kTcStages; ++s) {
       mbar_init(smem_u32(&sm.full_bar[s]), 1);
-      mbar_init(smem_u32(&sm.empty_bar[s]), 2);  // one commit per MMA warp
+      mbar_init(smem_u32(&sm.empty_bar[s]), 2);  // one commit per MMA warp, at the stage's last step
     }
     for (int b = 0; b < 2; ++b) {
       for (int q = 0; q < 2; ++q) {
@@ -325,25 +327,36 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
   if (warp == 8) {
     // ------------------------------------------------------------ bulk-copy producer
     if (lane == 0) {
+      // total number of steps of this CTA (for the byte count of the last, partial stage)
+      uint32_t total = 0;
+      for (uint64_t u = blockIdx.x; u < units; u += gridDim.x) {
+        uint32_t s_lo, s_hi;
+        slice_units(p, (uint32_t)(u % p.n_slices), &s_lo, &s_hi);
+        total += s_hi - s_lo;
+      }
       uint32_t it = 0;
       bool alive = true;
       for (uint64_t u = blockIdx.x; u < units && alive; u += gridDim.x) {
         uint32_t s_lo, s_hi;
         slice_units(p, (uint32_t)(u % p.n_slices), &s_lo, &s_hi);
         for (uint32_t st = s_lo; st < s_hi && alive; ++st, ++it) {
-          const uint32_t s = it % kTcStages;
-          if (it >= kTcStages)
-            alive = mbar_wait(smem_u32(&sm.empty_bar[s]), ((it / kTcStages) - 1) & 1, abort_flag, p.status);
-          if (!alive) break;
+          const uint32_t grp = it / kTcGroupSteps, sub = it % kTcGroupSteps, s = grp % kTcStages;
           const uint32_t fb = smem_u32(&sm.full_bar[s]);
-          mbar_expect_tx(fb, kTcStepBytes);
-          bulk_g2s(smem_u32(&sm.b[s][0]), bimg + (size_t)st * kTcStepBytes, kTcStepBytes, fb);
+          if (sub == 0) {
+            if (grp >= (uint32_t)kTcStages)
+              alive = mbar_wait(smem_u32(&sm.empty_bar[s]), ((grp / kTcStages) - 1) & 1, abort_flag, p.status);
+            if (!alive) break;
+            const uint32_t left = total - it;
+            mbar_expect_tx(fb, (left < (uint32_t)kTcGroupSteps ? left : (uint32_t)kTcGroupSteps) * kTcStepBytes);
+          }
+          bulk_g2s(smem_u32(&sm.b[s][sub][0]), bimg + (size_t)st * kTcStepBytes, kTcStepBytes, fb);
         }
       }
       if (!alive) {
         // let every copy that was issued land before the CTA may exit
-        for (uint32_t back = 1; back <= kTcStages && back <= it; ++back) {
-          const uint32_t j = it - back;
+        const uint32_t groups = (it + kTcGroupSteps - 1) / kTcGroupSteps;
+        for (uint32_t back = 1; back <= (uint32_t)kTcStages && back <= groups; ++back) {
+          const uint32_t j = groups - back;
           const uint32_t fb = smem_u32(&sm.full_bar[j % kTcStages]);
           for (uint32_t spin = 0; spin < kMaxSpins; ++spin) {
             if (mbar_try_wait(fb, (j / kTcStages) & 1)) break;
@@ -357,7 +370,18 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
     if (lane == 0) {
       const uint32_t q = (uint32_t)warp - 9u;
       const uint64_t a_desc = smem_desc(smem_u32(&sm.a[q][0]));
-      uint32_t it = 0, unit_i = 0;
+      // A lone thread pays about 150 cycles for a wait on an mbarrier (even on a finished phase) and about
+      // 50 per MMA or commit, and its loop is part of the hand-over ring of the accumulators: per step one wait
+      // (accumulator free), two MMAs, one commit; the codebook stage costs a wait and a commit per four steps.
+      uint32_t it = 0, unit_i = 0, total = 0;
+      for (uint64_t u = blockIdx.x; u < units; u += gridDim.x) {
+        uint32_t s_lo, s_hi;
+        slice_units(p, (uint32_t)(u % p.n_slices), &s_lo, &s_hi);
+        total += s_hi - s_lo;
+      }
+      const uint64_t b_desc0 = smem_desc(smem_u32(&sm.b[0][0][0]));
+      const uint32_t full0 = smem_u32(&sm.tmem_full[0][q]), full1 = smem_u32(&sm.tmem_full[1][q]);
+      const uint32_t empty0 = smem_u32(&sm.tmem_empty[0][q]), empty1 = smem_u32(&sm.tmem_empty[1][q]);
       bool alive = true;
       for (uint64_t u = blockIdx.x; u < units && alive; u += gridDim.x, ++unit_i) {
         uint32_t s_lo, s_hi;
@@ -365,18 +389,20 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
         alive = mbar_wait(smem_u32(&sm.a_ready), unit_i & 1, abort_flag, p.status);
         tc_fence_after();
         for (uint32_t st = s_lo; st < s_hi && alive; ++st, ++it) {
-          const uint32_t s = it % kTcStages, buf = it & 1;
-          alive = mbar_wait(smem_u32(&sm.full_bar[s]), (it / kTcStages) & 1, abort_flag, p.status);
-          if (alive) alive = mbar_wait(smem_u32(&sm.tmem_empty[buf][q]), ((it >> 1) & 1) ^ 1, abort_flag, p.status);
+          const uint32_t grp = it / kTcGroupSteps, sub = it % kTcGroupSteps, s = grp % kTcStages, buf = it & 1;
+          if (sub == 0 || it == 0)
+            alive = mbar_wait(smem_u32(&sm.full_bar[s]), (grp / kTcStages) & 1, abort_flag, p.status);
+          if (alive) alive = mbar_wait(buf ? empty1 : empty0, ((it >> 1) & 1) ^ 1, abort_flag, p.status);
           if (!alive) break;
           tc_fence_after();
-          const uint64_t b_desc = smem_desc(smem_u32(&sm.b[s][0]));
+          const uint64_t b_desc = b_desc0 + (uint64_t)((s * kTcGroupSteps + sub) * (kTcStepBytes >> 4));
           // K chunks 0-1 (hi, lo against c), then chunks 2-3 (the norm terms) on top
           const uint32_t d = tmem_base + buf * 256 + q * 128;
           umma_f16(d, a_desc, b_desc, kIdesc, 0);
           umma_f16(d, a_desc + kDescTwoChunks, b_desc + kDescTwoChunks, kIdesc, 1);
-          umma_commit(smem_u32(&sm.tmem_full[buf][q]));  // the accumulator is ready
-          umma_commit(smem_u32(&sm.empty_bar[s]));       // this warp no longer reads the stage
+          umma_commit(buf ? full1 : full0);  // the accumulator is ready
+          if (sub == (uint32_t)kTcGroupSteps - 1 && it + 1 < total)
+            umma_commit(smem_u32(&sm.empty_bar[s]));  // this warp has read the whole stage
         }
       }
       if (!alive) {
@@ -455,8 +481,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
       const float margin = sc * 1.52587890625e-5f /* 2^-16 */ * (sqrtf(nt2) * cnmax + hmax) +
                            4.76837158203125e-7f /* 2^-21 */ * cnmax + 1e-30f;
       float best = kNegInf, thr = kNegInf;
-      sm.list_cnt[tid] = 0;
-      sm.evicted_max[tid] = kNegInf;
 
       // Software-pipelined epilogue.  The 128 columns of a step are read as two halves into
       // two register sets; the first half of step i+1 is requested (if its MMAs are done)
@@ -464,14 +488,17 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
       // to the MMA warp as soon as both halves are in registers.
       uint32_t v[64], w[64];
       bool pending = false;  // the first half of step `st` is already in flight
+      // the list of remembered sub-chunks lives in shared memory, its fill count and the largest evicted maximum
+      // in registers: the common case of an event is two stores and no load
+      uint32_t list_cnt = 0;
+      float evicted_max = kNegInf;
       auto note = [&](float mx, uint32_t sub) {
         if (mx >= thr) {
-          const uint32_t cnt = sm.list_cnt[tid];
-          const uint32_t slot = cnt & (kListLen - 1);
-          if (cnt >= kListLen) sm.evicted_max[tid] = fmaxf(sm.evicted_max[tid], sm.list_max[slot][tid]);
+          const uint32_t slot = list_cnt & (kListLen - 1);
+          if (list_cnt >= kListLen) evicted_max = fmaxf(evicted_max, sm.list_max[slot][tid]);
           sm.list_id[slot][tid] = (uint16_t)sub;
           sm.list_max[slot][tid] = mx;
-          sm.list_cnt[tid] = (uint16_t)(cnt + 1);
+          ++list_cnt;
           best = fmaxf(best, mx);
           thr = best - margin;
         }
@@ -519,12 +546,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
         for (int q = 0; q < kListLen; ++q) rec.sub[q] = 0;
         if (in_range) {
           const float limit = best - margin;
-          const uint32_t cnt = sm.list_cnt[tid];
+          const uint32_t cnt = list_cnt;
 #pragma unroll
           for (int q = 0; q < kListLen; ++q)
             if ((uint32_t)q < cnt && sm.list_max[q][tid] >= limit) rec.sub[cnt_out++] = sm.list_id[q][tid];
           rec.best = -best;
-          rec.cnt = (cnt > (uint32_t)kListLen && sm.evicted_max[tid] >= limit) ? kCandOverflow : (uint16_t)cnt_out;
+          rec.cnt = (cnt > (uint32_t)kListLen && evicted_max >= limit) ? kCandOverflow : (uint16_t)cnt_out;
         } else {
           rec.best = kNegInf;  // passes every limit: the whole slice is rescored exactly
           rec.cnt = kCandOverflow;
