@@ -134,7 +134,10 @@ int pvt_vstep_select(const pvt_layer* layer, uint64_t k, uint32_t* idx_out, void
  *     from load until the process exits, whether or not this call is ever used.
  *   - The first call on each device looks up the array's device address (a
  *     host-side runtime query; the device must be current).  Make that first
- *     call outside any stream capture.
+ *     call outside any stream capture.  The address is kept for the life of
+ *     the process: a cudaDeviceReset unloads the array and leaves that address
+ *     dangling, so a process that resets a device must not call this
+ *     afterwards on that device.
  *   - Every call on a device uses the same array.  Calls whose kernels may
  *     overlap on the GPU (different streams, different host threads) race on it
  *     and give wrong results: issue them on one stream, or order them yourself.

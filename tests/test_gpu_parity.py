@@ -365,3 +365,24 @@ def test_whole_step_select_encode_dequant(M):
     helpers.check_codes_against_oracle(ref.t, L.codebooks, got_codes[ref.idx.astype(np.int64)], ref.enc, REL)
     want_W = oracle.dequant(got_codes, L.codebooks, L.scale, L.rows, L.cols)
     assert np.abs(to_np(W_hat) - want_W).max() <= DEQ_ABS
+
+
+# ------------------------------------------------------------------ ragged sizes of the work decomposition
+
+
+@pytest.mark.parametrize("engine", ["fp32", "tensor"])
+@pytest.mark.parametrize("k", [1, 2, 255, 257, 1023, 1025])
+def test_single_codebook_ragged_target_counts(engine, k):
+    """Target counts around the tile sizes of both engines (256 and 1024), down to a single group."""
+    L = synth.make_layer(64, 512, cfg=130, codebook_size=2048 + 37, codebook_fp16=True)  # K not a multiple of 128
+    idx = np.sort(np.random.default_rng(131 + k).choice(L.num_groups, size=k, replace=False)).astype(np.uint32)
+    with search_engine(engine):
+        check_encode(L, idx)
+
+
+@pytest.mark.parametrize("k", [1, 2, 3, 5, 31, 33])
+def test_two_codebook_ragged_target_counts(k):
+    """The beam search takes four targets per warp: counts that leave partial groups of four."""
+    L = synth.make_layer(32, 256, cfg=132, num_codebooks=2, codebook_size=200, codebook_fp16=True, nearest=oracle_nearest)
+    idx = np.sort(np.random.default_rng(133 + k).choice(L.num_groups, size=k, replace=False)).astype(np.uint32)
+    check_encode(L, idx)
