@@ -450,3 +450,63 @@ void pvt_oracle_adam_direction(const float* grad, float* exp_avg, float* exp_avg
     dir[i] = (m / bias1) / (sqrtf(v / bias2) + eps);
   }
 }
+
+/* ---- subspace size from a trust ratio (Section 4.3; Appendix J, "Hyperparameter tuning") --------------------
+ * The experiments behind Tables 1-2 do not fix tau: they take the largest number of weights, in the order of
+ * decreasing update norm, whose re-encoding keeps ||x_new - x_old|| / ||x_old|| below 0.01, x being the
+ * dequantised weights of one matrix.  The procedure the appendix describes -- re-encode a hundredth of the
+ * weights at a time until the change exceeds the bound, then put back codes from the end of the last portion
+ * until it holds again, always letting one change through -- is driven from pvt_oracle.py; the two functions
+ * below supply its arithmetic.
+ * Pins: a six-weight example worked by hand (bound met exactly, broken by the first change, never reached),
+ * the bound and its maximality recomputed from the dequantised matrices before and after, the longest-prefix
+ * form computed from one V step over all groups (which also shows the result does not depend on the portion
+ * size), ratio = 0 (one change) and a huge ratio (the plain V step).
+ */
+
+/* The order the portions are taken in: the first k groups by (norm descending, index ascending), NOT re-sorted. */
+int pvt_oracle_rank(const float* norms, int64_t G, int64_t k, uint32_t* rank_out) {
+  if (k < 1 || k > G || G >= ((int64_t)1 << 32)) return -1;
+  norm_entry* e = (norm_entry*)malloc((size_t)G * sizeof(norm_entry));
+  if (!e) return -1;
+  for (int64_t j = 0; j < G; ++j) {
+    if (!isfinite(norms[j]) || norms[j] < 0.0f) {
+      free(e);
+      return -1;
+    }
+    e[j].n = norms[j];
+    e[j].j = (uint32_t)j;
+  }
+  qsort(e, (size_t)G, sizeof(norm_entry), by_norm_desc_then_index);
+  for (int64_t i = 0; i < k; ++i) rank_out[i] = e[i].j;
+  free(e);
+  return 0;
+}
+
+/* Squared change of the dequantised weights of each listed group when its code tuple goes from codes_old to
+ * codes_new (both [k][M], one row per listed group): sum over the dg elements, in element order, of
+ * (w_new - w_old)^2 with w = s_row * (C_1[b_1] + ... ) formed in binary32 exactly as dequantisation forms it,
+ * the difference, the square and the sum in binary64.  sq_old (optional) receives sum w_old^2 of the same groups. */
+void pvt_oracle_group_change(const int32_t* codes_old, const int32_t* codes_new, const float* books,
+                             const float* scale, int64_t cols, int32_t dg, int32_t M, int32_t K,
+                             const uint32_t* idx, int64_t k, double* change_out, double* sq_old) {
+  const int64_t gpr = cols / dg;
+  for (int64_t n = 0; n < k; ++n) {
+    const int64_t r = (int64_t)idx[n] / gpr;
+    double acc = 0.0, own = 0.0;
+    for (int32_t i = 0; i < dg; ++i) {
+      float vo = books[((int64_t)0 * K + codes_old[n * M]) * dg + i];
+      float vn = books[((int64_t)0 * K + codes_new[n * M]) * dg + i];
+      for (int32_t q = 1; q < M; ++q) {
+        vo = vo + books[((int64_t)q * K + codes_old[n * M + q]) * dg + i];
+        vn = vn + books[((int64_t)q * K + codes_new[n * M + q]) * dg + i];
+      }
+      const float wo = scale[r] * vo, wn = scale[r] * vn;
+      const double diff = (double)wn - (double)wo;
+      acc = acc + diff * diff;
+      own = own + (double)wo * (double)wo;
+    }
+    change_out[n] = acc;
+    if (sq_old) sq_old[n] = own;
+  }
+}

@@ -40,6 +40,7 @@ def lib():
         L.pvt_oracle_num_threads.restype = ctypes.c_int
         L.pvt_oracle_select.restype = ctypes.c_int
         L.pvt_oracle_encode.restype = ctypes.c_int
+        L.pvt_oracle_rank.restype = ctypes.c_int
         _lib = L
     return _lib
 
@@ -229,3 +230,103 @@ def adam_direction(grad, exp_avg, exp_avg_sq, step: int, beta1: float = 0.9, bet
                                     ctypes.c_int64(grad.size), ctypes.c_float(beta1), ctypes.c_float(beta2),
                                     ctypes.c_float(eps), ctypes.c_float(bias1), ctypes.c_float(bias2))
     return out
+
+
+def rank(norms, k: int) -> np.ndarray:
+    """The k groups of largest norm in the order (norm descending, index ascending), uint32 [k]."""
+    norms = _f32(norms)
+    out = np.empty(k, dtype=np.uint32)
+    rc = lib().pvt_oracle_rank(_p(norms, ctypes.c_float), ctypes.c_int64(norms.size), ctypes.c_int64(k),
+                               _p(out, ctypes.c_uint32))
+    if rc != 0:
+        raise ValueError("pvt_oracle_rank rejected its arguments")
+    return out
+
+
+def group_change(codes_old, codes_new, codebooks, scale, cols: int, idx):
+    """Per listed group: squared change of its dequantised weights, and their squared norm before (float64 [k] each)."""
+    books = _f32(codebooks)
+    M, K, dg = books.shape
+    idx = np.ascontiguousarray(idx, dtype=np.uint32)
+    k = idx.size
+    co = np.ascontiguousarray(np.asarray(codes_old).reshape(k, M), dtype=np.int32)
+    cn = np.ascontiguousarray(np.asarray(codes_new).reshape(k, M), dtype=np.int32)
+    for c in (co, cn):
+        if k and (c.min() < 0 or c.max() >= K):
+            raise ValueError("code out of range")
+    scale = _f32(scale)
+    change = np.empty(k, dtype=np.float64)
+    own = np.empty(k, dtype=np.float64)
+    lib().pvt_oracle_group_change(_p(co, ctypes.c_int32), _p(cn, ctypes.c_int32), _p(books, ctypes.c_float),
+                                  _p(scale, ctypes.c_float), ctypes.c_int64(cols), ctypes.c_int32(dg),
+                                  ctypes.c_int32(M), ctypes.c_int32(K), _p(idx, ctypes.c_uint32), ctypes.c_int64(k),
+                                  _p(change, ctypes.c_double), _p(own, ctypes.c_double))
+    return change, own
+
+
+@dataclass
+class TrustResult:
+    order: np.ndarray  # uint32 [tried]: the groups that were re-encoded, in the order they were taken
+    n_kept: int  # how many of them (a prefix of ``order``) keep their new code
+    codes: np.ndarray  # full code array after the step
+    change: np.ndarray  # float64 [tried]: squared change of each tried group's dequantised weights
+    sq_norm: float  # ||x_old||^2 of the whole matrix
+    enc_codes: np.ndarray  # int32 [tried, M]: what the search returned for each tried group
+    gap_rel: np.ndarray  # float64 [tried]: (second - best) / second of each search (near-tie indicator)
+
+
+def vstep_trust(W, g, scale, codebooks, codes, eta: float, ratio: float = 0.01, portion: float = 0.01,
+                k_max: int | None = None, beam: int = 8) -> TrustResult:
+    """V step whose subspace size comes from the trust ratio (Section 4.3, Appendix J).
+
+    Groups are taken in the order of decreasing update norm, ``portion`` of all groups at a time, and
+    re-encoded; after each portion the total squared change of the dequantised matrix is compared with
+    ``ratio**2 * ||x_old||**2`` (the bound ``||x_new - x_old|| / ||x_old|| < ratio`` without the division and
+    the roots, in float64).  Once the bound fails, codes are put back one group at a time from the end of the
+    last portion until it holds; at least one group keeps its new code.  ``k_max`` stops the procedure after
+    that many groups (default: all of them).
+    """
+    books = _f32(codebooks)
+    M, K, dg = books.shape
+    W = _f32(W)
+    rows, cols = W.shape
+    G = rows * (cols // dg)
+    k_max = G if k_max is None else int(k_max)
+    codes = np.asarray(codes)
+    codes2 = codes.reshape(G, M)
+    order = rank(group_norms(g, eta, dg), k_max)
+    x_old = dequant(codes2, books, scale, rows, cols)
+    sq_norm = float(np.cumsum(x_old.astype(np.float64).ravel() ** 2)[-1]) if G else 0.0
+    limit = float(np.float64(np.float32(ratio)) * np.float64(np.float32(ratio))) * sq_norm
+    step = max(1, int(portion * G))
+    new_codes = codes2.copy()
+    changes, enc_all, gaps = [], [], []
+    total = 0.0
+    n_kept = 0
+    tried = 0
+    while tried < k_max:
+        part = order[tried:min(tried + step, k_max)]
+        j = part.astype(np.int64)
+        enc = encode(targets(W, g, scale, eta, part, dg), books, codes2[j], beam)
+        ch, _ = group_change(codes2[j], enc.codes, books, scale, cols, part)
+        new_codes[j] = enc.codes.astype(codes.dtype)
+        enc_all.append(enc.codes.reshape(-1, M))
+        gaps.append(np.where(enc.d_second > 0, (enc.d_second - enc.d_best) / np.where(enc.d_second > 0, enc.d_second, 1.0), 0.0))
+        running = total + np.cumsum(ch)  # total change after each group of this portion, in order
+        changes.append(ch)
+        tried += part.size
+        if running[-1] < limit:
+            total = float(running[-1])
+            n_kept = tried
+            continue
+        # the bound fails inside this portion: undo its groups from the end until it holds again
+        keep = part.size
+        while keep > 0 and not (running[keep - 1] < limit):
+            keep -= 1
+        n_kept = tried - part.size + keep
+        break
+    n_kept = max(n_kept, 1)  # one change is always let through
+    undo = order[n_kept:tried].astype(np.int64)
+    new_codes[undo] = codes2[undo]
+    return TrustResult(order[:tried], n_kept, new_codes.reshape(codes.shape), np.concatenate(changes), sq_norm,
+                       np.concatenate(enc_all), np.concatenate(gaps))
