@@ -174,6 +174,37 @@ int pvt_vstep_encode(const pvt_layer* layer, const uint32_t* idx, uint64_t k, fl
                      size_t ws_bytes, void* cuda_stream);
 
 /*
+ * V step whose subspace size comes from a trust ratio (Section 4.3: tau = "the
+ * number of weights such that the update satisfies ||x_new - x_old|| / ||x_old||
+ * <= 0.01"; Appendix J, "Hyperparameter tuning": the largest such number, found
+ * by re-encoding a hundredth of the weights at a time in the order of decreasing
+ * update norm and undoing codes from the end of the last portion; one weight is
+ * always allowed to change).  x is the dequantised matrix W_hat of this layer.
+ *
+ * What is computed: the k_max groups of largest ||eta*g_j||^2 are ranked by
+ * (norm descending, index ascending) and all re-encoded as by pvt_vstep_encode.
+ * With d_r the squared change of the dequantised weights of the group at rank r
+ * (binary64 sum, in element order, of squared differences of the binary32 values
+ * pvt_dequant would write before and after), n is the first rank at which
+ * d_0 + ... + d_r < ratio^2 * ||W_hat_old||^2 fails (binary64; k_max if it never
+ * fails; at least 1).  Ranks 0 .. n-1 keep their new codes, ranks n .. k_max-1
+ * get their previous codes back, every other group is untouched.  This equals
+ * the appendix's procedure whenever n < k_max; n == k_max says the cap was
+ * reached before the bound.
+ *
+ * idx_out: device, k_max uint32: group indices in rank order (the first *n_out
+ *          are the subspace).  n_out: device uint64.  stats_out: NULL or device
+ *          double[2]: ||W_hat_old||^2 and the squared change that was kept.
+ * ws: pvt_trust_workspace_bytes(layer, k_max) bytes, 256-byte aligned, header
+ *     cleared by pvt_workspace_init; status bits as for the other calls.
+ * Two codebooks need one-byte codes and 1 <= beam <= 8 (PVT_EUNSUPPORTED).
+ * Returns as pvt_vstep_encode; ratio must be finite and >= 0 (PVT_EINVAL).
+ */
+size_t pvt_trust_workspace_bytes(const pvt_layer* layer, uint64_t k_max);
+int pvt_vstep_trust(const pvt_layer* layer, uint64_t k_max, float ratio, uint32_t* idx_out, uint64_t* n_out,
+                    double* stats_out, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
  * dequantize_weights (Algorithm 3, first line): for every group
  *   W_hat[r, 8c+i] = scale[r] * (C_1[b_1][i] (+ C_2[b_2][i]))   in binary32, the
  *   sum rounded once, then the product rounded once; out_dtype PVT_F16 rounds that
@@ -270,6 +301,7 @@ void pvt_set_m1_search(int mode);
 #define PVT_KERNEL_ENCODE_RESCORE 4 /* exact rescoring and code write after the M = 1 search */
 #define PVT_KERNEL_PSTEP_GRAD 5  /* the kernel of pvt_pstep_grad */
 #define PVT_KERNEL_ADAM 6        /* the kernel of pvt_adam_update */
+#define PVT_KERNEL_TRUST 7       /* ranking, norm and code saving of pvt_vstep_trust (before its search) */
 void pvt_timing_enable(int on);
 /* Kernels this process has launched through the library so far (memsets not counted). */
 unsigned long long pvt_launch_count(void);

@@ -23,7 +23,7 @@ PVT_NOALLOC_MAX_GROUPS = 1 << 21
 PVT_DEV_BAD_INDEX, PVT_DEV_BAD_CODE, PVT_DEV_WAIT_EXPIRED, PVT_DEV_INTERNAL = 1, 2, 4, 8
 PVT_KERNEL_SELECT, PVT_KERNEL_ENCODE_MAIN, PVT_KERNEL_ENCODE_AUX, PVT_KERNEL_DEQUANT = 0, 1, 2, 3
 PVT_KERNEL_ENCODE_RESCORE = 4
-PVT_KERNEL_PSTEP_GRAD, PVT_KERNEL_ADAM = 5, 6
+PVT_KERNEL_PSTEP_GRAD, PVT_KERNEL_ADAM, PVT_KERNEL_TRUST = 5, 6, 7
 PVT_M1_AUTO, PVT_M1_FP32, PVT_M1_TENSOR = 0, 1, 2
 
 
@@ -64,7 +64,7 @@ def lib():
                 if not os.path.exists(path):
                     raise RuntimeError(f"libpvt.so is missing and could not be built: {exc}") from exc
         L = ctypes.CDLL(path)
-        vp, u64, sz = ctypes.c_void_p, ctypes.c_uint64, ctypes.c_size_t
+        vp, u64, sz, fl = ctypes.c_void_p, ctypes.c_uint64, ctypes.c_size_t, ctypes.c_float
         lp = ctypes.POINTER(pvt_layer)
         L.pvt_workspace_bytes.restype = sz
         L.pvt_workspace_bytes.argtypes = [lp, u64]
@@ -76,12 +76,15 @@ def lib():
         L.pvt_vstep_select_noalloc.argtypes = [lp, u64, vp, vp, vp]
         L.pvt_vstep_encode.restype = ctypes.c_int
         L.pvt_vstep_encode.argtypes = [lp, vp, u64, vp, vp, sz, vp]
+        L.pvt_trust_workspace_bytes.restype = sz
+        L.pvt_trust_workspace_bytes.argtypes = [lp, u64]
+        L.pvt_vstep_trust.restype = ctypes.c_int
+        L.pvt_vstep_trust.argtypes = [lp, u64, fl, vp, vp, vp, vp, sz, vp]
         L.pvt_dequant.restype = ctypes.c_int
         L.pvt_dequant.argtypes = [lp, vp, ctypes.c_int32, vp, vp]
         L.pvt_pstep_grad.restype = ctypes.c_int
         L.pvt_pstep_grad.argtypes = [lp, vp, vp, vp, vp]
         L.pvt_adam_update.restype = ctypes.c_int
-        fl = ctypes.c_float
         L.pvt_adam_update.argtypes = [vp, vp, vp, vp, vp, u64, fl, fl, fl, fl, fl, fl, vp]
         L.pvt_adam_direction.restype = ctypes.c_int
         L.pvt_adam_direction.argtypes = [vp, vp, vp, vp, u64, fl, fl, fl, fl, fl, vp]
@@ -177,6 +180,29 @@ def pvt_vstep_encode(layer: pvt_layer, idx: torch.Tensor, k: int, err_out: Optio
                      ws: torch.Tensor, stream=None) -> None:
     _check(lib().pvt_vstep_encode(ctypes.byref(layer), idx.data_ptr(), k, _ptr(err_out), ws.data_ptr(),
                                   ws.numel() * ws.element_size(), _stream_ptr(stream)), "pvt_vstep_encode")
+
+
+def pvt_trust_workspace_bytes(layer: pvt_layer, k_max: int) -> int:
+    n = int(lib().pvt_trust_workspace_bytes(ctypes.byref(layer), k_max))
+    if n == 0:
+        raise PvtError(PVT_EINVAL, "pvt_trust_workspace_bytes")
+    return n
+
+
+def new_trust_workspace(layer: pvt_layer, k_max: int, device=None) -> torch.Tensor:
+    ws = torch.empty(pvt_trust_workspace_bytes(layer, k_max), dtype=torch.uint8, device=device or "cuda")
+    pvt_workspace_init(ws)
+    return ws
+
+
+def pvt_vstep_trust(layer: pvt_layer, k_max: int, ratio: float, idx_out: torch.Tensor, n_out: torch.Tensor,
+                    stats_out: Optional[torch.Tensor], ws: torch.Tensor, stream=None) -> None:
+    """V step with the subspace size taken from the trust ratio: idx_out (uint32 [k_max]) receives the groups in
+    rank order, n_out (one int64/uint64) how many of them keep their new codes, stats_out (float64 [2] or None)
+    the squared norm of the dequantised matrix before and the squared change that was kept."""
+    _check(lib().pvt_vstep_trust(ctypes.byref(layer), k_max, ratio, idx_out.data_ptr(), n_out.data_ptr(),
+                                 _ptr(stats_out), ws.data_ptr(), ws.numel() * ws.element_size(),
+                                 _stream_ptr(stream)), "pvt_vstep_trust")
 
 
 def pvt_dequant(layer: pvt_layer, W_hat: torch.Tensor, status: Optional[torch.Tensor] = None, stream=None) -> None:

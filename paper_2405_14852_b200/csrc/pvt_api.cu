@@ -101,25 +101,34 @@ void timing_end(KernelId id, cudaStream_t stream) {
 
 using namespace pvt;
 
+namespace {
+
+// workspace of pvt_vstep_encode for k groups of this layer
+size_t encode_bytes(const pvt_layer& L, uint64_t k, int sms) {
+  if (L.num_codebooks != 1) return encode_m2_workspace_bytes();
+  return encode_m1_use_tc(L, k)
+             ? encode_m1_tc_layout((uint32_t)L.codebook_size, k, sms).bytes
+             : encode_m1_layout((uint32_t)L.codebook_size, k, sms, encode_m1_targets_per_thread(k, sms)).bytes;
+}
+
+}  // namespace
+
 extern "C" {
 
 size_t pvt_workspace_bytes(const pvt_layer* layer, uint64_t k) {
   uint64_t G = 0;
   if (check_layer(layer, &G) != PVT_OK || check_quantiser(layer) != PVT_OK) return 0;
   if (k < 1 || k > G) return 0;
+  const size_t s = select_layout(G).bytes, e = encode_bytes(*layer, k, sm_count());
+  return e > s ? e : s;
+}
+
+size_t pvt_trust_workspace_bytes(const pvt_layer* layer, uint64_t k_max) {
+  uint64_t G = 0;
+  if (check_layer(layer, &G) != PVT_OK || check_quantiser(layer) != PVT_OK) return 0;
+  if (k_max < 1 || k_max > G) return 0;
   const int sms = sm_count();
-  size_t need = select_layout(G).bytes;
-  if (layer->num_codebooks == 1) {
-    const size_t e =
-        encode_m1_use_tc(*layer, k)
-            ? encode_m1_tc_layout((uint32_t)layer->codebook_size, k, sms).bytes
-            : encode_m1_layout((uint32_t)layer->codebook_size, k, sms, encode_m1_targets_per_thread(k, sms)).bytes;
-    need = e > need ? e : need;
-  } else {
-    const size_t e = encode_m2_workspace_bytes();
-    need = e > need ? e : need;
-  }
-  return need;
+  return trust_layout(G, k_max, encode_bytes(*layer, k_max, sms), sms).bytes;
 }
 
 int pvt_workspace_init(void* ws, size_t ws_bytes, void* cuda_stream) {
@@ -167,6 +176,42 @@ int pvt_vstep_encode(const pvt_layer* layer, const uint32_t* idx, uint64_t k, fl
     if (ws_bytes < encode_m2_workspace_bytes()) return PVT_EWORKSPACE;
     e = launch_encode_m2(*layer, G, idx, k, err_out, ws, sms, static_cast<cudaStream_t>(cuda_stream));
   }
+  return e == cudaSuccess ? PVT_OK : fail_cuda(e);
+}
+
+int pvt_vstep_trust(const pvt_layer* layer, uint64_t k_max, float ratio, uint32_t* idx_out, uint64_t* n_out,
+                    double* stats_out, void* ws, size_t ws_bytes, void* cuda_stream) {
+  uint64_t G = 0;
+  int rc = check_layer(layer, &G);
+  if (rc != PVT_OK) return rc;
+  if ((rc = check_quantiser(layer)) != PVT_OK) return rc;
+  if (k_max < 1 || k_max > G) return PVT_EINVAL;
+  if (!(ratio >= 0.0f) || !(ratio <= 3.0e38f)) return PVT_EINVAL;
+  if (!layer->W || !layer->g || !layer->scale || !layer->codebooks || !layer->codes || !idx_out || !n_out || !ws)
+    return PVT_EINVAL;
+  if (!aligned16(layer->W) || !aligned16(layer->g) || !aligned16(layer->codebooks)) return PVT_EINVAL;
+  if ((reinterpret_cast<uintptr_t>(n_out) & 7u) || (reinterpret_cast<uintptr_t>(stats_out) & 7u)) return PVT_EINVAL;
+  if (reinterpret_cast<uintptr_t>(ws) & (kWsAlign - 1)) return PVT_EINVAL;
+  if (layer->num_codebooks == 2) {
+    if (layer->code_dtype != PVT_U8 || layer->beam < 1 || layer->beam > 8) return PVT_EUNSUPPORTED;
+    if (reinterpret_cast<uintptr_t>(layer->codes) & 1u) return PVT_EINVAL;
+  }
+  const int sms = sm_count();
+  const TrustLayout t = trust_layout(G, k_max, encode_bytes(*layer, k_max, sms), sms);
+  if (ws_bytes < t.bytes) return PVT_EWORKSPACE;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  char* base = static_cast<char*>(ws);
+  uint32_t* idx_sel = reinterpret_cast<uint32_t*>(base + t.idx_off);
+  cudaError_t e = launch_select(*layer, G, k_max, idx_sel, ws, sms, stream);
+  timing_begin(kKernTrust, stream);
+  if (e == cudaSuccess) e = launch_trust_rank(*layer, G, k_max, ws, t, stream);
+  if (e == cudaSuccess) e = launch_trust_before_search(*layer, G, k_max, ws, t, stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(base + t.encode_off, 0, kWsHeaderBytes, stream);
+  timing_end(kKernTrust, stream);
+  if (e != cudaSuccess) return fail_cuda(e);
+  rc = pvt_vstep_encode(layer, idx_sel, k_max, nullptr, base + t.encode_off, t.bytes - t.encode_off, cuda_stream);
+  if (rc != PVT_OK) return rc;
+  e = launch_trust_after_search(*layer, G, k_max, ratio, idx_out, n_out, stats_out, ws, t, stream);
   return e == cudaSuccess ? PVT_OK : fail_cuda(e);
 }
 

@@ -123,10 +123,32 @@ cudaError_t launch_adam_direction(const float* grad, float* exp_avg, float* exp_
                                   float beta1, float beta2, float eps, float bias1, float bias2, int sm_count,
                                   cudaStream_t stream);
 
+// V step with the subspace size taken from a trust ratio: scratch behind the selection's region
+struct TrustLayout {
+  size_t idx_off;       // u32 [k]: the selection, ascending
+  size_t pairs_a_off;   // u64 [k]: (inverted key, position) pairs; the sorted order ends here
+  size_t pairs_b_off;   // u64 [k]: second sort buffer, afterwards f64 [k] squared changes by rank
+  size_t counts_off;    // u32 [256 * sort_blocks]
+  size_t saved_off;     // u32 [k]: previous codes by position
+  size_t partial_off;   // f64 [norm_blocks]
+  size_t stats_off;     // f64 [2] + ticket
+  size_t encode_off;    // workspace of the search kernels (own header)
+  size_t bytes;
+  uint32_t sort_blocks, norm_blocks;
+};
+TrustLayout trust_layout(uint64_t G, uint64_t k, size_t encode_bytes, int sm_count);
+cudaError_t launch_trust_rank(const pvt_layer& L, uint64_t G, uint64_t k, void* ws, const TrustLayout& t,
+                              cudaStream_t stream);
+cudaError_t launch_trust_before_search(const pvt_layer& L, uint64_t G, uint64_t k, void* ws, const TrustLayout& t,
+                                       cudaStream_t stream);
+cudaError_t launch_trust_after_search(const pvt_layer& L, uint64_t G, uint64_t k, float ratio, uint32_t* idx_out,
+                                      uint64_t* n_out, double* stats_out, void* ws, const TrustLayout& t,
+                                      cudaStream_t stream);
+
 // optional per-kernel timing (benchmark instrumentation) ----------------------
 enum KernelId {
   kKernSelect = 0, kKernEncodeMain = 1, kKernEncodeAux = 2, kKernDequant = 3, kKernEncodeRescore = 4,
-  kKernPstepGrad = 5, kKernAdam = 6, kKernCount = 7
+  kKernPstepGrad = 5, kKernAdam = 6, kKernTrust = 7, kKernCount = 8
 };
 void timing_begin(KernelId id, cudaStream_t stream);
 void timing_end(KernelId id, cudaStream_t stream);

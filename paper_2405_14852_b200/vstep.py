@@ -70,5 +70,19 @@ class VStepLayer:
         self.encode(idx, err_out)
         return idx, self.dequant(W_hat) if W_hat is not None else None
 
+    def step_trust(self, k_max: int, ratio: float = 0.01):
+        """V step whose subspace size follows from the trust ratio (Section 4.3, Appendix J): returns the groups
+        in rank order (int32 [k_max]), the number kept (int64 [1]) and float64 [2] = squared norm of the
+        dequantised matrix before, squared change kept.  All three stay on the device."""
+        need = B.pvt_trust_workspace_bytes(self.desc, k_max)
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = torch.empty(need, dtype=torch.uint8, device=self.W.device)
+            B.pvt_workspace_init(self._ws)
+        idx = torch.empty(k_max, dtype=torch.int32, device=self.W.device)
+        n = torch.zeros(1, dtype=torch.int64, device=self.W.device)
+        stats = torch.zeros(2, dtype=torch.float64, device=self.W.device)
+        B.pvt_vstep_trust(self.desc, k_max, ratio, idx, n, stats, self._ws)
+        return idx, n, stats
+
     def status(self) -> int:
         return B.pvt_status(self.reserve(1))
