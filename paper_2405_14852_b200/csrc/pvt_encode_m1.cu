@@ -344,57 +344,83 @@ __device__ __forceinline__ void load_codeword(const void* book, uint32_t kappa, 
   }
 }
 
-// One warp per target.  Memory round trips are kept to three: (index, global minimum,
-// margin, one record per lane) -> (W, g, scale) -> codewords.
+// Eight lanes per target, four targets per warp: the kernel is a chain of dependent memory round trips
+// ((index, global minimum, margin, records) -> (W, g, scale) -> codewords), so what counts is how many targets
+// are in flight per warp, not how fast one of them is evaluated.
+constexpr int kRsLanes = 8;
+constexpr int kRsPerWarp = 32 / kRsLanes;
+constexpr int kRsPerBlock = 8 * kRsPerWarp;  // 256 threads
+static_assert(kMaxSlices <= 2 * kRsLanes, "two records per lane must cover every slice");
+
 template <bool CB_F16>
 __global__ void __launch_bounds__(256) rescore_m1_kernel(const EncM1Params p) {
+  constexpr uint32_t kFull = 0xffffffffu;
   const uint32_t sub_cw = p.sub_cw;
-  const int lane = threadIdx.x & 31;
-  const uint64_t n = (uint64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (n >= p.k) return;
-  const uint32_t tile = (uint32_t)(n / p.tile), s = (uint32_t)(n % p.tile);
-  const uint32_t j = __ldg(p.idx + n);
-  const float limit = unord(p.gbest[n]) + p.margin[n];
-  uint4 raw = make_uint4(0x7f800000u, 0, 0, 0);  // best = +inf: never within the limit
-  if ((uint32_t)lane < p.n_slices)
-    raw = __ldg(reinterpret_cast<const uint4*>(&p.rec[((size_t)tile * p.n_slices + lane) * p.tile + s]));
-  if (j >= p.G) {
-    if (lane == 0) atomicOr(p.status, PVT_DEV_BAD_INDEX);
-    return;
+  const int lane = threadIdx.x & 31, grp = lane / kRsLanes, l = lane % kRsLanes;
+  const int gshift = grp * kRsLanes;
+  const uint64_t n = ((uint64_t)blockIdx.x * 8 + (threadIdx.x >> 5)) * kRsPerWarp + grp;
+  bool active = n < p.k;
+  uint32_t j = 0;
+  float limit = 0.0f;
+  uint4 raw0 = make_uint4(0x7f800000u, 0, 0, 0), raw1 = raw0;  // best = +inf: never within the limit
+  if (active) {
+    const uint32_t tile = (uint32_t)(n / p.tile), s = (uint32_t)(n % p.tile);
+    j = __ldg(p.idx + n);
+    limit = unord(p.gbest[n]) + p.margin[n];
+    const uint4* rec = reinterpret_cast<const uint4*>(p.rec);
+    if ((uint32_t)l < p.n_slices) raw0 = __ldg(&rec[((size_t)tile * p.n_slices + l) * p.tile + s]);
+    if ((uint32_t)l + kRsLanes < p.n_slices)
+      raw1 = __ldg(&rec[((size_t)tile * p.n_slices + l + kRsLanes) * p.tile + s]);
+    if (j >= p.G) {
+      if (l == 0) atomicOr(p.status, PVT_DEV_BAD_INDEX);
+      active = false;
+    }
   }
-  float t[8];
-  form_target(p, j, t);
+  float t[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  if (active) form_target(p, j, t);
   const uint32_t subs_per_unit = p.unit_cw / sub_cw;
   double best_d = __longlong_as_double(0x7ff0000000000000ll);
   uint32_t best_code = 0xffffffffu;
 
-  auto visit = [&](uint32_t sub) {
-    for (uint32_t w = lane; w < sub_cw; w += 32) {
-      const uint32_t kappa = sub * sub_cw + w;
-      if (kappa < p.K) {
-        float c[8];
-        load_codeword<CB_F16>(p.book, kappa, c);
-        double d = 0.0;
+  auto score = [&](uint32_t kappa) {
+    float c[8];
+    load_codeword<CB_F16>(p.book, kappa, c);
+    double d = 0.0;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const double e = __dsub_rn((double)t[i], (double)c[i]);
-          d = __dadd_rn(d, __dmul_rn(e, e));
-        }
-        if (d < best_d || (d == best_d && kappa < best_code)) {
-          best_d = d;
-          best_code = kappa;
-        }
-      }
+    for (int i = 0; i < 8; ++i) {
+      const double e = __dsub_rn((double)t[i], (double)c[i]);
+      d = __dadd_rn(d, __dmul_rn(e, e));
+    }
+    if (d < best_d || (d == best_d && kappa < best_code)) {
+      best_d = d;
+      best_code = kappa;
+    }
+  };
+  auto visit = [&](uint32_t sub) {
+    for (uint32_t w = l; w < sub_cw; w += kRsLanes) {
+      const uint32_t kappa = sub * sub_cw + w;
+      if (kappa < p.K) score(kappa);
     }
   };
 
-  // slices whose minimum lies within the margin of the global minimum (kMaxSlices <= 32: one record per lane)
-  uint32_t live = __ballot_sync(0xffffffffu, __uint_as_float(raw.x) <= limit);
-  while (live) {
-    const int sl = __ffs(live) - 1;
+  // slices whose minimum lies within the margin of the global minimum: bit s of `live`, the same in the
+  // eight lanes of a target.  The loop runs while any target of the warp has a slice left, so that the
+  // shuffles are executed by the whole warp.
+  const uint32_t in0 = __ballot_sync(kFull, active && __uint_as_float(raw0.x) <= limit);
+  const uint32_t in1 = __ballot_sync(kFull, active && __uint_as_float(raw1.x) <= limit);
+  uint32_t live = ((in0 >> gshift) & 0xffu) | (((in1 >> gshift) & 0xffu) << kRsLanes);
+  while (__any_sync(kFull, live != 0)) {
+    const bool has = live != 0;
+    const int sl = has ? __ffs(live) - 1 : 0;
     live &= live - 1;
-    const uint32_t s01 = __shfl_sync(0xffffffffu, raw.y, sl), s23 = __shfl_sync(0xffffffffu, raw.z, sl);
-    const uint32_t cnt = __shfl_sync(0xffffffffu, raw.w, sl) & 0xffffu;
+    const int src = gshift + (sl & (kRsLanes - 1));
+    const bool upper = sl >= kRsLanes;
+    const uint32_t y0 = __shfl_sync(kFull, raw0.y, src), y1 = __shfl_sync(kFull, raw1.y, src);
+    const uint32_t z0 = __shfl_sync(kFull, raw0.z, src), z1 = __shfl_sync(kFull, raw1.z, src);
+    const uint32_t w0 = __shfl_sync(kFull, raw0.w, src), w1 = __shfl_sync(kFull, raw1.w, src);
+    if (!has) continue;
+    const uint32_t s01 = upper ? y1 : y0, s23 = upper ? z1 : z0;
+    const uint32_t cnt = (upper ? w1 : w0) & 0xffffu;
     if (cnt == kCandOverflow) {
       uint32_t u_lo, u_hi;
       slice_units(p, (uint32_t)sl, &u_lo, &u_hi);
@@ -406,39 +432,34 @@ __global__ void __launch_bounds__(256) rescore_m1_kernel(const EncM1Params p) {
       if (cnt > 3) visit(s23 >> 16);
     }
   }
-  if (p.exc_count) {  // codewords whose fast score is not trustworthy: always evaluated
+  if (p.exc_count && active) {  // codewords whose fast score is not trustworthy: always evaluated
     const uint32_t n_exc = __ldg(p.exc_count);
-    for (uint32_t e = lane; e < n_exc && e < p.K; e += 32) {
+    for (uint32_t e = l; e < n_exc && e < p.K; e += kRsLanes) {
       const uint32_t kappa = __ldg(p.exc_list + e);
-      if (kappa < p.K) {
-        float c[8];
-        load_codeword<CB_F16>(p.book, kappa, c);
-        double d = 0.0;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const double df = __dsub_rn((double)t[i], (double)c[i]);
-          d = __dadd_rn(d, __dmul_rn(df, df));
-        }
-        if (d < best_d || (d == best_d && kappa < best_code)) {
-          best_d = d;
-          best_code = kappa;
-        }
-      }
+      if (kappa < p.K) score(kappa);
     }
   }
-  // warp-wide lexicographic minimum of (distance, code); distances are >= 0 so their bits order like u64
+  // lexicographic minimum of (distance, code) over the eight lanes of the target; distances are >= 0 so their
+  // bits order like u64
   const uint64_t bits = (uint64_t)__double_as_longlong(best_d);
-  const uint32_t hi = (uint32_t)(bits >> 32), lo = (uint32_t)bits;
-  const uint32_t mhi = __reduce_min_sync(0xffffffffu, hi);
-  const uint32_t mlo = __reduce_min_sync(0xffffffffu, hi == mhi ? lo : 0xffffffffu);
-  const uint32_t mk = __reduce_min_sync(0xffffffffu, (hi == mhi && lo == mlo) ? best_code : 0xffffffffu);
-  if (lane == 0) {
-    if (mk < p.K) {
+  uint32_t hi = (uint32_t)(bits >> 32), lo = (uint32_t)bits, code = best_code;
+#pragma unroll
+  for (int off = kRsLanes / 2; off > 0; off >>= 1) {
+    const uint32_t ohi = __shfl_xor_sync(kFull, hi, off), olo = __shfl_xor_sync(kFull, lo, off);
+    const uint32_t ocode = __shfl_xor_sync(kFull, code, off);
+    if (ohi < hi || (ohi == hi && (olo < lo || (olo == lo && ocode < code)))) {
+      hi = ohi;
+      lo = olo;
+      code = ocode;
+    }
+  }
+  if (l == 0 && active) {
+    if (code < p.K) {
       if (p.code_u16)
-        reinterpret_cast<uint16_t*>(p.codes)[j] = (uint16_t)mk;
+        reinterpret_cast<uint16_t*>(p.codes)[j] = (uint16_t)code;
       else
-        reinterpret_cast<uint8_t*>(p.codes)[j] = (uint8_t)mk;
-      if (p.err_out) p.err_out[n] = (float)__longlong_as_double((long long)(((uint64_t)mhi << 32) | mlo));
+        reinterpret_cast<uint8_t*>(p.codes)[j] = (uint8_t)code;
+      if (p.err_out) p.err_out[n] = (float)__longlong_as_double((long long)(((uint64_t)hi << 32) | lo));
     } else {
       atomicOr(p.status, PVT_DEV_INTERNAL);  // no candidate survived: the search did not complete
     }
@@ -515,7 +536,7 @@ cudaError_t launch_encode_m1(const pvt_layer& L, uint64_t G, const uint32_t* idx
 
 cudaError_t launch_rescore_m1(const EncM1Params& p, bool codebook_f16, cudaStream_t stream) {
   timing_begin(kKernEncodeRescore, stream);
-  const unsigned blocks = (unsigned)((p.k + 7) / 8);
+  const unsigned blocks = (unsigned)((p.k + kRsPerBlock - 1) / kRsPerBlock);
   if (codebook_f16)
     rescore_m1_kernel<true><<<blocks, 256, 0, stream>>>(p);
   else
