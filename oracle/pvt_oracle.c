@@ -510,3 +510,64 @@ void pvt_oracle_group_change(const int32_t* codes_old, const int32_t* codes_new,
     if (sq_old) sq_old[n] = own;
   }
 }
+
+/* ---- local search over single-index changes (Appendix D) ---------------------------------------------------
+ * Appendix D's neighbourhood N_1 holds every assignment that differs from the current one in exactly one
+ * index, and its local search moves to the best neighbour while that lowers the squared error.  The error is
+ * a sum over weight groups, so the search separates: for one group with code tuple (b_1..b_M) the neighbours
+ * are the M*(K-1) tuples that differ in one code.  One move = the neighbour that is smallest under
+ * (error, tuple), taken only if its error is strictly below the current one; at most max_moves moves.
+ * Errors are evaluated exactly as everywhere else in this file (residual carried in binary64 through the
+ * codebooks in order), so a run started from the beam search's result can only improve on it.
+ * Pins: a two-codebook scalar example worked by hand (two moves to the optimum; a start that is stuck in a
+ * local optimum), Appendix D's difference formula hat_x^2 - x^2 - 2 (hat_x - x) B for the scalar case,
+ * M = 1 (one move reaches the exhaustive optimum), enumeration of all neighbours by an independent routine
+ * (the result has no better neighbour), monotonicity.
+ */
+int pvt_oracle_local_search(const float* t, int64_t k, int32_t dg, int32_t M, int32_t K, const float* books,
+                            int32_t* codes, int32_t max_moves, double* d_out, int32_t* moves_out) {
+  if (M < 1 || M > PVT_ORACLE_MAX_M || K < 1 || dg < 1 || dg > 64 || max_moves < 0) return -1;
+  int bad = 0;
+#pragma omp parallel for schedule(dynamic, 16)
+  for (int64_t n = 0; n < k; ++n) {
+    beam_entry cur;
+    memset(&cur, 0, sizeof cur);
+    int ok = 1;
+    for (int32_t q = 0; q < M; ++q) {
+      cur.code[q] = codes[n * M + q];
+      if (cur.code[q] < 0 || cur.code[q] >= K) ok = 0;
+    }
+    if (!ok) {
+      bad = 1;
+      continue;
+    }
+    double r[64];
+    residual_of(t + n * dg, books, dg, K, cur.code, M - 1, r);
+    cur.d = sqdist(r, books + ((int64_t)(M - 1) * K + cur.code[M - 1]) * dg, dg);
+    int32_t moves = 0;
+    while (moves < max_moves) {
+      beam_entry best = cur;
+      int found = 0;
+      for (int32_t m = 0; m < M; ++m) {
+        for (int32_t q = 0; q < K; ++q) {
+          if (q == cur.code[m]) continue;
+          beam_entry e = cur;
+          e.code[m] = q;
+          residual_of(t + n * dg, books, dg, K, e.code, M - 1, r);
+          e.d = sqdist(r, books + ((int64_t)(M - 1) * K + e.code[M - 1]) * dg, dg);
+          if (!found || entry_less(&e, &best, M)) {
+            best = e;
+            found = 1;
+          }
+        }
+      }
+      if (!found || !(best.d < cur.d)) break;
+      cur = best;
+      ++moves;
+    }
+    for (int32_t q = 0; q < M; ++q) codes[n * M + q] = cur.code[q];
+    if (d_out) d_out[n] = cur.d;
+    if (moves_out) moves_out[n] = moves;
+  }
+  return bad ? -1 : 0;
+}

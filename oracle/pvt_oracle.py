@@ -41,6 +41,7 @@ def lib():
         L.pvt_oracle_select.restype = ctypes.c_int
         L.pvt_oracle_encode.restype = ctypes.c_int
         L.pvt_oracle_rank.restype = ctypes.c_int
+        L.pvt_oracle_local_search.restype = ctypes.c_int
         _lib = L
     return _lib
 
@@ -330,3 +331,22 @@ def vstep_trust(W, g, scale, codebooks, codes, eta: float, ratio: float = 0.01, 
     new_codes[undo] = codes2[undo]
     return TrustResult(order[:tried], n_kept, new_codes.reshape(codes.shape), np.concatenate(changes), sq_norm,
                        np.concatenate(enc_all), np.concatenate(gaps))
+
+
+def local_search(t, codebooks, codes, max_moves: int = 64):
+    """Local search over single-code changes (Appendix D) from the given code tuples: returns
+    (codes int32 [k, M], error float64 [k], moves int32 [k])."""
+    books = _f32(codebooks)
+    M, K, dg = books.shape
+    t = _f32(t).reshape(-1, dg)
+    k = t.shape[0]
+    out = np.ascontiguousarray(np.asarray(codes).reshape(k, M), dtype=np.int32).copy()
+    d = np.empty(k, dtype=np.float64)
+    moves = np.empty(k, dtype=np.int32)
+    rc = lib().pvt_oracle_local_search(_p(t, ctypes.c_float), ctypes.c_int64(k), ctypes.c_int32(dg),
+                                       ctypes.c_int32(M), ctypes.c_int32(K), _p(books, ctypes.c_float),
+                                       _p(out, ctypes.c_int32), ctypes.c_int32(max_moves), _p(d, ctypes.c_double),
+                                       _p(moves, ctypes.c_int32))
+    if rc != 0:
+        raise ValueError("pvt_oracle_local_search rejected its arguments")
+    return out, d, moves
