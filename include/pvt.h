@@ -205,6 +205,28 @@ int pvt_vstep_trust(const pvt_layer* layer, uint64_t k_max, float ratio, uint32_
                     double* stats_out, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * Local search over single-code changes (Appendix D: the neighbourhood N_1 of
+ * assignments that differ in one index, and the search that moves to the best
+ * neighbour while the squared error drops) for the groups listed in idx, started
+ * from the codes that are stored -- e.g. right after pvt_vstep_encode, whose
+ * two-codebook beam search is a heuristic.  The squared error is a sum over
+ * groups, so each group is searched on its own:
+ *   error(b) = ||t - sum_m C_m[b_m]||^2 with the target t of pvt_vstep_encode, in
+ *   binary64 (residual through the codebooks in order, elements in order);
+ *   one move: among the M*(K-1) tuples that differ from the current one in one
+ *   code, the smallest under (error, tuple); taken only if its error is strictly
+ *   below the current error; at most max_moves moves (0 <= max_moves <= 65535).
+ * The error never rises; for one codebook a single move reaches the exhaustive
+ * optimum.  codes[idx[i]] is rewritten when the group moved.
+ * err_out: NULL or device float[k], final error rounded to binary32.  moves_out:
+ * NULL or device uint32[k], moves taken.  status: NULL or a device uint32 into
+ * which PVT_DEV_BAD_INDEX / PVT_DEV_BAD_CODE are OR-ed (such groups are skipped).
+ * No workspace.  Two codebooks need one-byte codes (PVT_EUNSUPPORTED).
+ */
+int pvt_vstep_refine(const pvt_layer* layer, const uint32_t* idx, uint64_t k, int32_t max_moves, float* err_out,
+                     uint32_t* moves_out, uint32_t* status, void* cuda_stream);
+
+/*
  * dequantize_weights (Algorithm 3, first line): for every group
  *   W_hat[r, 8c+i] = scale[r] * (C_1[b_1][i] (+ C_2[b_2][i]))   in binary32, the
  *   sum rounded once, then the product rounded once; out_dtype PVT_F16 rounds that
@@ -302,6 +324,7 @@ void pvt_set_m1_search(int mode);
 #define PVT_KERNEL_PSTEP_GRAD 5  /* the kernel of pvt_pstep_grad */
 #define PVT_KERNEL_ADAM 6        /* the kernel of pvt_adam_update */
 #define PVT_KERNEL_TRUST 7       /* ranking, norm and code saving of pvt_vstep_trust (before its search) */
+#define PVT_KERNEL_REFINE 8      /* the kernel of pvt_vstep_refine */
 void pvt_timing_enable(int on);
 /* Kernels this process has launched through the library so far (memsets not counted). */
 unsigned long long pvt_launch_count(void);

@@ -23,7 +23,7 @@ PVT_NOALLOC_MAX_GROUPS = 1 << 21
 PVT_DEV_BAD_INDEX, PVT_DEV_BAD_CODE, PVT_DEV_WAIT_EXPIRED, PVT_DEV_INTERNAL = 1, 2, 4, 8
 PVT_KERNEL_SELECT, PVT_KERNEL_ENCODE_MAIN, PVT_KERNEL_ENCODE_AUX, PVT_KERNEL_DEQUANT = 0, 1, 2, 3
 PVT_KERNEL_ENCODE_RESCORE = 4
-PVT_KERNEL_PSTEP_GRAD, PVT_KERNEL_ADAM, PVT_KERNEL_TRUST = 5, 6, 7
+PVT_KERNEL_PSTEP_GRAD, PVT_KERNEL_ADAM, PVT_KERNEL_TRUST, PVT_KERNEL_REFINE = 5, 6, 7, 8
 PVT_M1_AUTO, PVT_M1_FP32, PVT_M1_TENSOR = 0, 1, 2
 
 
@@ -80,6 +80,8 @@ def lib():
         L.pvt_trust_workspace_bytes.argtypes = [lp, u64]
         L.pvt_vstep_trust.restype = ctypes.c_int
         L.pvt_vstep_trust.argtypes = [lp, u64, fl, vp, vp, vp, vp, sz, vp]
+        L.pvt_vstep_refine.restype = ctypes.c_int
+        L.pvt_vstep_refine.argtypes = [lp, vp, u64, ctypes.c_int32, vp, vp, vp, vp]
         L.pvt_dequant.restype = ctypes.c_int
         L.pvt_dequant.argtypes = [lp, vp, ctypes.c_int32, vp, vp]
         L.pvt_pstep_grad.restype = ctypes.c_int
@@ -203,6 +205,14 @@ def pvt_vstep_trust(layer: pvt_layer, k_max: int, ratio: float, idx_out: torch.T
     _check(lib().pvt_vstep_trust(ctypes.byref(layer), k_max, ratio, idx_out.data_ptr(), n_out.data_ptr(),
                                  _ptr(stats_out), ws.data_ptr(), ws.numel() * ws.element_size(),
                                  _stream_ptr(stream)), "pvt_vstep_trust")
+
+
+def pvt_vstep_refine(layer: pvt_layer, idx: torch.Tensor, k: int, max_moves: int,
+                     err_out: Optional[torch.Tensor] = None, moves_out: Optional[torch.Tensor] = None,
+                     status: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Local search over single-code changes (Appendix D) on the listed groups, from the stored codes."""
+    _check(lib().pvt_vstep_refine(ctypes.byref(layer), idx.data_ptr(), k, max_moves, _ptr(err_out), _ptr(moves_out),
+                                  _ptr(status), _stream_ptr(stream)), "pvt_vstep_refine")
 
 
 def pvt_dequant(layer: pvt_layer, W_hat: torch.Tensor, status: Optional[torch.Tensor] = None, stream=None) -> None:

@@ -215,6 +215,24 @@ int pvt_vstep_trust(const pvt_layer* layer, uint64_t k_max, float ratio, uint32_
   return e == cudaSuccess ? PVT_OK : fail_cuda(e);
 }
 
+int pvt_vstep_refine(const pvt_layer* layer, const uint32_t* idx, uint64_t k, int32_t max_moves, float* err_out,
+                     uint32_t* moves_out, uint32_t* status, void* cuda_stream) {
+  uint64_t G = 0;
+  int rc = check_layer(layer, &G);
+  if (rc != PVT_OK) return rc;
+  if ((rc = check_quantiser(layer)) != PVT_OK) return rc;
+  if (k < 1 || k > G || max_moves < 0 || max_moves > 65535) return PVT_EINVAL;
+  if (!layer->W || !layer->g || !layer->scale || !layer->codebooks || !layer->codes || !idx) return PVT_EINVAL;
+  if (!aligned16(layer->W) || !aligned16(layer->g) || !aligned16(layer->codebooks)) return PVT_EINVAL;
+  if (layer->num_codebooks == 2) {
+    if (layer->code_dtype != PVT_U8) return PVT_EUNSUPPORTED;
+    if (reinterpret_cast<uintptr_t>(layer->codes) & 1u) return PVT_EINVAL;
+  }
+  const cudaError_t e = launch_refine(*layer, G, idx, k, max_moves, err_out, moves_out, status,
+                                      static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? PVT_OK : fail_cuda(e);
+}
+
 int pvt_dequant(const pvt_layer* layer, void* W_hat, int32_t out_dtype, uint32_t* status, void* cuda_stream) {
   uint64_t G = 0;
   int rc = check_layer(layer, &G);

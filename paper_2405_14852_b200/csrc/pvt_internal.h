@@ -145,10 +145,13 @@ cudaError_t launch_trust_after_search(const pvt_layer& L, uint64_t G, uint64_t k
                                       uint64_t* n_out, double* stats_out, void* ws, const TrustLayout& t,
                                       cudaStream_t stream);
 
+cudaError_t launch_refine(const pvt_layer& L, uint64_t G, const uint32_t* idx, uint64_t k, int max_moves,
+                          float* err_out, uint32_t* moves_out, uint32_t* status, cudaStream_t stream);
+
 // optional per-kernel timing (benchmark instrumentation) ----------------------
 enum KernelId {
   kKernSelect = 0, kKernEncodeMain = 1, kKernEncodeAux = 2, kKernDequant = 3, kKernEncodeRescore = 4,
-  kKernPstepGrad = 5, kKernAdam = 6, kKernTrust = 7, kKernCount = 8
+  kKernPstepGrad = 5, kKernAdam = 6, kKernTrust = 7, kKernRefine = 8, kKernCount = 9
 };
 void timing_begin(KernelId id, cudaStream_t stream);
 void timing_end(KernelId id, cudaStream_t stream);
