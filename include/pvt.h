@@ -69,8 +69,9 @@ extern "C" {
  * each, one code per group and codebook, per-output-channel scale:
  *     W_hat[r, 8c + i] = scale[r] * sum_m codebooks[m][codes[j][m]][i].
  * Supported: group_dim 8; M = 1 with 2 <= K <= 65536 (codes U8 if K <= 256, else
- * U16; U16 is accepted for any K); M = 2 with 2 <= K <= 256, codes U8, 1 <= beam
- * <= 8.
+ * U16; U16 is accepted for any K); M = 2, 3, 4 with 2 <= K <= 256, codes U8, 1 <=
+ * beam <= 8 (M = 3, 4: select, encode and dequant only; the other calls return
+ * PVT_EUNSUPPORTED).
  */
 typedef struct pvt_layer {
   int32_t rows, cols;     /* cols % group_dim == 0 */
@@ -79,7 +80,7 @@ typedef struct pvt_layer {
   int32_t codebook_size;  /* K */
   int32_t codebook_dtype; /* PVT_F32 | PVT_F16 */
   int32_t code_dtype;     /* PVT_U8 | PVT_U16 */
-  int32_t beam;           /* beam width of the M = 2 search; ignored for M = 1 */
+  int32_t beam;           /* beam width of the M >= 2 search; ignored for M = 1 */
   float eta;              /* step size 1/L_S of Eq. 8; finite, >= 0 */
   int32_t reserved_;      /* set to 0 */
   const float* W;         /* [rows][cols] current dense weight y (16-byte aligned) */
@@ -162,6 +163,10 @@ int pvt_vstep_select_noalloc(const pvt_layer* layer, uint64_t k, uint32_t* idx_o
  *          nearest to t under (distance, code); each is extended by every
  *          codeword of codebook 2; the pool is those beam*K pairs plus the
  *          previous pair; codes[j] = argmin of (||t - c1 - c2||^2, code1, code2).
+ *   M = 3, 4: the same search carried through more stages: after each stage but
+ *          the last the `beam` smallest partial tuples under (||t - c1 - ... -
+ *          cm||^2, tuple) are kept; the pool is the last stage's beam*K tuples
+ *          plus the previous tuple.  Every score is the binary64 value itself.
  *   A fast binary32 score shortlists candidates; the decision among shortlisted
  *   candidates is taken on binary64 distances sum_i (t_i - c_i)^2 accumulated in
  *   index order, so ties break exactly as stated above.

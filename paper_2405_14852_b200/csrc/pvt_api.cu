@@ -48,10 +48,11 @@ int check_quantiser(const pvt_layer* L) {
   if (M < 1 || K < 1) return PVT_EINVAL;
   if (L->codebook_dtype != PVT_F32 && L->codebook_dtype != PVT_F16) return PVT_EINVAL;
   if (L->code_dtype != PVT_U8 && L->code_dtype != PVT_U16) return PVT_EINVAL;
-  if (M > 2 || K < 2) return PVT_EUNSUPPORTED;
+  if (M > 4 || K < 2) return PVT_EUNSUPPORTED;
   if (M == 1 && K > 65536) return PVT_EUNSUPPORTED;
   if (L->code_dtype == PVT_U8 && K > 256) return PVT_EINVAL;
-  if (M == 2 && K > 256) return PVT_EUNSUPPORTED;
+  if (M >= 2 && K > 256) return PVT_EUNSUPPORTED;
+  if (M >= 3 && L->code_dtype != PVT_U8) return PVT_EUNSUPPORTED;
   return PVT_OK;
 }
 
@@ -105,6 +106,7 @@ namespace {
 
 // workspace of pvt_vstep_encode for k groups of this layer
 size_t encode_bytes(const pvt_layer& L, uint64_t k, int sms) {
+  if (L.num_codebooks >= 3) return kWsHeaderBytes;
   if (L.num_codebooks != 1) return encode_m2_workspace_bytes();
   return encode_m1_use_tc(L, k)
              ? encode_m1_tc_layout((uint32_t)L.codebook_size, k, sms).bytes
@@ -170,11 +172,15 @@ int pvt_vstep_encode(const pvt_layer* layer, const uint32_t* idx, uint64_t k, fl
         encode_m1_layout((uint32_t)layer->codebook_size, k, sms, encode_m1_targets_per_thread(k, sms));
     if (ws_bytes < lay.bytes) return PVT_EWORKSPACE;
     e = launch_encode_m1(*layer, G, idx, k, err_out, ws, sms, static_cast<cudaStream_t>(cuda_stream));
-  } else {
+  } else if (layer->num_codebooks == 2) {
     if (layer->code_dtype != PVT_U8) return PVT_EUNSUPPORTED;
     if (layer->beam < 1 || layer->beam > 8) return PVT_EUNSUPPORTED;
     if (ws_bytes < encode_m2_workspace_bytes()) return PVT_EWORKSPACE;
     e = launch_encode_m2(*layer, G, idx, k, err_out, ws, sms, static_cast<cudaStream_t>(cuda_stream));
+  } else {
+    if (layer->beam < 1 || layer->beam > 8) return PVT_EUNSUPPORTED;
+    if (ws_bytes < kWsHeaderBytes) return PVT_EWORKSPACE;
+    e = launch_encode_mx(*layer, G, idx, k, err_out, ws, static_cast<cudaStream_t>(cuda_stream));
   }
   return e == cudaSuccess ? PVT_OK : fail_cuda(e);
 }
@@ -192,6 +198,7 @@ int pvt_vstep_trust(const pvt_layer* layer, uint64_t k_max, float ratio, uint32_
   if (!aligned16(layer->W) || !aligned16(layer->g) || !aligned16(layer->codebooks)) return PVT_EINVAL;
   if ((reinterpret_cast<uintptr_t>(n_out) & 7u) || (reinterpret_cast<uintptr_t>(stats_out) & 7u)) return PVT_EINVAL;
   if (reinterpret_cast<uintptr_t>(ws) & (kWsAlign - 1)) return PVT_EINVAL;
+  if (layer->num_codebooks > 2) return PVT_EUNSUPPORTED;
   if (layer->num_codebooks == 2) {
     if (layer->code_dtype != PVT_U8 || layer->beam < 1 || layer->beam > 8) return PVT_EUNSUPPORTED;
     if (reinterpret_cast<uintptr_t>(layer->codes) & 1u) return PVT_EINVAL;
@@ -224,6 +231,7 @@ int pvt_vstep_refine(const pvt_layer* layer, const uint32_t* idx, uint64_t k, in
   if (k < 1 || k > G || max_moves < 0 || max_moves > 65535) return PVT_EINVAL;
   if (!layer->W || !layer->g || !layer->scale || !layer->codebooks || !layer->codes || !idx) return PVT_EINVAL;
   if (!aligned16(layer->W) || !aligned16(layer->g) || !aligned16(layer->codebooks)) return PVT_EINVAL;
+  if (layer->num_codebooks > 2) return PVT_EUNSUPPORTED;
   if (layer->num_codebooks == 2) {
     if (layer->code_dtype != PVT_U8) return PVT_EUNSUPPORTED;
     if (reinterpret_cast<uintptr_t>(layer->codes) & 1u) return PVT_EINVAL;
@@ -253,6 +261,7 @@ int pvt_pstep_grad(const pvt_layer* layer, double* grad_codebooks, double* grad_
   int rc = check_layer(layer, &G);
   if (rc != PVT_OK) return rc;
   if ((rc = check_quantiser(layer)) != PVT_OK) return rc;
+  if (layer->num_codebooks > 2) return PVT_EUNSUPPORTED;
   if (!layer->g || !layer->scale || !layer->codebooks || !layer->codes || !grad_codebooks) return PVT_EINVAL;
   if (!aligned16(layer->g) || !aligned16(layer->codebooks)) return PVT_EINVAL;
   if ((reinterpret_cast<uintptr_t>(grad_codebooks) & 7u) || (reinterpret_cast<uintptr_t>(grad_scale) & 7u))

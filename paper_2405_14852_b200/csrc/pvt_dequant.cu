@@ -73,7 +73,9 @@ __global__ void __launch_bounds__(kDqThreads) dequant_kernel(const void* __restr
           b[u][0] = both & 0xffu;
           b[u][M - 1] = both >> 8;
         } else {
-          b[u][0] = __ldg(reinterpret_cast<const uint8_t*>(codes) + j);
+          const uint8_t* c = reinterpret_cast<const uint8_t*>(codes) + (size_t)j * M;
+#pragma unroll
+          for (int m = 0; m < M; ++m) b[u][m] = __ldg(c + m);
         }
 #pragma unroll
         for (int m = 0; m < M; ++m) {
@@ -92,8 +94,9 @@ __global__ void __launch_bounds__(kDqThreads) dequant_kernel(const void* __restr
       const uint64_t h = base + (uint64_t)u * kDqThreads + threadIdx.x;
       const uint32_t j = (uint32_t)(h >> 1), half = (uint32_t)h & 1u;
       v[u] = load_half_codeword<CB_F16>(book, b[u][0], half);
-      if (M == 2) {
-        const float4 v2 = load_half_codeword<CB_F16>(book, K + b[u][M - 1], half);
+#pragma unroll
+      for (int m = 1; m < M; ++m) {  // codebooks added left to right, each sum rounded once
+        const float4 v2 = load_half_codeword<CB_F16>(book, m * K + b[u][m], half);
         v[u].x = __fadd_rn(v[u].x, v2.x);
         v[u].y = __fadd_rn(v[u].y, v2.y);
         v[u].z = __fadd_rn(v[u].z, v2.z);
@@ -166,12 +169,24 @@ cudaError_t launch_dequant(const pvt_layer& L, uint64_t G, void* W_hat, int32_t 
   timing_begin(kKernDequant, stream);
   cudaError_t err;
   const bool f16 = L.codebook_dtype == PVT_F16;
-  if (L.num_codebooks == 1)
-    err = f16 ? launch_c<1, true>(L, G, W_hat, out_dtype, status, sm_count, stream)
-              : launch_c<1, false>(L, G, W_hat, out_dtype, status, sm_count, stream);
-  else
-    err = f16 ? launch_c<2, true>(L, G, W_hat, out_dtype, status, sm_count, stream)
-              : launch_c<2, false>(L, G, W_hat, out_dtype, status, sm_count, stream);
+  switch (L.num_codebooks) {
+    case 1:
+      err = f16 ? launch_c<1, true>(L, G, W_hat, out_dtype, status, sm_count, stream)
+                : launch_c<1, false>(L, G, W_hat, out_dtype, status, sm_count, stream);
+      break;
+    case 2:
+      err = f16 ? launch_c<2, true>(L, G, W_hat, out_dtype, status, sm_count, stream)
+                : launch_c<2, false>(L, G, W_hat, out_dtype, status, sm_count, stream);
+      break;
+    case 3:
+      err = f16 ? launch_c<3, true>(L, G, W_hat, out_dtype, status, sm_count, stream)
+                : launch_c<3, false>(L, G, W_hat, out_dtype, status, sm_count, stream);
+      break;
+    default:
+      err = f16 ? launch_c<4, true>(L, G, W_hat, out_dtype, status, sm_count, stream)
+                : launch_c<4, false>(L, G, W_hat, out_dtype, status, sm_count, stream);
+      break;
+  }
   count_launches(1);
   timing_end(kKernDequant, stream);
   return err;

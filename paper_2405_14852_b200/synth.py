@@ -127,16 +127,20 @@ def make_layer(
     pick = np.random.default_rng(seed + 2).choice(G, size=K, replace=False)
     C1 = _scaled_groups(W, scale, pick, group_dim).astype(cb_dtype)
     books = [C1]
-    if num_codebooks == 2:
+    if num_codebooks >= 2:
         if nearest is None:
-            raise ValueError("a nearest(X, C) routine is needed to build the second codebook")
-        pick2 = np.random.default_rng(seed + 4).choice(G, size=K, replace=False)
-        X = _scaled_groups(W, scale, pick2, group_dim)
-        a = np.asarray(nearest(X, C1.astype(np.float32)), dtype=np.int64)
-        C2 = (np.float32(0.3) * (X - C1.astype(np.float32)[a])).astype(cb_dtype)
-        books.append(C2)
-    elif num_codebooks != 1:
-        raise ValueError("num_codebooks must be 1 or 2")
+            raise ValueError("a nearest(X, C) routine is needed to build the further codebooks")
+        if num_codebooks > 4:
+            raise ValueError("num_codebooks must be 1..4")
+        # codebook m+1 = 0.3 x what is left of K further sampled groups after their greedy assignment to
+        # codebooks 1..m (streams 4, 5, 6 for codebooks 2, 3, 4)
+        for m in range(1, num_codebooks):
+            pick_m = np.random.default_rng(seed + 3 + m).choice(G, size=K, replace=False)
+            X = _scaled_groups(W, scale, pick_m, group_dim)
+            for Cq in books:
+                Cq32 = Cq.astype(np.float32)
+                X = X - Cq32[np.asarray(nearest(X, Cq32), dtype=np.int64)]
+            books.append((np.float32(0.3) * X).astype(cb_dtype))
     codebooks = np.stack(books, axis=0)
 
     code_np = np.uint8 if K <= 256 else np.uint16

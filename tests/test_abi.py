@@ -63,7 +63,9 @@ def test_select_rejects_bad_arguments_before_launch(kw, k, code):
 
 
 @pytest.mark.parametrize("kw,code", [
-    (dict(num_codebooks=3), B.PVT_EUNSUPPORTED),
+    (dict(num_codebooks=5), B.PVT_EUNSUPPORTED),
+    (dict(num_codebooks=3, beam=9), B.PVT_EUNSUPPORTED),
+    (dict(num_codebooks=4, codebook_size=64, code_dtype=B.PVT_U16), B.PVT_EUNSUPPORTED),
     (dict(codebook_size=1), B.PVT_EUNSUPPORTED),
     (dict(codebook_size=70000, code_dtype=B.PVT_U16), B.PVT_EUNSUPPORTED),
     (dict(codebook_size=512), B.PVT_EINVAL),        # 512 codewords do not fit U8 codes

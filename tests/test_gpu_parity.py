@@ -386,3 +386,48 @@ def test_two_codebook_ragged_target_counts(k):
     L = synth.make_layer(32, 256, cfg=132, num_codebooks=2, codebook_size=200, codebook_fp16=True, nearest=oracle_nearest)
     idx = np.sort(np.random.default_rng(133 + k).choice(L.num_groups, size=k, replace=False)).astype(np.uint32)
     check_encode(L, idx)
+
+
+# ------------------------------------------------------------------ three and four codebooks
+
+
+@pytest.mark.parametrize("M,K,f16,rows,cols,k,beam", [
+    (3, 64, True, 64, 256, 700, 8),
+    (3, 256, True, 64, 512, 600, 8),
+    (4, 32, False, 33, 72, 297, 8),     # every group, ragged sizes
+    (4, 256, True, 32, 512, 300, 4),
+    (3, 16, True, 32, 128, 512, 1),     # greedy
+])
+def test_three_and_four_codebooks_match_checker(M, K, f16, rows, cols, k, beam):
+    L = synth.make_layer(rows, cols, cfg=210 + M, num_codebooks=M, codebook_size=K, codebook_fp16=f16,
+                         nearest=oracle_nearest, beam=beam)
+    idx = np.sort(np.random.default_rng(k + M).choice(L.num_groups, size=k, replace=False)).astype(np.uint32)
+    exact, band = check_encode(L, idx)
+    assert band == 0  # every decision is taken on the checker's own binary64 values
+
+
+@pytest.mark.parametrize("M,K,f16,rows,cols", [(3, 100, True, 96, 136), (4, 256, True, 64, 512), (4, 50, False, 33, 72)])
+@pytest.mark.parametrize("out_f16", [False, True])
+def test_dequant_three_and_four_codebooks_bit_exact(M, K, f16, rows, cols, out_f16):
+    L = synth.make_layer(rows, cols, cfg=220 + M, num_codebooks=M, codebook_size=K, codebook_fp16=f16,
+                         nearest=oracle_nearest)
+    want = oracle.dequant(L.codes, L.codebooks, L.scale, rows, cols)
+    dev = VStepLayer.from_host(L)
+    out = dev.dequant(dtype=torch.float16 if out_f16 else torch.float32)
+    torch.cuda.synchronize()
+    got = to_np(out)
+    assert got.tobytes() == (want.astype(np.float16) if out_f16 else want).tobytes()
+
+
+def test_whole_step_with_three_codebooks():
+    L = synth.make_layer(64, 512, cfg=225, num_codebooks=3, codebook_size=128, codebook_fp16=True,
+                         nearest=oracle_nearest)
+    k = 400
+    want = oracle.vstep(L.W, L.g, L.scale, L.codebooks, L.codes, L.eta, k, L.beam)
+    dev = VStepLayer.from_host(L)
+    idx, W_hat = dev.step(k, W_hat=torch.empty(64, 512, device="cuda"))
+    torch.cuda.synchronize()
+    assert dev.status() == 0
+    assert np.array_equal(to_np(idx).astype(np.uint32), want.idx)
+    assert np.array_equal(to_np(dev.codes), want.codes)
+    assert to_np(W_hat).tobytes() == oracle.dequant(want.codes, L.codebooks, L.scale, 64, 512).tobytes()
