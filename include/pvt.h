@@ -71,11 +71,13 @@ extern "C" {
  * Supported: group_dim 8; M = 1 with 2 <= K <= 65536 (codes U8 if K <= 256, else
  * U16; U16 is accepted for any K); M = 2, 3, 4 with 2 <= K <= 256, codes U8, 1 <=
  * beam <= 8 (M = 3, 4: select, encode and dequant only; the other calls return
- * PVT_EUNSUPPORTED).
+ * PVT_EUNSUPPORTED).  group_dim 16 (Appendix J's one-codebook representations
+ * with groups of 16 weights): M = 1 only, select, encode and dequant only; read
+ * "8" as "16" in the layouts below.
  */
 typedef struct pvt_layer {
   int32_t rows, cols;     /* cols % group_dim == 0 */
-  int32_t group_dim;      /* 8 */
+  int32_t group_dim;      /* 8 (or 16 with one codebook) */
   int32_t num_codebooks;  /* M */
   int32_t codebook_size;  /* K */
   int32_t codebook_dtype; /* PVT_F32 | PVT_F16 */

@@ -34,9 +34,9 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 int check_layer(const pvt_layer* L, uint64_t* G_out) {
   if (!L) return PVT_EINVAL;
   if (L->rows <= 0 || L->cols <= 0) return PVT_EINVAL;
-  if (L->group_dim != kGroupDim) return L->group_dim > 0 ? PVT_EUNSUPPORTED : PVT_EINVAL;
-  if (L->cols % kGroupDim != 0) return PVT_EINVAL;
-  const uint64_t G = (uint64_t)L->rows * (uint64_t)(L->cols / kGroupDim);
+  if (L->group_dim != 8 && L->group_dim != 16) return L->group_dim > 0 ? PVT_EUNSUPPORTED : PVT_EINVAL;
+  if (L->cols % L->group_dim != 0) return PVT_EINVAL;
+  const uint64_t G = (uint64_t)L->rows * (uint64_t)(L->cols / L->group_dim);
   if (G >= (1ull << 32)) return PVT_EINVAL;
   if (!(L->eta >= 0.0f) || !(L->eta <= 3.0e38f)) return PVT_EINVAL;
   *G_out = G;
@@ -53,6 +53,7 @@ int check_quantiser(const pvt_layer* L) {
   if (L->code_dtype == PVT_U8 && K > 256) return PVT_EINVAL;
   if (M >= 2 && K > 256) return PVT_EUNSUPPORTED;
   if (M >= 3 && L->code_dtype != PVT_U8) return PVT_EUNSUPPORTED;
+  if (L->group_dim == 16 && M != 1) return PVT_EUNSUPPORTED;  // groups of 16 weights: one codebook
   return PVT_OK;
 }
 
@@ -106,7 +107,7 @@ namespace {
 
 // workspace of pvt_vstep_encode for k groups of this layer
 size_t encode_bytes(const pvt_layer& L, uint64_t k, int sms) {
-  if (L.num_codebooks >= 3) return kWsHeaderBytes;
+  if (L.num_codebooks >= 3 || L.group_dim == 16) return kWsHeaderBytes;
   if (L.num_codebooks != 1) return encode_m2_workspace_bytes();
   return encode_m1_use_tc(L, k)
              ? encode_m1_tc_layout((uint32_t)L.codebook_size, k, sms).bytes
@@ -164,7 +165,10 @@ int pvt_vstep_encode(const pvt_layer* layer, const uint32_t* idx, uint64_t k, fl
   if (reinterpret_cast<uintptr_t>(ws) & (kWsAlign - 1)) return PVT_EINVAL;
   const int sms = sm_count();
   cudaError_t e;
-  if (layer->num_codebooks == 1 && encode_m1_use_tc(*layer, k)) {
+  if (layer->group_dim == 16) {
+    if (ws_bytes < kWsHeaderBytes) return PVT_EWORKSPACE;
+    e = launch_encode_g16(*layer, G, idx, k, err_out, ws, static_cast<cudaStream_t>(cuda_stream));
+  } else if (layer->num_codebooks == 1 && encode_m1_use_tc(*layer, k)) {
     if (ws_bytes < encode_m1_tc_layout((uint32_t)layer->codebook_size, k, sms).bytes) return PVT_EWORKSPACE;
     e = launch_encode_m1_tc(*layer, G, idx, k, err_out, ws, sms, static_cast<cudaStream_t>(cuda_stream));
   } else if (layer->num_codebooks == 1) {
@@ -198,7 +202,7 @@ int pvt_vstep_trust(const pvt_layer* layer, uint64_t k_max, float ratio, uint32_
   if (!aligned16(layer->W) || !aligned16(layer->g) || !aligned16(layer->codebooks)) return PVT_EINVAL;
   if ((reinterpret_cast<uintptr_t>(n_out) & 7u) || (reinterpret_cast<uintptr_t>(stats_out) & 7u)) return PVT_EINVAL;
   if (reinterpret_cast<uintptr_t>(ws) & (kWsAlign - 1)) return PVT_EINVAL;
-  if (layer->num_codebooks > 2) return PVT_EUNSUPPORTED;
+  if (layer->num_codebooks > 2 || layer->group_dim != kGroupDim) return PVT_EUNSUPPORTED;
   if (layer->num_codebooks == 2) {
     if (layer->code_dtype != PVT_U8 || layer->beam < 1 || layer->beam > 8) return PVT_EUNSUPPORTED;
     if (reinterpret_cast<uintptr_t>(layer->codes) & 1u) return PVT_EINVAL;
@@ -231,7 +235,7 @@ int pvt_vstep_refine(const pvt_layer* layer, const uint32_t* idx, uint64_t k, in
   if (k < 1 || k > G || max_moves < 0 || max_moves > 65535) return PVT_EINVAL;
   if (!layer->W || !layer->g || !layer->scale || !layer->codebooks || !layer->codes || !idx) return PVT_EINVAL;
   if (!aligned16(layer->W) || !aligned16(layer->g) || !aligned16(layer->codebooks)) return PVT_EINVAL;
-  if (layer->num_codebooks > 2) return PVT_EUNSUPPORTED;
+  if (layer->num_codebooks > 2 || layer->group_dim != kGroupDim) return PVT_EUNSUPPORTED;
   if (layer->num_codebooks == 2) {
     if (layer->code_dtype != PVT_U8) return PVT_EUNSUPPORTED;
     if (reinterpret_cast<uintptr_t>(layer->codes) & 1u) return PVT_EINVAL;
@@ -261,7 +265,7 @@ int pvt_pstep_grad(const pvt_layer* layer, double* grad_codebooks, double* grad_
   int rc = check_layer(layer, &G);
   if (rc != PVT_OK) return rc;
   if ((rc = check_quantiser(layer)) != PVT_OK) return rc;
-  if (layer->num_codebooks > 2) return PVT_EUNSUPPORTED;
+  if (layer->num_codebooks > 2 || layer->group_dim != kGroupDim) return PVT_EUNSUPPORTED;
   if (!layer->g || !layer->scale || !layer->codebooks || !layer->codes || !grad_codebooks) return PVT_EINVAL;
   if (!aligned16(layer->g) || !aligned16(layer->codebooks)) return PVT_EINVAL;
   if ((reinterpret_cast<uintptr_t>(grad_codebooks) & 7u) || (reinterpret_cast<uintptr_t>(grad_scale) & 7u))

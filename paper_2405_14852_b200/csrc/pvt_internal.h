@@ -112,6 +112,8 @@ cudaError_t launch_encode_m2(const pvt_layer& L, uint64_t G, const uint32_t* idx
                              void* ws, int sm_count, cudaStream_t stream);
 cudaError_t launch_encode_mx(const pvt_layer& L, uint64_t G, const uint32_t* idx, uint64_t k, float* err_out,
                              void* ws, cudaStream_t stream);
+cudaError_t launch_encode_g16(const pvt_layer& L, uint64_t G, const uint32_t* idx, uint64_t k, float* err_out,
+                              void* ws, cudaStream_t stream);
 cudaError_t launch_dequant(const pvt_layer& L, uint64_t G, void* W_hat, int32_t out_dtype, uint32_t* status,
                            int sm_count, cudaStream_t stream);
 

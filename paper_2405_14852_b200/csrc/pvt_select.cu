@@ -100,25 +100,36 @@ __device__ void find_digit(const uint32_t* hist, uint64_t k_left, uint32_t* digi
 }
 
 constexpr int kNormPer = 4;                              // 16-byte loads per thread and iteration of the norm pass
-constexpr int kNormTile = kSelThreads * kNormPer / 2;    // 512 groups: two threads per group
 
-// Two adjacent lanes share a group: the even lane holds elements 0..3, the odd lane 4..7,
-// so a warp reads 512 contiguous bytes per load instruction.  The sum is a single chain
-// in index order: the even lane runs its four steps from 0, hands the partial sum to the
-// odd lane, which runs the remaining four.
+// LP adjacent lanes share a group (LP = group size / 4: 2 or 4), lane q of them holding elements 4q..4q+3,
+// so a warp reads 512 contiguous bytes per load instruction.  The sum is a single chain in index order:
+// lane 0 runs its four steps from 0 and hands the partial sum to lane 1, which runs the next four, and so
+// on; every lane computes every round (the work is free, the pass is bound by memory), the value is
+// kept only where it is the group's own partial sum.
+__device__ __forceinline__ float norm_chain(float acc, const float4& a, float eta) {
+  float u;
+  u = __fmul_rn(eta, a.x); acc = __fmaf_rn(u, u, acc);
+  u = __fmul_rn(eta, a.y); acc = __fmaf_rn(u, u, acc);
+  u = __fmul_rn(eta, a.z); acc = __fmaf_rn(u, u, acc);
+  u = __fmul_rn(eta, a.w); acc = __fmaf_rn(u, u, acc);
+  return acc;
+}
+
+template <int LP>
 __global__ void __launch_bounds__(kSelThreads) norm_hist_kernel(const float* __restrict__ g, uint64_t G, float eta,
                                                                  uint64_t k, uint32_t* __restrict__ keys,
                                                                  uint32_t* __restrict__ hist0, SelectState* st) {
+  constexpr int kTile = kSelThreads * kNormPer / LP;  // groups per block and iteration
   __shared__ uint32_t sh_hist[kSelBins0];
   __shared__ uint64_t sh_scan[kSelThreads / 32];
   for (int b = threadIdx.x; b < kSelBins0; b += kSelThreads) sh_hist[b] = 0;
   __syncthreads();
   const float4* g4 = reinterpret_cast<const float4*>(g);
-  const uint64_t F = 2 * G;  // 16-byte pieces
-  const uint32_t n_tiles = (uint32_t)((G + kNormTile - 1) / kNormTile);
-  const bool odd = threadIdx.x & 1;
+  const uint64_t F = (uint64_t)LP * G;  // 16-byte pieces
+  const uint32_t n_tiles = (uint32_t)((G + kTile - 1) / kTile);
+  const int q = threadIdx.x & (LP - 1);  // position of this lane within its group
   for (uint32_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
-    const uint64_t f0 = (uint64_t)tile * (2 * kNormTile) + threadIdx.x;
+    const uint64_t f0 = (uint64_t)tile * (LP * kTile) + threadIdx.x;
     float4 a[kNormPer];
 #pragma unroll
     for (int i = 0; i < kNormPer; ++i) {  // all loads of the iteration first
@@ -128,19 +139,16 @@ __global__ void __launch_bounds__(kSelThreads) norm_hist_kernel(const float* __r
 #pragma unroll
     for (int i = 0; i < kNormPer; ++i) {
       const uint64_t f = f0 + (uint64_t)i * kSelThreads;
-      float u, lo = 0.0f;
-      u = __fmul_rn(eta, a[i].x); lo = __fmaf_rn(u, u, lo);
-      u = __fmul_rn(eta, a[i].y); lo = __fmaf_rn(u, u, lo);
-      u = __fmul_rn(eta, a[i].z); lo = __fmaf_rn(u, u, lo);
-      u = __fmul_rn(eta, a[i].w); lo = __fmaf_rn(u, u, lo);
-      float acc = __shfl_up_sync(0xffffffffu, lo, 1);  // odd lanes: the sum over elements 0..3 of their group
-      u = __fmul_rn(eta, a[i].x); acc = __fmaf_rn(u, u, acc);
-      u = __fmul_rn(eta, a[i].y); acc = __fmaf_rn(u, u, acc);
-      u = __fmul_rn(eta, a[i].z); acc = __fmaf_rn(u, u, acc);
-      u = __fmul_rn(eta, a[i].w); acc = __fmaf_rn(u, u, acc);
-      if (odd && f < F) {
+      float acc = norm_chain(0.0f, a[i], eta);  // valid on lane 0 of the group
+#pragma unroll
+      for (int r = 1; r < LP; ++r) {
+        const float in = __shfl_up_sync(0xffffffffu, acc, 1);  // lane r: the sum over elements 0..4r-1
+        const float next = norm_chain(in, a[i], eta);
+        acc = q >= r ? next : acc;
+      }
+      if (q == LP - 1 && f < F) {
         const uint32_t key = __float_as_uint(acc);
-        keys[f >> 1] = key;
+        keys[f / LP] = key;
         atomicAdd(&sh_hist[key >> 20], 1u);
       }
     }
@@ -414,18 +422,25 @@ cudaError_t launch_select(const pvt_layer& L, uint64_t G, uint64_t k, uint32_t* 
   uint32_t* cand = reinterpret_cast<uint32_t*>(base + lay.cand_off);
   // persistent grids: exactly the blocks that are resident at once
   int norm_per_sm = 0, mid_per_sm = 0;
-  if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&norm_per_sm, norm_hist_kernel, kSelThreads, 0)) !=
+  const int lp = L.group_dim / 4;  // lanes per group in the norm pass: 2 or 4
+  if ((err = (lp == 2 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&norm_per_sm, norm_hist_kernel<2>, kSelThreads, 0)
+                      : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&norm_per_sm, norm_hist_kernel<4>, kSelThreads,
+                                                                      0))) !=
           cudaSuccess ||
       (err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&mid_per_sm, refine_mid_kernel, kSelThreads, 0)) !=
           cudaSuccess)
     return err;
-  const uint64_t norm_tiles = (G + kNormTile - 1) / kNormTile;
+  const uint64_t norm_tile = (uint64_t)kSelThreads * kNormPer / lp;
+  const uint64_t norm_tiles = (G + norm_tile - 1) / norm_tile;
   const uint64_t norm_res = (uint64_t)sm_count * (uint64_t)(norm_per_sm > 0 ? norm_per_sm : 1);
   const unsigned norm_grid = (unsigned)(norm_tiles < norm_res ? norm_tiles : norm_res);
   const uint64_t quad_blocks = ((G + 3) / 4 + 2 * kSelThreads - 1) / (2 * kSelThreads);
   const uint64_t mid_res = (uint64_t)sm_count * (uint64_t)(mid_per_sm > 0 ? mid_per_sm : 1);
   const unsigned mid_grid = (unsigned)(quad_blocks < mid_res ? quad_blocks : mid_res);
-  norm_hist_kernel<<<norm_grid, kSelThreads, 0, stream>>>(L.g, G, L.eta, k, keys, hist0, st);
+  if (lp == 2)
+    norm_hist_kernel<2><<<norm_grid, kSelThreads, 0, stream>>>(L.g, G, L.eta, k, keys, hist0, st);
+  else
+    norm_hist_kernel<4><<<norm_grid, kSelThreads, 0, stream>>>(L.g, G, L.eta, k, keys, hist0, st);
   refine_mid_kernel<<<mid_grid, kSelThreads, 0, stream>>>(keys, G, hist1, cand, lay.cand_cap, st);
   const unsigned low_grid = (unsigned)(lay.cand_cap / 8192 < (uint32_t)sm_count ? lay.cand_cap / 8192 + 1 : sm_count);
   refine_low_kernel<<<low_grid, kSelThreads, 0, stream>>>(keys, G, cand, lay.cand_cap, hist2, st);

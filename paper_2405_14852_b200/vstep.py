@@ -21,12 +21,14 @@ def _codes_to_torch(codes: np.ndarray) -> torch.Tensor:
 
 
 class VStepLayer:
-    def __init__(self, rows, cols, W, g, scale, codebooks, codes, *, eta=1.0, beam=8, max_k=None):
+    def __init__(self, rows, cols, W, g, scale, codebooks, codes, *, eta=1.0, beam=8, max_k=None, group_dim=8):
         self.rows, self.cols = int(rows), int(cols)
         self.W, self.g, self.scale, self.codebooks, self.codes = W, g, scale, codebooks, codes
         self.eta, self.beam = float(eta), int(beam)
-        self.num_groups = self.rows * (self.cols // 8)
-        self.desc = B.make_layer(self.rows, self.cols, W, g, scale, codebooks, codes, eta=self.eta, beam=self.beam)
+        self.group_dim = int(group_dim)
+        self.num_groups = self.rows * (self.cols // self.group_dim)
+        self.desc = B.make_layer(self.rows, self.cols, W, g, scale, codebooks, codes, eta=self.eta, beam=self.beam,
+                                 group_dim=self.group_dim)
         self._ws = None
         self._ws_k = 0
         if max_k is not None:
@@ -37,7 +39,7 @@ class VStepLayer:
         dev = torch.device(device)
         up = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
         return cls(L.rows, L.cols, up(L.W), up(L.g), up(L.scale), up(L.codebooks), _codes_to_torch(L.codes).to(dev),
-                   eta=L.eta, beam=L.beam, max_k=max_k)
+                   eta=L.eta, beam=L.beam, max_k=max_k, group_dim=L.group_dim)
 
     def reserve(self, k: int) -> torch.Tensor:
         """Workspace large enough for select/encode with this k (grown on demand)."""

@@ -50,7 +50,8 @@ def test_workspace_bytes_depends_on_shape_not_on_a_device():
     (dict(), 0, B.PVT_EINVAL),                      # k = 0
     (dict(), 16 * 8 + 1, B.PVT_EINVAL),             # k > G
     (dict(cols=60), 1, B.PVT_EINVAL),               # cols % 8
-    (dict(group_dim=16), 1, B.PVT_EUNSUPPORTED),
+    (dict(group_dim=12), 1, B.PVT_EUNSUPPORTED),
+    (dict(group_dim=16, cols=72), 1, B.PVT_EINVAL),  # cols % 16
     (dict(eta=-1.0), 1, B.PVT_EINVAL),
     (dict(eta=float("nan")), 1, B.PVT_EINVAL),
     (dict(g=None), 1, B.PVT_EINVAL),
@@ -64,6 +65,7 @@ def test_select_rejects_bad_arguments_before_launch(kw, k, code):
 
 @pytest.mark.parametrize("kw,code", [
     (dict(num_codebooks=5), B.PVT_EUNSUPPORTED),
+    (dict(group_dim=16, num_codebooks=2), B.PVT_EUNSUPPORTED),   # groups of 16: one codebook
     (dict(num_codebooks=3, beam=9), B.PVT_EUNSUPPORTED),
     (dict(num_codebooks=4, codebook_size=64, code_dtype=B.PVT_U16), B.PVT_EUNSUPPORTED),
     (dict(codebook_size=1), B.PVT_EUNSUPPORTED),

@@ -1,0 +1,100 @@
+"""Groups of 16 weights with one codebook (Appendix J's representations with group size 16): selection, search and
+dequantisation of the CUDA library against the CPU checker.  The search scores every codeword in binary64, so
+codes are compared exactly."""
+import numpy as np
+import pytest
+import torch
+
+import helpers
+from oracle import pvt_oracle as oracle
+from paper_2405_14852_b200 import binding as B
+from paper_2405_14852_b200 import synth
+from paper_2405_14852_b200.vstep import VStepLayer
+
+pytestmark = pytest.mark.gpu
+
+
+def layer(rows, cols, K, f16, cfg=240):
+    return synth.make_layer(rows, cols, cfg=cfg, codebook_size=K, codebook_fp16=f16, group_dim=16)
+
+
+@pytest.mark.parametrize("rows,cols,k", [(64, 512, 1), (64, 512, 100), (100, 272, 333), (256, 4096, 655), (33, 48, 99)])
+def test_select_group_size_16(rows, cols, k):
+    L = layer(rows, cols, 16, True)
+    want = oracle.select(oracle.group_norms(L.g, L.eta, 16), k)
+    dev = VStepLayer.from_host(L)
+    idx = dev.select(k)
+    torch.cuda.synchronize()
+    assert dev.status() == 0
+    assert np.array_equal(idx.cpu().numpy().astype(np.uint32), want)
+
+
+def test_select_group_size_16_ties_take_lowest_index():
+    L = layer(64, 512, 16, True)
+    L.g[:] = np.tile(L.g[0, :16].copy(), 32)[None, :]
+    dev = VStepLayer.from_host(L)
+    idx = dev.select(77)
+    torch.cuda.synchronize()
+    assert np.array_equal(idx.cpu().numpy(), np.arange(77))
+
+
+@pytest.mark.parametrize("K,f16,rows,cols,k", [
+    (256, False, 64, 256, 500),
+    (300, True, 64, 512, 700),       # two-byte codes, K not a multiple of the staged chunk
+    (1500, True, 100, 272, 333),     # ragged sizes
+    (65536, True, 256, 4096, 40),    # the full-size codebook, a few targets
+])
+def test_encode_group_size_16_matches_checker(K, f16, rows, cols, k):
+    L = layer(rows, cols, K, f16)
+    G = L.num_groups
+    idx = np.sort(np.random.default_rng(K + k).choice(G, size=k, replace=False)).astype(np.uint32)
+    t = oracle.targets(L.W, L.g, L.scale, L.eta, idx, 16)
+    enc = oracle.encode(t, L.codebooks, L.codes[idx.astype(np.int64)])
+    dev = VStepLayer.from_host(L)
+    err = torch.full((k,), -1.0, device="cuda")
+    dev.encode(torch.from_numpy(idx.astype(np.int32)).cuda(), err)
+    torch.cuda.synchronize()
+    assert dev.status() == 0
+    got = dev.codes.cpu().numpy().reshape(G, 1)
+    assert np.array_equal(got[idx.astype(np.int64), 0].astype(np.int32), enc.codes[:, 0])
+    assert np.array_equal(err.cpu().numpy(), enc.d_best.astype(np.float32))
+    rest = np.setdiff1d(np.arange(G), idx.astype(np.int64))
+    assert np.array_equal(got[rest], L.codes.reshape(G, 1)[rest])
+
+
+@pytest.mark.parametrize("K,f16,rows,cols", [(256, False, 64, 256), (200, True, 100, 272), (65536, True, 256, 4096)])
+@pytest.mark.parametrize("out_f16", [False, True])
+def test_dequant_group_size_16_bit_exact(K, f16, rows, cols, out_f16):
+    L = layer(rows, cols, K, f16)
+    want = oracle.dequant(L.codes, L.codebooks, L.scale, rows, cols)
+    dev = VStepLayer.from_host(L)
+    out = dev.dequant(dtype=torch.float16 if out_f16 else torch.float32)
+    torch.cuda.synchronize()
+    assert out.cpu().numpy().tobytes() == (want.astype(np.float16) if out_f16 else want).tobytes()
+
+
+def test_whole_step_group_size_16():
+    L = layer(128, 1024, 2048, True)
+    k = 300
+    want = oracle.vstep(L.W, L.g, L.scale, L.codebooks, L.codes, L.eta, k)
+    dev = VStepLayer.from_host(L)
+    idx, W_hat = dev.step(k, W_hat=torch.empty(128, 1024, device="cuda"))
+    torch.cuda.synchronize()
+    assert dev.status() == 0
+    assert np.array_equal(idx.cpu().numpy().astype(np.uint32), want.idx)
+    assert np.array_equal(dev.codes.cpu().numpy(), want.codes)
+    assert W_hat.cpu().numpy().tobytes() == oracle.dequant(want.codes, L.codebooks, L.scale, 128, 1024).tobytes()
+
+
+def test_group_size_16_rejections():
+    L = layer(64, 256, 64, True)
+    dev = VStepLayer.from_host(L)
+    idx = torch.zeros(4, dtype=torch.int32, device="cuda")
+    with pytest.raises(B.PvtError) as e:
+        B.pvt_vstep_refine(dev.desc, idx, 4, 1)
+    assert e.value.code == B.PVT_EUNSUPPORTED
+    with pytest.raises(B.PvtError) as e:
+        B.pvt_trust_workspace_bytes(dev.desc, 4) and B.pvt_vstep_trust(dev.desc, 4, 0.01, idx, torch.zeros(1, dtype=torch.int64, device="cuda"), None, B.new_workspace(dev.desc, 4))
+    with pytest.raises(B.PvtError) as e:
+        B.pvt_vstep_select_noalloc(dev.desc, 4, idx)
+    assert e.value.code == B.PVT_EUNSUPPORTED

@@ -503,3 +503,47 @@ def test_adam_direction_first_step_and_library():
         opt.step()
     # directions are O(1) and each carries a few binary32 roundings; their sum may cancel, so the bound is absolute
     assert np.allclose(-acc, tp.detach().numpy(), rtol=0, atol=2e-6)
+
+
+# ---------------------------------------------------------------- groups of 16 weights
+
+
+def test_group_size_16_norm_is_one_chain_over_sixteen_elements():
+    g = (_rng(31).normal(0, 1e-3, size=(4, 48)) * np.array([1, 1e-19, 1e3, 7])[:, None]).astype(np.float32)
+    for eta in (1.0, 0.3):
+        n = oracle.group_norms(g, eta, group_dim=16)
+        assert n.shape == (12,)
+        for j in range(12):
+            r, c = divmod(j, 3)
+            want = helpers.exact_group_norm(g[r, 16 * c:16 * c + 16], eta)
+            assert n[j].tobytes() == want.tobytes(), (eta, j)
+
+
+def test_group_size_16_search_equals_brute_force_and_library():
+    r = _rng(32)
+    book = r.normal(size=(1, 300, 16)).astype(np.float32)
+    t = r.normal(size=(200, 16)).astype(np.float32)
+    enc = oracle.encode(t, book, np.zeros((200, 1)))
+    d = ((t[:, None, :].astype(np.float64) - book[0][None].astype(np.float64)) ** 2).sum(axis=2)
+    assert np.array_equal(enc.codes[:, 0], d.argmin(axis=1))
+    assert np.allclose(enc.d_best, d.min(axis=1), rtol=1e-13)
+    lib_codes, _ = vq(t.astype(np.float64), book[0].astype(np.float64))
+    assert np.array_equal(enc.codes[:, 0], lib_codes)
+
+
+def test_group_size_16_step_dequant_and_fixed_point():
+    L = synth.make_layer(32, 256, cfg=230, codebook_size=128, codebook_fp16=True, group_dim=16)
+    G = L.num_groups
+    assert G == 32 * 16 and L.codebooks.shape == (1, 128, 16)
+    W_hat = oracle.dequant(L.codes, L.codebooks, L.scale, L.rows, L.cols)
+    want = L.scale[:, None, None] * L.codebooks[0].astype(np.float32)[L.codes[:, 0].astype(int)].reshape(32, 16, 16)
+    assert W_hat.tobytes() == want.reshape(32, 256).astype(np.float32).tobytes()
+    # the dequantised matrix is its own nearest assignment (distinct codewords), and the step is local
+    again = oracle.vstep(W_hat, np.zeros_like(W_hat), L.scale, L.codebooks, L.codes, eta=0.0, k=G)
+    assert np.array_equal(again.codes, L.codes) and np.all(again.enc.d_best < 1e-12)
+    res = oracle.vstep(L.W, L.g, L.scale, L.codebooks, L.codes, L.eta, k=40)
+    rest = np.setdiff1d(np.arange(G), res.idx.astype(int))
+    assert np.array_equal(res.codes[rest], L.codes[rest])
+    t = oracle.targets(L.W, L.g, L.scale, L.eta, res.idx, 16)
+    assert np.all(helpers.recon_error(t, L.codebooks, res.codes[res.idx.astype(int)]) <=
+                  helpers.recon_error(t, L.codebooks, L.codes[res.idx.astype(int)]) * (1 + 1e-12))
