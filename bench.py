@@ -346,7 +346,7 @@ def run_ours(args):
                                                   (props.multi_processor_count * 128 * sm_max_mhz * 1e6),
                         "epilogue_bound_is": "one accumulator read per pair: 128 lanes per SM per clock",
                         # dram__bytes_read + dram__bytes_write of one launch (ncu, this kernel, default workload)
-                        "traffic": 9.72e6 if args.workload == DEFAULT_WORKLOAD else None}
+                        "traffic": 9.73e6 if args.workload == DEFAULT_WORKLOAD else None}
         else:
             roofline = {"kernel": "encode search (M=1, fp32 pipe)" if M == 1 else "encode beam search (M=2)",
                         "bound": "alu", "achieved": achieved, "peak": alu_peak, "unit": "TFLOP/s",
@@ -354,7 +354,8 @@ def run_ours(args):
                         "peak_is": f"{props.multi_processor_count} SMs x 128 FP32 lanes x 2 flop x "
                                    f"{sm_max_mhz:.0f} MHz (derived; no measured FP32 peak)",
                         "flop_per_pair": FLOP_PER_PAIR, "avg_launch_ms": enc_avg_ms, "launches": enc_n,
-                        "traffic": None}
+                        # dram__bytes_read + dram__bytes_write of one launch (ncu, FP32 engine, default workload)
+                        "traffic": 7.87e6 if (M == 1 and args.workload == DEFAULT_WORKLOAD) else None}
         line = {
             "metric": METRIC, "value": job_value(k, world, ms_per_step), "unit": UNIT,
             "pairs_per_s": world * pairs / (ms_per_step * 1e-3),
