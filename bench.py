@@ -535,6 +535,87 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+# --------------------------------------------------------------------------- the calls beyond the V step proper
+
+
+def run_next_rows(args):
+    """Times the calls that widen the path (trust-ratio step, local search, three and four codebooks, groups of
+    16 weights) on synthetic layers of the benchmark shapes and prints one JSON line.  Not the headline metric."""
+    import numpy as np
+    import torch
+
+    from paper_2405_14852_b200 import binding as B
+    from paper_2405_14852_b200 import synth
+    from paper_2405_14852_b200.vstep import VStepLayer
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the V step has no CPU path")
+    flush = torch.empty(64 << 20, dtype=torch.int32, device="cuda")
+
+    def timed(fn, reps=5):
+        spans = []
+        for i in range(reps + 2):
+            flush.fill_(1)
+            flush.sum()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            b.synchronize()
+            if i >= 2:
+                spans.append(a.elapsed_time(b))
+        return sorted(spans)[len(spans) // 2]
+
+    out = {"what": "median of 5 cold-L2 calls each, CUDA events; synthetic layers of the benchmark shapes"}
+
+    # trust-ratio step on the default workload's layer (its random previous codes make every change large, so
+    # the cut falls early; the cost is that of ranking and re-encoding k_max groups either way)
+    L = synth.make_layer(4096, 4096, cfg=2, codebook_size=65536, codebook_fp16=True)
+    dev = VStepLayer.from_host(L)
+    k = synth.subspace_size("0.01", L.num_groups)
+    dev.step_trust(k, 0.01)
+    out["trust_step_4096x4096_1x16_kmax20971"] = {"ms": timed(lambda: dev.step_trust(k, 0.01))}
+    out["plain_select_plus_encode_same_layer"] = {"ms": timed(lambda: dev.encode(dev.select(k)))}
+    del dev
+
+    # local search after the two-codebook beam search
+    L = synth.make_layer(11008, 4096, cfg=3, num_codebooks=2, codebook_size=256, codebook_fp16=True,
+                         nearest=_nearest_on_gpu)
+    dev = VStepLayer.from_host(L)
+    k = synth.subspace_size("0.01", L.num_groups)
+    idx = dev.select(k)
+    dev.encode(idx)
+    out["local_search_11008x4096_2x8_k56360"] = {"ms": timed(lambda: B.pvt_vstep_refine(dev.desc, idx, k, 64))}
+    out["beam_search_same_layer"] = {"ms": timed(lambda: dev.encode(idx))}
+    del dev
+
+    # three and four codebooks
+    for M in (3, 4):
+        L = synth.make_layer(11008, 4096, cfg=3, num_codebooks=M, codebook_size=256, codebook_fp16=True,
+                             nearest=_nearest_on_gpu)
+        dev = VStepLayer.from_host(L)
+        idx = dev.select(k)
+        ms = timed(lambda: dev.encode(idx))
+        pairs = k * L.pairs_per_group()
+        out[f"beam_search_11008x4096_{M}x8_k56360"] = {"ms": ms, "pairs_per_s": pairs / (ms * 1e-3)}
+        out[f"dequant_11008x4096_{M}x8"] = {"ms": timed(lambda: dev.dequant())}
+        del dev
+
+    # groups of 16 weights, one codebook of 65 536
+    L = synth.make_layer(4096, 4096, cfg=2, codebook_size=65536, codebook_fp16=True, group_dim=16)
+    dev = VStepLayer.from_host(L)
+    k = synth.subspace_size("0.01", L.num_groups)
+    idx = dev.select(k)
+    ms = timed(lambda: dev.encode(idx), reps=3)
+    out["g16_4096x4096_1x16_k10485"] = {"select_ms": timed(lambda: dev.select(k)), "search_ms": ms,
+                                        "pairs_per_s": k * 65536 / (ms * 1e-3),
+                                        "dequant_ms": timed(lambda: dev.dequant())}
+    torch.cuda.synchronize()
+    if dev.status() != 0:
+        raise SystemExit("bench.py: device status word set")
+    print(json.dumps({"next_rows": out}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -549,9 +630,15 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of a CUDA graph replay")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--list", action="store_true")
+    ap.add_argument("--next-rows", action="store_true",
+                    help="time the calls beyond the V step proper (trust-ratio step, local search, 3-4 codebooks, "
+                         "groups of 16) instead of the headline metric")
     args = ap.parse_args()
     if args.list:
         print("\n".join(workloads()))
+        return
+    if args.next_rows:
+        run_next_rows(args)
         return
     if args.workload not in workloads():
         raise SystemExit(f"unknown workload {args.workload}; --list shows the names")
