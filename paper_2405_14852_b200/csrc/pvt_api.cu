@@ -107,7 +107,9 @@ namespace {
 
 // workspace of pvt_vstep_encode for k groups of this layer
 size_t encode_bytes(const pvt_layer& L, uint64_t k, int sms) {
-  if (L.num_codebooks >= 3 || L.group_dim == 16) return kWsHeaderBytes;
+  if (L.num_codebooks >= 3) return kWsHeaderBytes;
+  if (L.group_dim == 16)
+    return encode_m1_use_tc(L, k) ? encode_m1_tc_layout((uint32_t)L.codebook_size, k, sms, 16).bytes : kWsHeaderBytes;
   if (L.num_codebooks != 1) return encode_m2_workspace_bytes();
   return encode_m1_use_tc(L, k)
              ? encode_m1_tc_layout((uint32_t)L.codebook_size, k, sms).bytes
@@ -165,9 +167,12 @@ int pvt_vstep_encode(const pvt_layer* layer, const uint32_t* idx, uint64_t k, fl
   if (reinterpret_cast<uintptr_t>(ws) & (kWsAlign - 1)) return PVT_EINVAL;
   const int sms = sm_count();
   cudaError_t e;
-  if (layer->group_dim == 16) {
+  if (layer->group_dim == 16 && !encode_m1_use_tc(*layer, k)) {
     if (ws_bytes < kWsHeaderBytes) return PVT_EWORKSPACE;
     e = launch_encode_g16(*layer, G, idx, k, err_out, ws, static_cast<cudaStream_t>(cuda_stream));
+  } else if (layer->group_dim == 16) {
+    if (ws_bytes < encode_m1_tc_layout((uint32_t)layer->codebook_size, k, sms, 16).bytes) return PVT_EWORKSPACE;
+    e = launch_encode_m1_tc(*layer, G, idx, k, err_out, ws, sms, static_cast<cudaStream_t>(cuda_stream));
   } else if (layer->num_codebooks == 1 && encode_m1_use_tc(*layer, k)) {
     if (ws_bytes < encode_m1_tc_layout((uint32_t)layer->codebook_size, k, sms).bytes) return PVT_EWORKSPACE;
     e = launch_encode_m1_tc(*layer, G, idx, k, err_out, ws, sms, static_cast<cudaStream_t>(cuda_stream));

@@ -325,22 +325,27 @@ __global__ void __launch_bounds__(kEncThreads + 32, 1) encode_m1_kernel(const En
 }
 
 // ---- rescoring --------------------------------------------------------------------
-template <bool CB_F16>
+template <bool CB_F16, int DG>
 __device__ __forceinline__ void load_codeword(const void* book, uint32_t kappa, float* c) {
   if (CB_F16) {
-    const uint4 raw = __ldg(reinterpret_cast<const uint4*>(book) + kappa);
-    const __half2* h = reinterpret_cast<const __half2*>(&raw);
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const float2 f = __half22float2(h[i]);
-      c[2 * i] = f.x;
-      c[2 * i + 1] = f.y;
+    for (int part = 0; part < DG / 8; ++part) {
+      const uint4 raw = __ldg(reinterpret_cast<const uint4*>(book) + (size_t)kappa * (DG / 8) + part);
+      const __half2* h = reinterpret_cast<const __half2*>(&raw);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float2 f = __half22float2(h[i]);
+        c[8 * part + 2 * i] = f.x;
+        c[8 * part + 2 * i + 1] = f.y;
+      }
     }
   } else {
-    const float4* q = reinterpret_cast<const float4*>(book) + 2 * (size_t)kappa;
-    const float4 a = __ldg(q), b = __ldg(q + 1);
-    c[0] = a.x; c[1] = a.y; c[2] = a.z; c[3] = a.w;
-    c[4] = b.x; c[5] = b.y; c[6] = b.z; c[7] = b.w;
+    const float4* q = reinterpret_cast<const float4*>(book) + (size_t)kappa * (DG / 4);
+#pragma unroll
+    for (int part = 0; part < DG / 4; ++part) {
+      const float4 a = __ldg(q + part);
+      c[4 * part] = a.x; c[4 * part + 1] = a.y; c[4 * part + 2] = a.z; c[4 * part + 3] = a.w;
+    }
   }
 }
 
@@ -352,7 +357,7 @@ constexpr int kRsPerWarp = 32 / kRsLanes;
 constexpr int kRsPerBlock = 8 * kRsPerWarp;  // 256 threads
 static_assert(kMaxSlices <= 2 * kRsLanes, "two records per lane must cover every slice");
 
-template <bool CB_F16>
+template <bool CB_F16, int DG>
 __global__ void __launch_bounds__(256) rescore_m1_kernel(const EncM1Params p) {
   constexpr uint32_t kFull = 0xffffffffu;
   const uint32_t sub_cw = p.sub_cw;
@@ -376,18 +381,25 @@ __global__ void __launch_bounds__(256) rescore_m1_kernel(const EncM1Params p) {
       active = false;
     }
   }
-  float t[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-  if (active) form_target(p, j, t);
+  float t[DG];
+#pragma unroll
+  for (int i = 0; i < DG; ++i) t[i] = 0.0f;
+  if (active) {
+    if (DG == 8)
+      form_target(p, j, t);
+    else
+      form_target16(p, j, t);
+  }
   const uint32_t subs_per_unit = p.unit_cw / sub_cw;
   double best_d = __longlong_as_double(0x7ff0000000000000ll);
   uint32_t best_code = 0xffffffffu;
 
   auto score = [&](uint32_t kappa) {
-    float c[8];
-    load_codeword<CB_F16>(p.book, kappa, c);
+    float c[DG];
+    load_codeword<CB_F16, DG>(p.book, kappa, c);
     double d = 0.0;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
+    for (int i = 0; i < DG; ++i) {
       const double e = __dsub_rn((double)t[i], (double)c[i]);
       d = __dadd_rn(d, __dmul_rn(e, e));
     }
@@ -493,6 +505,7 @@ cudaError_t launch_encode_m1(const pvt_layer& L, uint64_t G, const uint32_t* idx
   p.k = k;
   p.G = G;
   p.gpr = (uint32_t)(L.cols / kGroupDim);
+  p.dg = kGroupDim;
   p.eta = L.eta;
   p.cbx = reinterpret_cast<const float*>(base + lay.cbx_off);
   p.n2max_bits = reinterpret_cast<const uint32_t*>(base + lay.n2max_off);
@@ -537,10 +550,13 @@ cudaError_t launch_encode_m1(const pvt_layer& L, uint64_t G, const uint32_t* idx
 cudaError_t launch_rescore_m1(const EncM1Params& p, bool codebook_f16, cudaStream_t stream) {
   timing_begin(kKernEncodeRescore, stream);
   const unsigned blocks = (unsigned)((p.k + kRsPerBlock - 1) / kRsPerBlock);
-  if (codebook_f16)
-    rescore_m1_kernel<true><<<blocks, 256, 0, stream>>>(p);
-  else
-    rescore_m1_kernel<false><<<blocks, 256, 0, stream>>>(p);
+  if (p.dg == 16) {  // groups of 16 weights come from the tensor engine only: fp16 codebooks
+    rescore_m1_kernel<true, 16><<<blocks, 256, 0, stream>>>(p);
+  } else if (codebook_f16) {
+    rescore_m1_kernel<true, 8><<<blocks, 256, 0, stream>>>(p);
+  } else {
+    rescore_m1_kernel<false, 8><<<blocks, 256, 0, stream>>>(p);
+  }
   count_launches(1);
   timing_end(kKernEncodeRescore, stream);
   return cudaGetLastError();

@@ -19,6 +19,7 @@ struct EncM1Params {
   const uint32_t* idx;
   uint64_t k, G;
   uint32_t gpr;
+  uint32_t dg;  // weights per group: 8, or 16 (tensor engine and rescoring only)
   float eta;
   const float* cbx;
   const uint32_t* n2max_bits;
@@ -30,7 +31,7 @@ struct EncM1Params {
   uint32_t* gbest;
   float* margin;
   CandRecord* rec;
-  const void* book;  // the caller's codebook [K][8]
+  const void* book;  // the caller's codebook [K][dg]
   void* codes;
   int code_u16;
   float* err_out;
@@ -62,6 +63,22 @@ __device__ __forceinline__ void form_target(const EncM1Params& p, uint32_t j, fl
   t[5] = __fdiv_rn(__fmaf_rn(neg_eta, g1.y, w1.y), sc);
   t[6] = __fdiv_rn(__fmaf_rn(neg_eta, g1.z, w1.z), sc);
   t[7] = __fdiv_rn(__fmaf_rn(neg_eta, g1.w, w1.w), sc);
+}
+
+// the same for a group of 16 weights
+__device__ __forceinline__ void form_target16(const EncM1Params& p, uint32_t j, float* t) {
+  const float4* W4 = reinterpret_cast<const float4*>(p.W) + 4 * (size_t)j;
+  const float4* g4 = reinterpret_cast<const float4*>(p.g) + 4 * (size_t)j;
+  const float sc = __ldg(p.scale + j / p.gpr);
+  const float neg_eta = -p.eta;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const float4 w = __ldg(W4 + q), gg = __ldg(g4 + q);
+    t[4 * q + 0] = __fdiv_rn(__fmaf_rn(neg_eta, gg.x, w.x), sc);
+    t[4 * q + 1] = __fdiv_rn(__fmaf_rn(neg_eta, gg.y, w.y), sc);
+    t[4 * q + 2] = __fdiv_rn(__fmaf_rn(neg_eta, gg.z, w.z), sc);
+    t[4 * q + 3] = __fdiv_rn(__fmaf_rn(neg_eta, gg.w, w.w), sc);
+  }
 }
 
 // ---- PTX helpers ---------------------------------------------------------------

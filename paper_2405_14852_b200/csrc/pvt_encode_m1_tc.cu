@@ -43,6 +43,10 @@
 // that can never win and are listed as "exceptions": the rescoring kernel always
 // evaluates them exactly.  Targets outside the range the scaling can serve
 // (non-finite, or max |t_i| >= 256) are rescored against the whole codebook.
+//
+// Groups of 16 weights (Appendix J) use the same kernel with rows of 48 halves: [ hi x 16 | lo x 16 | 2^e x 8 |
+// 0 x 8 ] against [ c x 16 | c x 16 | norm terms | 0 x 8 ], six K chunks, three instructions per step and A
+// block, 12 KB per step.  Everything described for eight weights above holds with these sizes.
 #include <atomic>
 
 #include "pvt_encode_m1.cuh"
@@ -55,9 +59,18 @@ namespace {
 
 constexpr int kTcTile = 256;            // targets per CTA tile
 constexpr int kTcStepCw = 128;          // codewords per MMA step (the N of one instruction)
-constexpr int kTcRowBytes = 64;         // 32 halves
-constexpr int kTcStepBytes = kTcStepCw * kTcRowBytes;  // 8192
-constexpr int kTcGroupBytes = 8 * kTcRowBytes;         // one 8-row group: 4 core matrices of 128 bytes
+// Operand geometry for groups of DG weights: a row holds the two halves of the target (or the codeword
+// twice), eight norm slots and eight zeros: 32 halves for DG = 8, 48 for DG = 16.
+template <int DG>
+struct TcDim {
+  static constexpr int kRowBytes = 2 * (2 * DG + 16);          // 64 or 96
+  static constexpr int kStepBytes = kTcStepCw * kRowBytes;     // 8192 or 12288
+  static constexpr int kGroupBytes = 8 * kRowBytes;            // one 8-row group: kChunks core matrices of 128 bytes
+  static constexpr int kChunks = kRowBytes / 16;               // 16-byte K chunks per row: 4 or 6
+  static constexpr int kMmas = kChunks / 2;                    // instructions per step and A block
+  static constexpr int kPart = DG / 8;                         // K chunks per copy of the codeword
+};
+constexpr int kTcStepBytes = TcDim<8>::kStepBytes;
 constexpr int kTcSubCw = 64;            // tracking granularity of the running maximum
 constexpr int kTcGroupSteps = 4;        // steps per codebook stage: the MMA threads wait for the codebook once per four steps
 constexpr int kTcStages = 3;            // codebook stages (32 KB each)
@@ -84,7 +97,7 @@ bool encode_m1_use_tc(const pvt_layer& L, uint64_t k) {
   return L.codebook_size >= 1024;  // below that the FP32 pipe with its larger target tiles is as fast
 }
 
-EncodeM1TcLayout encode_m1_tc_layout(uint32_t K, uint64_t k, int sm_count) {
+EncodeM1TcLayout encode_m1_tc_layout(uint32_t K, uint64_t k, int sm_count, int group_dim) {
   EncodeM1TcLayout e;
   e.n_steps = (K + kTcStepCw - 1) / kTcStepCw;
   e.n_tiles = (uint32_t)((k + kTcTile - 1) / kTcTile);
@@ -107,7 +120,8 @@ EncodeM1TcLayout encode_m1_tc_layout(uint32_t K, uint64_t k, int sm_count) {
   const uint64_t units = (uint64_t)e.n_tiles * e.n_slices;
   e.n_ctas = (uint32_t)(units < (uint64_t)sm_count ? units : (uint64_t)sm_count);
   e.bimg_off = kWsHeaderBytes;
-  e.stats_off = align_up(e.bimg_off + (size_t)e.n_steps * kTcStepBytes, kWsAlign);
+  e.stats_off = align_up(e.bimg_off + (size_t)e.n_steps * (group_dim == 16 ? TcDim<16>::kStepBytes : kTcStepBytes),
+                         kWsAlign);
   e.exc_off = e.stats_off + kWsAlign;
   e.gbest_off = align_up(e.exc_off + sizeof(uint32_t) * K, kWsAlign);
   e.margin_off = align_up(e.gbest_off + sizeof(uint32_t) * k, kWsAlign);
@@ -125,23 +139,29 @@ struct TcStats {
 };
 
 // ---- codebook image ------------------------------------------------------------
+template <int DG>
 __global__ void __launch_bounds__(256) tc_prep_kernel(const uint4* __restrict__ book, uint32_t K, uint32_t n_steps,
                                                        unsigned char* __restrict__ bimg, TcStats* stats,
                                                        uint32_t* __restrict__ exc_list) {
+  using D = TcDim<DG>;
   const uint32_t kappa = blockIdx.x * blockDim.x + threadIdx.x;
   uint32_t n2bits = 0;
   if (kappa < n_steps * kTcStepCw) {
     const bool real = kappa < K;
-    uint4 raw = make_uint4(0, 0, 0, 0);
+    uint4 raw[D::kPart];
     float n2 = 0.0f;
-    if (real) {
-      raw = __ldg(book + kappa);
-      const __half2* h = reinterpret_cast<const __half2*>(&raw);
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const float2 f = __half22float2(h[i]);
-        n2 = __fmaf_rn(f.x, f.x, n2);
-        n2 = __fmaf_rn(f.y, f.y, n2);
+    for (int part = 0; part < D::kPart; ++part) {
+      raw[part] = make_uint4(0, 0, 0, 0);
+      if (real) {
+        raw[part] = __ldg(book + (size_t)kappa * D::kPart + part);
+        const __half2* h = reinterpret_cast<const __half2*>(&raw[part]);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float2 f = __half22float2(h[i]);
+          n2 = __fmaf_rn(f.x, f.x, n2);
+          n2 = __fmaf_rn(f.y, f.y, n2);
+        }
       }
     }
     const float hn = 0.5f * n2;
@@ -150,7 +170,7 @@ __global__ void __launch_bounds__(256) tc_prep_kernel(const uint4* __restrict__ 
       const uint32_t pos = atomicAdd(&stats->exc_count, 1u);
       if (pos < K) exc_list[pos] = kappa;
     }
-    uint4 k0, k1;
+    uint4 k1;
     if (rep) {
       const __half h_hi = __float2half_rn(hn);
       const float r1 = hn - __half2float(h_hi);
@@ -159,20 +179,23 @@ __global__ void __launch_bounds__(256) tc_prep_kernel(const uint4* __restrict__ 
       const __half h_lo2 = __float2half_rn(r2);
       const __half2 a = __halves2half2(__hneg(h_hi), __hneg(h_lo));
       const __half2 b = __halves2half2(__hneg(h_lo2), __float2half_rn(0.0f));
-      k0 = raw;
       k1 = make_uint4(*reinterpret_cast<const uint32_t*>(&a), *reinterpret_cast<const uint32_t*>(&b), 0u, 0u);
       n2bits = __float_as_uint(n2);
     } else {
       // padding and exceptions: zero codeword with the most negative norm terms, never a maximum
-      k0 = make_uint4(0, 0, 0, 0);
+#pragma unroll
+      for (int part = 0; part < D::kPart; ++part) raw[part] = make_uint4(0, 0, 0, 0);
       k1 = make_uint4(0xfbfffbffu, 0xfbfffbffu, 0xfbfffbffu, 0xfbfffbffu);  // -65504 x 8
     }
     const uint32_t step = kappa / kTcStepCw, r = kappa % kTcStepCw;
-    unsigned char* row = bimg + (size_t)step * kTcStepBytes + (r >> 3) * kTcGroupBytes + (r & 7) * 16;
-    *reinterpret_cast<uint4*>(row) = k0;        // pairs with hi
-    *reinterpret_cast<uint4*>(row + 128) = k0;  // pairs with lo
-    *reinterpret_cast<uint4*>(row + 256) = k1;  // norm terms
-    *reinterpret_cast<uint4*>(row + 384) = make_uint4(0, 0, 0, 0);
+    unsigned char* row = bimg + (size_t)step * D::kStepBytes + (r >> 3) * D::kGroupBytes + (r & 7) * 16;
+#pragma unroll
+    for (int part = 0; part < D::kPart; ++part) {
+      *reinterpret_cast<uint4*>(row + 128 * part) = raw[part];                 // pairs with hi
+      *reinterpret_cast<uint4*>(row + 128 * (D::kPart + part)) = raw[part];    // pairs with lo
+    }
+    *reinterpret_cast<uint4*>(row + 128 * (2 * D::kPart)) = k1;  // norm terms
+    *reinterpret_cast<uint4*>(row + 128 * (2 * D::kPart + 1)) = make_uint4(0, 0, 0, 0);
   }
   n2bits = __reduce_max_sync(0xffffffffu, n2bits);
   if ((threadIdx.x & 31) == 0 && n2bits > __ldcg(&stats->n2max_bits)) atomicMax(&stats->n2max_bits, n2bits);
@@ -205,10 +228,10 @@ __device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint6
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// shared-memory operand descriptor: K-major, no swizzle, K chunks 128 B apart, 8-row groups kTcGroupBytes apart
-__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr) {
+// shared-memory operand descriptor: K-major, no swizzle, K chunks 128 B apart, 8-row groups group_bytes apart
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t group_bytes) {
   return (uint64_t)((saddr & 0x3ffffu) >> 4) | ((uint64_t)(128u >> 4) << 16) |
-         ((uint64_t)((uint32_t)kTcGroupBytes >> 4) << 32) | (1ull << 46);
+         ((uint64_t)(group_bytes >> 4) << 32) | (1ull << 46);
 }
 // instruction descriptor: D fp32, A and B fp16, both K-major, N = 128, M = 128
 constexpr uint64_t kDescTwoChunks = 256u >> 4;  // start-address field advance for two K chunks
@@ -273,9 +296,10 @@ __device__ __forceinline__ float max64(const uint32_t* v) {
 }
 
 // ---- shared memory -----------------------------------------------------------------
+template <int DG>
 struct TcSmem {
-  alignas(128) unsigned char a[2][kTcStepBytes];  // two A blocks of 128 targets
-  alignas(128) unsigned char b[kTcStages][kTcGroupSteps][kTcStepBytes];
+  alignas(128) unsigned char a[2][TcDim<DG>::kStepBytes];  // two A blocks of 128 targets
+  alignas(128) unsigned char b[kTcStages][kTcGroupSteps][TcDim<DG>::kStepBytes];
   alignas(8) uint64_t full_bar[kTcStages];
   uint64_t empty_bar[kTcStages];
   uint64_t tmem_full[2][2];   // per buffer and A block
@@ -288,11 +312,14 @@ struct TcSmem {
   uint32_t abort_flag;
 };
 
+template <int DG>
 __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1Params p,
                                                                       const unsigned char* __restrict__ bimg,
                                                                       const TcStats* __restrict__ stats) {
+  using D = TcDim<DG>;
+  constexpr int kStepBytes = D::kStepBytes;
   extern __shared__ __align__(128) unsigned char smem_raw[];
-  TcSmem& sm = *reinterpret_cast<TcSmem*>(smem_raw);
+  TcSmem<DG>& sm = *reinterpret_cast<TcSmem<DG>*>(smem_raw);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   volatile uint32_t* abort_flag = &sm.abort_flag;
 
@@ -347,9 +374,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
               alive = mbar_wait(smem_u32(&sm.empty_bar[s]), ((grp / kTcStages) - 1) & 1, abort_flag, p.status);
             if (!alive) break;
             const uint32_t left = total - it;
-            mbar_expect_tx(fb, (left < (uint32_t)kTcGroupSteps ? left : (uint32_t)kTcGroupSteps) * kTcStepBytes);
+            mbar_expect_tx(fb, (left < (uint32_t)kTcGroupSteps ? left : (uint32_t)kTcGroupSteps) * kStepBytes);
           }
-          bulk_g2s(smem_u32(&sm.b[s][sub][0]), bimg + (size_t)st * kTcStepBytes, kTcStepBytes, fb);
+          bulk_g2s(smem_u32(&sm.b[s][sub][0]), bimg + (size_t)st * kStepBytes, kStepBytes, fb);
         }
       }
       if (!alive) {
@@ -369,7 +396,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
     // ------------------------------------------------------------ MMA issuers: warp 9 -> A block 0, warp 10 -> A block 1
     if (lane == 0) {
       const uint32_t q = (uint32_t)warp - 9u;
-      const uint64_t a_desc = smem_desc(smem_u32(&sm.a[q][0]));
+      const uint64_t a_desc = smem_desc(smem_u32(&sm.a[q][0]), D::kGroupBytes);
       // A lone thread pays about 150 cycles for a wait on an mbarrier (even on a finished phase) and about
       // 50 per MMA or commit, and its loop is part of the hand-over ring of the accumulators: per step one wait
       // (accumulator free), two MMAs, one commit; the codebook stage costs a wait and a commit per four steps.
@@ -379,7 +406,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
         slice_units(p, (uint32_t)(u % p.n_slices), &s_lo, &s_hi);
         total += s_hi - s_lo;
       }
-      const uint64_t b_desc0 = smem_desc(smem_u32(&sm.b[0][0][0]));
+      const uint64_t b_desc0 = smem_desc(smem_u32(&sm.b[0][0][0]), D::kGroupBytes);
       const uint32_t full0 = smem_u32(&sm.tmem_full[0][q]), full1 = smem_u32(&sm.tmem_full[1][q]);
       const uint32_t empty0 = smem_u32(&sm.tmem_empty[0][q]), empty1 = smem_u32(&sm.tmem_empty[1][q]);
       bool alive = true;
@@ -395,11 +422,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
           if (alive) alive = mbar_wait(buf ? empty1 : empty0, ((it >> 1) & 1) ^ 1, abort_flag, p.status);
           if (!alive) break;
           tc_fence_after();
-          const uint64_t b_desc = b_desc0 + (uint64_t)((s * kTcGroupSteps + sub) * (kTcStepBytes >> 4));
-          // K chunks 0-1 (hi, lo against c), then chunks 2-3 (the norm terms) on top
+          const uint64_t b_desc = b_desc0 + (uint64_t)((s * kTcGroupSteps + sub) * (kStepBytes >> 4));
+          // two K chunks per instruction: the halves of the target against the codeword, then the norm terms on top
           const uint32_t d = tmem_base + buf * 256 + q * 128;
           umma_f16(d, a_desc, b_desc, kIdesc, 0);
-          umma_f16(d, a_desc + kDescTwoChunks, b_desc + kDescTwoChunks, kIdesc, 1);
+#pragma unroll
+          for (int m = 1; m < D::kMmas; ++m)
+            umma_f16(d, a_desc + m * kDescTwoChunks, b_desc + m * kDescTwoChunks, kIdesc, 1);
           umma_commit(buf ? full1 : full0);  // the accumulator is ready
           if (sub == (uint32_t)kTcGroupSteps - 1 && it + 1 < total)
             umma_commit(smem_u32(&sm.empty_bar[s]));  // this warp has read the whole stage
@@ -419,7 +448,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
     const float n2max = __uint_as_float(stats->n2max_bits);
     const float cnmax = sqrtf(n2max), hmax = 0.5f * n2max;
     const uint32_t rb = (uint32_t)tid >> 7, r = (uint32_t)tid & 127u;
-    unsigned char* a_row = &sm.a[rb][(r >> 3) * kTcGroupBytes + (r & 7) * 16];
+    unsigned char* a_row = &sm.a[rb][(r >> 3) * D::kGroupBytes + (r & 7) * 16];
     const uint32_t lane_base = ((uint32_t)(warp & 3) * 32u) << 16;
     uint32_t it = 0;
     bool alive = true;
@@ -431,20 +460,23 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
       const uint64_t n = (uint64_t)tile * kTcTile + tid;
 
       // the target of this thread, its scaling, its A row
-      float t[8];
+      float t[DG];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) t[i] = 0.0f;
+      for (int i = 0; i < DG; ++i) t[i] = 0.0f;
       bool have = false;
       if (n < p.k) {
         const uint32_t j = p.idx[n];
         if (j < p.G) {  // an index out of range is reported by the rescoring kernel
-          form_target(p, j, t);
+          if (DG == 8)
+            form_target(p, j, t);
+          else
+            form_target16(p, j, t);
           have = true;
         }
       }
       float m = 0.0f, nt2 = 0.0f;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
+      for (int i = 0; i < DG; ++i) {
         m = fmaxf(m, fabsf(t[i]));
         nt2 = fmaf(t[i], t[i], nt2);
       }
@@ -456,9 +488,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
       }
       const float sc = in_range ? scalbnf(1.0f, e) : 0.0f;
       {
-        __half2 hi[4], lo[4];
+        __half2 hi[DG / 2], lo[DG / 2];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < DG / 2; ++i) {
           const float x = in_range ? t[2 * i] * sc : 0.0f, y = in_range ? t[2 * i + 1] * sc : 0.0f;  // exact products
           hi[i] = __floats2half2_rn(x, y);
           const float2 back = __half22float2(hi[i]);
@@ -466,10 +498,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
         }
         const __half2 s2 = __floats2half2_rn(sc, sc);
         const uint32_t sb = *reinterpret_cast<const uint32_t*>(&s2);
-        *reinterpret_cast<uint4*>(a_row) = *reinterpret_cast<const uint4*>(hi);
-        *reinterpret_cast<uint4*>(a_row + 128) = *reinterpret_cast<const uint4*>(lo);
-        *reinterpret_cast<uint4*>(a_row + 256) = make_uint4(sb, sb, sb, sb);
-        *reinterpret_cast<uint4*>(a_row + 384) = make_uint4(0, 0, 0, 0);
+#pragma unroll
+        for (int part = 0; part < D::kPart; ++part) {
+          *reinterpret_cast<uint4*>(a_row + 128 * part) = reinterpret_cast<const uint4*>(hi)[part];
+          *reinterpret_cast<uint4*>(a_row + 128 * (D::kPart + part)) = reinterpret_cast<const uint4*>(lo)[part];
+        }
+        *reinterpret_cast<uint4*>(a_row + 128 * (2 * D::kPart)) = make_uint4(sb, sb, sb, sb);
+        *reinterpret_cast<uint4*>(a_row + 128 * (2 * D::kPart + 1)) = make_uint4(0, 0, 0, 0);
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the MMA
       mbar_arrive(smem_u32(&sm.a_ready));
@@ -478,7 +513,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
       // |hi + lo - 2^e t_i| <= 2^-22 |2^e t_i| (2^-25 where lo is subnormal); the norm split is exact to
       // 2^-33 h; products of halves are exact in fp32; the accumulation of at most 32 terms in fp32, rounded
       // or truncated, stays below 2^-19 of the sum of magnitudes 2^e (||t|| ||c|| + h)
-      const float margin = sc * 1.52587890625e-5f /* 2^-16 */ * (sqrtf(nt2) * cnmax + hmax) +
+      // (48 terms instead of 32 for groups of 16: the factor is doubled there)
+      const float margin = sc * (DG == 8 ? 1.52587890625e-5f /* 2^-16 */ : 3.0517578125e-5f /* 2^-15 */) *
+                               (sqrtf(nt2) * cnmax + hmax) +
                            4.76837158203125e-7f /* 2^-21 */ * cnmax + 1e-30f;
       float best = kNegInf, thr = kNegInf;
 
@@ -574,9 +611,37 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
 
 }  // namespace
 
+namespace {
+
+template <int DG>
+cudaError_t launch_tc(const pvt_layer& L, const EncM1Params& p, const EncodeM1TcLayout& lay, char* base, TcStats* stats,
+                      cudaStream_t stream) {
+  timing_begin(kKernEncodeAux, stream);
+  const uint32_t n_cw = lay.n_steps * kTcStepCw;
+  tc_prep_kernel<DG><<<(n_cw + 255) / 256, 256, 0, stream>>>(
+      reinterpret_cast<const uint4*>(L.codebooks), p.K, lay.n_steps,
+      reinterpret_cast<unsigned char*>(base + lay.bimg_off), stats, reinterpret_cast<uint32_t*>(base + lay.exc_off));
+  count_launches(1);
+  timing_end(kKernEncodeAux, stream);
+  cudaError_t err = cudaGetLastError();
+  if (err != cudaSuccess) return err;
+  const size_t smem = sizeof(TcSmem<DG>);
+  if ((err = cudaFuncSetAttribute(encode_m1_tc_kernel<DG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) !=
+      cudaSuccess)
+    return err;
+  timing_begin(kKernEncodeMain, stream);
+  encode_m1_tc_kernel<DG><<<lay.n_ctas, kTcThreads, smem, stream>>>(
+      p, reinterpret_cast<const unsigned char*>(base + lay.bimg_off), stats);
+  timing_end(kKernEncodeMain, stream);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
 cudaError_t launch_encode_m1_tc(const pvt_layer& L, uint64_t G, const uint32_t* idx, uint64_t k, float* err_out,
                                 void* ws, int sm_count, cudaStream_t stream) {
-  const EncodeM1TcLayout lay = encode_m1_tc_layout((uint32_t)L.codebook_size, k, sm_count);
+  const EncodeM1TcLayout lay = encode_m1_tc_layout((uint32_t)L.codebook_size, k, sm_count, L.group_dim);
   char* base = static_cast<char*>(ws);
   TcStats* stats = reinterpret_cast<TcStats*>(base + lay.stats_off);
   EncM1Params p;
@@ -586,7 +651,8 @@ cudaError_t launch_encode_m1_tc(const pvt_layer& L, uint64_t G, const uint32_t* 
   p.idx = idx;
   p.k = k;
   p.G = G;
-  p.gpr = (uint32_t)(L.cols / kGroupDim);
+  p.gpr = (uint32_t)(L.cols / L.group_dim);
+  p.dg = (uint32_t)L.group_dim;
   p.eta = L.eta;
   p.cbx = nullptr;
   p.n2max_bits = &stats->n2max_bits;
@@ -611,25 +677,8 @@ cudaError_t launch_encode_m1_tc(const pvt_layer& L, uint64_t G, const uint32_t* 
   cudaError_t err = cudaMemsetAsync(stats, 0, sizeof(TcStats), stream);
   if (err != cudaSuccess) return err;
   if ((err = cudaMemsetAsync(p.gbest, 0xff, sizeof(uint32_t) * k, stream)) != cudaSuccess) return err;
-  timing_begin(kKernEncodeAux, stream);
-  const uint32_t n_cw = lay.n_steps * kTcStepCw;
-  tc_prep_kernel<<<(n_cw + 255) / 256, 256, 0, stream>>>(reinterpret_cast<const uint4*>(L.codebooks), p.K, lay.n_steps,
-                                                         reinterpret_cast<unsigned char*>(base + lay.bimg_off), stats,
-                                                         reinterpret_cast<uint32_t*>(base + lay.exc_off));
-  count_launches(1);
-  timing_end(kKernEncodeAux, stream);
-  if ((err = cudaGetLastError()) != cudaSuccess) return err;
-
-  const size_t smem = sizeof(TcSmem);
-  if ((err = cudaFuncSetAttribute(encode_m1_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) !=
-      cudaSuccess)
-    return err;
-  timing_begin(kKernEncodeMain, stream);
-  encode_m1_tc_kernel<<<lay.n_ctas, kTcThreads, smem, stream>>>(
-      p, reinterpret_cast<const unsigned char*>(base + lay.bimg_off), stats);
-  timing_end(kKernEncodeMain, stream);
-  count_launches(1);
-  if ((err = cudaGetLastError()) != cudaSuccess) return err;
+  err = L.group_dim == 16 ? launch_tc<16>(L, p, lay, base, stats, stream) : launch_tc<8>(L, p, lay, base, stats, stream);
+  if (err != cudaSuccess) return err;
   return launch_rescore_m1(p, true, stream);
 }
 

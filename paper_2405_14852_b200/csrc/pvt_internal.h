@@ -99,7 +99,7 @@ struct EncodeM1TcLayout {
 };
 bool encode_m1_use_tc(const pvt_layer& L, uint64_t k);
 void set_m1_search(int mode);
-EncodeM1TcLayout encode_m1_tc_layout(uint32_t K, uint64_t k, int sm_count);
+EncodeM1TcLayout encode_m1_tc_layout(uint32_t K, uint64_t k, int sm_count, int group_dim = 8);
 
 // launchers (each returns a cudaError_t) --------------------------------------
 cudaError_t launch_select(const pvt_layer& L, uint64_t G, uint64_t k, uint32_t* idx_out, void* ws, int sm_count,

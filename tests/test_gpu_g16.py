@@ -38,16 +38,49 @@ def test_select_group_size_16_ties_take_lowest_index():
     assert np.array_equal(idx.cpu().numpy(), np.arange(77))
 
 
-@pytest.mark.parametrize("K,f16,rows,cols,k", [
-    (256, False, 64, 256, 500),
-    (300, True, 64, 512, 700),       # two-byte codes, K not a multiple of the staged chunk
-    (1500, True, 100, 272, 333),     # ragged sizes
-    (65536, True, 256, 4096, 40),    # the full-size codebook, a few targets
+ENGINE = {"binary64": B.PVT_M1_FP32, "tensor": B.PVT_M1_TENSOR, "auto": B.PVT_M1_AUTO}
+
+
+@pytest.mark.parametrize("K,f16,rows,cols,k,engine", [
+    (256, False, 64, 256, 500, "auto"),
+    (300, True, 64, 512, 700, "binary64"),     # two-byte codes, K not a multiple of the staged chunk
+    (300, True, 64, 512, 700, "tensor"),       # K not a multiple of the 128-codeword step
+    (1500, True, 100, 272, 333, "auto"),       # ragged sizes; tensor cores from 1024 codewords on
+    (1500, True, 100, 272, 333, "binary64"),
+    (4096, True, 256, 4096, 3000, "tensor"),   # several tiles of 256 targets and a ragged last one
+    (65536, True, 256, 4096, 40, "auto"),      # the full-size codebook, a few targets
+    (200, True, 64, 512, 1, "tensor"),         # a single target
 ])
-def test_encode_group_size_16_matches_checker(K, f16, rows, cols, k):
-    L = layer(rows, cols, K, f16)
+def test_encode_group_size_16_matches_checker(K, f16, rows, cols, k, engine):
+    B.pvt_set_m1_search(ENGINE[engine])
+    try:
+        _encode_case(K, f16, rows, cols, k)
+    finally:
+        B.pvt_set_m1_search(B.PVT_M1_AUTO)
+
+
+def test_encode_group_size_16_extreme_scales_on_the_tensor_engine():
+    """Targets outside the range the operand scaling serves (huge, tiny, zero) and a codeword whose norm does not
+    fit the operand image: the tensor engine must hand these to exact rescoring."""
+    L = layer(64, 512, 2048, True, cfg=241)
+    L.W[3] *= 1e4      # |t| >= 256 after the division by the (unchanged) scale
+    L.W[5] *= 1e-12    # tiny targets
+    L.W[7] = 0.0
+    L.g[7] = 0.0       # zero targets
+    L.codebooks[0, 17] = 300.0   # half squared norm 16 * 300^2 / 2 > 60000: an exception row
+    idx = np.arange(0, L.num_groups, 3, dtype=np.uint32)
+    B.pvt_set_m1_search(B.PVT_M1_TENSOR)
+    try:
+        _encode_case(None, None, None, None, idx.size, L=L, idx=idx)
+    finally:
+        B.pvt_set_m1_search(B.PVT_M1_AUTO)
+
+
+def _encode_case(K, f16, rows, cols, k, L=None, idx=None):
+    L = layer(rows, cols, K, f16) if L is None else L
     G = L.num_groups
-    idx = np.sort(np.random.default_rng(K + k).choice(G, size=k, replace=False)).astype(np.uint32)
+    if idx is None:
+        idx = np.sort(np.random.default_rng(K + k).choice(G, size=k, replace=False)).astype(np.uint32)
     t = oracle.targets(L.W, L.g, L.scale, L.eta, idx, 16)
     enc = oracle.encode(t, L.codebooks, L.codes[idx.astype(np.int64)])
     dev = VStepLayer.from_host(L)
@@ -56,8 +89,10 @@ def test_encode_group_size_16_matches_checker(K, f16, rows, cols, k):
     torch.cuda.synchronize()
     assert dev.status() == 0
     got = dev.codes.cpu().numpy().reshape(G, 1)
-    assert np.array_equal(got[idx.astype(np.int64), 0].astype(np.int32), enc.codes[:, 0])
-    assert np.array_equal(err.cpu().numpy(), enc.d_best.astype(np.float32))
+    helpers.check_codes_against_oracle(t, L.codebooks, got[idx.astype(np.int64)], enc, 1e-6)
+    decisive = (enc.d_second - enc.d_best) > 1e-6 * enc.d_second
+    assert np.array_equal(got[idx.astype(np.int64), 0].astype(np.int32)[decisive], enc.codes[decisive, 0])
+    assert np.allclose(err.cpu().numpy(), enc.d_best, rtol=1e-5, atol=1e-30)
     rest = np.setdiff1d(np.arange(G), idx.astype(np.int64))
     assert np.array_equal(got[rest], L.codes.reshape(G, 1)[rest])
 
