@@ -78,3 +78,63 @@ def test_full_size_step_against_checker(cfg, which, tau, wdtype):
         assert got_W.tobytes() == want_W.astype(np.float16).tobytes()
     else:
         assert got_W.tobytes() == want_W.tobytes()
+
+
+def test_full_size_trust_step_against_checker():
+    """pvt_vstep_trust on the benchmark's default layer (4096 x 4096, one codebook of 65 536, k_max = 1 % of the
+    groups): rank order in full, kept count, codes of the kept groups, everything else untouched."""
+    L = synth.make_config_layer(2, 0)
+    G = L.num_groups
+    k_max = synth.subspace_size("0.01", G)
+    ratio = 0.1  # the layer's previous codes are random, so every change is large: the cut falls inside k_max
+    want = oracle.vstep_trust(L.W, L.g, L.scale, L.codebooks, L.codes, L.eta, ratio=ratio, k_max=k_max)
+    order = oracle.rank(oracle.group_norms(L.g, L.eta), k_max)
+    dev = VStepLayer.from_host(L)
+    idx, n, stats = dev.step_trust(k_max, ratio)
+    torch.cuda.synchronize()
+    assert dev.status() == 0
+    n = int(n.item())
+    assert np.array_equal(idx.cpu().numpy().astype(np.uint32), order)
+    assert 1 < want.n_kept < k_max
+    near_tie = np.any(want.gap_rel <= REL)
+    if not near_tie:
+        assert n == want.n_kept
+        assert np.array_equal(dev.codes.cpu().numpy(), want.codes)
+    else:
+        assert abs(n - want.n_kept) <= 2
+    got = dev.codes.cpu().numpy().reshape(G, 1)
+    rest = np.setdiff1d(np.arange(G), order[:n].astype(np.int64))
+    assert np.array_equal(got[rest], L.codes.reshape(G, 1)[rest])
+    s = stats.cpu().numpy()
+    # both sides add rows*cols non-negative binary64 terms, in different orders: each within n * 2^-53 of the sum
+    assert abs(s[0] - want.sq_norm) <= (L.rows * L.cols) * 2.0 ** -52 * want.sq_norm
+    assert s[1] < ratio ** 2 * s[0]
+
+
+def test_full_size_step_with_groups_of_16():
+    """4096 x 4096 in groups of 16 weights, one fp16 codebook of 65 536, tau = 0.01: the tensor engine's 48-half
+    operand rows at the full codebook size; codes of a seeded sample against the checker."""
+    L = synth.make_layer(4096, 4096, cfg=2, codebook_size=65536, codebook_fp16=True, group_dim=16)
+    G = L.num_groups
+    k = synth.subspace_size("0.01", G)
+    dev = VStepLayer.from_host(L)
+    W_hat = torch.empty(4096, 4096, device="cuda")
+    idx, _ = dev.step(k, W_hat=W_hat)
+    torch.cuda.synchronize()
+    assert dev.status() == 0
+    want_idx = oracle.select(oracle.group_norms(L.g, L.eta, 16), k)
+    assert np.array_equal(idx.cpu().numpy().astype(np.uint32), want_idx)
+    got = dev.codes.cpu().numpy().reshape(G, 1)
+    pick = np.sort(np.random.default_rng(960).choice(k, size=4096, replace=False))
+    sel = want_idx[pick]
+    t = oracle.targets(L.W, L.g, L.scale, L.eta, sel, 16)
+    enc = oracle.encode(t, L.codebooks, L.codes[sel.astype(np.int64)])
+    exact, band = helpers.check_codes_against_oracle(t, L.codebooks, got[sel.astype(np.int64)], enc, REL)
+    assert exact >= 4096 - 8
+    mask = np.ones(G, bool)
+    mask[want_idx.astype(np.int64)] = False
+    assert np.array_equal(got[mask], L.codes.reshape(G, 1)[mask])
+    rows = np.unique(np.random.default_rng(961).integers(0, 4096, size=8))
+    sub = np.concatenate([got[r * 256:(r + 1) * 256] for r in rows])
+    want_W = oracle.dequant(sub, L.codebooks, L.scale[rows], len(rows), 4096)
+    assert W_hat[torch.from_numpy(rows).cuda()].cpu().numpy().tobytes() == want_W.tobytes()
