@@ -141,11 +141,197 @@ __global__ void __launch_bounds__(kPsThreads) pstep_grad_kernel(const float* __r
   }
 }
 
+
+// Small codebooks with one-byte codes (M K <= 512): no floating-point atomics in the block.  A block takes tiles
+// of 512 groups; per tile it stages the exact products s * g in shared memory, counting-sorts the tile's groups by
+// code (integer shared-memory atomics hand out the slots), and then every accumulator (codebook, code, element)
+// is owned by one thread, which adds the products of the code's groups in binary64 with plain
+// additions.  The accumulators go to the L2 once per block.
+constexpr int kPsTile = 512;
+
+template <int M, bool CB_F16>
+__global__ void __launch_bounds__(kPsThreads) pstep_grad_sorted_kernel(const float* __restrict__ g,
+                                                                        const float* __restrict__ scale,
+                                                                        const uint8_t* __restrict__ codes,
+                                                                        const void* __restrict__ codebooks, uint64_t G,
+                                                                        uint32_t gpr, uint32_t K,
+                                                                        double* __restrict__ grad_books,
+                                                                        double* __restrict__ grad_scale,
+                                                                        uint32_t* status) {
+  extern __shared__ __align__(16) unsigned char ps_smem[];
+  double* sh_acc = reinterpret_cast<double*>(ps_smem);                       // [M*K*8]
+  double* sh_p = sh_acc + (size_t)M * K * 8;                                 // [tile][8]: the exact products s * g
+  uint32_t* sh_cnt = reinterpret_cast<uint32_t*>(sh_p + kPsTile * 8);        // [M][256] counts
+  uint32_t* sh_start = sh_cnt + M * 256;                                     // [M][256]
+  uint16_t* sh_sorted = reinterpret_cast<uint16_t*>(sh_start + M * 256);     // [M][tile]
+  uint16_t* sh_slot = sh_sorted + M * kPsTile;                               // [M][tile]: slot of group in its bin
+  uint8_t* sh_code = reinterpret_cast<uint8_t*>(sh_slot + M * kPsTile);      // [M][tile]
+
+  for (uint32_t i = threadIdx.x; i < (uint32_t)M * K * 8; i += kPsThreads) sh_acc[i] = 0.0;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const float4* g4 = reinterpret_cast<const float4*>(g);
+  const uint64_t n_tiles = (G + kPsTile - 1) / kPsTile;
+  for (uint64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+    const uint64_t j0 = tile * kPsTile;
+    const uint32_t n_here = (uint32_t)(G - j0 < (uint64_t)kPsTile ? G - j0 : (uint64_t)kPsTile);
+    __syncthreads();  // the previous tile has been consumed
+    for (uint32_t i = threadIdx.x; i < (uint32_t)M * 256; i += kPsThreads) sh_cnt[i] = 0;
+    __syncthreads();
+    // stage the tile: two threads per group (512 contiguous bytes per warp load); all loads of the tile are
+    // issued before the first use, the pass is bound by memory latency otherwise
+    constexpr int kIter = 2 * kPsTile / kPsThreads;  // 8 half-groups per thread
+    float4 gv_all[kIter];
+    uint32_t b_all[kIter][M];
+#pragma unroll
+    for (int it = 0; it < kIter; ++it) {
+      const uint32_t hh = it * kPsThreads + threadIdx.x, slot = hh >> 1, half = hh & 1u;
+      gv_all[it] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int m = 0; m < M; ++m) b_all[it][m] = 0;
+      if (slot < n_here) {
+        const uint64_t j = j0 + slot;
+        gv_all[it] = __ldcs(g4 + 2 * j + half);
+#pragma unroll
+        for (int m = 0; m < M; ++m) b_all[it][m] = __ldg(codes + j * M + m);
+      }
+    }
+#pragma unroll
+    for (int it = 0; it < kIter; ++it) {
+      const uint32_t hh = it * kPsThreads + threadIdx.x, slot = hh >> 1, half = hh & 1u;
+      const uint64_t j = j0 + slot;
+      uint32_t row = 0xffffffffu;
+      double ds = 0.0;
+      if (slot < n_here) {
+        const float4 gv = gv_all[it];
+        row = (uint32_t)j / gpr;
+        uint32_t b[M];
+        bool bad = false;
+#pragma unroll
+        for (int m = 0; m < M; ++m) {
+          b[m] = b_all[it][m];
+          if (b[m] >= K) {
+            bad = true;
+            b[m] = 0;
+          }
+        }
+        {
+          const double sd = bad ? 0.0 : (double)__ldg(scale + row);  // a group with a bad code contributes nothing
+          double* dst = &sh_p[slot * 8 + half * 4];
+          dst[0] = sd * (double)gv.x;
+          dst[1] = sd * (double)gv.y;
+          dst[2] = sd * (double)gv.z;
+          dst[3] = sd * (double)gv.w;
+        }
+        if (half == 0) {
+#pragma unroll
+          for (int m = 0; m < M; ++m) {
+            sh_code[m * kPsTile + slot] = (uint8_t)b[m];
+            sh_slot[m * kPsTile + slot] = (uint16_t)atomicAdd(&sh_cnt[m * 256 + b[m]], 1u);
+          }
+        }
+        if (bad) {
+          if (status) atomicOr(status, PVT_DEV_BAD_CODE);
+        } else if (grad_scale) {
+          float4 v = half_codeword<CB_F16>(codebooks, b[0], half);
+#pragma unroll
+          for (int m = 1; m < M; ++m) {
+            const float4 v2 = half_codeword<CB_F16>(codebooks, m * K + b[m], half);
+            v.x = __fadd_rn(v.x, v2.x);
+            v.y = __fadd_rn(v.y, v2.y);
+            v.z = __fadd_rn(v.z, v2.z);
+            v.w = __fadd_rn(v.w, v2.w);
+          }
+          ds = (double)gv.x * (double)v.x;
+          ds = __dadd_rn(ds, (double)gv.y * (double)v.y);
+          ds = __dadd_rn(ds, (double)gv.z * (double)v.z);
+          ds = __dadd_rn(ds, (double)gv.w * (double)v.w);
+        }
+      }
+      if (grad_scale) {
+        const uint32_t row0 = __shfl_sync(0xffffffffu, row, 0);
+        if (__all_sync(0xffffffffu, row == row0)) {
+#pragma unroll
+          for (int o = 16; o; o >>= 1) ds = __dadd_rn(ds, __shfl_xor_sync(0xffffffffu, ds, o));
+          if (lane == 0 && row0 != 0xffffffffu) red_add_f64(grad_scale + row0, ds);
+        } else if (row != 0xffffffffu) {
+          red_add_f64(grad_scale + row, ds);
+        }
+      }
+    }
+    __syncthreads();
+    // exclusive prefix of the counts per codebook: one warp per codebook, eight bins per lane
+    if (warp < M) {
+      uint32_t c[8], sum = 0;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        c[q] = sh_cnt[warp * 256 + lane * 8 + q];
+        sum += c[q];
+      }
+      uint32_t incl = sum;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+      }
+      uint32_t run = incl - sum;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        sh_start[warp * 256 + lane * 8 + q] = run;
+        run += c[q];
+      }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int m = 0; m < M; ++m)
+      for (uint32_t slot = threadIdx.x; slot < n_here; slot += kPsThreads) {
+        const uint32_t code = sh_code[m * kPsTile + slot];
+        sh_sorted[m * kPsTile + sh_start[m * 256 + code] + sh_slot[m * kPsTile + slot]] = (uint16_t)slot;
+      }
+    __syncthreads();
+    // every accumulator (codebook, code, element) is owned by one thread: plain binary64 additions over the
+    // code's groups; eight adjacent threads share a code, so its group list is a broadcast load
+#pragma unroll
+    for (int m = 0; m < M; ++m)
+      for (uint32_t bin = threadIdx.x; bin < K * 8; bin += kPsThreads) {
+        const uint32_t code = bin >> 3, e = bin & 7u;
+        const uint32_t cnt = sh_cnt[m * 256 + code];
+        if (cnt == 0) continue;
+        const uint16_t* list = &sh_sorted[m * kPsTile + sh_start[m * 256 + code]];
+        double acc = 0.0;
+        for (uint32_t i = 0; i < cnt; ++i) acc = __dadd_rn(acc, sh_p[(uint32_t)list[i] * 8 + e]);
+        sh_acc[((size_t)m * K + code) * 8 + e] += acc;
+      }
+  }
+  __syncthreads();
+  for (uint32_t i = threadIdx.x; i < (uint32_t)M * K * 8; i += kPsThreads)
+    if (sh_acc[i] != 0.0) red_add_f64(grad_books + i, sh_acc[i]);
+}
+
+template <int M, bool CB_F16>
+cudaError_t launch_grad_sorted(const pvt_layer& L, uint64_t G, double* grad_books, double* grad_scale, uint32_t* status,
+                               int sm_count, cudaStream_t stream) {
+  const uint32_t gpr = (uint32_t)(L.cols / kGroupDim), K = (uint32_t)L.codebook_size;
+  const size_t smem = sizeof(double) * M * K * 8 + sizeof(double) * kPsTile * 8 + sizeof(uint32_t) * M * 512 +
+                      sizeof(uint16_t) * M * kPsTile * 2 + (size_t)M * kPsTile;
+  cudaError_t e = cudaFuncSetAttribute(pstep_grad_sorted_kernel<M, CB_F16>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  int per_sm = 0;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, pstep_grad_sorted_kernel<M, CB_F16>, kPsThreads, smem);
+  if (e != cudaSuccess) return e;
+  if (per_sm < 1) per_sm = 1;
+  const uint64_t tiles = (G + kPsTile - 1) / kPsTile, cap = (uint64_t)sm_count * per_sm;
+  pstep_grad_sorted_kernel<M, CB_F16><<<(unsigned)(tiles < cap ? tiles : cap), kPsThreads, smem, stream>>>(
+      L.g, L.scale, static_cast<const uint8_t*>(L.codes), L.codebooks, G, gpr, K, grad_books, grad_scale, status);
+  return cudaGetLastError();
+}
+
 template <int M, bool CB_F16, bool CODE_U16>
 cudaError_t launch_grad(const pvt_layer& L, uint64_t G, double* grad_books, double* grad_scale, uint32_t* status,
                         int sm_count, cudaStream_t stream) {
   const uint32_t gpr = (uint32_t)(L.cols / kGroupDim), K = (uint32_t)L.codebook_size;
   const bool smem_acc = (uint32_t)M * K <= (uint32_t)kPsSmemCodewords;
+  if (smem_acc && !CODE_U16) return launch_grad_sorted<M, CB_F16>(L, G, grad_books, grad_scale, status, sm_count, stream);
   const uint64_t want = (2 * G + kPsThreads - 1) / kPsThreads;
   const uint64_t cap = (uint64_t)sm_count * (smem_acc ? 4 : 8);
   const unsigned blocks = (unsigned)(want < cap ? want : cap);
