@@ -33,6 +33,7 @@ CASES = [
     (4, 2, "0.01", torch.float16),
     (5, 1, "0.01", torch.float32),
     (5, 3, "0.01", torch.float32),
+    (5, 1, "1.0", torch.float32),   # every group re-encoded (1 048 576 targets): the selection is the index list
 ]
 
 

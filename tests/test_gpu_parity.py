@@ -431,3 +431,53 @@ def test_whole_step_with_three_codebooks():
     assert np.array_equal(to_np(idx).astype(np.uint32), want.idx)
     assert np.array_equal(to_np(dev.codes), want.codes)
     assert to_np(W_hat).tobytes() == oracle.dequant(want.codes, L.codebooks, L.scale, 64, 512).tobytes()
+
+
+# ------------------------------------------------------------------ repeatability and graph replay
+
+
+@pytest.mark.parametrize("M,K", [(1, 4096), (2, 256)])
+def test_step_is_repeatable_and_replays_from_a_cuda_graph(M, K):
+    """The three calls of a step give the same indices, codes and weights when run again on the same inputs, and
+    when captured once into a CUDA graph and replayed (the calls only enqueue work on the given stream)."""
+    L = synth.make_layer(128, 1024, cfg=250 + M, num_codebooks=M, codebook_size=K, codebook_fp16=True,
+                         nearest=oracle_nearest)
+    k = 900
+    results = []
+    for _ in range(2):
+        dev = VStepLayer.from_host(L, max_k=k)
+        idx, W_hat = dev.step(k, W_hat=torch.empty(128, 1024, device="cuda"))
+        torch.cuda.synchronize()
+        assert dev.status() == 0
+        results.append((to_np(idx), to_np(dev.codes), to_np(W_hat)))
+    for a, b in zip(results[0], results[1]):
+        assert a.tobytes() == b.tobytes()
+
+    dev = VStepLayer.from_host(L, max_k=k)
+    codes0 = dev.codes.clone()
+    idx = torch.empty(k, dtype=torch.int32, device="cuda")
+    W_hat = torch.empty(128, 1024, device="cuda")
+    ws = dev.reserve(k)
+    stream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        # one eager pass first: anything the library sets up lazily happens outside the capture
+        B.pvt_vstep_select(dev.desc, k, idx, ws, stream=stream)
+        B.pvt_vstep_encode(dev.desc, idx, k, None, ws, stream=stream)
+        B.pvt_dequant(dev.desc, W_hat, stream=stream)
+        stream.synchronize()
+        with torch.cuda.graph(graph, stream=stream):
+            B.pvt_vstep_select(dev.desc, k, idx, ws, stream=stream)
+            B.pvt_vstep_encode(dev.desc, idx, k, None, ws, stream=stream)
+            B.pvt_dequant(dev.desc, W_hat, stream=stream)
+    for _ in range(2):
+        dev.codes.copy_(codes0)
+        idx.zero_()
+        W_hat.zero_()
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert dev.status() == 0
+        assert to_np(idx).tobytes() == results[0][0].tobytes()
+        assert to_np(dev.codes).tobytes() == results[0][1].tobytes()
+        assert to_np(W_hat).tobytes() == results[0][2].tobytes()
