@@ -59,16 +59,25 @@ namespace {
 
 constexpr int kTcTile = 256;            // targets per CTA tile
 constexpr int kTcStepCw = 128;          // codewords per MMA step (the N of one instruction)
-// Operand geometry for groups of DG weights: a row holds the two halves of the target (or the codeword
-// twice), eight norm slots and eight zeros: 32 halves for DG = 8, 48 for DG = 16.
+// Operand geometry for groups of DG weights.  The codeword appears once per row of the codebook image; the two
+// halves of the target meet it in separate instructions that read the same K chunks of B:
+//   DG = 8:   A row = [ hi | 2^e x 8 | lo | 0 ]  (4 chunks),  B row = [ c | norm terms ]  (2 chunks)
+//             instruction 0: A chunks 0-1 x B chunks 0-1;  instruction 1: A chunks 2-3 x B chunks 0-1
+//   DG = 16:  A row = [ hi x 16 | lo x 16 | 2^e x 8 | 0 ]  (6 chunks),  B row = [ c x 16 | norm terms | 0 ]  (4 chunks)
+//             instructions: A 0-1 x B 0-1, A 2-3 x B 0-1, A 4-5 x B 2-3
 template <int DG>
 struct TcDim {
-  static constexpr int kRowBytes = 2 * (2 * DG + 16);          // 64 or 96
-  static constexpr int kStepBytes = kTcStepCw * kRowBytes;     // 8192 or 12288
-  static constexpr int kGroupBytes = 8 * kRowBytes;            // one 8-row group: kChunks core matrices of 128 bytes
-  static constexpr int kChunks = kRowBytes / 16;               // 16-byte K chunks per row: 4 or 6
-  static constexpr int kMmas = kChunks / 2;                    // instructions per step and A block
-  static constexpr int kPart = DG / 8;                         // K chunks per copy of the codeword
+  static constexpr int kARowBytes = 2 * (2 * DG + 16);         // 64 or 96
+  static constexpr int kAGroupBytes = 8 * kARowBytes;          // one 8-row group of A
+  static constexpr int kABlockBytes = 128 * kARowBytes;        // one A block of 128 targets
+  static constexpr int kBRowBytes = DG == 8 ? 32 : 64;
+  static constexpr int kBGroupBytes = 8 * kBRowBytes;
+  static constexpr int kStepBytes = kTcStepCw * kBRowBytes;    // codebook image per step: 4096 or 8192
+  static constexpr int kMmas = DG == 8 ? 2 : 3;                // instructions per step and A block
+  static constexpr int kPart = DG / 8;                         // K chunks per codeword
+  // K chunk at which instruction m starts reading A and B
+  __host__ __device__ static constexpr int a_chunk(int m) { return 2 * m; }
+  __host__ __device__ static constexpr int b_chunk(int m) { return (DG == 16 && m == 2) ? 2 : 0; }
 };
 constexpr int kTcStepBytes = TcDim<8>::kStepBytes;
 constexpr int kTcSubCw = 64;            // tracking granularity of the running maximum
@@ -188,14 +197,11 @@ __global__ void __launch_bounds__(256) tc_prep_kernel(const uint4* __restrict__ 
       k1 = make_uint4(0xfbfffbffu, 0xfbfffbffu, 0xfbfffbffu, 0xfbfffbffu);  // -65504 x 8
     }
     const uint32_t step = kappa / kTcStepCw, r = kappa % kTcStepCw;
-    unsigned char* row = bimg + (size_t)step * D::kStepBytes + (r >> 3) * D::kGroupBytes + (r & 7) * 16;
+    unsigned char* row = bimg + (size_t)step * D::kStepBytes + (r >> 3) * D::kBGroupBytes + (r & 7) * 16;
 #pragma unroll
-    for (int part = 0; part < D::kPart; ++part) {
-      *reinterpret_cast<uint4*>(row + 128 * part) = raw[part];                 // pairs with hi
-      *reinterpret_cast<uint4*>(row + 128 * (D::kPart + part)) = raw[part];    // pairs with lo
-    }
-    *reinterpret_cast<uint4*>(row + 128 * (2 * D::kPart)) = k1;  // norm terms
-    *reinterpret_cast<uint4*>(row + 128 * (2 * D::kPart + 1)) = make_uint4(0, 0, 0, 0);
+    for (int part = 0; part < D::kPart; ++part) *reinterpret_cast<uint4*>(row + 128 * part) = raw[part];
+    *reinterpret_cast<uint4*>(row + 128 * D::kPart) = k1;  // norm terms
+    if (DG == 16) *reinterpret_cast<uint4*>(row + 128 * (D::kPart + 1)) = make_uint4(0, 0, 0, 0);
   }
   n2bits = __reduce_max_sync(0xffffffffu, n2bits);
   if ((threadIdx.x & 31) == 0 && n2bits > __ldcg(&stats->n2max_bits)) atomicMax(&stats->n2max_bits, n2bits);
@@ -298,7 +304,7 @@ __device__ __forceinline__ float max64(const uint32_t* v) {
 // ---- shared memory -----------------------------------------------------------------
 template <int DG>
 struct TcSmem {
-  alignas(128) unsigned char a[2][TcDim<DG>::kStepBytes];  // two A blocks of 128 targets
+  alignas(128) unsigned char a[2][TcDim<DG>::kABlockBytes];  // two A blocks of 128 targets
   alignas(128) unsigned char b[kTcStages][kTcGroupSteps][TcDim<DG>::kStepBytes];
   alignas(8) uint64_t full_bar[kTcStages];
   uint64_t empty_bar[kTcStages];
@@ -396,7 +402,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
     // ------------------------------------------------------------ MMA issuers: warp 9 -> A block 0, warp 10 -> A block 1
     if (lane == 0) {
       const uint32_t q = (uint32_t)warp - 9u;
-      const uint64_t a_desc = smem_desc(smem_u32(&sm.a[q][0]), D::kGroupBytes);
+      const uint64_t a_desc = smem_desc(smem_u32(&sm.a[q][0]), D::kAGroupBytes);
       // A lone thread pays about 150 cycles for a wait on an mbarrier (even on a finished phase) and about
       // 50 per MMA or commit, and its loop is part of the hand-over ring of the accumulators: per step one wait
       // (accumulator free), two MMAs, one commit; the codebook stage costs a wait and a commit per four steps.
@@ -406,7 +412,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
         slice_units(p, (uint32_t)(u % p.n_slices), &s_lo, &s_hi);
         total += s_hi - s_lo;
       }
-      const uint64_t b_desc0 = smem_desc(smem_u32(&sm.b[0][0][0]), D::kGroupBytes);
+      const uint64_t b_desc0 = smem_desc(smem_u32(&sm.b[0][0][0]), D::kBGroupBytes);
       const uint32_t full0 = smem_u32(&sm.tmem_full[0][q]), full1 = smem_u32(&sm.tmem_full[1][q]);
       const uint32_t empty0 = smem_u32(&sm.tmem_empty[0][q]), empty1 = smem_u32(&sm.tmem_empty[1][q]);
       bool alive = true;
@@ -423,12 +429,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
           if (!alive) break;
           tc_fence_after();
           const uint64_t b_desc = b_desc0 + (uint64_t)((s * kTcGroupSteps + sub) * (kStepBytes >> 4));
-          // two K chunks per instruction: the halves of the target against the codeword, then the norm terms on top
+          // two K chunks per instruction (see TcDim for which chunks of A meet which chunks of B)
           const uint32_t d = tmem_base + buf * 256 + q * 128;
-          umma_f16(d, a_desc, b_desc, kIdesc, 0);
 #pragma unroll
-          for (int m = 1; m < D::kMmas; ++m)
-            umma_f16(d, a_desc + m * kDescTwoChunks, b_desc + m * kDescTwoChunks, kIdesc, 1);
+          for (int m = 0; m < D::kMmas; ++m)
+            umma_f16(d, a_desc + (uint64_t)(D::a_chunk(m) * (128 >> 4)), b_desc + (uint64_t)(D::b_chunk(m) * (128 >> 4)),
+                     kIdesc, m > 0);
           umma_commit(buf ? full1 : full0);  // the accumulator is ready
           if (sub == (uint32_t)kTcGroupSteps - 1 && it + 1 < total)
             umma_commit(smem_u32(&sm.empty_bar[s]));  // this warp has read the whole stage
@@ -448,7 +454,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
     const float n2max = __uint_as_float(stats->n2max_bits);
     const float cnmax = sqrtf(n2max), hmax = 0.5f * n2max;
     const uint32_t rb = (uint32_t)tid >> 7, r = (uint32_t)tid & 127u;
-    unsigned char* a_row = &sm.a[rb][(r >> 3) * D::kGroupBytes + (r & 7) * 16];
+    unsigned char* a_row = &sm.a[rb][(r >> 3) * D::kAGroupBytes + (r & 7) * 16];
     const uint32_t lane_base = ((uint32_t)(warp & 3) * 32u) << 16;
     uint32_t it = 0;
     bool alive = true;
@@ -498,13 +504,20 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
         }
         const __half2 s2 = __floats2half2_rn(sc, sc);
         const uint32_t sb = *reinterpret_cast<const uint32_t*>(&s2);
+        if (DG == 8) {  // [ hi | 2^e | lo | 0 ]
+          *reinterpret_cast<uint4*>(a_row) = reinterpret_cast<const uint4*>(hi)[0];
+          *reinterpret_cast<uint4*>(a_row + 128) = make_uint4(sb, sb, sb, sb);
+          *reinterpret_cast<uint4*>(a_row + 256) = reinterpret_cast<const uint4*>(lo)[0];
+          *reinterpret_cast<uint4*>(a_row + 384) = make_uint4(0, 0, 0, 0);
+        } else {        // [ hi x 16 | lo x 16 | 2^e | 0 ]
 #pragma unroll
-        for (int part = 0; part < D::kPart; ++part) {
-          *reinterpret_cast<uint4*>(a_row + 128 * part) = reinterpret_cast<const uint4*>(hi)[part];
-          *reinterpret_cast<uint4*>(a_row + 128 * (D::kPart + part)) = reinterpret_cast<const uint4*>(lo)[part];
+          for (int part = 0; part < D::kPart; ++part) {
+            *reinterpret_cast<uint4*>(a_row + 128 * part) = reinterpret_cast<const uint4*>(hi)[part];
+            *reinterpret_cast<uint4*>(a_row + 128 * (D::kPart + part)) = reinterpret_cast<const uint4*>(lo)[part];
+          }
+          *reinterpret_cast<uint4*>(a_row + 128 * (2 * D::kPart)) = make_uint4(sb, sb, sb, sb);
+          *reinterpret_cast<uint4*>(a_row + 128 * (2 * D::kPart + 1)) = make_uint4(0, 0, 0, 0);
         }
-        *reinterpret_cast<uint4*>(a_row + 128 * (2 * D::kPart)) = make_uint4(sb, sb, sb, sb);
-        *reinterpret_cast<uint4*>(a_row + 128 * (2 * D::kPart + 1)) = make_uint4(0, 0, 0, 0);
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the MMA
       mbar_arrive(smem_u32(&sm.a_ready));
