@@ -240,7 +240,6 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t group_byt
          ((uint64_t)(group_bytes >> 4) << 32) | (1ull << 46);
 }
 // instruction descriptor: D fp32, A and B fp16, both K-major, N = 128, M = 128
-constexpr uint64_t kDescTwoChunks = 256u >> 4;  // start-address field advance for two K chunks
 constexpr uint32_t kIdesc = (1u << 4) | ((uint32_t)(kTcStepCw >> 3) << 17) | ((128u >> 4) << 24);
 
 // 32 lanes x 64 consecutive columns of 32-bit accumulators -> 64 registers per thread
