@@ -346,7 +346,7 @@ def run_ours(args):
                                                   (props.multi_processor_count * 128 * sm_max_mhz * 1e6),
                         "epilogue_bound_is": "one accumulator read per pair: 128 lanes per SM per clock",
                         # dram__bytes_read + dram__bytes_write of one launch (ncu, this kernel, default workload)
-                        "traffic": 9.73e6 if args.workload == DEFAULT_WORKLOAD else None}
+                        "traffic": 7.64e6 if args.workload == DEFAULT_WORKLOAD else None}
         else:
             roofline = {"kernel": "encode search (M=1, fp32 pipe)" if M == 1 else "encode beam search (M=2)",
                         "bound": "alu", "achieved": achieved, "peak": alu_peak, "unit": "TFLOP/s",
