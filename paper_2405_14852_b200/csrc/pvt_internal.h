@@ -152,6 +152,33 @@ cudaError_t launch_trust_after_search(const pvt_layer& L, uint64_t G, uint64_t k
 cudaError_t launch_refine(const pvt_layer& L, uint64_t G, const uint32_t* idx, uint64_t k, int max_moves,
                           float* err_out, uint32_t* moves_out, uint32_t* status, cudaStream_t stream);
 
+// ---- programmatic dependent launch --------------------------------------------------------------------
+// Consecutive kernels of a call depend on one another, so between two of them the GPU would idle for a launch
+// latency.  A kernel launched with launch_dependent() may be scheduled while the kernel before it on the stream
+// is still running; it must execute pdl_wait() before its first access to global memory, which returns once
+// that kernel has completed and its writes are visible.  Every kernel of a chain calls pdl_trigger() at its
+// start to allow the one after it to be scheduled early.  Both are no-ops for a kernel launched the plain way.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_dependent(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem, cudaStream_t stream,
+                             Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(block);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+#endif
+
 // optional per-kernel timing (benchmark instrumentation) ----------------------
 enum KernelId {
   kKernSelect = 0, kKernEncodeMain = 1, kKernEncodeAux = 2, kKernDequant = 3, kKernEncodeRescore = 4,

@@ -119,6 +119,8 @@ template <int LP>
 __global__ void __launch_bounds__(kSelThreads) norm_hist_kernel(const float* __restrict__ g, uint64_t G, float eta,
                                                                  uint64_t k, uint32_t* __restrict__ keys,
                                                                  uint32_t* __restrict__ hist0, SelectState* st) {
+  pdl_trigger();
+  pdl_wait();
   constexpr int kTile = kSelThreads * kNormPer / LP;  // groups per block and iteration
   __shared__ uint32_t sh_hist[kSelBins0];
   __shared__ uint64_t sh_scan[kSelThreads / 32];
@@ -168,6 +170,8 @@ __global__ void __launch_bounds__(kSelThreads) refine_mid_kernel(const uint32_t*
                                                                   uint32_t* __restrict__ hist1,
                                                                   uint32_t* __restrict__ cand, uint32_t cand_cap,
                                                                   SelectState* st) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ uint32_t sh_hist[kSelBins1];
   __shared__ uint64_t sh_scan[kSelThreads / 32];
   __shared__ uint32_t sh_stage[kMidStage + 8 * kSelThreads];  // room for one more iteration after the check
@@ -243,6 +247,8 @@ __global__ void __launch_bounds__(kSelThreads) refine_low_kernel(const uint32_t*
                                                                   const uint32_t* __restrict__ cand,
                                                                   uint32_t cand_cap, uint32_t* __restrict__ hist2,
                                                                   SelectState* st) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ uint32_t sh_hist[kSelBins2];
   __shared__ uint64_t sh_scan[kSelThreads / 32];
   for (int b = threadIdx.x; b < kSelBins2; b += kSelThreads) sh_hist[b] = 0;
@@ -276,6 +282,8 @@ __global__ void __launch_bounds__(kSelThreads) refine_low_kernel(const uint32_t*
 __global__ void __launch_bounds__(kSelThreads) tile_count_kernel(const uint32_t* __restrict__ keys, uint64_t G,
                                                                   uint32_t* __restrict__ tiles, uint32_t ntiles,
                                                                   uint64_t k, SelectState* st, uint32_t* status) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ uint32_t sh_gt, sh_eq;
   __shared__ uint64_t sh_scan[kSelThreads / 32];
   if (threadIdx.x == 0) sh_gt = sh_eq = 0;
@@ -344,6 +352,8 @@ __global__ void __launch_bounds__(kSelThreads) scatter_kernel(const uint32_t* __
                                                                const uint32_t* __restrict__ tiles,
                                                                const SelectState* st, uint64_t k,
                                                                uint32_t* __restrict__ idx_out) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ uint64_t sh_scan[kSelThreads / 32];
   const uint32_t T = st->threshold, need_eq = st->need_eq;
   constexpr int PER = kSelTile / kSelThreads;  // consecutive groups per thread: keeps index order
@@ -441,12 +451,15 @@ cudaError_t launch_select(const pvt_layer& L, uint64_t G, uint64_t k, uint32_t* 
     norm_hist_kernel<2><<<norm_grid, kSelThreads, 0, stream>>>(L.g, G, L.eta, k, keys, hist0, st);
   else
     norm_hist_kernel<4><<<norm_grid, kSelThreads, 0, stream>>>(L.g, G, L.eta, k, keys, hist0, st);
-  refine_mid_kernel<<<mid_grid, kSelThreads, 0, stream>>>(keys, G, hist1, cand, lay.cand_cap, st);
+  err = launch_dependent(refine_mid_kernel, mid_grid, kSelThreads, 0, stream, keys, G, hist1, cand, lay.cand_cap, st);
+  if (err != cudaSuccess) return err;
   const unsigned low_grid = (unsigned)(lay.cand_cap / 8192 < (uint32_t)sm_count ? lay.cand_cap / 8192 + 1 : sm_count);
-  refine_low_kernel<<<low_grid, kSelThreads, 0, stream>>>(keys, G, cand, lay.cand_cap, hist2, st);
-  tile_count_kernel<<<lay.ntiles, kSelThreads, 0, stream>>>(keys, G, tiles, lay.ntiles, k, st, status);
-  scatter_kernel<<<lay.ntiles, kSelThreads, 0, stream>>>(keys, G, tiles, st, k, idx_out);
-  err = cudaGetLastError();
+  err = launch_dependent(refine_low_kernel, low_grid, kSelThreads, 0, stream, keys, G, cand, lay.cand_cap, hist2, st);
+  if (err != cudaSuccess) return err;
+  err = launch_dependent(tile_count_kernel, lay.ntiles, kSelThreads, 0, stream, keys, G, tiles, lay.ntiles, k, st, status);
+  if (err != cudaSuccess) return err;
+  err = launch_dependent(scatter_kernel, lay.ntiles, kSelThreads, 0, stream, keys, G, tiles, st, k, idx_out);
+  if (err == cudaSuccess) err = cudaGetLastError();
   count_launches(5);
   timing_end(kKernSelect, stream);
   return err;
