@@ -99,7 +99,7 @@ __device__ void find_digit(const uint32_t* hist, uint64_t k_left, uint32_t* digi
   }
 }
 
-constexpr int kNormPer = 4;                              // 16-byte loads per thread and iteration of the norm pass
+constexpr int kNormPer = 8;                              // 16-byte loads per thread and iteration of the norm pass
 
 // LP adjacent lanes share a group (LP = group size / 4: 2 or 4), lane q of them holding elements 4q..4q+3,
 // so a warp reads 512 contiguous bytes per load instruction.  The sum is a single chain in index order:
