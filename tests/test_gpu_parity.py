@@ -481,3 +481,30 @@ def test_step_is_repeatable_and_replays_from_a_cuda_graph(M, K):
         assert to_np(idx).tobytes() == results[0][0].tobytes()
         assert to_np(dev.codes).tobytes() == results[0][1].tobytes()
         assert to_np(W_hat).tobytes() == results[0][2].tobytes()
+
+
+# ------------------------------------------------------------------ small codebooks on the tensor engine, negative scales
+
+
+@pytest.mark.parametrize("K", [2, 3, 100, 129])
+def test_tiny_codebooks_on_the_tensor_engine(K):
+    """Codebooks far below one 128-codeword step: padding rows must never win."""
+    L = synth.make_layer(64, 256, cfg=260, codebook_size=K, codebook_fp16=True)
+    idx = np.arange(0, L.num_groups, 2, dtype=np.uint32)
+    with search_engine("tensor"):
+        check_encode(L, idx)
+
+
+@pytest.mark.parametrize("engine", ["fp32", "tensor"])
+def test_negative_row_scales(engine):
+    """Row scales only have to be finite and non-zero: the target divides by them, the dequantised weight
+    multiplies by them."""
+    L = synth.make_layer(64, 512, cfg=261, codebook_size=2048, codebook_fp16=True)
+    L.scale[::3] *= -1.0
+    idx = oracle.select(oracle.group_norms(L.g, L.eta), 700)
+    with search_engine(engine):
+        check_encode(L, idx)
+    dev = VStepLayer.from_host(L)
+    out = dev.dequant()
+    torch.cuda.synchronize()
+    assert to_np(out).tobytes() == oracle.dequant(L.codes, L.codebooks, L.scale, 64, 512).tobytes()
