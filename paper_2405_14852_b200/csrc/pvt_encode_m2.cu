@@ -192,32 +192,40 @@ __global__ void __launch_bounds__(kM2Threads, 2) encode_m2_kernel(const EncM2Par
     uint32_t my_j = 0xffffffffu, my_prev = 0;
     float my_margin2 = 0.0f;
 
+    // the four targets of the group, one element per lane (lane = 8 * target + element): index, W, g, row scale
+    // and previous pair are fetched for all four at once, one fma and one division per lane (binary32)
+    uint32_t lane_j = 0xffffffffu, lane_prev = 0;
+    {
+      const uint64_t n_mine = gi * kM2Group + my_q;
+      if (n_mine < p.k) lane_j = __ldg(p.idx + n_mine);
+      float tv = 0.0f;
+      if (lane_j < p.G) {
+        const float wv = __ldg(p.W + (size_t)lane_j * 8 + my_b), gv = __ldg(p.g + (size_t)lane_j * 8 + my_b);
+        const float sc = __ldg(p.scale + lane_j / p.gpr);
+        lane_prev = p.codes[lane_j];
+        tv = __fdiv_rn(__fmaf_rn(-p.eta, gv, wv), sc);
+      }
+      sm.wt[warp][my_q][my_b] = tv;
+    }
+    __syncwarp();
+
     // ---- stage 1, one target after the other, the whole warp on each
 #pragma unroll 1
     for (uint32_t q = 0; q < (uint32_t)kM2Group; ++q) {
       const uint64_t n = gi * kM2Group + q;
       if (n >= p.k) break;
-      const uint32_t j = __ldg(p.idx + n);
+      const uint32_t j = __shfl_sync(0xffffffffu, lane_j, 8 * q);
+      const uint32_t prev = __shfl_sync(0xffffffffu, lane_prev, 8 * q);
       if (j >= p.G) {
         if (lane == 0) atomicOr(p.status, PVT_DEV_BAD_INDEX);
         continue;
       }
-      // target, binary32: one fma, one division (every lane holds all 8 values)
       float t[8];
       {
-        const float4 w0 = __ldg(W4 + 2 * (size_t)j), w1 = __ldg(W4 + 2 * (size_t)j + 1);
-        const float4 g0 = __ldg(g4 + 2 * (size_t)j), g1 = __ldg(g4 + 2 * (size_t)j + 1);
-        const float sc = __ldg(p.scale + j / p.gpr), ne = -p.eta;
-        t[0] = __fdiv_rn(__fmaf_rn(ne, g0.x, w0.x), sc);
-        t[1] = __fdiv_rn(__fmaf_rn(ne, g0.y, w0.y), sc);
-        t[2] = __fdiv_rn(__fmaf_rn(ne, g0.z, w0.z), sc);
-        t[3] = __fdiv_rn(__fmaf_rn(ne, g0.w, w0.w), sc);
-        t[4] = __fdiv_rn(__fmaf_rn(ne, g1.x, w1.x), sc);
-        t[5] = __fdiv_rn(__fmaf_rn(ne, g1.y, w1.y), sc);
-        t[6] = __fdiv_rn(__fmaf_rn(ne, g1.z, w1.z), sc);
-        t[7] = __fdiv_rn(__fmaf_rn(ne, g1.w, w1.w), sc);
+        const float4 ta = *reinterpret_cast<const float4*>(&sm.wt[warp][q][0]);
+        const float4 tb = *reinterpret_cast<const float4*>(&sm.wt[warp][q][4]);
+        t[0] = ta.x, t[1] = ta.y, t[2] = ta.z, t[3] = ta.w, t[4] = tb.x, t[5] = tb.y, t[6] = tb.z, t[7] = tb.w;
       }
-      const uint32_t prev = p.codes[j];
       float nt2 = 0.0f;
 #pragma unroll
       for (int i = 0; i < 8; ++i) nt2 = fmaf(t[i], t[i], nt2);
@@ -317,8 +325,6 @@ __global__ void __launch_bounds__(kM2Threads, 2) encode_m2_kernel(const EncM2Par
       }
       // hand the target and its beam to the lanes of stage 2
       if (lane == 0) {
-        *reinterpret_cast<float4*>(&sm.wt[warp][q][0]) = make_float4(t[0], t[1], t[2], t[3]);
-        *reinterpret_cast<float4*>(&sm.wt[warp][q][4]) = make_float4(t[4], t[5], t[6], t[7]);
         *reinterpret_cast<uint4*>(&sm.wk[warp][q][0]) = make_uint4(beam_code[0], beam_code[1], beam_code[2], beam_code[3]);
         *reinterpret_cast<uint4*>(&sm.wk[warp][q][4]) = make_uint4(beam_code[4], beam_code[5], beam_code[6], beam_code[7]);
       }
