@@ -70,8 +70,7 @@ extern "C" {
  *     W_hat[r, 8c + i] = scale[r] * sum_m codebooks[m][codes[j][m]][i].
  * Supported: group_dim 8; M = 1 with 2 <= K <= 65536 (codes U8 if K <= 256, else
  * U16; U16 is accepted for any K); M = 2, 3, 4 with 2 <= K <= 256, codes U8, 1 <=
- * beam <= 8 (M = 3, 4: select, encode and dequant only; the other calls return
- * PVT_EUNSUPPORTED).  group_dim 16 (Appendix J's one-codebook representations
+ * beam <= 8.  group_dim 16 (Appendix J's one-codebook representations
  * with groups of 16 weights): M = 1 only, select, encode and dequant only; read
  * "8" as "16" in the layouts below.
  */
@@ -204,7 +203,7 @@ int pvt_vstep_encode(const pvt_layer* layer, const uint32_t* idx, uint64_t k, fl
  *          double[2]: ||W_hat_old||^2 and the squared change that was kept.
  * ws: pvt_trust_workspace_bytes(layer, k_max) bytes, 256-byte aligned, header
  *     cleared by pvt_workspace_init; status bits as for the other calls.
- * Two codebooks need one-byte codes and 1 <= beam <= 8 (PVT_EUNSUPPORTED).
+ * Two to four codebooks need one-byte codes and 1 <= beam <= 8 (PVT_EUNSUPPORTED).
  * Returns as pvt_vstep_encode; ratio must be finite and >= 0 (PVT_EINVAL).
  */
 size_t pvt_trust_workspace_bytes(const pvt_layer* layer, uint64_t k_max);
@@ -228,7 +227,7 @@ int pvt_vstep_trust(const pvt_layer* layer, uint64_t k_max, float ratio, uint32_
  * err_out: NULL or device float[k], final error rounded to binary32.  moves_out:
  * NULL or device uint32[k], moves taken.  status: NULL or a device uint32 into
  * which PVT_DEV_BAD_INDEX / PVT_DEV_BAD_CODE are OR-ed (such groups are skipped).
- * No workspace.  Two codebooks need one-byte codes (PVT_EUNSUPPORTED).
+ * No workspace.  Two to four codebooks need one-byte codes (PVT_EUNSUPPORTED).
  */
 int pvt_vstep_refine(const pvt_layer* layer, const uint32_t* idx, uint64_t k, int32_t max_moves, float* err_out,
                      uint32_t* moves_out, uint32_t* status, void* cuda_stream);

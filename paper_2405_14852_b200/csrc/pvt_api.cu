@@ -207,10 +207,10 @@ int pvt_vstep_trust(const pvt_layer* layer, uint64_t k_max, float ratio, uint32_
   if (!aligned16(layer->W) || !aligned16(layer->g) || !aligned16(layer->codebooks)) return PVT_EINVAL;
   if ((reinterpret_cast<uintptr_t>(n_out) & 7u) || (reinterpret_cast<uintptr_t>(stats_out) & 7u)) return PVT_EINVAL;
   if (reinterpret_cast<uintptr_t>(ws) & (kWsAlign - 1)) return PVT_EINVAL;
-  if (layer->num_codebooks > 2 || layer->group_dim != kGroupDim) return PVT_EUNSUPPORTED;
-  if (layer->num_codebooks == 2) {
+  if (layer->group_dim != kGroupDim) return PVT_EUNSUPPORTED;
+  if (layer->num_codebooks >= 2) {
     if (layer->code_dtype != PVT_U8 || layer->beam < 1 || layer->beam > 8) return PVT_EUNSUPPORTED;
-    if (reinterpret_cast<uintptr_t>(layer->codes) & 1u) return PVT_EINVAL;
+    if (layer->num_codebooks == 2 && (reinterpret_cast<uintptr_t>(layer->codes) & 1u)) return PVT_EINVAL;
   }
   const int sms = sm_count();
   const TrustLayout t = trust_layout(G, k_max, encode_bytes(*layer, k_max, sms), sms);
@@ -240,11 +240,8 @@ int pvt_vstep_refine(const pvt_layer* layer, const uint32_t* idx, uint64_t k, in
   if (k < 1 || k > G || max_moves < 0 || max_moves > 65535) return PVT_EINVAL;
   if (!layer->W || !layer->g || !layer->scale || !layer->codebooks || !layer->codes || !idx) return PVT_EINVAL;
   if (!aligned16(layer->W) || !aligned16(layer->g) || !aligned16(layer->codebooks)) return PVT_EINVAL;
-  if (layer->num_codebooks > 2 || layer->group_dim != kGroupDim) return PVT_EUNSUPPORTED;
-  if (layer->num_codebooks == 2) {
-    if (layer->code_dtype != PVT_U8) return PVT_EUNSUPPORTED;
-    if (reinterpret_cast<uintptr_t>(layer->codes) & 1u) return PVT_EINVAL;
-  }
+  if (layer->group_dim != kGroupDim) return PVT_EUNSUPPORTED;
+  if (layer->num_codebooks >= 2 && layer->code_dtype != PVT_U8) return PVT_EUNSUPPORTED;
   const cudaError_t e = launch_refine(*layer, G, idx, k, max_moves, err_out, moves_out, status,
                                       static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? PVT_OK : fail_cuda(e);
@@ -270,7 +267,7 @@ int pvt_pstep_grad(const pvt_layer* layer, double* grad_codebooks, double* grad_
   int rc = check_layer(layer, &G);
   if (rc != PVT_OK) return rc;
   if ((rc = check_quantiser(layer)) != PVT_OK) return rc;
-  if (layer->num_codebooks > 2 || layer->group_dim != kGroupDim) return PVT_EUNSUPPORTED;
+  if (layer->group_dim != kGroupDim) return PVT_EUNSUPPORTED;
   if (!layer->g || !layer->scale || !layer->codebooks || !layer->codes || !grad_codebooks) return PVT_EINVAL;
   if (!aligned16(layer->g) || !aligned16(layer->codebooks)) return PVT_EINVAL;
   if ((reinterpret_cast<uintptr_t>(grad_codebooks) & 7u) || (reinterpret_cast<uintptr_t>(grad_scale) & 7u))

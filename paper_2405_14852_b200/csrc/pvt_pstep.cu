@@ -75,7 +75,9 @@ __global__ void __launch_bounds__(kPsThreads) pstep_grad_kernel(const float* __r
         b[0] = both & 0xffu;
         b[M - 1] = both >> 8;
       } else {
-        b[0] = __ldg(reinterpret_cast<const uint8_t*>(codes) + j);
+        const uint8_t* c = reinterpret_cast<const uint8_t*>(codes) + (size_t)j * M;
+#pragma unroll
+        for (int m = 0; m < M; ++m) b[m] = __ldg(c + m);
       }
       bool bad = false;
 #pragma unroll
@@ -108,8 +110,9 @@ __global__ void __launch_bounds__(kPsThreads) pstep_grad_kernel(const float* __r
         }
         if (grad_scale) {
           float4 v = half_codeword<CB_F16>(codebooks, b[0], half);
-          if (M == 2) {
-            const float4 v2 = half_codeword<CB_F16>(codebooks, K + b[M - 1], half);
+#pragma unroll
+          for (int m = 1; m < M; ++m) {
+            const float4 v2 = half_codeword<CB_F16>(codebooks, m * K + b[m], half);
             v.x = __fadd_rn(v.x, v2.x);
             v.y = __fadd_rn(v.y, v2.y);
             v.z = __fadd_rn(v.z, v2.z);
@@ -420,13 +423,19 @@ cudaError_t launch_pstep_grad(const pvt_layer& L, uint64_t G, double* grad_books
     else
       err = u16 ? launch_grad<1, false, true>(L, G, grad_books, grad_scale, status, sm_count, stream)
                 : launch_grad<1, false, false>(L, G, grad_books, grad_scale, status, sm_count, stream);
-  } else {
+  } else if (L.num_codebooks == 2) {
     if (f16)
       err = u16 ? launch_grad<2, true, true>(L, G, grad_books, grad_scale, status, sm_count, stream)
                 : launch_grad<2, true, false>(L, G, grad_books, grad_scale, status, sm_count, stream);
     else
       err = u16 ? launch_grad<2, false, true>(L, G, grad_books, grad_scale, status, sm_count, stream)
                 : launch_grad<2, false, false>(L, G, grad_books, grad_scale, status, sm_count, stream);
+  } else if (L.num_codebooks == 3) {  // three and four codebooks: one-byte codes
+    err = f16 ? launch_grad<3, true, false>(L, G, grad_books, grad_scale, status, sm_count, stream)
+              : launch_grad<3, false, false>(L, G, grad_books, grad_scale, status, sm_count, stream);
+  } else {
+    err = f16 ? launch_grad<4, true, false>(L, G, grad_books, grad_scale, status, sm_count, stream)
+              : launch_grad<4, false, false>(L, G, grad_books, grad_scale, status, sm_count, stream);
   }
   count_launches(1);
   timing_end(kKernPstepGrad, stream);

@@ -3,7 +3,7 @@
 // codebooks.  A move replaces one code of the group's tuple by the value that lowers ||t - sum_m C_m[b_m]||^2
 // most (the neighbour that is smallest under (error, tuple)), and is taken only if the error strictly drops.
 //
-// One warp per target.  Every error is the binary64 sum the final decision of the search kernels uses
+// One warp per target, one to four codebooks.  Every error is the binary64 sum the final decision of the search kernels uses
 // (residual through the codebooks in order, terms added in element order), so the moves are decided on exact
 // values and the error can only fall.  All M*K neighbours are evaluated per move: M*K*8 binary64 multiply-adds
 // per target and move, a few moves per target.
@@ -51,14 +51,16 @@ __device__ __forceinline__ void global_codeword(const void* books, uint32_t row,
   }
 }
 
-// ||t - c||^2 (M = 1) or ||(t - c1) - c2||^2 (M = 2), binary64, element order
+// ||t - c_1 - ... - c_M||^2 with the residual carried in binary64 through the codebooks in order and the terms
+// added in element order; cw[m] = the codeword of codebook m
 template <int M>
-__device__ __forceinline__ double tuple_error(const float t[8], const float c1[8], const float c2[8]) {
+__device__ __forceinline__ double tuple_error(const float t[8], const float (*cw)[8]) {
   double d = 0.0;
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
-    double e = __dsub_rn((double)t[i], (double)c1[i]);
-    if (M == 2) e = __dsub_rn(e, (double)c2[i]);
+    double e = (double)t[i];
+#pragma unroll
+    for (int m = 0; m < M; ++m) e = __dsub_rn(e, (double)cw[m][i]);
     d = __dadd_rn(d, __dmul_rn(e, e));
   }
   return d;
@@ -106,79 +108,98 @@ __global__ void __launch_bounds__(kRfThreads) refine_kernel(const RefineParams p
 #pragma unroll
     for (int i = 0; i < 8; ++i) t[i] = __fdiv_rn(__fmaf_rn(ne, gg[i], w[i]), s);
   }
-  uint32_t b[2] = {0, 0};
+  uint32_t b[M];
+  bool ok = true;
   if (M == 1) {
     b[0] = CODE_U16 ? reinterpret_cast<const uint16_t*>(p.codes)[j] : reinterpret_cast<const uint8_t*>(p.codes)[j];
   } else {
-    const uint16_t both = reinterpret_cast<const uint16_t*>(p.codes)[j];  // two adjacent bytes
-    b[0] = both & 0xffu;
-    b[1] = both >> 8;
+    const uint8_t* c = reinterpret_cast<const uint8_t*>(p.codes) + (size_t)j * M;
+#pragma unroll
+    for (int m = 0; m < M; ++m) b[m] = c[m];
   }
-  if (b[0] >= K || (M == 2 && b[1] >= K)) {
+#pragma unroll
+  for (int m = 0; m < M; ++m) ok = ok && b[m] < K;
+  if (!ok) {
     if (lane == 0 && p.status) atomicOr(p.status, PVT_DEV_BAD_CODE);
     return;
   }
-  float c1[8], c2[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-  codeword(b[0], c1);
-  if (M == 2) codeword(K + b[1], c2);
-  double d_cur = tuple_error<M>(t, c1, c2);
+  float cw[M][8];
+#pragma unroll
+  for (int m = 0; m < M; ++m) codeword((uint32_t)m * K + b[m], cw[m]);
+  double d_cur = tuple_error<M>(t, cw);
   uint32_t moves = 0;
   while (moves < (uint32_t)p.max_moves) {
-    // best neighbour of this lane under (error, tuple); tuple key = b1 * K + b2 (b1 alone for one codebook)
+    // best neighbour of this lane under (error, tuple); a neighbour is named by (codebook changed, new code)
     double ld = __longlong_as_double(0x7ff0000000000000ll);
-    uint32_t lkey = 0xffffffffu;
-    for (uint32_t q = lane; q < K; q += 32) {  // change the first code
-      if (q == b[0]) continue;
-      float c[8];
-      codeword(q, c);
-      const double d = tuple_error<M>(t, c, c2);
-      const uint32_t key = M == 2 ? q * K + b[1] : q;
-      if (d < ld || (d == ld && key < lkey)) {
-        ld = d;
-        lkey = key;
+    uint32_t lm = 0, lq = 0;
+    bool lhave = false;
+    auto tuple_less = [&](uint32_t m1, uint32_t q1, uint32_t m2, uint32_t q2) {
+      // lexicographic order of the two neighbours' tuples (both differ from the current tuple in one place)
+#pragma unroll
+      for (int m = 0; m < M; ++m) {
+        const uint32_t x = (uint32_t)m == m1 ? q1 : b[m], y = (uint32_t)m == m2 ? q2 : b[m];
+        if (x != y) return x < y;
       }
-    }
-    if (M == 2) {
-      for (uint32_t q = lane; q < K; q += 32) {  // change the second code
-        if (q == b[1]) continue;
-        float c[8];
-        codeword(K + q, c);
-        const double d = tuple_error<M>(t, c1, c);
-        const uint32_t key = b[0] * K + q;
-        if (d < ld || (d == ld && key < lkey)) {
+      return false;
+    };
+#pragma unroll
+    for (int m = 0; m < M; ++m) {
+      float keep[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) keep[i] = cw[m][i];
+      for (uint32_t q = lane; q < K; q += 32) {
+        if (q == b[m]) continue;
+        codeword((uint32_t)m * K + q, cw[m]);
+        const double d = tuple_error<M>(t, cw);
+        if (!lhave || d < ld || (d == ld && tuple_less((uint32_t)m, q, lm, lq))) {
           ld = d;
-          lkey = key;
+          lm = (uint32_t)m;
+          lq = q;
+          lhave = true;
         }
       }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) cw[m][i] = keep[i];
     }
-    // warp-wide minimum of (error, key); errors are >= 0, so their bits order like u64
+    // warp-wide minimum of (error, tuple); errors are >= 0, so their bits order like u64
     const uint64_t bits = (uint64_t)__double_as_longlong(ld);
     const uint32_t hi = (uint32_t)(bits >> 32), lo = (uint32_t)bits;
     const uint32_t mhi = __reduce_min_sync(0xffffffffu, hi);
     const uint32_t mlo = __reduce_min_sync(0xffffffffu, hi == mhi ? lo : 0xffffffffu);
-    const uint32_t mkey = __reduce_min_sync(0xffffffffu, (hi == mhi && lo == mlo) ? lkey : 0xffffffffu);
-    const double md = __longlong_as_double((long long)(((uint64_t)mhi << 32) | mlo));
-    if (mkey == 0xffffffffu || !(md < d_cur)) break;  // warp-uniform
-    if (M == 2) {
-      b[0] = mkey / K;
-      b[1] = mkey % K;
-      codeword(b[0], c1);
-      codeword(K + b[1], c2);
-    } else {
-      b[0] = mkey;
-      codeword(b[0], c1);
+    const bool tied = lhave && hi == mhi && lo == mlo;
+    // among the lanes that hold the minimum error: the smallest tuple, codebook by codebook
+    uint32_t alive_mask = __ballot_sync(0xffffffffu, tied);
+    if (alive_mask == 0 || !(__longlong_as_double((long long)(((uint64_t)mhi << 32) | mlo)) < d_cur)) break;
+    bool mine = tied;
+#pragma unroll
+    for (int m = 0; m < M; ++m) {
+      const uint32_t x = mine ? ((uint32_t)m == lm ? lq : b[m]) : 0xffffffffu;
+      const uint32_t mx = __reduce_min_sync(0xffffffffu, x);
+      mine = mine && x == mx;
     }
-    d_cur = md;
+    const int winner = __ffs(__ballot_sync(0xffffffffu, mine)) - 1;  // exactly one lane (tuples are distinct)
+    const uint32_t wm = __shfl_sync(0xffffffffu, lm, winner), wq = __shfl_sync(0xffffffffu, lq, winner);
+#pragma unroll
+    for (int m = 0; m < M; ++m)
+      if ((uint32_t)m == wm) {
+        b[m] = wq;
+        codeword((uint32_t)m * K + wq, cw[m]);
+      }
+    d_cur = __longlong_as_double((long long)(((uint64_t)mhi << 32) | mlo));
     ++moves;
   }
   if (lane == 0) {
     if (moves) {
-      if (M == 2)
-        reinterpret_cast<uint16_t*>(p.codes)[j] = (uint16_t)(b[0] | (b[1] << 8));
-      else if (CODE_U16)
-        reinterpret_cast<uint16_t*>(p.codes)[j] = (uint16_t)b[0];
-      else
-        reinterpret_cast<uint8_t*>(p.codes)[j] = (uint8_t)b[0];
+      if (M == 1) {
+        if (CODE_U16)
+          reinterpret_cast<uint16_t*>(p.codes)[j] = (uint16_t)b[0];
+        else
+          reinterpret_cast<uint8_t*>(p.codes)[j] = (uint8_t)b[0];
+      } else {
+        uint8_t* c = reinterpret_cast<uint8_t*>(p.codes) + (size_t)j * M;
+#pragma unroll
+        for (int m = 0; m < M; ++m) c[m] = (uint8_t)b[m];
+      }
     }
     if (p.err_out) p.err_out[n] = (float)d_cur;
     if (p.moves_out) p.moves_out[n] = moves;
@@ -221,6 +242,10 @@ cudaError_t launch_refine(const pvt_layer& L, uint64_t G, const uint32_t* idx, u
   cudaError_t e;
   if (L.num_codebooks == 2)
     e = f16 ? launch_staged<2, true, false>(p, stream) : launch_staged<2, false, false>(p, stream);
+  else if (L.num_codebooks == 3)
+    e = f16 ? launch_staged<3, true, false>(p, stream) : launch_staged<3, false, false>(p, stream);
+  else if (L.num_codebooks == 4)
+    e = f16 ? launch_staged<4, true, false>(p, stream) : launch_staged<4, false, false>(p, stream);
   else if (f16)
     e = u16 ? launch_staged<1, true, true>(p, stream) : launch_staged<1, true, false>(p, stream);
   else

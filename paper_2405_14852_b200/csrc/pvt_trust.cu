@@ -147,19 +147,26 @@ __global__ void __launch_bounds__(kSortThreads) sort_scatter_kernel(const uint64
 
 // ---- codes and dequantised values ------------------------------------------------------------------------------
 
+// codes of a group packed into one word: the two-byte code itself for two-byte codes (one codebook), otherwise
+// byte m = code of codebook m
 template <bool CODE_U16>
 __device__ __forceinline__ uint32_t load_codes(const void* codes, uint32_t j, int M) {
   if (CODE_U16) return reinterpret_cast<const uint16_t*>(codes)[j];  // M == 1
   if (M == 2) return reinterpret_cast<const uint16_t*>(codes)[j];    // two adjacent bytes: first | second << 8
-  return reinterpret_cast<const uint8_t*>(codes)[j];
+  const uint8_t* c = reinterpret_cast<const uint8_t*>(codes) + (size_t)j * M;
+  uint32_t packed = 0;
+  for (int m = 0; m < M; ++m) packed |= (uint32_t)c[m] << (8 * m);
+  return packed;
 }
 
 template <bool CODE_U16>
 __device__ __forceinline__ void store_codes(void* codes, uint32_t j, int M, uint32_t packed) {
-  if (CODE_U16 || M == 2)
+  if (CODE_U16 || M == 2) {
     reinterpret_cast<uint16_t*>(codes)[j] = (uint16_t)packed;
-  else
-    reinterpret_cast<uint8_t*>(codes)[j] = (uint8_t)packed;
+  } else {
+    uint8_t* c = reinterpret_cast<uint8_t*>(codes) + (size_t)j * M;
+    for (int m = 0; m < M; ++m) c[m] = (uint8_t)(packed >> (8 * m));
+  }
 }
 
 template <bool CB_F16>
@@ -184,14 +191,14 @@ __device__ __forceinline__ void codeword(const void* book, uint32_t code, float 
 template <bool CB_F16>
 __device__ __forceinline__ bool group_weights(const void* books, uint32_t K, int M, uint32_t packed, bool code_u16,
                                               float s, float w[8]) {
-  const uint32_t b0 = (M == 2 && !code_u16) ? (packed & 0xffu) : packed;
-  const uint32_t b1 = packed >> 8;
-  bool ok = b0 < K && (M == 1 || b1 < K);
+  const uint32_t b0 = (M >= 2 && !code_u16) ? (packed & 0xffu) : packed;
+  bool ok = b0 < K;
+  for (int m = 1; m < M; ++m) ok = ok && ((packed >> (8 * m)) & 0xffu) < K;
   float v[8];
   codeword<CB_F16>(books, ok ? b0 : 0, v);
-  if (M == 2) {
+  for (int m = 1; m < M; ++m) {  // codebooks added left to right, each sum rounded once
     float v2[8];
-    codeword<CB_F16>(books, K + (ok ? b1 : 0), v2);
+    codeword<CB_F16>(books, (uint32_t)m * K + (ok ? ((packed >> (8 * m)) & 0xffu) : 0u), v2);
 #pragma unroll
     for (int i = 0; i < 8; ++i) v[i] = __fadd_rn(v[i], v2[i]);
   }

@@ -23,6 +23,9 @@ def oracle_nearest(X, C):
     (1, 65536, True, 512, 1024),   # accumulation straight in L2
     (2, 256, True, 96, 136),
     (2, 64, False, 33, 72),
+    (3, 128, True, 64, 256),       # three codebooks, sorted tiles (384 codewords)
+    (4, 256, True, 64, 512),       # four codebooks: 1024 codewords, accumulation straight in L2
+    (4, 64, False, 33, 72),
 ])
 def test_pstep_grad_matches_checker(M, K, f16, rows, cols):
     L = synth.make_layer(rows, cols, cfg=110 + M, num_codebooks=M, codebook_size=K, codebook_fp16=f16,

@@ -36,6 +36,9 @@ def gpu_refine(L, idx_np, max_moves, encode_first=False):
     (2, 256, True, 64, 512, 1500),
     (2, 200, False, 33, 72, 297),      # every group, ragged sizes
     (1, 256, False, 64, 256, 900),
+    (3, 64, True, 64, 256, 600),
+    (4, 256, True, 32, 512, 300),      # codebooks read through L2 (1024 codewords)
+    (4, 16, False, 32, 128, 512),
     (1, 2048, True, 64, 512, 333),     # two-byte codes; codebook read through L2 instead of shared memory
 ])
 @pytest.mark.parametrize("max_moves", [0, 1, 64])

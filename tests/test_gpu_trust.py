@@ -74,6 +74,8 @@ def run_case(L, k_max, ratio):
     (1, 2048, True, 100, 264, 3300, 0.05),      # ragged sizes
     (2, 256, True, 128, 1024, 3000, 0.03),
     (2, 200, True, 96, 136, 1632, 0.1),
+    (3, 64, True, 128, 512, 2000, 0.05),
+    (4, 32, False, 64, 512, 1500, 0.05),
 ])
 def test_trust_step_matches_checker(M, K, f16, rows, cols, k_max, ratio):
     L = settle(synth.make_layer(rows, cols, cfg=180 + M, num_codebooks=M, codebook_size=K, codebook_fp16=f16,
