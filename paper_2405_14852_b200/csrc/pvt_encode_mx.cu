@@ -50,6 +50,7 @@ __global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p)
   extern __shared__ __align__(16) unsigned char smem_raw[];
   float* book = reinterpret_cast<float*>(smem_raw);                               // [M][K][8]
   double* resid = reinterpret_cast<double*>(smem_raw + (size_t)M * p.K * 32);     // [warps][beam][8]
+  float* resid_f = reinterpret_cast<float*>(resid + kMxWarps * kMxBeam * 8);      // the same, rounded to binary32
   const uint32_t K = p.K;
   for (uint32_t row = threadIdx.x; row < M * K; row += kMxThreads) {
     float c[8];
@@ -93,6 +94,7 @@ __global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p)
     for (int i = 0; i < 8; ++i) t[i] = __fdiv_rn(__fmaf_rn(ne, gg[i], w[i]), s);
   }
   double* my_resid = resid + (size_t)warp * kMxBeam * 8;
+  float* my_resid_f = resid_f + (size_t)warp * kMxBeam * 8;
   const int beam = p.beam;
 
   // kept partial tuples: key = code_1 << 24 | code_2 << 16 | ... (lexicographic order of tuples = numeric order)
@@ -123,6 +125,7 @@ __global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p)
         r = __dsub_rn(r, (double)book[((size_t)q * K + code) * 8 + i]);
       }
       my_resid[b * 8 + i] = r;
+      my_resid_f[b * 8 + i] = (float)r;
     }
     __syncwarp();
 
@@ -137,10 +140,24 @@ __global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p)
     const int keep = (m == M - 1) ? 1 : beam;
     const uint32_t n_cand = (uint32_t)n_kept * K;
     const int shift = 24 - 8 * m;
+    float worst_fl = __int_as_float(0x7f800000);  // binary32 bound above which a candidate cannot enter this lane's list
     for (uint32_t cnd = lane; cnd < n_cand; cnd += 32) {
       const uint32_t b = cnd / K, q = cnd - b * K;
       const float* c = &book[((size_t)m * K + q) * 8];
       const double* r = &my_resid[b * 8];
+      const float* rf = &my_resid_f[b * 8];
+      // binary32 estimate first: |d_fl - d| <= 2^-20 d (eight roundings of the residual to binary32, eight
+      // differences, squares and sums), so a candidate whose estimate exceeds (1 + 2^-19) x the worst kept
+      // score cannot belong to the list, ties included
+      {
+        float dfl = 0.0f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const float e = rf[i] - c[i];
+          dfl = fmaf(e, e, dfl);
+        }
+        if (dfl > worst_fl) continue;
+      }
       double d = 0.0;
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
@@ -164,6 +181,12 @@ __global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p)
           key = tk;
         }
       }
+      // the list's last kept score, once the list is full, bounds what can still enter
+      double worst = ld[0];
+#pragma unroll
+      for (int x = 1; x < kMxBeam; ++x)
+        if (x < keep) worst = ld[x];
+      if (worst < __longlong_as_double(kInfBits)) worst_fl = __double2float_ru(worst) * 1.0000020f;  // > 1 + 2^-19
     }
 
     // the warp's `keep` smallest: repeated minimum over the lanes' current heads
@@ -250,7 +273,7 @@ __global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p)
 
 template <int M, bool CB_F16>
 cudaError_t launch_m(const MxParams& p, cudaStream_t stream) {
-  const size_t smem = (size_t)M * p.K * 32 + (size_t)kMxWarps * kMxBeam * 8 * sizeof(double);
+  const size_t smem = (size_t)M * p.K * 32 + (size_t)kMxWarps * kMxBeam * 8 * (sizeof(double) + sizeof(float));
   cudaError_t e = cudaFuncSetAttribute(encode_mx_kernel<M, CB_F16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)smem);
   if (e != cudaSuccess) return e;
