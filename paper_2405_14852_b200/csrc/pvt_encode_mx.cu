@@ -129,7 +129,65 @@ __global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p)
     }
     __syncwarp();
 
-    // this lane's `beam` smallest extensions (only the smallest matters at the last stage)
+    const int keep = (m == M - 1) ? 1 : beam;
+    const int shift = 24 - 8 * m;
+
+    // Pass 1, binary32 and branch-free: the estimate d_fl = sum_i (fl32(r_i) - c_i)^2 of every extension; each lane
+    // keeps its smallest estimate, the warp derives a threshold theta from the 32 minima.  With R = the largest residual norm, |d_fl - d| <= 2^-22 sqrt(d) R + 2^-20 d: the residual is
+    // rounded to binary32 (2^-24 |r_i| per element, which matters when the codeword nearly cancels it), the
+    // differences, squares and sums add relative roundings.
+    float r2max = 0.0f;
+    if (lane < n_kept) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) r2max = fmaf(my_resid_f[lane * 8 + i], my_resid_f[lane * 8 + i], r2max);
+    }
+    r2max = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(r2max)));  // non-negative: bits order like values
+    auto estimate = [&](const float4& ra, const float4& rb, const float* c) {
+      const float4 ca = *reinterpret_cast<const float4*>(c), cb = *reinterpret_cast<const float4*>(c + 4);
+      float e, dfl;
+      e = ra.x - ca.x; dfl = e * e;
+      e = ra.y - ca.y; dfl = fmaf(e, e, dfl);
+      e = ra.z - ca.z; dfl = fmaf(e, e, dfl);
+      e = ra.w - ca.w; dfl = fmaf(e, e, dfl);
+      e = rb.x - cb.x; dfl = fmaf(e, e, dfl);
+      e = rb.y - cb.y; dfl = fmaf(e, e, dfl);
+      e = rb.z - cb.z; dfl = fmaf(e, e, dfl);
+      e = rb.w - cb.w; dfl = fmaf(e, e, dfl);
+      return dfl;
+    };
+    uint32_t est_min = 0x7f800000u;  // this lane's smallest estimate (non-negative: bits order like values)
+    for (int b = 0; b < n_kept; ++b) {
+      const float4 ra = *reinterpret_cast<const float4*>(&my_resid_f[b * 8]);
+      const float4 rb = *reinterpret_cast<const float4*>(&my_resid_f[b * 8 + 4]);
+      for (uint32_t q = lane; q < K; q += 32)
+        est_min = min(est_min, __float_as_uint(estimate(ra, rb, &book[((size_t)m * K + q) * 8])));
+    }
+    // theta: the keep-th smallest of the 32 lane minima -- `keep` different extensions have an estimate of at
+    // most theta, so the exact keep-th smallest score lies within the error bound of it (a little looser than
+    // the keep-th smallest estimate overall, at one instruction per extension instead of a sorted insertion)
+    uint32_t theta_bits = 0x7f800000u;
+    {
+      uint32_t hv = est_min;
+      for (int round = 0; round < keep; ++round) {
+        const uint32_t mv = __reduce_min_sync(0xffffffffu, hv);
+        if (mv == 0x7f800000u) {  // fewer than `keep` lanes have an extension: everything survives
+          theta_bits = mv;
+          break;
+        }
+        theta_bits = mv;
+        const uint32_t owners = __ballot_sync(0xffffffffu, hv == mv);
+        if (lane == __ffs(owners) - 1) hv = 0x7f800000u;  // equal minima in several lanes: one leaves per round
+      }
+    }
+    // every member of the exact `keep` smallest has an estimate within the two error bounds of theta
+    const float theta = __uint_as_float(theta_bits);
+    const float bound = theta_bits == 0x7f800000u
+                            ? theta
+                            : theta + 4.0f * (2.3841858e-7f /* 2^-22 */ * sqrtf(theta * r2max) + 9.5367432e-7f /* 2^-20 */ * theta) +
+                                  1e-37f;
+
+    // Pass 2: the same estimates again (bit for bit); the few extensions within the bound are scored in binary64
+    // and kept in this lane's sorted list
     double ld[kMxBeam];
     uint32_t lk[kMxBeam];
 #pragma unroll
@@ -137,56 +195,37 @@ __global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p)
       ld[q] = __longlong_as_double(kInfBits);
       lk[q] = kNoKey;
     }
-    const int keep = (m == M - 1) ? 1 : beam;
-    const uint32_t n_cand = (uint32_t)n_kept * K;
-    const int shift = 24 - 8 * m;
-    float worst_fl = __int_as_float(0x7f800000);  // binary32 bound above which a candidate cannot enter this lane's list
-    for (uint32_t cnd = lane; cnd < n_cand; cnd += 32) {
-      const uint32_t b = cnd / K, q = cnd - b * K;
-      const float* c = &book[((size_t)m * K + q) * 8];
-      const double* r = &my_resid[b * 8];
-      const float* rf = &my_resid_f[b * 8];
-      // binary32 estimate first: |d_fl - d| <= 2^-20 d (eight roundings of the residual to binary32, eight
-      // differences, squares and sums), so a candidate whose estimate exceeds (1 + 2^-19) x the worst kept
-      // score cannot belong to the list, ties included
-      {
-        float dfl = 0.0f;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const float e = rf[i] - c[i];
-          dfl = fmaf(e, e, dfl);
-        }
-        if (dfl > worst_fl) continue;
-      }
-      double d = 0.0;
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const double e = __dsub_rn(r[i], (double)c[i]);
-        d = __dadd_rn(d, __dmul_rn(e, e));
-      }
+    for (int b = 0; b < n_kept; ++b) {
+      const float4 ra = *reinterpret_cast<const float4*>(&my_resid_f[b * 8]);
+      const float4 rb = *reinterpret_cast<const float4*>(&my_resid_f[b * 8 + 4]);
       uint32_t kb = kept_key[0];
 #pragma unroll
       for (int x = 1; x < kMxBeam; ++x)
-        if ((uint32_t)x == b) kb = kept_key[x];
-      uint32_t key = kb | (q << shift);
-      // insertion into the sorted list of `keep` entries: the new entry sinks to its place, the last one drops
+        if (x == b) kb = kept_key[x];
+      const double* r = &my_resid[b * 8];
+      for (uint32_t q = lane; q < K; q += 32) {
+        const float* c = &book[((size_t)m * K + q) * 8];
+        if (!(estimate(ra, rb, c) <= bound)) continue;
+        double d = 0.0;
 #pragma unroll
-      for (int x = 0; x < kMxBeam; ++x) {
-        if (x < keep && less_than(d, key, ld[x], lk[x])) {
-          const double td = ld[x];
-          const uint32_t tk = lk[x];
-          ld[x] = d;
-          lk[x] = key;
-          d = td;
-          key = tk;
+        for (int i = 0; i < 8; ++i) {
+          const double ee = __dsub_rn(r[i], (double)c[i]);
+          d = __dadd_rn(d, __dmul_rn(ee, ee));
+        }
+        uint32_t key = kb | (q << shift);
+        // insertion into the sorted list of `keep` entries: the new entry sinks to its place, the last one drops
+#pragma unroll
+        for (int x = 0; x < kMxBeam; ++x) {
+          if (x < keep && less_than(d, key, ld[x], lk[x])) {
+            const double td = ld[x];
+            const uint32_t tk = lk[x];
+            ld[x] = d;
+            lk[x] = key;
+            d = td;
+            key = tk;
+          }
         }
       }
-      // the list's last kept score, once the list is full, bounds what can still enter
-      double worst = ld[0];
-#pragma unroll
-      for (int x = 1; x < kMxBeam; ++x)
-        if (x < keep) worst = ld[x];
-      if (worst < __longlong_as_double(kInfBits)) worst_fl = __double2float_ru(worst) * 1.0000020f;  // > 1 + 2^-19
     }
 
     // the warp's `keep` smallest: repeated minimum over the lanes' current heads
