@@ -71,8 +71,8 @@ extern "C" {
  * Supported: group_dim 8; M = 1 with 2 <= K <= 65536 (codes U8 if K <= 256, else
  * U16; U16 is accepted for any K); M = 2, 3, 4 with 2 <= K <= 256, codes U8, 1 <=
  * beam <= 8.  group_dim 16 (Appendix J's one-codebook representations
- * with groups of 16 weights): M = 1 only, select, encode and dequant only; read
- * "8" as "16" in the layouts below.
+ * with groups of 16 weights): M = 1 only; every call but pvt_vstep_refine and
+ * pvt_vstep_select_noalloc takes it; read "8" as "16" in the layouts below.
  */
 typedef struct pvt_layer {
   int32_t rows, cols;     /* cols % group_dim == 0 */

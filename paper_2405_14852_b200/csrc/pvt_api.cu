@@ -207,7 +207,6 @@ int pvt_vstep_trust(const pvt_layer* layer, uint64_t k_max, float ratio, uint32_
   if (!aligned16(layer->W) || !aligned16(layer->g) || !aligned16(layer->codebooks)) return PVT_EINVAL;
   if ((reinterpret_cast<uintptr_t>(n_out) & 7u) || (reinterpret_cast<uintptr_t>(stats_out) & 7u)) return PVT_EINVAL;
   if (reinterpret_cast<uintptr_t>(ws) & (kWsAlign - 1)) return PVT_EINVAL;
-  if (layer->group_dim != kGroupDim) return PVT_EUNSUPPORTED;
   if (layer->num_codebooks >= 2) {
     if (layer->code_dtype != PVT_U8 || layer->beam < 1 || layer->beam > 8) return PVT_EUNSUPPORTED;
     if (layer->num_codebooks == 2 && (reinterpret_cast<uintptr_t>(layer->codes) & 1u)) return PVT_EINVAL;
@@ -267,7 +266,6 @@ int pvt_pstep_grad(const pvt_layer* layer, double* grad_codebooks, double* grad_
   int rc = check_layer(layer, &G);
   if (rc != PVT_OK) return rc;
   if ((rc = check_quantiser(layer)) != PVT_OK) return rc;
-  if (layer->group_dim != kGroupDim) return PVT_EUNSUPPORTED;
   if (!layer->g || !layer->scale || !layer->codebooks || !layer->codes || !grad_codebooks) return PVT_EINVAL;
   if (!aligned16(layer->g) || !aligned16(layer->codebooks)) return PVT_EINVAL;
   if ((reinterpret_cast<uintptr_t>(grad_codebooks) & 7u) || (reinterpret_cast<uintptr_t>(grad_scale) & 7u))

@@ -23,15 +23,16 @@ namespace {
 constexpr int kPsThreads = 256;
 constexpr int kPsSmemCodewords = 512;
 
-template <bool CB_F16>
+// elements 4*half .. 4*half+3 of a codeword of 4*PARTS elements (PARTS = 2 for groups of 8 weights, 4 for 16)
+template <bool CB_F16, int PARTS = 2>
 __device__ __forceinline__ float4 half_codeword(const void* book, uint32_t code, uint32_t half) {
   if (CB_F16) {
-    const uint2 raw = __ldg(reinterpret_cast<const uint2*>(book) + 2 * (size_t)code + half);
+    const uint2 raw = __ldg(reinterpret_cast<const uint2*>(book) + PARTS * (size_t)code + half);
     const float2 lo = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
     const float2 hi = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
     return make_float4(lo.x, lo.y, hi.x, hi.y);
   } else {
-    return __ldg(reinterpret_cast<const float4*>(book) + 2 * (size_t)code + half);
+    return __ldg(reinterpret_cast<const float4*>(book) + PARTS * (size_t)code + half);
   }
 }
 
@@ -39,7 +40,7 @@ __device__ __forceinline__ void red_add_f64(double* p, double v) {
   asm volatile("red.global.add.f64 [%0], %1;" ::"l"(p), "d"(v) : "memory");
 }
 
-template <int M, bool CB_F16, bool CODE_U16, bool SMEM_ACC>
+template <int M, bool CB_F16, bool CODE_U16, bool SMEM_ACC, int PARTS = 2>
 __global__ void __launch_bounds__(kPsThreads) pstep_grad_kernel(const float* __restrict__ g,
                                                                  const float* __restrict__ scale,
                                                                  const void* __restrict__ codes,
@@ -52,13 +53,13 @@ __global__ void __launch_bounds__(kPsThreads) pstep_grad_kernel(const float* __r
     for (uint32_t i = threadIdx.x; i < (uint32_t)M * K * 8; i += kPsThreads) sh_acc[i] = 0.0;
     __syncthreads();
   }
-  const uint64_t H = 2 * G;
+  const uint64_t H = (uint64_t)PARTS * G;  // PARTS threads per group, four weights each
   const float4* g4 = reinterpret_cast<const float4*>(g);
   const int lane = threadIdx.x & 31;
   for (uint64_t h0 = (uint64_t)blockIdx.x * kPsThreads; h0 < H; h0 += (uint64_t)gridDim.x * kPsThreads) {
     const uint64_t h = h0 + threadIdx.x;
     const bool valid = h < H;
-    const uint32_t j = (uint32_t)(h >> 1), half = (uint32_t)h & 1u;
+    const uint32_t j = (uint32_t)(h / PARTS), half = (uint32_t)h & (uint32_t)(PARTS - 1);
     uint32_t row = 0xffffffffu;
     double ds = 0.0;
     if (valid) {
@@ -95,7 +96,7 @@ __global__ void __launch_bounds__(kPsThreads) pstep_grad_kernel(const float* __r
         const double p0 = sd * (double)gv.x, p1 = sd * (double)gv.y, p2 = sd * (double)gv.z, p3 = sd * (double)gv.w;
 #pragma unroll
         for (int m = 0; m < M; ++m) {
-          const size_t at = ((size_t)m * K + b[m]) * 8 + half * 4;
+          const size_t at = ((size_t)m * K + b[m]) * (4 * PARTS) + half * 4;
           if (SMEM_ACC) {
             atomicAdd(&sh_acc[at], p0);
             atomicAdd(&sh_acc[at + 1], p1);
@@ -109,10 +110,10 @@ __global__ void __launch_bounds__(kPsThreads) pstep_grad_kernel(const float* __r
           }
         }
         if (grad_scale) {
-          float4 v = half_codeword<CB_F16>(codebooks, b[0], half);
+          float4 v = half_codeword<CB_F16, PARTS>(codebooks, b[0], half);
 #pragma unroll
           for (int m = 1; m < M; ++m) {
-            const float4 v2 = half_codeword<CB_F16>(codebooks, m * K + b[m], half);
+            const float4 v2 = half_codeword<CB_F16, PARTS>(codebooks, m * K + b[m], half);
             v.x = __fadd_rn(v.x, v2.x);
             v.y = __fadd_rn(v.y, v2.y);
             v.z = __fadd_rn(v.z, v2.z);
@@ -333,6 +334,12 @@ template <int M, bool CB_F16, bool CODE_U16>
 cudaError_t launch_grad(const pvt_layer& L, uint64_t G, double* grad_books, double* grad_scale, uint32_t* status,
                         int sm_count, cudaStream_t stream) {
   const uint32_t gpr = (uint32_t)(L.cols / kGroupDim), K = (uint32_t)L.codebook_size;
+  if (L.group_dim == 16) {  // groups of 16 weights (one codebook): four threads per group, reductions in the L2
+    const uint64_t want16 = (4 * G + kPsThreads - 1) / kPsThreads, cap16 = (uint64_t)sm_count * 8;
+    pstep_grad_kernel<M, CB_F16, CODE_U16, false, 4><<<(unsigned)(want16 < cap16 ? want16 : cap16), kPsThreads, 0, stream>>>(
+        L.g, L.scale, L.codes, L.codebooks, G, (uint32_t)(L.cols / 16), K, grad_books, grad_scale, status);
+    return cudaGetLastError();
+  }
   const bool smem_acc = (uint32_t)M * K <= (uint32_t)kPsSmemCodewords;
   if (smem_acc && !CODE_U16) return launch_grad_sorted<M, CB_F16>(L, G, grad_books, grad_scale, status, sm_count, stream);
   const uint64_t want = (2 * G + kPsThreads - 1) / kPsThreads;
@@ -410,7 +417,7 @@ cudaError_t launch_adam_direction(const float* grad, float* exp_avg, float* exp_
 cudaError_t launch_pstep_grad(const pvt_layer& L, uint64_t G, double* grad_books, double* grad_scale, uint32_t* status,
                               int sm_count, cudaStream_t stream) {
   cudaError_t err = cudaMemsetAsync(grad_books, 0,
-                                    sizeof(double) * (size_t)L.num_codebooks * (size_t)L.codebook_size * kGroupDim, stream);
+                                    sizeof(double) * (size_t)L.num_codebooks * (size_t)L.codebook_size * (size_t)L.group_dim, stream);
   if (err != cudaSuccess) return err;
   if (grad_scale && (err = cudaMemsetAsync(grad_scale, 0, sizeof(double) * (size_t)L.rows, stream)) != cudaSuccess)
     return err;

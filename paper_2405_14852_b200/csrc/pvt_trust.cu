@@ -38,6 +38,7 @@ constexpr int kCutThreads = 1024;
 
 // pair = (~key) << 32 | position in the ascending index list.  Sorting the pairs by their upper half in ascending
 // order, stably, gives (norm descending, index ascending).
+template <int DG>
 __global__ void __launch_bounds__(256) rank_init_kernel(const float* __restrict__ g, uint64_t G, float eta,
                                                         const uint32_t* __restrict__ idx, uint64_t k,
                                                         uint64_t* __restrict__ pairs, uint32_t* status) {
@@ -46,14 +47,16 @@ __global__ void __launch_bounds__(256) rank_init_kernel(const float* __restrict_
   const uint32_t j = __ldg(idx + a);
   uint32_t key = 0;
   if (j < G) {
-    const float4* src = reinterpret_cast<const float4*>(g) + 2 * (size_t)j;
-    const float4 lo = __ldg(src), hi = __ldg(src + 1);
-    const float v[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+    const float4* src = reinterpret_cast<const float4*>(g) + (DG / 4) * (size_t)j;
     float acc = 0.0f;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const float u = __fmul_rn(eta, v[i]);
-      acc = __fmaf_rn(u, u, acc);
+    for (int q = 0; q < DG / 4; ++q) {  // one chain over the DG elements in index order
+      const float4 x = __ldg(src + q);
+      float u;
+      u = __fmul_rn(eta, x.x); acc = __fmaf_rn(u, u, acc);
+      u = __fmul_rn(eta, x.y); acc = __fmaf_rn(u, u, acc);
+      u = __fmul_rn(eta, x.z); acc = __fmaf_rn(u, u, acc);
+      u = __fmul_rn(eta, x.w); acc = __fmaf_rn(u, u, acc);
     }
     key = __float_as_uint(acc);
   } else {
@@ -169,41 +172,47 @@ __device__ __forceinline__ void store_codes(void* codes, uint32_t j, int M, uint
   }
 }
 
-template <bool CB_F16>
-__device__ __forceinline__ void codeword(const void* book, uint32_t code, float c[8]) {
+template <bool CB_F16, int DG>
+__device__ __forceinline__ void codeword(const void* book, uint32_t code, float* c) {
   if (CB_F16) {
-    const uint4 raw = __ldg(reinterpret_cast<const uint4*>(book) + code);
-    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
-      c[2 * i] = f.x;
-      c[2 * i + 1] = f.y;
+    for (int part = 0; part < DG / 8; ++part) {
+      const uint4 raw = __ldg(reinterpret_cast<const uint4*>(book) + (size_t)code * (DG / 8) + part);
+      const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+        c[8 * part + 2 * i] = f.x;
+        c[8 * part + 2 * i + 1] = f.y;
+      }
     }
   } else {
-    const float4* src = reinterpret_cast<const float4*>(book) + 2 * (size_t)code;
-    const float4 lo = __ldg(src), hi = __ldg(src + 1);
-    c[0] = lo.x, c[1] = lo.y, c[2] = lo.z, c[3] = lo.w, c[4] = hi.x, c[5] = hi.y, c[6] = hi.z, c[7] = hi.w;
+    const float4* src = reinterpret_cast<const float4*>(book) + (size_t)code * (DG / 4);
+#pragma unroll
+    for (int part = 0; part < DG / 4; ++part) {
+      const float4 x = __ldg(src + part);
+      c[4 * part] = x.x, c[4 * part + 1] = x.y, c[4 * part + 2] = x.z, c[4 * part + 3] = x.w;
+    }
   }
 }
 
-// the eight dequantised weights of a group, binary32 exactly as dequantisation forms them: v = c1 (+ c2), w = s * v
-template <bool CB_F16>
+// the dequantised weights of a group, binary32 exactly as dequantisation forms them: v = c1 (+ c2 ...), w = s * v
+template <bool CB_F16, int DG>
 __device__ __forceinline__ bool group_weights(const void* books, uint32_t K, int M, uint32_t packed, bool code_u16,
-                                              float s, float w[8]) {
+                                              float s, float* w) {
   const uint32_t b0 = (M >= 2 && !code_u16) ? (packed & 0xffu) : packed;
   bool ok = b0 < K;
   for (int m = 1; m < M; ++m) ok = ok && ((packed >> (8 * m)) & 0xffu) < K;
-  float v[8];
-  codeword<CB_F16>(books, ok ? b0 : 0, v);
+  float v[DG];
+  codeword<CB_F16, DG>(books, ok ? b0 : 0, v);
   for (int m = 1; m < M; ++m) {  // codebooks added left to right, each sum rounded once
-    float v2[8];
-    codeword<CB_F16>(books, (uint32_t)m * K + (ok ? ((packed >> (8 * m)) & 0xffu) : 0u), v2);
+    float v2[DG];
+    codeword<CB_F16, DG>(books, (uint32_t)m * K + (ok ? ((packed >> (8 * m)) & 0xffu) : 0u), v2);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] = __fadd_rn(v[i], v2[i]);
+    for (int i = 0; i < DG; ++i) v[i] = __fadd_rn(v[i], v2[i]);
   }
 #pragma unroll
-  for (int i = 0; i < 8; ++i) w[i] = __fmul_rn(s, v[i]);
+  for (int i = 0; i < DG; ++i) w[i] = __fmul_rn(s, v[i]);
   return ok;
 }
 
@@ -238,7 +247,7 @@ __global__ void __launch_bounds__(256) save_codes_kernel(const TrustParams p) {
 
 // ||W_hat||^2: every thread adds its groups in index order, the block adds its threads in a fixed tree, the last
 // block to finish adds the block sums in block order -- the same binary64 result on every run
-template <bool CB_F16, bool CODE_U16>
+template <bool CB_F16, bool CODE_U16, int DG>
 __global__ void __launch_bounds__(kNormThreads) sq_norm_kernel(const TrustParams p) {
   __shared__ double sh[kNormThreads];
   __shared__ bool last;
@@ -246,11 +255,11 @@ __global__ void __launch_bounds__(kNormThreads) sq_norm_kernel(const TrustParams
   bool bad = false;
   const uint64_t stride = (uint64_t)gridDim.x * kNormThreads;
   for (uint64_t j = (uint64_t)blockIdx.x * kNormThreads + threadIdx.x; j < p.G; j += stride) {
-    float w[8];
+    float w[DG];
     const uint32_t packed = load_codes<CODE_U16>(p.codes, (uint32_t)j, p.M);
-    bad |= !group_weights<CB_F16>(p.books, p.K, p.M, packed, CODE_U16, __ldg(p.scale + (uint32_t)j / p.gpr), w);
+    bad |= !group_weights<CB_F16, DG>(p.books, p.K, p.M, packed, CODE_U16, __ldg(p.scale + (uint32_t)j / p.gpr), w);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) acc = __fma_rn((double)w[i], (double)w[i], acc);
+    for (int i = 0; i < DG; ++i) acc = __fma_rn((double)w[i], (double)w[i], acc);
   }
   if (bad) atomicOr(p.status, PVT_DEV_BAD_CODE);
   sh[threadIdx.x] = acc;
@@ -275,7 +284,7 @@ __global__ void __launch_bounds__(kNormThreads) sq_norm_kernel(const TrustParams
 }
 
 // squared change of the dequantised weights of the group at every rank; the group index in rank order
-template <bool CB_F16, bool CODE_U16>
+template <bool CB_F16, bool CODE_U16, int DG>
 __global__ void __launch_bounds__(256) change_kernel(const TrustParams p) {
   const uint64_t r = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (r >= p.k) return;
@@ -284,12 +293,12 @@ __global__ void __launch_bounds__(256) change_kernel(const TrustParams p) {
   double acc = 0.0;
   if (j < p.G) {
     const float s = __ldg(p.scale + j / p.gpr);
-    float wo[8], wn[8];
-    bool ok = group_weights<CB_F16>(p.books, p.K, p.M, p.saved[a], CODE_U16, s, wo);
-    ok &= group_weights<CB_F16>(p.books, p.K, p.M, load_codes<CODE_U16>(p.codes, j, p.M), CODE_U16, s, wn);
+    float wo[DG], wn[DG];
+    bool ok = group_weights<CB_F16, DG>(p.books, p.K, p.M, p.saved[a], CODE_U16, s, wo);
+    ok &= group_weights<CB_F16, DG>(p.books, p.K, p.M, load_codes<CODE_U16>(p.codes, j, p.M), CODE_U16, s, wn);
     if (!ok) atomicOr(p.status, PVT_DEV_BAD_CODE);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
+    for (int i = 0; i < DG; ++i) {
       const double diff = __dsub_rn((double)wn[i], (double)wo[i]);
       acc = __dadd_rn(acc, __dmul_rn(diff, diff));
     }
@@ -382,7 +391,10 @@ cudaError_t launch_trust_rank(const pvt_layer& L, uint64_t G, uint64_t k, void* 
   uint64_t* b = reinterpret_cast<uint64_t*>(base + t.pairs_b_off);
   uint32_t* counts = reinterpret_cast<uint32_t*>(base + t.counts_off);
   const unsigned flat = (unsigned)((k + 255) / 256);
-  rank_init_kernel<<<flat, 256, 0, stream>>>(L.g, G, L.eta, idx, k, a, status);
+  if (L.group_dim == 16)
+    rank_init_kernel<16><<<flat, 256, 0, stream>>>(L.g, G, L.eta, idx, k, a, status);
+  else
+    rank_init_kernel<8><<<flat, 256, 0, stream>>>(L.g, G, L.eta, idx, k, a, status);
   for (int pass = 0; pass < 4; ++pass) {
     sort_count_kernel<<<t.sort_blocks, kSortThreads, 0, stream>>>(a, k, pass, counts, t.sort_blocks);
     sort_scan_kernel<<<1, kScanThreads, 0, stream>>>(counts, kSortBins * t.sort_blocks);
@@ -406,7 +418,7 @@ TrustParams make_params(const pvt_layer& L, uint64_t G, uint64_t k, float ratio,
   p.scale = L.scale;
   p.G = G;
   p.k = k;
-  p.gpr = (uint32_t)(L.cols / kGroupDim);
+  p.gpr = (uint32_t)(L.cols / L.group_dim);
   p.K = (uint32_t)L.codebook_size;
   p.M = L.num_codebooks;
   p.idx = reinterpret_cast<const uint32_t*>(base + t.idx_off);
@@ -425,18 +437,24 @@ TrustParams make_params(const pvt_layer& L, uint64_t G, uint64_t k, float ratio,
 }
 
 template <bool CB_F16, bool CODE_U16>
-cudaError_t before_search(const TrustParams& p, unsigned norm_blocks, cudaStream_t stream) {
+cudaError_t before_search(const TrustParams& p, int dg, unsigned norm_blocks, cudaStream_t stream) {
   const unsigned flat = (unsigned)((p.k + 255) / 256);
   save_codes_kernel<CODE_U16><<<flat, 256, 0, stream>>>(p);
-  sq_norm_kernel<CB_F16, CODE_U16><<<norm_blocks, kNormThreads, 0, stream>>>(p);
+  if (dg == 16)
+    sq_norm_kernel<CB_F16, CODE_U16, 16><<<norm_blocks, kNormThreads, 0, stream>>>(p);
+  else
+    sq_norm_kernel<CB_F16, CODE_U16, 8><<<norm_blocks, kNormThreads, 0, stream>>>(p);
   count_launches(2);
   return cudaGetLastError();
 }
 
 template <bool CB_F16, bool CODE_U16>
-cudaError_t after_search(const TrustParams& p, cudaStream_t stream) {
+cudaError_t after_search(const TrustParams& p, int dg, cudaStream_t stream) {
   const unsigned flat = (unsigned)((p.k + 255) / 256);
-  change_kernel<CB_F16, CODE_U16><<<flat, 256, 0, stream>>>(p);
+  if (dg == 16)
+    change_kernel<CB_F16, CODE_U16, 16><<<flat, 256, 0, stream>>>(p);
+  else
+    change_kernel<CB_F16, CODE_U16, 8><<<flat, 256, 0, stream>>>(p);
   cut_kernel<<<1, kCutThreads, 0, stream>>>(p);
   restore_kernel<CODE_U16><<<flat, 256, 0, stream>>>(p);
   count_launches(3);
@@ -451,8 +469,12 @@ cudaError_t launch_trust_before_search(const pvt_layer& L, uint64_t G, uint64_t 
   cudaError_t e = cudaMemsetAsync(static_cast<char*>(ws) + t.stats_off, 0, 64, stream);
   if (e != cudaSuccess) return e;
   const bool f16 = L.codebook_dtype == PVT_F16, u16 = L.code_dtype == PVT_U16;
-  if (f16) return u16 ? before_search<true, true>(p, t.norm_blocks, stream) : before_search<true, false>(p, t.norm_blocks, stream);
-  return u16 ? before_search<false, true>(p, t.norm_blocks, stream) : before_search<false, false>(p, t.norm_blocks, stream);
+  const int dg = L.group_dim;
+  if (f16)
+    return u16 ? before_search<true, true>(p, dg, t.norm_blocks, stream)
+               : before_search<true, false>(p, dg, t.norm_blocks, stream);
+  return u16 ? before_search<false, true>(p, dg, t.norm_blocks, stream)
+             : before_search<false, false>(p, dg, t.norm_blocks, stream);
 }
 
 cudaError_t launch_trust_after_search(const pvt_layer& L, uint64_t G, uint64_t k, float ratio, uint32_t* idx_out,
@@ -462,9 +484,9 @@ cudaError_t launch_trust_after_search(const pvt_layer& L, uint64_t G, uint64_t k
   const bool f16 = L.codebook_dtype == PVT_F16, u16 = L.code_dtype == PVT_U16;
   cudaError_t e;
   if (f16)
-    e = u16 ? after_search<true, true>(p, stream) : after_search<true, false>(p, stream);
+    e = u16 ? after_search<true, true>(p, L.group_dim, stream) : after_search<true, false>(p, L.group_dim, stream);
   else
-    e = u16 ? after_search<false, true>(p, stream) : after_search<false, false>(p, stream);
+    e = u16 ? after_search<false, true>(p, L.group_dim, stream) : after_search<false, false>(p, L.group_dim, stream);
   if (e == cudaSuccess && stats_out)
     e = cudaMemcpyAsync(stats_out, p.stats, 2 * sizeof(double), cudaMemcpyDeviceToDevice, stream);
   return e;

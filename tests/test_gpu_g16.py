@@ -121,6 +121,47 @@ def test_whole_step_group_size_16():
     assert W_hat.cpu().numpy().tobytes() == oracle.dequant(want.codes, L.codebooks, L.scale, 128, 1024).tobytes()
 
 
+def settle(L):
+    L.codes = oracle.vstep(L.W, np.zeros_like(L.g), L.scale, L.codebooks, L.codes, eta=0.0, k=L.num_groups).codes
+    return L
+
+
+@pytest.mark.parametrize("K,f16,rows,cols,k_max,ratio", [(256, False, 128, 1024, 2000, 0.05), (2048, True, 128, 2048, 3000, 0.03)])
+def test_trust_step_group_size_16(K, f16, rows, cols, k_max, ratio):
+    L = settle(layer(rows, cols, K, f16, cfg=242))
+    G = L.num_groups
+    want = oracle.vstep_trust(L.W, L.g, L.scale, L.codebooks, L.codes, L.eta, ratio=ratio, k_max=k_max)
+    order = oracle.rank(oracle.group_norms(L.g, L.eta, 16), k_max)
+    dev = VStepLayer.from_host(L)
+    idx, n, stats = dev.step_trust(k_max, ratio)
+    torch.cuda.synchronize()
+    assert dev.status() == 0
+    assert np.array_equal(idx.cpu().numpy().astype(np.uint32), order)
+    assert 1 < want.n_kept < k_max
+    if not np.any(want.gap_rel <= 1e-6):
+        assert int(n.item()) == want.n_kept
+        assert np.array_equal(dev.codes.cpu().numpy(), want.codes)
+    s = stats.cpu().numpy()
+    assert abs(s[0] - want.sq_norm) <= max(1e-12, rows * cols * 2.0 ** -52) * want.sq_norm
+
+
+@pytest.mark.parametrize("K,f16,rows,cols", [(256, False, 64, 256), (1500, True, 100, 272)])
+def test_pstep_grad_group_size_16(K, f16, rows, cols):
+    L = layer(rows, cols, K, f16, cfg=243)
+    want_b, want_s = oracle.pstep_grad(L.g, L.scale, L.codes, L.codebooks, rows, cols)
+    dev = VStepLayer.from_host(L)
+    gb = torch.full((1, K, 16), 7.0, dtype=torch.float64, device="cuda")
+    gs = torch.full((rows,), 7.0, dtype=torch.float64, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B.pvt_pstep_grad(dev.desc, gb, gs, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    a_b = float(np.abs(L.scale).max()) * float(np.abs(L.g).max())
+    a_s = float(np.abs(L.g).max()) * float(np.abs(L.codebooks.astype(np.float32)).max())
+    assert np.abs(gb.cpu().numpy() - want_b).max() <= L.num_groups * a_b * 2.0 ** -50
+    assert np.abs(gs.cpu().numpy() - want_s).max() <= cols * a_s * 2.0 ** -50
+
+
 def test_group_size_16_rejections():
     L = layer(64, 256, 64, True)
     dev = VStepLayer.from_host(L)
@@ -128,8 +169,6 @@ def test_group_size_16_rejections():
     with pytest.raises(B.PvtError) as e:
         B.pvt_vstep_refine(dev.desc, idx, 4, 1)
     assert e.value.code == B.PVT_EUNSUPPORTED
-    with pytest.raises(B.PvtError) as e:
-        B.pvt_trust_workspace_bytes(dev.desc, 4) and B.pvt_vstep_trust(dev.desc, 4, 0.01, idx, torch.zeros(1, dtype=torch.int64, device="cuda"), None, B.new_workspace(dev.desc, 4))
     with pytest.raises(B.PvtError) as e:
         B.pvt_vstep_select_noalloc(dev.desc, 4, idx)
     assert e.value.code == B.PVT_EUNSUPPORTED
