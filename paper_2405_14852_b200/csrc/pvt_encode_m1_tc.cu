@@ -11,19 +11,21 @@
 // code)) is taken afterwards by the rescoring kernel on those sub-chunks, so the
 // fp16 rounding of the operands only has to be bounded, not small.
 //
-// Operands (K = 32 halves per row = four 16-byte K chunks, no swizzle, K-major
-// "interleaved" core-matrix layout: 8 rows x 16 bytes per core matrix, K chunks
-// 128 bytes apart, 8-row groups 512 bytes apart; one MMA instruction consumes two
-// K chunks, so a step is two instructions per A block, the second accumulating):
-//   A row n     = [ hi_0 .. hi_7 | lo_0 .. lo_7 | 2^e x 8 | 0 x 8 ]
+// Operands (16-byte K chunks of 8 halves, no swizzle, K-major "interleaved" core-matrix
+// layout: 8 rows x 16 bytes per core matrix, K chunks 128 bytes apart, 8-row groups of
+// A 512 and of B 256 bytes apart; one MMA instruction consumes two K chunks, so a step is
+// two instructions per A block, the second accumulating onto the first):
+//   A row n     = [ hi_0 .. hi_7 | 2^e x 8 | lo_0 .. lo_7 | 0 x 8 ]
 //                 hi_i = fp16(2^e t_i), lo_i = fp16(2^e t_i - hi_i)
-//   B row kappa = [ c_0 .. c_7   | c_0 .. c_7   | -h_hi, -h_lo, -h_lo2, 0 x 5 | 0 x 8 ]
+//   B row kappa = [ c_0 .. c_7   | -h_hi, -h_lo, -h_lo2, 0 x 5 ]
 //                 h = ||c||^2/2 = h_hi + h_lo + h_lo2
+//   instruction 1: A chunks 0-1 x B chunks 0-1 (hi . c - 2^e h);  instruction 2: A chunks 2-3 x
+//   the same B chunks (lo . c + 0): the codeword is stored and streamed once.
 // Splitting t into two halves keeps 22 of its 24 significant bits, so the fast
 // score is about as accurate as a binary32 evaluation and very few sub-chunks
 // come within the margin.  The codebook image is written once per call by a small
 // kernel in exactly the shared-memory byte order, so every 128-codeword step
-// arrives with one 1-D bulk copy (8 KB); the A rows are written by the threads
+// arrives with one 1-D bulk copy (4 KB); the A rows are written by the threads
 // that own the targets.  e_n is chosen per target so that max_i |2^e t_i| lies in
 // [1/2, 1).
 //
@@ -44,9 +46,10 @@
 // evaluates them exactly.  Targets outside the range the scaling can serve
 // (non-finite, or max |t_i| >= 256) are rescored against the whole codebook.
 //
-// Groups of 16 weights (Appendix J) use the same kernel with rows of 48 halves: [ hi x 16 | lo x 16 | 2^e x 8 |
-// 0 x 8 ] against [ c x 16 | c x 16 | norm terms | 0 x 8 ], six K chunks, three instructions per step and A
-// block, 12 KB per step.  Everything described for eight weights above holds with these sizes.
+// Groups of 16 weights (Appendix J) use the same kernel with A rows of 48 halves, [ hi x 16 | lo x 16 | 2^e x 8 |
+// 0 x 8 ], against B rows of 32 halves, [ c x 16 | norm terms | 0 x 8 ]: three instructions per step and A block
+// (hi . c, lo . c, 2^e x norm terms), 8 KB per step.  Everything described for eight weights above holds with
+// these sizes.
 #include <atomic>
 
 #include "pvt_encode_m1.cuh"
@@ -82,7 +85,7 @@ struct TcDim {
 constexpr int kTcStepBytes = TcDim<8>::kStepBytes;
 constexpr int kTcSubCw = 64;            // tracking granularity of the running maximum
 constexpr int kTcGroupSteps = 4;        // steps per codebook stage: the MMA threads wait for the codebook once per four steps
-constexpr int kTcStages = 3;            // codebook stages (32 KB each)
+constexpr int kTcStages = 3;            // codebook stages (four steps each: 16 KB, or 32 KB for groups of 16)
 constexpr int kTcEpiThreads = 256;
 constexpr int kTcThreads = kTcEpiThreads + 96;  // + producer warp + one MMA warp per A block
 constexpr uint32_t kTmemCols = 512;
