@@ -167,7 +167,7 @@ int pvt_vstep_select_noalloc(const pvt_layer* layer, uint64_t k, uint32_t* idx_o
  *   M = 3, 4: the same search carried through more stages: after each stage but
  *          the last the `beam` smallest partial tuples under (||t - c1 - ... -
  *          cm||^2, tuple) are kept; the pool is the last stage's beam*K tuples
- *          plus the previous tuple.  Every score is the binary64 value itself.
+ *          plus the previous tuple.
  *   A fast binary32 score shortlists candidates; the decision among shortlisted
  *   candidates is taken on binary64 distances sum_i (t_i - c_i)^2 accumulated in
  *   index order, so ties break exactly as stated above.
@@ -234,9 +234,10 @@ int pvt_vstep_refine(const pvt_layer* layer, const uint32_t* idx, uint64_t k, in
 
 /*
  * dequantize_weights (Algorithm 3, first line): for every group
- *   W_hat[r, 8c+i] = scale[r] * (C_1[b_1][i] (+ C_2[b_2][i]))   in binary32, the
- *   sum rounded once, then the product rounded once; out_dtype PVT_F16 rounds that
- *   binary32 value to nearest-even binary16.
+ *   W_hat[r, 8c+i] = scale[r] * (C_1[b_1][i] (+ C_2[b_2][i] + ...))   in binary32,
+ *   the codebooks added left to right with each sum rounded once, then the product
+ *   rounded once; out_dtype PVT_F16 rounds that binary32 value to nearest-even
+ *   binary16.
  * W_hat: device, rows x cols of out_dtype, 16-byte aligned.  `status` may be NULL
  * or a device uint32 into which PVT_DEV_BAD_CODE is OR-ed.
  */
@@ -249,9 +250,10 @@ int pvt_dequant(const pvt_layer* layer, void* W_hat, int32_t out_dtype, uint32_t
  * pvt_dequant forms):
  *   grad_codebooks[m][kappa][i] = sum over groups j with codes[j][m] == kappa of scale[r(j)] * g[j][i]
  *   grad_scale[r]               = sum over the groups j of row r and over i of g[j][i] * v[j][i]
- * Products are exact in binary64; sums are accumulated in binary64 by atomic adds, so
+ * Products are exact in binary64; sums are accumulated in binary64 in an order that
+ * is not fixed (atomic adds, or per-block sorted partial sums for small codebooks), so
  * results vary from run to run in the order of binary64 roundings only.
- * Reads layer->g, scale, codes, codebooks, shape.  grad_codebooks: device, M*K*8 doubles;
+ * Reads layer->g, scale, codes, codebooks, shape.  grad_codebooks: device, M*K*group_dim doubles;
  * grad_scale: device, rows doubles, or NULL.  Both are overwritten.  `status` may be NULL
  * or a device uint32 into which PVT_DEV_BAD_CODE is OR-ed (such groups contribute nothing).
  */
