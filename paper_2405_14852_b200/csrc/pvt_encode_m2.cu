@@ -181,8 +181,6 @@ __global__ void __launch_bounds__(kM2Threads, 2) encode_m2_kernel(const EncM2Par
   const float s1max = sqrtf(n1max), s2max = sqrtf(n2max);
   const uint32_t B = p.beam;  // already min(beam, K)
 
-  const float4* W4 = reinterpret_cast<const float4*>(p.W);
-  const float4* g4 = reinterpret_cast<const float4*>(p.g);
   const uint64_t nwarps = (uint64_t)gridDim.x * (kM2Threads / 32);
   const uint64_t n_groups = (p.k + kM2Group - 1) / kM2Group;
   const uint32_t my_q = (uint32_t)lane >> 3, my_b = (uint32_t)lane & 7u;
