@@ -52,7 +52,7 @@ extern "C" {
 /* host-side return codes */
 #define PVT_OK 0
 #define PVT_EINVAL (-1)       /* null / misaligned pointer, k = 0, k > G, cols % 8 != 0, G >= 2^32, bad eta */
-#define PVT_EUNSUPPORTED (-2) /* group_dim / M / K / dtype / beam combination this build has no kernel for */
+#define PVT_EUNSUPPORTED (-2) /* group_dim / M / K / dtype / beam combination the library has no kernel for */
 #define PVT_EWORKSPACE (-3)   /* ws_bytes smaller than pvt_workspace_bytes() */
 #define PVT_ECUDA (-4)        /* a CUDA runtime call or kernel launch failed; see pvt_last_cuda_error() */
 #define PVT_ETOOLARGE (-5)    /* pvt_vstep_select_noalloc only: the layer exceeds the built-in scratch */
