@@ -23,7 +23,9 @@
  *     consecutive elements of a row (input dimension); group j = r * (cols/8) + c
  *     covers W[r, 8c .. 8c+7].  G = rows * cols / 8 groups, G < 2^32.
  *   - Every pointer is DEVICE memory owned by the caller (16-byte aligned where
- *     stated).  The library allocates nothing and keeps no state between calls.
+ *     stated; index, error, move-count and status arrays 4-byte aligned; codes
+ *     2-byte aligned when they are two-byte codes or pairs of one-byte codes).
+ *     The library allocates nothing and keeps no state between calls.
  *   - Every call only enqueues work on `cuda_stream` (a cudaStream_t passed as
  *     void*; NULL = the legacy default stream) and returns without synchronising,
  *     except pvt_status.  Calls on one stream execute in order.

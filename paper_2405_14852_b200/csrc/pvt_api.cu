@@ -29,6 +29,13 @@ int sm_count() {
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }  // true for NULL
+
+// codes are read two bytes at a time when they are two-byte codes, or a pair of one-byte codes
+bool codes_aligned(const pvt_layer* L) {
+  const bool two_byte_access = L->code_dtype == PVT_U16 || L->num_codebooks == 2;
+  return !two_byte_access || (reinterpret_cast<uintptr_t>(L->codes) & 1u) == 0;
+}
 
 // Shape / type checks shared by every entry point.  Returns PVT_OK and G, or the error.
 int check_layer(const pvt_layer* L, uint64_t* G_out) {
@@ -148,7 +155,7 @@ int pvt_vstep_select(const pvt_layer* layer, uint64_t k, uint32_t* idx_out, void
   int rc = check_layer(layer, &G);
   if (rc != PVT_OK) return rc;
   if (k < 1 || k > G) return PVT_EINVAL;
-  if (!layer->g || !aligned16(layer->g) || !idx_out || !ws) return PVT_EINVAL;
+  if (!layer->g || !aligned16(layer->g) || !idx_out || !aligned4(idx_out) || !ws) return PVT_EINVAL;
   if (reinterpret_cast<uintptr_t>(ws) & (kWsAlign - 1)) return PVT_EINVAL;
   if (ws_bytes < select_layout(G).bytes) return PVT_EWORKSPACE;
   const cudaError_t e = launch_select(*layer, G, k, idx_out, ws, sm_count(), static_cast<cudaStream_t>(cuda_stream));
@@ -164,6 +171,7 @@ int pvt_vstep_encode(const pvt_layer* layer, const uint32_t* idx, uint64_t k, fl
   if (k < 1 || k > G) return PVT_EINVAL;
   if (!layer->W || !layer->g || !layer->scale || !layer->codebooks || !layer->codes || !idx || !ws) return PVT_EINVAL;
   if (!aligned16(layer->W) || !aligned16(layer->g) || !aligned16(layer->codebooks)) return PVT_EINVAL;
+  if (!codes_aligned(layer) || !aligned4(idx) || !aligned4(err_out)) return PVT_EINVAL;
   if (reinterpret_cast<uintptr_t>(ws) & (kWsAlign - 1)) return PVT_EINVAL;
   const int sms = sm_count();
   cudaError_t e;
@@ -206,6 +214,7 @@ int pvt_vstep_trust(const pvt_layer* layer, uint64_t k_max, float ratio, uint32_
     return PVT_EINVAL;
   if (!aligned16(layer->W) || !aligned16(layer->g) || !aligned16(layer->codebooks)) return PVT_EINVAL;
   if ((reinterpret_cast<uintptr_t>(n_out) & 7u) || (reinterpret_cast<uintptr_t>(stats_out) & 7u)) return PVT_EINVAL;
+  if (!codes_aligned(layer) || !aligned4(idx_out)) return PVT_EINVAL;
   if (reinterpret_cast<uintptr_t>(ws) & (kWsAlign - 1)) return PVT_EINVAL;
   if (layer->num_codebooks >= 2) {
     if (layer->code_dtype != PVT_U8 || layer->beam < 1 || layer->beam > 8) return PVT_EUNSUPPORTED;
@@ -241,6 +250,8 @@ int pvt_vstep_refine(const pvt_layer* layer, const uint32_t* idx, uint64_t k, in
   if (!aligned16(layer->W) || !aligned16(layer->g) || !aligned16(layer->codebooks)) return PVT_EINVAL;
   if (layer->group_dim != kGroupDim) return PVT_EUNSUPPORTED;
   if (layer->num_codebooks >= 2 && layer->code_dtype != PVT_U8) return PVT_EUNSUPPORTED;
+  if (!codes_aligned(layer) || !aligned4(idx) || !aligned4(err_out) || !aligned4(moves_out) || !aligned4(status))
+    return PVT_EINVAL;
   const cudaError_t e = launch_refine(*layer, G, idx, k, max_moves, err_out, moves_out, status,
                                       static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? PVT_OK : fail_cuda(e);
@@ -254,8 +265,7 @@ int pvt_dequant(const pvt_layer* layer, void* W_hat, int32_t out_dtype, uint32_t
   if (out_dtype != PVT_F32 && out_dtype != PVT_F16) return PVT_EINVAL;
   if (!layer->scale || !layer->codebooks || !layer->codes || !W_hat) return PVT_EINVAL;
   if (!aligned16(layer->codebooks) || !aligned16(W_hat)) return PVT_EINVAL;
-  if (layer->num_codebooks == 2 && layer->code_dtype == PVT_U8 && (reinterpret_cast<uintptr_t>(layer->codes) & 1u))
-    return PVT_EINVAL;
+  if (!codes_aligned(layer) || !aligned4(status)) return PVT_EINVAL;
   const cudaError_t e = launch_dequant(*layer, G, W_hat, out_dtype, status, sm_count(), static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? PVT_OK : fail_cuda(e);
 }
@@ -270,8 +280,7 @@ int pvt_pstep_grad(const pvt_layer* layer, double* grad_codebooks, double* grad_
   if (!aligned16(layer->g) || !aligned16(layer->codebooks)) return PVT_EINVAL;
   if ((reinterpret_cast<uintptr_t>(grad_codebooks) & 7u) || (reinterpret_cast<uintptr_t>(grad_scale) & 7u))
     return PVT_EINVAL;
-  if (layer->num_codebooks == 2 && layer->code_dtype == PVT_U8 && (reinterpret_cast<uintptr_t>(layer->codes) & 1u))
-    return PVT_EINVAL;
+  if (!codes_aligned(layer) || !aligned4(status)) return PVT_EINVAL;
   const cudaError_t e = launch_pstep_grad(*layer, G, grad_codebooks, grad_scale, status, sm_count(),
                                           static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? PVT_OK : fail_cuda(e);

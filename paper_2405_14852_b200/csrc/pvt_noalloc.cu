@@ -70,6 +70,7 @@ extern "C" int pvt_vstep_select_noalloc(const pvt_layer* layer, uint64_t k, uint
   if (!(layer->eta >= 0.0f) || !(layer->eta <= 3.0e38f)) return PVT_EINVAL;
   if (k < 1 || k > G) return PVT_EINVAL;
   if (!layer->g || (reinterpret_cast<uintptr_t>(layer->g) & 15u) || !idx_out) return PVT_EINVAL;
+  if ((reinterpret_cast<uintptr_t>(idx_out) & 3u) || (reinterpret_cast<uintptr_t>(status_out) & 3u)) return PVT_EINVAL;
   if (G > kNoAllocMaxGroups || select_layout(G).bytes > kNoAllocScratchBytes) return PVT_ETOOLARGE;
 
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);

@@ -75,6 +75,8 @@ def test_select_rejects_bad_arguments_before_launch(kw, k, code):
     (dict(num_codebooks=2, beam=9), B.PVT_EUNSUPPORTED),
     (dict(codebook_dtype=7), B.PVT_EINVAL),
     (dict(W=None), B.PVT_EINVAL),
+    (dict(num_codebooks=2, codes=0x1001), B.PVT_EINVAL),          # pairs of one-byte codes are read two bytes at a time
+    (dict(codebook_size=1024, code_dtype=B.PVT_U16, codes=0x1001), B.PVT_EINVAL),
 ])
 def test_encode_rejects_bad_arguments_before_launch(kw, code):
     L = _layer(**kw)
@@ -93,3 +95,14 @@ def test_dequant_rejects_bad_arguments():
     L = _layer()
     assert B.lib().pvt_dequant(ctypes.byref(L), None, B.PVT_F32, None, None) == B.PVT_EINVAL
     assert B.lib().pvt_dequant(ctypes.byref(L), 0x2000, 5, None, None) == B.PVT_EINVAL
+
+
+def test_misaligned_index_and_output_pointers_are_rejected():
+    L = _layer()
+    lib = B.lib()
+    assert lib.pvt_vstep_select(ctypes.byref(L), 4, 0x2002, 0x4000, 1 << 30, None) == B.PVT_EINVAL
+    assert lib.pvt_vstep_encode(ctypes.byref(L), 0x2002, 4, None, 0x4000, 1 << 30, None) == B.PVT_EINVAL
+    assert lib.pvt_vstep_encode(ctypes.byref(L), 0x2000, 4, 0x3002, 0x4000, 1 << 30, None) == B.PVT_EINVAL
+    assert lib.pvt_vstep_refine(ctypes.byref(L), 0x2000, 4, 1, None, 0x3001, None, None) == B.PVT_EINVAL
+    assert lib.pvt_vstep_select_noalloc(ctypes.byref(L), 4, 0x2002, None, None) == B.PVT_EINVAL
+    assert lib.pvt_dequant(ctypes.byref(_layer(num_codebooks=2, codes=0x1001)), 0x4000, B.PVT_F32, None, None) == B.PVT_EINVAL
