@@ -289,6 +289,9 @@ int pvt_pstep_grad(const pvt_layer* layer, double* grad_codebooks, double* grad_
 int pvt_adam_update(float* param, void* param_f16, const double* grad, float* exp_avg, float* exp_avg_sq, uint64_t n,
                     float lr, float beta1, float beta2, float eps, float bias1, float bias2, void* cuda_stream) {
   if (!param || !grad || !exp_avg || !exp_avg_sq || n == 0) return PVT_EINVAL;
+  if (!aligned4(param) || !aligned4(exp_avg) || !aligned4(exp_avg_sq) || (reinterpret_cast<uintptr_t>(grad) & 7u) ||
+      (reinterpret_cast<uintptr_t>(param_f16) & 1u))
+    return PVT_EINVAL;
   if (!(lr >= 0.0f) || !(beta1 >= 0.0f && beta1 < 1.0f) || !(beta2 >= 0.0f && beta2 < 1.0f) || !(eps >= 0.0f))
     return PVT_EINVAL;
   if (!(bias1 > 0.0f && bias1 <= 1.0f) || !(bias2 > 0.0f && bias2 <= 1.0f)) return PVT_EINVAL;
