@@ -466,7 +466,17 @@ def cpu_baseline(L, k, tau, budget_s=15.0):
     oracle.dequant(L.codes, L.codebooks, L.scale, L.rows, L.cols)
     t_deq = time.perf_counter() - t0
     t_step = t_sel + t_enc * (k / n) + t_deq
-    return {"value": k / t_step, "unit": UNIT, "cores": threads, "kind": "oracle",
+    # the same search on one thread, on a sample smaller by the thread count (a few seconds)
+    one_thread = None
+    if threads > 1:
+        n1 = max(1, min(n, n // threads))
+        oracle.set_num_threads(1)
+        try:
+            t1 = _time_oracle_encode(oracle, L, idx[:n1], codes2)
+        finally:
+            oracle.set_num_threads(threads)
+        one_thread = {"pairs_per_s": n1 * L.pairs_per_group() / t1, "sample_groups": n1, "seconds": t1}
+    return {"value": k / t_step, "unit": UNIT, "cores": threads, "kind": "oracle", "search_on_one_thread": one_thread,
             "sample": f"norms+selection over all {L.num_groups} groups ({t_sel:.2f} s), search of the first {n} of "
                       f"{k} selected groups ({t_enc:.2f} s, scaled by k/n), dequantisation of the whole layer "
                       f"({t_deq:.2f} s)",
