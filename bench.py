@@ -318,6 +318,13 @@ def run_ours(args):
         stages["dequant"] = {"ms": dq_ms / max(dq_n, 1), "algorithmic_bytes": dq_bytes,
                              "gbs": dq_bytes / (dq_ms / max(dq_n, 1) * 1e-3) / 1e9 if dq_n else None}
         stages["dequant"]["library_fill_of_the_same_output_ms"] = fill_ms
+        # per-stage rates: the whole encode call (codebook preparation + search + rescoring), alone and with
+        # the selection in front of it
+        t_enc_call = (aux_ms / max(aux_n, 1) + enc_avg_ms + rs_ms / max(rs_n, 1)) * 1e-3
+        t_sel_call = sel_ms / max(sel_n, 1) * 1e-3
+        stages["rates"] = {"groups_per_s_encode": k / t_enc_call if t_enc_call > 0 else None,
+                           "groups_per_s_select_plus_encode": k / (t_enc_call + t_sel_call) if t_enc_call > 0 else None,
+                           "pairs_per_s_encode": pairs / t_enc_call if t_enc_call > 0 else None}
         pg_ms, pg_n = kern[B.PVT_KERNEL_PSTEP_GRAD]
         ad_ms, ad_n = kern[B.PVT_KERNEL_ADAM]
         pg_bytes = G * (32 + code_bytes) + M * K * 8 * 8 + rows * 12
