@@ -296,6 +296,7 @@ def run_ours(args):
         props = torch.cuda.get_device_properties(local)
         sm_max_mhz = (clocks or {}).get("sm_max_mhz") or peaks.get("sm_max_mhz") or 1965.0
         alu_peak = props.multi_processor_count * FP32_LANES_PER_SM * 2 * sm_max_mhz * 1e6 / 1e12  # TFLOP/s
+        ffma_measured = B.pvt_probe_fp32_tflops()  # the same pipe, measured in this job
         enc_ms, enc_n = kern[B.PVT_KERNEL_ENCODE_MAIN]
         enc_avg_ms = enc_ms / max(enc_n, 1)
         pairs = k * pairs_per_group
@@ -349,6 +350,7 @@ def run_ours(args):
                         "flop_per_pair": FLOP_PER_PAIR, "avg_launch_ms": enc_avg_ms, "launches": enc_n,
                         "executed_tflops": achieved * 4.0,  # operands are padded from depth 8 to depth 32
                         "frac_of_fp32_alu_roofline": achieved / alu_peak,
+                        "fp32_fma_microbenchmark_tflops": ffma_measured,
                         "frac_of_epilogue_bound": (pairs / (enc_avg_ms * 1e-3)) /
                                                   (props.multi_processor_count * 128 * sm_max_mhz * 1e6),
                         "epilogue_bound_is": "one accumulator read per pair: 128 lanes per SM per clock",
@@ -361,6 +363,7 @@ def run_ours(args):
                         "peak_is": f"{props.multi_processor_count} SMs x 128 FP32 lanes x 2 flop x "
                                    f"{sm_max_mhz:.0f} MHz (derived; no measured FP32 peak)",
                         "flop_per_pair": FLOP_PER_PAIR, "avg_launch_ms": enc_avg_ms, "launches": enc_n,
+                        "fp32_fma_microbenchmark_tflops": ffma_measured,
                         # dram__bytes_read + dram__bytes_write of one launch (ncu, FP32 engine, default workload)
                         "traffic": 7.87e6 if (M == 1 and args.workload == DEFAULT_WORKLOAD) else None}
         line = {

@@ -336,6 +336,9 @@ void pvt_set_m1_search(int mode);
 #define PVT_KERNEL_TRUST 7       /* ranking, norm and code saving of pvt_vstep_trust (before its search) */
 #define PVT_KERNEL_REFINE 8      /* the kernel of pvt_vstep_refine */
 void pvt_timing_enable(int on);
+/* FP32 FMA throughput of the current device, measured: a kernel of independent FMA chains on every SM, timed with
+ * CUDA events (synchronises).  scratch: device, at least 2048 floats per SM.  tflops_out: host. */
+int pvt_probe_fp32_tflops(float* scratch, size_t scratch_floats, float* tflops_out, void* cuda_stream);
 /* Kernels this process has launched through the library so far (memsets not counted). */
 unsigned long long pvt_launch_count(void);
 int pvt_timing_read(int kernel_id, float* total_ms, int* launches);

@@ -100,6 +100,8 @@ def lib():
         L.pvt_set_m1_search.argtypes = [ctypes.c_int]
         L.pvt_timing_enable.restype = None
         L.pvt_timing_enable.argtypes = [ctypes.c_int]
+        L.pvt_probe_fp32_tflops.restype = ctypes.c_int
+        L.pvt_probe_fp32_tflops.argtypes = [vp, sz, ctypes.POINTER(ctypes.c_float), vp]
         L.pvt_launch_count.restype = ctypes.c_ulonglong
         L.pvt_timing_read.restype = ctypes.c_int
         L.pvt_timing_read.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int)]
@@ -273,6 +275,16 @@ def pvt_version() -> int:
 def pvt_set_m1_search(mode: int) -> None:
     """Engine of the single-codebook search: PVT_M1_AUTO, PVT_M1_FP32 or PVT_M1_TENSOR."""
     lib().pvt_set_m1_search(mode)
+
+
+def pvt_probe_fp32_tflops(stream=None) -> float:
+    """Measured FP32 FMA throughput of the current device in TFLOP/s (a short kernel of independent FMA chains)."""
+    props = torch.cuda.get_device_properties(torch.cuda.current_device())
+    scratch = torch.empty(props.multi_processor_count * 2048, dtype=torch.float32, device="cuda")
+    out = ctypes.c_float(0.0)
+    _check(lib().pvt_probe_fp32_tflops(scratch.data_ptr(), scratch.numel(), ctypes.byref(out), _stream_ptr(stream)),
+           "pvt_probe_fp32_tflops")
+    return float(out.value)
 
 
 def pvt_launch_count() -> int:

@@ -108,6 +108,25 @@ void timing_end(KernelId id, cudaStream_t stream) {
 
 }  // namespace pvt
 
+namespace pvt {
+// 16 independent chains of dependent FMAs per thread: nothing but the FP32 pipe is busy
+__global__ void __launch_bounds__(256) ffma_probe_kernel(float* out, int iters) {
+  float x[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) x[i] = 1.0f + 1e-3f * (float)(threadIdx.x + i);
+  const float a = 1.0000001f, b = 1e-7f;
+  for (int it = 0; it < iters; ++it) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) x[i] = __fmaf_rn(x[i], a, b);
+  }
+  float s = 0.0f;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) s += x[i];
+  out[(size_t)blockIdx.x * blockDim.x + threadIdx.x] = s;
+}
+
+}  // namespace pvt
+
 using namespace pvt;
 
 namespace {
@@ -343,6 +362,30 @@ void pvt_set_m1_search(int mode) {
 }
 
 unsigned long long pvt_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int pvt_probe_fp32_tflops(float* scratch, size_t scratch_floats, float* tflops_out, void* cuda_stream) {
+  if (!scratch || !tflops_out) return PVT_EINVAL;
+  const int blocks = sm_count() * 8, iters = 8192;
+  if (scratch_floats < (size_t)blocks * 256) return PVT_EWORKSPACE;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  cudaError_t e = cudaEventCreate(&e0);
+  if (e == cudaSuccess) e = cudaEventCreate(&e1);
+  if (e == cudaSuccess) {
+    ffma_probe_kernel<<<blocks, 256, 0, s>>>(scratch, iters);  // warm-up
+    cudaEventRecord(e0, s);
+    ffma_probe_kernel<<<blocks, 256, 0, s>>>(scratch, iters);
+    cudaEventRecord(e1, s);
+    e = cudaEventSynchronize(e1);
+  }
+  float ms = 0.0f;
+  if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+  if (e0) cudaEventDestroy(e0);
+  if (e1) cudaEventDestroy(e1);
+  if (e != cudaSuccess) return fail_cuda(e);
+  *tflops_out = (float)(2.0 * 16.0 * iters * 256.0 * blocks / (ms * 1e-3) / 1e12);
+  return PVT_OK;
+}
 
 void pvt_timing_enable(int on) {
   Timing& t = timing();
