@@ -61,9 +61,19 @@ struct M2Smem {
   alignas(16) float c2[kM2K][8];
   alignas(16) uint64_t p1[4][8][32];  // stage-1 operands: (c1[l+64q][i], c1[l+64q+32][i])
   uint64_t h1[4][32];                 // (||c1||^2/2) pairs in the same order
-  alignas(16) float x2[kM2K / 2][16]; // stage-2 operands: pair p holds (c2[2p][0], c2[2p+1][0], c2[2p][1], ...)
-  alignas(8) float hx2[kM2K / 2][2];  // (||c2||^2/2) of the pair
-  float h2[kM2K];
+  union {
+    struct {
+      alignas(16) float x2[kM2K / 2][16];  // FP32 stage 2: pair p holds (c2[2p][0], c2[2p+1][0], c2[2p][1], ...)
+      alignas(8) float hx2[kM2K / 2][2];   // (||c2||^2/2) of the pair
+    };
+    struct {
+      // tensor stage 2: B fragments of codebook 2, word [n-tile][lane] = halves (c2[8 nt + lane/4][2 (lane%4)], [.. + 1]);
+      // and the sub-chunk minima of a warp's 32 residual rows on their way to the lanes that own the rows
+      uint32_t b2[kM2K / 8][32];
+      alignas(16) float wmin[kM2Threads / 32][32][8];
+    };
+  };
+  alignas(8) float h2[kM2K];
   alignas(16) float wt[kM2Threads / 32][kM2Group][8];     // the targets of a warp's group
   alignas(16) uint32_t wk[kM2Threads / 32][kM2Group][8];  // their beam entries (codes of codebook 1)
   float red[kM2Threads / 32][2];
@@ -84,6 +94,14 @@ __device__ __forceinline__ float min3(float a, float b, float c) {
   float d;
   asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
   return d;
+}
+// D = A (16 x 16, rows = residuals) x B (16 x 8, columns = codewords) + C, fp16 operands, fp32 accumulation
+__device__ __forceinline__ void mma_16x8x16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1, float c0,
+                                            float c1) {
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+      "{%10, %11, %10, %11};"
+      : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(c0), "f"(c1));
 }
 __device__ __forceinline__ uint64_t pack2(float lo, float hi) {
   return (uint64_t)__float_as_uint(lo) | ((uint64_t)__float_as_uint(hi) << 32);
@@ -126,6 +144,8 @@ __device__ __forceinline__ float load_cb(const void* books, int f16, uint32_t m,
   return f16 ? __half2float(reinterpret_cast<const __half*>(books)[off]) : reinterpret_cast<const float*>(books)[off];
 }
 
+// TC2: stage 2 on the tensor cores (fp16 codebooks: the codewords are exact halves), else on the FP32 pipe.
+template <bool TC2>
 __global__ void __launch_bounds__(kM2Threads, 2) encode_m2_kernel(const EncM2Params p) {
   __shared__ M2Smem sm;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -150,10 +170,18 @@ __global__ void __launch_bounds__(kM2Threads, 2) encode_m2_kernel(const EncM2Par
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       p1f[(((q * 8 + i) * 32) + l) * 2 + half] = c1[i];
-      sm.x2[tid >> 1][2 * i + (tid & 1)] = c2[i];
+      if (!TC2) sm.x2[tid >> 1][2 * i + (tid & 1)] = c2[i];
     }
     reinterpret_cast<float*>(&sm.h1[0][0])[(q * 32 + l) * 2 + half] = h1;
-    sm.hx2[tid >> 1][tid & 1] = h2;
+    if (TC2) {
+#pragma unroll
+      for (int qq = 0; qq < 4; ++qq) {
+        const __half2 v = __floats2half2_rn(c2[2 * qq], c2[2 * qq + 1]);  // exact: the codebook is fp16
+        sm.b2[tid >> 3][4 * (tid & 7) + qq] = *reinterpret_cast<const uint32_t*>(&v);
+      }
+    } else {
+      sm.hx2[tid >> 1][tid & 1] = h2;
+    }
     sm.h2[tid] = h2;
     float m1 = n1, m2 = n2;
 #pragma unroll
@@ -348,36 +376,110 @@ __global__ void __launch_bounds__(kM2Threads, 2) encode_m2_kernel(const EncM2Par
       c1v[0] = ca.x; c1v[1] = ca.y; c1v[2] = ca.z; c1v[3] = ca.w; c1v[4] = cb.x; c1v[5] = cb.y; c1v[6] = cb.z; c1v[7] = cb.w;
     }
     float rho = 0.0f;
-    uint64_t nrd[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       r[i] = active ? __fsub_rn(t[i], c1v[i]) : 0.0f;
       rho = __fmaf_rn(r[i], r[i], rho);
-      nrd[i] = pack2(-r[i], -r[i]);
     }
     rho = __fmul_rn(0.5f, rho);
-    const uint64_t rho2 = pack2(rho, rho);
     float sub_min[8];
+    if (TC2) {
+      // The 32 residuals of the group are the rows of two 16-row A tiles, each row [ -hi(2^e r) | -lo(2^e r) ] in fp16
+      // (hi + lo keeps 22 significant bits of r, or all bits above 2^-25 in scaled units); the columns of B are the
+      // codewords of codebook 2, [ c2 | c2 ]; C starts at 2^e ||c2||^2/2.  e is common to the group: the largest
+      // residual element becomes [1/2, 1).  A thread holds elements 2 qd, 2 qd + 1 of rows g8, g8 + 8 of each tile.
+      const uint32_t g8 = (uint32_t)lane >> 2, qd = (uint32_t)lane & 3u;
+      float2 nr[4];  // -r of the four rows of this thread
+      float rmax = 0.0f;
 #pragma unroll
-    for (int sub = 0; sub < 8; ++sub) {
-      float cmin = kInf;
-      const ulonglong2* vals = reinterpret_cast<const ulonglong2*>(&sm.x2[0][0]) + sub * 16 * 4;
-      const uint64_t* norms = reinterpret_cast<const uint64_t*>(&sm.hx2[0][0]) + sub * 16;
-#pragma unroll 4
-      for (int pr = 0; pr < 16; ++pr) {
-        const ulonglong2 q0 = vals[4 * pr], q1 = vals[4 * pr + 1], q2 = vals[4 * pr + 2], q3 = vals[4 * pr + 3];
-        uint64_t acc = add2(norms[pr], rho2);
-        acc = fma2(nrd[0], q0.x, acc);
-        acc = fma2(nrd[1], q0.y, acc);
-        acc = fma2(nrd[2], q1.x, acc);
-        acc = fma2(nrd[3], q1.y, acc);
-        acc = fma2(nrd[4], q2.x, acc);
-        acc = fma2(nrd[5], q2.y, acc);
-        acc = fma2(nrd[6], q3.x, acc);
-        acc = fma2(nrd[7], q3.y, acc);
-        cmin = min3(cmin, lo_of(acc), hi_of(acc));
+      for (int r4 = 0; r4 < 4; ++r4) {
+        const uint32_t row = 16u * (r4 >> 1) + 8u * (r4 & 1) + g8, tq = row >> 3, b = row & 7u;
+        const uint32_t tj = __shfl_sync(0xffffffffu, my_j, 8 * tq);
+        const bool valid = tj != 0xffffffffu && b < B;
+        const uint32_t kr = valid ? sm.wk[warp][tq][b] : 0u;  // the beam of a skipped target was never written
+        const float2 tt = *reinterpret_cast<const float2*>(&sm.wt[warp][tq][2 * qd]);
+        const float2 cc = *reinterpret_cast<const float2*>(&sm.c1[kr][2 * qd]);
+        nr[r4].x = valid ? __fsub_rn(cc.x, tt.x) : 0.0f;  // -(t - c1), exactly
+        nr[r4].y = valid ? __fsub_rn(cc.y, tt.y) : 0.0f;
+        rmax = fmaxf(rmax, fmaxf(fabsf(nr[r4].x), fabsf(nr[r4].y)));
       }
-      sub_min[sub] = active ? cmin : kInf;
+      const uint32_t rbits = __reduce_max_sync(0xffffffffu, __float_as_uint(rmax));  // non-negative floats order as u32
+      int e = 126 - (int)((rbits >> 23) & 0xffu);
+      e = e > 15 ? 15 : (e < -100 ? -100 : e);
+      const float sc = __uint_as_float((uint32_t)(e + 127) << 23), inv = __uint_as_float((uint32_t)(127 - e) << 23);
+      uint32_t a[2][4];
+#pragma unroll
+      for (int r4 = 0; r4 < 4; ++r4) {
+        const float x = nr[r4].x * sc, y = nr[r4].y * sc;
+        const __half2 hi = __floats2half2_rn(x, y);
+        const float2 back = __half22float2(hi);
+        const __half2 lo = __floats2half2_rn(x - back.x, y - back.y);
+        a[r4 >> 1][r4 & 1] = *reinterpret_cast<const uint32_t*>(&hi);
+        a[r4 >> 1][2 + (r4 & 1)] = *reinterpret_cast<const uint32_t*>(&lo);
+      }
+#pragma unroll 2
+      for (int sub = 0; sub < 8; ++sub) {
+        float m[4] = {kInf, kInf, kInf, kInf};
+#pragma unroll
+        for (int n4 = 0; n4 < 4; ++n4) {
+          const int nt = 4 * sub + n4;
+          const uint32_t b = sm.b2[nt][lane];
+          const float2 hh = *reinterpret_cast<const float2*>(&sm.h2[8 * nt + 2 * qd]);
+          const float hx = hh.x * sc, hy = hh.y * sc;
+          float d0[4], d1[4];
+          mma_16x8x16(d0, a[0], b, b, hx, hy);
+          mma_16x8x16(d1, a[1], b, b, hx, hy);
+          m[0] = min3(m[0], d0[0], d0[1]);
+          m[1] = min3(m[1], d0[2], d0[3]);
+          m[2] = min3(m[2], d1[0], d1[1]);
+          m[3] = min3(m[3], d1[2], d1[3]);
+        }
+#pragma unroll
+        for (int r4 = 0; r4 < 4; ++r4) {
+          m[r4] = fminf(m[r4], __shfl_xor_sync(0xffffffffu, m[r4], 1));
+          m[r4] = fminf(m[r4], __shfl_xor_sync(0xffffffffu, m[r4], 2));
+        }
+        if (qd == 0) {
+#pragma unroll
+          for (int r4 = 0; r4 < 4; ++r4) sm.wmin[warp][16 * (r4 >> 1) + 8 * (r4 & 1) + g8][sub] = m[r4];
+        }
+      }
+      __syncwarp();
+      {
+        const float4 ma = *reinterpret_cast<const float4*>(&sm.wmin[warp][lane][0]);
+        const float4 mb = *reinterpret_cast<const float4*>(&sm.wmin[warp][lane][4]);
+        const float mm[8] = {ma.x, ma.y, ma.z, ma.w, mb.x, mb.y, mb.z, mb.w};
+#pragma unroll
+        for (int sub = 0; sub < 8; ++sub) sub_min[sub] = active ? __fmaf_rn(mm[sub], inv, rho) : kInf;
+      }
+      // the halves' absolute rounding floor (2^-25 per element in scaled units), doubled, with a factor 4 to spare
+      my_margin2 += 4.76837158203125e-7f /* 2^-21 */ * inv * s2max;
+    } else {
+      uint64_t nrd[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) nrd[i] = pack2(-r[i], -r[i]);
+      const uint64_t rho2 = pack2(rho, rho);
+#pragma unroll
+      for (int sub = 0; sub < 8; ++sub) {
+        float cmin = kInf;
+        const ulonglong2* vals = reinterpret_cast<const ulonglong2*>(&sm.x2[0][0]) + sub * 16 * 4;
+        const uint64_t* norms = reinterpret_cast<const uint64_t*>(&sm.hx2[0][0]) + sub * 16;
+#pragma unroll 4
+        for (int pr = 0; pr < 16; ++pr) {
+          const ulonglong2 q0 = vals[4 * pr], q1 = vals[4 * pr + 1], q2 = vals[4 * pr + 2], q3 = vals[4 * pr + 3];
+          uint64_t acc = add2(norms[pr], rho2);
+          acc = fma2(nrd[0], q0.x, acc);
+          acc = fma2(nrd[1], q0.y, acc);
+          acc = fma2(nrd[2], q1.x, acc);
+          acc = fma2(nrd[3], q1.y, acc);
+          acc = fma2(nrd[4], q2.x, acc);
+          acc = fma2(nrd[5], q2.y, acc);
+          acc = fma2(nrd[6], q3.x, acc);
+          acc = fma2(nrd[7], q3.y, acc);
+          cmin = min3(cmin, lo_of(acc), hi_of(acc));
+        }
+        sub_min[sub] = active ? cmin : kInf;
+      }
     }
     float gmin = sub_min[0];
 #pragma unroll
@@ -504,7 +606,10 @@ cudaError_t launch_encode_m2(const pvt_layer& L, uint64_t G, const uint32_t* idx
   uint64_t ctas = (groups + warps_per_cta - 1) / warps_per_cta;
   if (ctas > 2 * (uint64_t)sm_count) ctas = 2 * (uint64_t)sm_count;  // two CTAs (16 warps) per SM
   timing_begin(kKernEncodeMain, stream);
-  encode_m2_kernel<<<(unsigned)ctas, kM2Threads, 0, stream>>>(p);
+  if (p.cb_f16)
+    encode_m2_kernel<true><<<(unsigned)ctas, kM2Threads, 0, stream>>>(p);
+  else
+    encode_m2_kernel<false><<<(unsigned)ctas, kM2Threads, 0, stream>>>(p);
   count_launches(1);
   timing_end(kKernEncodeMain, stream);
   return cudaGetLastError();
