@@ -281,35 +281,45 @@ __global__ void __launch_bounds__(kM2Threads, 2) encode_m2_kernel(const EncM2Par
           f[2 * qq + 1] = hi_of(acc[qq]);
         }
       }
-      // extract the B smallest (score truncated to 24 bits | code): a first guess of the beam
+      // extract the B smallest (score truncated to 24 bits | code): a first guess of the beam.  Every lane sorts
+      // its eight keys once (19 compare-exchanges); a round is then one warp minimum of the lanes' heads and a shift
+      // of the winning lane's list.
       uint32_t key[8];
 #pragma unroll
       for (int jj = 0; jj < 8; ++jj) key[jj] = (ord(f[jj]) & 0xffffff00u) | (uint32_t)(lane + 32 * jj);
+#define PVT_CE(a, b)                               \
+  {                                                \
+    const uint32_t lo_ = min(key[a], key[b]);      \
+    key[b] = max(key[a], key[b]);                  \
+    key[a] = lo_;                                  \
+  }
+      PVT_CE(0, 2) PVT_CE(1, 3) PVT_CE(4, 6) PVT_CE(5, 7)
+      PVT_CE(0, 4) PVT_CE(1, 5) PVT_CE(2, 6) PVT_CE(3, 7)
+      PVT_CE(0, 1) PVT_CE(2, 3) PVT_CE(4, 5) PVT_CE(6, 7)
+      PVT_CE(2, 4) PVT_CE(3, 5)
+      PVT_CE(1, 4) PVT_CE(3, 6)
+      PVT_CE(1, 2) PVT_CE(3, 4) PVT_CE(5, 6)
+#undef PVT_CE
       uint32_t beam_code[8];
+      uint32_t last = 0;  // the key extracted last
 #pragma unroll
       for (int b = 0; b < 8; ++b) {
         beam_code[b] = 0;
         if ((uint32_t)b < B) {
-          uint32_t lm = key[0];
+          last = __reduce_min_sync(0xffffffffu, key[0]);
+          beam_code[b] = last & 0xffu;
+          const bool own = key[0] == last;  // keys are distinct: they end in the code
 #pragma unroll
-          for (int jj = 1; jj < 8; ++jj) lm = min(lm, key[jj]);
-          const uint32_t m = __reduce_min_sync(0xffffffffu, lm);
-          beam_code[b] = m & 0xffu;
-#pragma unroll
-          for (int jj = 0; jj < 8; ++jj)
-            if (key[jj] == m) key[jj] = 0xffffffffu;
+          for (int jj = 0; jj < 7; ++jj) key[jj] = own ? key[jj + 1] : key[jj];
+          key[7] = own ? 0xffffffffu : key[7];
         }
       }
-      // is that guess provably the exact beam?  theta = largest score in the guess;
-      // every member of the exact beam scores <= theta + margin1; if exactly B
-      // codewords do, they are the guess and the exact beam at once.
+      // is that guess provably the exact beam?  theta = an upper bound of the scores in the guess (the top of the
+      // truncation bucket of the key extracted last); every member of the exact beam scores <= theta + margin1; if
+      // exactly B codewords do, they are the guess and the exact beam at once.
       {
-        float th = -kInf;
         uint32_t cnt = 0;
-#pragma unroll
-        for (int jj = 0; jj < 8; ++jj)
-          if (key[jj] == 0xffffffffu) th = fmaxf(th, f[jj]);
-        const float theta = unord(__reduce_max_sync(0xffffffffu, ord(th)));
+        const float theta = unord(last | 0xffu);
         const float limit1 = theta + margin1;
         uint32_t member = 0;
 #pragma unroll
