@@ -499,59 +499,67 @@ __global__ void __launch_bounds__(kM2Threads, 2) encode_m2_kernel(const EncM2Par
     const float limit2 = gmin + my_margin2;
 
     // ---- decision in binary64 among the pairs within the margin, plus the previous pair.
-    // A sub-chunk within the margin is revisited by the whole warp, one codeword per lane, on behalf of the
-    // lane (target, beam entry) that found it; that lane keeps the best (distance, code pair).
+    // The eight lanes of a target revisit its sub-chunks within the margin one after the other, four codewords per
+    // lane, the four targets of the group side by side; every lane keeps the best (distance, code pair) it has seen.
+    // (The fast score is evaluated again here, in another order: both evaluations lie within half the margin of the
+    // true score, so the pair the definition selects passes both tests.)
     double bd = __longlong_as_double(0x7ff0000000000000ll);
     uint32_t bk = 0xffffffffu;  // code1 << 8 | code2: orders like (code1, code2)
+    {
+      uint32_t hm = 0;  // sub-chunks of this lane's beam entry within the margin
 #pragma unroll
-    for (int sub = 0; sub < 8; ++sub) {
-      uint32_t hits = __ballot_sync(0xffffffffu, sub_min[sub] <= limit2);  // false for inactive lanes
-      while (hits) {
-        const int src = __ffs(hits) - 1;
-        hits &= hits - 1;
-        const uint32_t sq = (uint32_t)src >> 3;
-        const uint32_t sk1 = __shfl_sync(0xffffffffu, k1, src);
-        const float slimit = __shfl_sync(0xffffffffu, limit2, src);
-        // the owner's target, codeword of codebook 1, residual and its half norm: the same operations
-        float st[8], sc1[8], sr[8], srho = 0.0f;
+      for (int sub = 0; sub < 8; ++sub) hm |= (active && sub_min[sub] <= limit2) ? (1u << sub) : 0u;
+      // the target's 64 (beam entry, sub-chunk) flags: byte b belongs to beam entry b
+      uint32_t hlo = my_b < 4 ? hm << (8 * my_b) : 0u, hhi = my_b >= 4 ? hm << (8 * (my_b - 4)) : 0u;
+#pragma unroll
+      for (int o = 1; o < 8; o <<= 1) {
+        hlo |= __shfl_xor_sync(0xffffffffu, hlo, o);
+        hhi |= __shfl_xor_sync(0xffffffffu, hhi, o);
+      }
+      while (__any_sync(0xffffffffu, (hlo | hhi) != 0u)) {
+        const bool work = (hlo | hhi) != 0u;
+        uint32_t pos = 0;
+        if (hlo) {
+          pos = (uint32_t)__ffs(hlo) - 1u;
+          hlo &= hlo - 1u;
+        } else if (hhi) {
+          pos = 32u + (uint32_t)__ffs(hhi) - 1u;
+          hhi &= hhi - 1u;
+        }
+        const uint32_t hb = pos >> 3, hsub = pos & 7u;
+        const uint32_t hk1 = work ? sm.wk[warp][my_q][hb] : 0u;
+        float sc1[8], sr[8], srho = 0.0f;
         {
-          const float4 ta = *reinterpret_cast<const float4*>(&sm.wt[warp][sq][0]);
-          const float4 tb = *reinterpret_cast<const float4*>(&sm.wt[warp][sq][4]);
-          const float4 ca = *reinterpret_cast<const float4*>(&sm.c1[sk1][0]);
-          const float4 cb = *reinterpret_cast<const float4*>(&sm.c1[sk1][4]);
-          st[0] = ta.x; st[1] = ta.y; st[2] = ta.z; st[3] = ta.w; st[4] = tb.x; st[5] = tb.y; st[6] = tb.z; st[7] = tb.w;
+          const float4 ca = *reinterpret_cast<const float4*>(&sm.c1[hk1][0]);
+          const float4 cb = *reinterpret_cast<const float4*>(&sm.c1[hk1][4]);
           sc1[0] = ca.x; sc1[1] = ca.y; sc1[2] = ca.z; sc1[3] = ca.w;
           sc1[4] = cb.x; sc1[5] = cb.y; sc1[6] = cb.z; sc1[7] = cb.w;
         }
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-          sr[i] = __fsub_rn(st[i], sc1[i]);
+          sr[i] = __fsub_rn(t[i], sc1[i]);
           srho = __fmaf_rn(sr[i], sr[i], srho);
         }
         srho = __fmul_rn(0.5f, srho);
-        const uint32_t k2 = sub * 32 + lane;
-        float s2 = __fadd_rn(sm.h2[k2], srho);  // the same operations as the packed evaluation
 #pragma unroll
-        for (int i = 0; i < 8; ++i) s2 = __fmaf_rn(-sr[i], sm.c2[k2][i], s2);
-        const bool cand = s2 <= slimit && k2 < p.K;
-        if (__any_sync(0xffffffffu, cand)) {
-          double d = __longlong_as_double(0x7ff0000000000000ll);
-          uint32_t kk = 0xffffffffu;
-          if (cand) {
-            d = exact2(st, sc1, sm.c2[k2]);
-            kk = (sk1 << 8) | k2;
+        for (int c = 0; c < 4; ++c) {
+          const uint32_t k2 = hsub * 32u + 8u * c + my_b;
+          float c2v[8];
+          {
+            const float4 ca = *reinterpret_cast<const float4*>(&sm.c2[k2][0]);
+            const float4 cb = *reinterpret_cast<const float4*>(&sm.c2[k2][4]);
+            c2v[0] = ca.x; c2v[1] = ca.y; c2v[2] = ca.z; c2v[3] = ca.w;
+            c2v[4] = cb.x; c2v[5] = cb.y; c2v[6] = cb.z; c2v[7] = cb.w;
           }
-          // warp-wide lexicographic minimum of (d, kk); distances are >= 0 so their bits order like u64
-          const uint64_t bits = (uint64_t)__double_as_longlong(d);
-          const uint32_t hi = (uint32_t)(bits >> 32), lo = (uint32_t)bits;
-          const uint32_t mhi = __reduce_min_sync(0xffffffffu, hi);
-          const uint32_t mlo = __reduce_min_sync(0xffffffffu, hi == mhi ? lo : 0xffffffffu);
-          const uint32_t mk = __reduce_min_sync(0xffffffffu, (hi == mhi && lo == mlo) ? kk : 0xffffffffu);
-          if (lane == src) {
-            const double md = __longlong_as_double((long long)(((uint64_t)mhi << 32) | mlo));
-            if (md < bd || (md == bd && mk < bk)) {
-              bd = md;
-              bk = mk;
+          float s2 = __fadd_rn(sm.h2[k2], srho);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) s2 = __fmaf_rn(-sr[i], c2v[i], s2);
+          if (work && s2 <= limit2 && k2 < p.K) {
+            const double d = exact2(t, sc1, c2v);
+            const uint32_t kk = (hk1 << 8) | k2;
+            if (d < bd || (d == bd && kk < bk)) {
+              bd = d;
+              bk = kk;
             }
           }
         }
