@@ -1,6 +1,5 @@
 // Beam search for three or four additive codebooks (Appendix C / Appendix J: beam search, beam size 8; the
-// residual form of the two-codebook kernel carried through more stages).  First version: every candidate is
-// scored directly in binary64, exactly as the decision is defined, so there is no fast filter and no rescoring:
+// residual form of the two-codebook kernel carried through more stages).
 //
 //   stage m (m = 1..M): each kept partial tuple (one empty tuple before stage 1) is extended by every codeword
 //     of codebook m; the score of an extension is ||t - c^1 - ... - c^m||^2 with the residual carried in binary64
@@ -8,10 +7,15 @@
 //   after stages 1..M-1 the `beam` smallest extensions under (score, tuple) are kept;
 //   the result is the smallest member of the last stage's extensions and the previous tuple.
 //
-// One warp per target.  Codebooks sit in shared memory as binary32 (M * K * 32 bytes).  Per stage a lane scores
-// the candidates lane, lane+32, ... and keeps its own `beam` smallest in registers (sorted by insertion); the
-// warp then extracts the overall `beam` smallest by repeated warp minimum over the lanes' heads.
-// Cost per target: (1 + (M-1) * beam) * K candidates of 24 binary64 operations.
+// One warp per target.  Codebooks sit in shared memory as binary32 (M * K * 32 bytes).  A stage makes two passes
+// over fast estimates of all extensions: the first finds a threshold (the keep-th smallest of the lanes' minima),
+// the second gives every extension within the estimates' error bound of it its binary64 score and keeps the
+// lane's `beam` smallest in registers (sorted by insertion); the warp then extracts the overall `beam` smallest by
+// repeated warp minimum over the lanes' heads.  For fp16 codebooks the estimates come from the tensor pipe: the
+// kept residuals are the rows of a 16 x 16 fp16 tile [ -hi(2^e r) | -lo(2^e r) ], the codewords the columns
+// [ c | c ], the accumulator starts at 2^e ||c||^2 / 2 (mma.sync m16n8k16, fp32 accumulation); with fewer than
+// eight kept residuals the rows repeat them and the copies share the codebook between them.  For binary32
+// codebooks the estimate is sum_i (fl32(r_i) - c_i)^2 on the FP32 pipe.
 #include <cuda_fp16.h>
 
 #include "pvt_internal.h"
@@ -45,13 +49,45 @@ __device__ __forceinline__ bool less_than(double da, uint32_t ka, double db, uin
   return da < db || (da == db && ka < kb);
 }
 
+constexpr int kMxPadK = 256;              // codewords per codebook in the tensor-pipe image (padded)
+constexpr float kMxPadHalfNorm = 3.0e38f;  // half norm of a padding codeword: never within any bound
+
+// D = A (16 x 16, rows = residuals) x B (16 x 8, columns = codewords) + C, fp16 operands, fp32 accumulation;
+// rows 8..15 of A are zero
+__device__ __forceinline__ void mma_rows8(float& d0, float& d1, uint32_t a_hi, uint32_t a_lo, uint32_t b, float c0,
+                                          float c1) {
+  float d2 __attribute__((unused)), d3 __attribute__((unused));  // rows 8..15: nothing
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %5}, {%7, %7}, "
+      "{%8, %9, %8, %9};"
+      : "=f"(d0), "=f"(d1), "=f"(d2), "=f"(d3)
+      : "r"(a_hi), "r"(0u), "r"(a_lo), "r"(b), "f"(c0), "f"(c1));
+}
+
+// bytes of the tensor-pipe image of the codebooks: B fragments, half norms, largest norm per codebook
+__host__ __device__ constexpr size_t mx_image_bytes(int M) {
+  return (size_t)M * (kMxPadK / 8) * 32 * 4 + (size_t)M * kMxPadK * 4 + 16;
+}
+
 template <int M, bool CB_F16>
 __global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   float* book = reinterpret_cast<float*>(smem_raw);                               // [M][K][8]
   double* resid = reinterpret_cast<double*>(smem_raw + (size_t)M * p.K * 32);     // [warps][beam][8]
   float* resid_f = reinterpret_cast<float*>(resid + kMxWarps * kMxBeam * 8);      // the same, rounded to binary32
+  // fp16 codebooks only: word [m][n-tile][lane] = halves (c[8 nt + lane/4][2 (lane%4)], [.. + 1]); ||c||^2/2; max ||c||^2
+  uint32_t* bfrag = reinterpret_cast<uint32_t*>(resid_f + kMxWarps * kMxBeam * 8);
+  float* hnorm = reinterpret_cast<float*>(bfrag + M * (kMxPadK / 8) * 32);
+  uint32_t* n2max_bits = reinterpret_cast<uint32_t*>(hnorm + M * kMxPadK);
   const uint32_t K = p.K;
+  if (CB_F16) {
+    for (uint32_t e = threadIdx.x; e < (uint32_t)M * kMxPadK; e += kMxThreads) {
+      hnorm[e] = kMxPadHalfNorm;
+#pragma unroll
+      for (int qq = 0; qq < 4; ++qq) bfrag[4 * e + qq] = 0u;
+    }
+    if (threadIdx.x < M) n2max_bits[threadIdx.x] = 0u;
+    __syncthreads();
+  }
   for (uint32_t row = threadIdx.x; row < M * K; row += kMxThreads) {
     float c[8];
     if (CB_F16) {
@@ -70,6 +106,19 @@ __global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p)
     }
 #pragma unroll
     for (int i = 0; i < 8; ++i) book[(size_t)row * 8 + i] = c[i];
+    if (CB_F16) {
+      const uint32_t m = row / K, kap = row % K;
+      float n2 = 0.0f;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) n2 = fmaf(c[i], c[i], n2);
+      hnorm[m * kMxPadK + kap] = 0.5f * n2;
+      atomicMax(&n2max_bits[m], __float_as_uint(n2));  // non-negative: bits order like values
+#pragma unroll
+      for (int qq = 0; qq < 4; ++qq) {
+        const __half2 v = __floats2half2_rn(c[2 * qq], c[2 * qq + 1]);  // exact: the codebook is fp16
+        bfrag[(m * (kMxPadK / 8) + (kap >> 3)) * 32 + 4 * (kap & 7u) + qq] = *reinterpret_cast<const uint32_t*>(&v);
+      }
+    }
   }
   __syncthreads();
 
@@ -132,62 +181,6 @@ __global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p)
     const int keep = (m == M - 1) ? 1 : beam;
     const int shift = 24 - 8 * m;
 
-    // Pass 1, binary32 and branch-free: the estimate d_fl = sum_i (fl32(r_i) - c_i)^2 of every extension; each lane
-    // keeps its smallest estimate, the warp derives a threshold theta from the 32 minima.  With R = the largest residual norm, |d_fl - d| <= 2^-22 sqrt(d) R + 2^-20 d: the residual is
-    // rounded to binary32 (2^-24 |r_i| per element, which matters when the codeword nearly cancels it), the
-    // differences, squares and sums add relative roundings.
-    float r2max = 0.0f;
-    if (lane < n_kept) {
-#pragma unroll
-      for (int i = 0; i < 8; ++i) r2max = fmaf(my_resid_f[lane * 8 + i], my_resid_f[lane * 8 + i], r2max);
-    }
-    r2max = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(r2max)));  // non-negative: bits order like values
-    auto estimate = [&](const float4& ra, const float4& rb, const float* c) {
-      const float4 ca = *reinterpret_cast<const float4*>(c), cb = *reinterpret_cast<const float4*>(c + 4);
-      float e, dfl;
-      e = ra.x - ca.x; dfl = e * e;
-      e = ra.y - ca.y; dfl = fmaf(e, e, dfl);
-      e = ra.z - ca.z; dfl = fmaf(e, e, dfl);
-      e = ra.w - ca.w; dfl = fmaf(e, e, dfl);
-      e = rb.x - cb.x; dfl = fmaf(e, e, dfl);
-      e = rb.y - cb.y; dfl = fmaf(e, e, dfl);
-      e = rb.z - cb.z; dfl = fmaf(e, e, dfl);
-      e = rb.w - cb.w; dfl = fmaf(e, e, dfl);
-      return dfl;
-    };
-    uint32_t est_min = 0x7f800000u;  // this lane's smallest estimate (non-negative: bits order like values)
-    for (int b = 0; b < n_kept; ++b) {
-      const float4 ra = *reinterpret_cast<const float4*>(&my_resid_f[b * 8]);
-      const float4 rb = *reinterpret_cast<const float4*>(&my_resid_f[b * 8 + 4]);
-      for (uint32_t q = lane; q < K; q += 32)
-        est_min = min(est_min, __float_as_uint(estimate(ra, rb, &book[((size_t)m * K + q) * 8])));
-    }
-    // theta: the keep-th smallest of the 32 lane minima -- `keep` different extensions have an estimate of at
-    // most theta, so the exact keep-th smallest score lies within the error bound of it (a little looser than
-    // the keep-th smallest estimate overall, at one instruction per extension instead of a sorted insertion)
-    uint32_t theta_bits = 0x7f800000u;
-    {
-      uint32_t hv = est_min;
-      for (int round = 0; round < keep; ++round) {
-        const uint32_t mv = __reduce_min_sync(0xffffffffu, hv);
-        if (mv == 0x7f800000u) {  // fewer than `keep` lanes have an extension: everything survives
-          theta_bits = mv;
-          break;
-        }
-        theta_bits = mv;
-        const uint32_t owners = __ballot_sync(0xffffffffu, hv == mv);
-        if (lane == __ffs(owners) - 1) hv = 0x7f800000u;  // equal minima in several lanes: one leaves per round
-      }
-    }
-    // every member of the exact `keep` smallest has an estimate within the two error bounds of theta
-    const float theta = __uint_as_float(theta_bits);
-    const float bound = theta_bits == 0x7f800000u
-                            ? theta
-                            : theta + 4.0f * (2.3841858e-7f /* 2^-22 */ * sqrtf(theta * r2max) + 9.5367432e-7f /* 2^-20 */ * theta) +
-                                  1e-37f;
-
-    // Pass 2: the same estimates again (bit for bit); the few extensions within the bound are scored in binary64
-    // and kept in this lane's sorted list
     double ld[kMxBeam];
     uint32_t lk[kMxBeam];
 #pragma unroll
@@ -195,35 +188,194 @@ __global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p)
       ld[q] = __longlong_as_double(kInfBits);
       lk[q] = kNoKey;
     }
-    for (int b = 0; b < n_kept; ++b) {
-      const float4 ra = *reinterpret_cast<const float4*>(&my_resid_f[b * 8]);
-      const float4 rb = *reinterpret_cast<const float4*>(&my_resid_f[b * 8 + 4]);
+    // sorted insertion of an extension into this lane's list of `keep` entries: the new entry sinks to its place,
+    // the last one drops
+    auto insert = [&](double d, uint32_t key) {
+#pragma unroll
+      for (int x = 0; x < kMxBeam; ++x) {
+        if (x < keep && less_than(d, key, ld[x], lk[x])) {
+          const double td = ld[x];
+          const uint32_t tk = lk[x];
+          ld[x] = d;
+          lk[x] = key;
+          d = td;
+          key = tk;
+        }
+      }
+    };
+    // theta: the keep-th smallest of the lanes' smallest estimates (one or two per lane, sorted) -- `keep` different
+    // extensions have an estimate of at most theta, so the exact keep-th smallest score lies within the error bound
+    // of it (a little looser than the keep-th smallest estimate overall, at a few instructions per extension instead
+    // of a sorted insertion)
+    auto kth_of_lane_minima = [&](uint32_t first, uint32_t second) {
+      uint32_t theta_bits = 0x7f800000u;
+      for (int round = 0; round < keep; ++round) {
+        const uint32_t mv = __reduce_min_sync(0xffffffffu, first);
+        theta_bits = mv;
+        if (mv == 0x7f800000u) break;  // fewer than `keep` extensions on offer: everything survives
+        const uint32_t owners = __ballot_sync(0xffffffffu, first == mv);
+        if (lane == __ffs(owners) - 1) {  // equal minima in several lanes: one leaves per round
+          first = second;
+          second = 0x7f800000u;
+        }
+      }
+      return theta_bits;
+    };
+    if (CB_F16) {
+      // Estimates from the tensor pipe.  Row rho of the A tile (rho = lane / 4) holds kept residual b = rho mod
+      // n_kept; the copies of a residual take the n-tiles of the codebook in turn.  A thread sees, per n-tile of
+      // eight codewords, the estimates of its row against codewords 8 nt + 2 (lane % 4) and the next one:
+      //   est = ||r_f||^2 + 2 * 2^-e * D,   D = 2^e (||c||^2/2 - <r_f, c>)  up to rounding.
+      // Error against the binary64 score d (R = largest residual norm, C = largest codeword norm, S = (R + C)^2):
+      // rounding r to binary32 2^-23 sqrt(d) R; the halves 2^-21 R C, or 2^-24 2^-e sqrt(8) C where the low half is
+      // subnormal; 17 accumulations of the products 2^-17.9 (R C + C^2/2); the norms 2^-20 C^2 + 2^-21 R^2:
+      // below 2^-17 S + 2^-22 2^-e C in all.
+      const uint32_t g8 = (uint32_t)lane >> 2, qd = (uint32_t)lane & 3u;
+      const uint32_t nk = (uint32_t)n_kept;
+      const uint32_t b = g8 % nk, rep = g8 / nk, nrep = (7u - b) / nk + 1u;  // copies of residual b among the 8 rows
+      const float2 rv = *reinterpret_cast<const float2*>(&my_resid_f[b * 8 + 2 * qd]);
+      float rr = 0.0f;
+      {
+        const float4 ra = *reinterpret_cast<const float4*>(&my_resid_f[b * 8]);
+        const float4 rb = *reinterpret_cast<const float4*>(&my_resid_f[b * 8 + 4]);
+        rr = ra.x * ra.x;
+        rr = fmaf(ra.y, ra.y, rr); rr = fmaf(ra.z, ra.z, rr); rr = fmaf(ra.w, ra.w, rr);
+        rr = fmaf(rb.x, rb.x, rr); rr = fmaf(rb.y, rb.y, rr); rr = fmaf(rb.z, rb.z, rr); rr = fmaf(rb.w, rb.w, rr);
+      }
+      const float rmax = fmaxf(fabsf(rv.x), fabsf(rv.y));
+      const uint32_t rbits = __reduce_max_sync(0xffffffffu, __float_as_uint(rmax));
+      const float r2max = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(rr)));
+      int e = 126 - (int)((rbits >> 23) & 0xffu);
+      e = e > 15 ? 15 : (e < -100 ? -100 : e);
+      const float sc = __uint_as_float((uint32_t)(e + 127) << 23), inv = __uint_as_float((uint32_t)(127 - e) << 23);
+      uint32_t a_hi, a_lo;
+      {
+        const float x = -rv.x * sc, y = -rv.y * sc;  // exact
+        const __half2 hi = __floats2half2_rn(x, y);
+        const float2 back = __half22float2(hi);
+        const __half2 lo = __floats2half2_rn(x - back.x, y - back.y);
+        a_hi = *reinterpret_cast<const uint32_t*>(&hi);
+        a_lo = *reinterpret_cast<const uint32_t*>(&lo);
+      }
+      const uint32_t* bf = bfrag + (size_t)m * (kMxPadK / 8) * 32 + lane;
+      const float* hn = hnorm + (size_t)m * kMxPadK + 2 * qd;
+      const float two_inv = 2.0f * inv;
+      const uint32_t n_tiles = (K + 7u) >> 3;
+      // pass 1: this lane's two smallest estimates (all of a lane's extensions belong to one residual, so the
+      // best residual's lanes must be able to offer more than one each)
+      float m0 = __uint_as_float(0x7f800000u), m1 = m0;
+      {
+        uint32_t next = rep;
+        for (uint32_t nt = 0; nt < n_tiles; ++nt) {
+          const float2 hh = *reinterpret_cast<const float2*>(hn + 8 * nt);
+          float d0, d1;
+          mma_rows8(d0, d1, a_hi, a_lo, bf[32 * nt], hh.x * sc, hh.y * sc);
+          if (nt == next) {
+            next += nrep;
+            const float e0 = fmaf(d0, two_inv, rr), e1 = fmaf(d1, two_inv, rr);
+            const float lo = fminf(e0, e1), hi = fmaxf(e0, e1);
+            const float t0 = fmaxf(m0, lo);
+            m0 = fminf(m0, lo);
+            m1 = fminf(fminf(m1, hi), t0);
+          }
+        }
+      }
+      // an estimate can come out slightly negative; the order of the bit patterns needs non-negative values
+      const uint32_t theta_bits =
+          kth_of_lane_minima(__float_as_uint(fmaxf(m0, 0.0f)), __float_as_uint(fmaxf(m1, 0.0f)));
+      const float theta = __uint_as_float(theta_bits);
+      const float cmax = sqrtf(__uint_as_float(n2max_bits[m]));
+      const float reach = sqrtf(r2max) + cmax;
+      // twice the error bound, with a factor 2 to spare
+      const float bound = theta_bits == 0x7f800000u
+                              ? theta
+                              : theta + 3.0517578e-5f /* 2^-15 */ * reach * reach + 9.5367432e-7f /* 2^-20 */ * inv * cmax + 1e-37f;
+      // pass 2: the same estimates again (bit for bit); the few extensions within the bound are scored in binary64
       uint32_t kb = kept_key[0];
 #pragma unroll
       for (int x = 1; x < kMxBeam; ++x)
-        if (x == b) kb = kept_key[x];
+        if ((uint32_t)x == b) kb = kept_key[x];
       const double* r = &my_resid[b * 8];
-      for (uint32_t q = lane; q < K; q += 32) {
-        const float* c = &book[((size_t)m * K + q) * 8];
-        if (!(estimate(ra, rb, c) <= bound)) continue;
-        double d = 0.0;
+      uint32_t next = rep;
+      for (uint32_t nt = 0; nt < n_tiles; ++nt) {
+        const float2 hh = *reinterpret_cast<const float2*>(hn + 8 * nt);
+        float d0, d1;
+        mma_rows8(d0, d1, a_hi, a_lo, bf[32 * nt], hh.x * sc, hh.y * sc);
+        if (nt != next) continue;
+        next += nrep;
+        const float e0 = fmaf(d0, two_inv, rr), e1 = fmaf(d1, two_inv, rr);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const double ee = __dsub_rn(r[i], (double)c[i]);
-          d = __dadd_rn(d, __dmul_rn(ee, ee));
-        }
-        uint32_t key = kb | (q << shift);
-        // insertion into the sorted list of `keep` entries: the new entry sinks to its place, the last one drops
+        for (int h = 0; h < 2; ++h) {
+          const uint32_t q = 8 * nt + 2 * qd + h;
+          if (!((h ? e1 : e0) <= bound) || q >= K) continue;
+          const float* c = &book[((size_t)m * K + q) * 8];
+          double d = 0.0;
 #pragma unroll
-        for (int x = 0; x < kMxBeam; ++x) {
-          if (x < keep && less_than(d, key, ld[x], lk[x])) {
-            const double td = ld[x];
-            const uint32_t tk = lk[x];
-            ld[x] = d;
-            lk[x] = key;
-            d = td;
-            key = tk;
+          for (int i = 0; i < 8; ++i) {
+            const double ee = __dsub_rn(r[i], (double)c[i]);
+            d = __dadd_rn(d, __dmul_rn(ee, ee));
           }
+          insert(d, kb | (q << shift));
+        }
+      }
+    } else {
+      // Pass 1, binary32 and branch-free: the estimate d_fl = sum_i (fl32(r_i) - c_i)^2 of every extension.  With
+      // R = the largest residual norm, |d_fl - d| <= 2^-22 sqrt(d) R + 2^-20 d: the residual is rounded to binary32
+      // (2^-24 |r_i| per element, which matters when the codeword nearly cancels it), the differences, squares and
+      // sums add relative roundings.
+      float r2max = 0.0f;
+      if (lane < n_kept) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) r2max = fmaf(my_resid_f[lane * 8 + i], my_resid_f[lane * 8 + i], r2max);
+      }
+      r2max = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(r2max)));  // non-negative: bits order like values
+      auto estimate = [&](const float4& ra, const float4& rb, const float* c) {
+        const float4 ca = *reinterpret_cast<const float4*>(c), cb = *reinterpret_cast<const float4*>(c + 4);
+        float e, dfl;
+        e = ra.x - ca.x; dfl = e * e;
+        e = ra.y - ca.y; dfl = fmaf(e, e, dfl);
+        e = ra.z - ca.z; dfl = fmaf(e, e, dfl);
+        e = ra.w - ca.w; dfl = fmaf(e, e, dfl);
+        e = rb.x - cb.x; dfl = fmaf(e, e, dfl);
+        e = rb.y - cb.y; dfl = fmaf(e, e, dfl);
+        e = rb.z - cb.z; dfl = fmaf(e, e, dfl);
+        e = rb.w - cb.w; dfl = fmaf(e, e, dfl);
+        return dfl;
+      };
+      uint32_t est_min = 0x7f800000u;  // this lane's smallest estimate (non-negative: bits order like values)
+      for (int b = 0; b < n_kept; ++b) {
+        const float4 ra = *reinterpret_cast<const float4*>(&my_resid_f[b * 8]);
+        const float4 rb = *reinterpret_cast<const float4*>(&my_resid_f[b * 8 + 4]);
+        for (uint32_t q = lane; q < K; q += 32)
+          est_min = min(est_min, __float_as_uint(estimate(ra, rb, &book[((size_t)m * K + q) * 8])));
+      }
+      // every member of the exact `keep` smallest has an estimate within the two error bounds of theta
+      const uint32_t theta_bits = kth_of_lane_minima(est_min, 0x7f800000u);
+      const float theta = __uint_as_float(theta_bits);
+      const float bound = theta_bits == 0x7f800000u
+                              ? theta
+                              : theta + 4.0f * (2.3841858e-7f /* 2^-22 */ * sqrtf(theta * r2max) + 9.5367432e-7f /* 2^-20 */ * theta) +
+                                    1e-37f;
+      // Pass 2: the same estimates again (bit for bit); the few extensions within the bound are scored in binary64
+      // and kept in this lane's sorted list
+      for (int b = 0; b < n_kept; ++b) {
+        const float4 ra = *reinterpret_cast<const float4*>(&my_resid_f[b * 8]);
+        const float4 rb = *reinterpret_cast<const float4*>(&my_resid_f[b * 8 + 4]);
+        uint32_t kb = kept_key[0];
+#pragma unroll
+        for (int x = 1; x < kMxBeam; ++x)
+          if (x == b) kb = kept_key[x];
+        const double* r = &my_resid[b * 8];
+        for (uint32_t q = lane; q < K; q += 32) {
+          const float* c = &book[((size_t)m * K + q) * 8];
+          if (!(estimate(ra, rb, c) <= bound)) continue;
+          double d = 0.0;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const double ee = __dsub_rn(r[i], (double)c[i]);
+            d = __dadd_rn(d, __dmul_rn(ee, ee));
+          }
+          insert(d, kb | (q << shift));
         }
       }
     }
@@ -312,7 +464,8 @@ __global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p)
 
 template <int M, bool CB_F16>
 cudaError_t launch_m(const MxParams& p, cudaStream_t stream) {
-  const size_t smem = (size_t)M * p.K * 32 + (size_t)kMxWarps * kMxBeam * 8 * (sizeof(double) + sizeof(float));
+  const size_t smem = (size_t)M * p.K * 32 + (size_t)kMxWarps * kMxBeam * 8 * (sizeof(double) + sizeof(float)) +
+                      (CB_F16 ? mx_image_bytes(M) : 0);
   cudaError_t e = cudaFuncSetAttribute(encode_mx_kernel<M, CB_F16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)smem);
   if (e != cudaSuccess) return e;
