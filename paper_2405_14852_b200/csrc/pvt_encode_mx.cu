@@ -49,6 +49,7 @@ __device__ __forceinline__ bool less_than(double da, uint32_t ka, double db, uin
   return da < db || (da == db && ka < kb);
 }
 
+constexpr int kMxCand = 256;              // capacity of a warp's candidate list
 constexpr int kMxPadK = 256;              // codewords per codebook in the tensor-pipe image (padded)
 constexpr float kMxPadHalfNorm = 3.0e38f;  // half norm of a padding codeword: never within any bound
 
@@ -75,7 +76,10 @@ __global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p)
   double* resid = reinterpret_cast<double*>(smem_raw + (size_t)M * p.K * 32);     // [warps][beam][8]
   float* resid_f = reinterpret_cast<float*>(resid + kMxWarps * kMxBeam * 8);      // the same, rounded to binary32
   // fp16 codebooks only: word [m][n-tile][lane] = halves (c[8 nt + lane/4][2 (lane%4)], [.. + 1]); ||c||^2/2; max ||c||^2
-  uint32_t* bfrag = reinterpret_cast<uint32_t*>(resid_f + kMxWarps * kMxBeam * 8);
+  // per warp: the extensions that pass the filter of a stage, (kept tuple << 8 | code), and their count
+  uint16_t* cand = reinterpret_cast<uint16_t*>(resid_f + kMxWarps * kMxBeam * 8);
+  uint32_t* cand_n = reinterpret_cast<uint32_t*>(cand + kMxWarps * kMxCand);
+  uint32_t* bfrag = cand_n + kMxWarps;
   float* hnorm = reinterpret_cast<float*>(bfrag + M * (kMxPadK / 8) * 32);
   uint32_t* n2max_bits = reinterpret_cast<uint32_t*>(hnorm + M * kMxPadK);
   const uint32_t K = p.K;
@@ -144,6 +148,8 @@ __global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p)
   }
   double* my_resid = resid + (size_t)warp * kMxBeam * 8;
   float* my_resid_f = resid_f + (size_t)warp * kMxBeam * 8;
+  uint16_t* my_cand = cand + (size_t)warp * kMxCand;
+  uint32_t* my_cand_n = cand_n + warp;
   const int beam = p.beam;
 
   // kept partial tuples: key = code_1 << 24 | code_2 << 16 | ... (lexicographic order of tuples = numeric order)
@@ -201,6 +207,36 @@ __global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p)
           d = td;
           key = tk;
         }
+      }
+    };
+    // an extension that passed the filter goes on the warp's list (any order: the decision below does not depend
+    // on it); a list that overflows is detected by its count
+    if (lane == 0) *my_cand_n = 0u;
+    __syncwarp();
+    auto collect = [&](uint32_t b, uint32_t q) {
+      const uint32_t pos = atomicAdd(my_cand_n, 1u);
+      if (pos < (uint32_t)kMxCand) my_cand[pos] = (uint16_t)((b << 8) | q);
+    };
+    // binary64 score of extension (kept tuple b, codeword q of this stage's codebook) into this lane's list
+    auto score_exact = [&](uint32_t b, uint32_t q, bool first) {
+      const double* r = &my_resid[b * 8];
+      const float* c = &book[((size_t)m * K + q) * 8];
+      double d = 0.0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const double ee = __dsub_rn(r[i], (double)c[i]);
+        d = __dadd_rn(d, __dmul_rn(ee, ee));
+      }
+      uint32_t kb = kept_key[0];
+#pragma unroll
+      for (int x = 1; x < kMxBeam; ++x)
+        if ((uint32_t)x == b) kb = kept_key[x];
+      const uint32_t key = kb | (q << shift);
+      if (first) {  // the list is still empty
+        ld[0] = d;
+        lk[0] = key;
+      } else {
+        insert(d, key);
       }
     };
     // theta: the keep-th smallest of the lanes' smallest estimates (one or two per lane, sorted) -- `keep` different
@@ -290,12 +326,7 @@ __global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p)
       const float bound = theta_bits == 0x7f800000u
                               ? theta
                               : theta + 3.0517578e-5f /* 2^-15 */ * reach * reach + 9.5367432e-7f /* 2^-20 */ * inv * cmax + 1e-37f;
-      // pass 2: the same estimates again (bit for bit); the few extensions within the bound are scored in binary64
-      uint32_t kb = kept_key[0];
-#pragma unroll
-      for (int x = 1; x < kMxBeam; ++x)
-        if ((uint32_t)x == b) kb = kept_key[x];
-      const double* r = &my_resid[b * 8];
+      // pass 2: the same estimates again (bit for bit); the few extensions within the bound go on the list
       uint32_t next = rep;
       for (uint32_t nt = 0; nt < n_tiles; ++nt) {
         const float2 hh = *reinterpret_cast<const float2*>(hn + 8 * nt);
@@ -304,19 +335,9 @@ __global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p)
         if (nt != next) continue;
         next += nrep;
         const float e0 = fmaf(d0, two_inv, rr), e1 = fmaf(d1, two_inv, rr);
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const uint32_t q = 8 * nt + 2 * qd + h;
-          if (!((h ? e1 : e0) <= bound) || q >= K) continue;
-          const float* c = &book[((size_t)m * K + q) * 8];
-          double d = 0.0;
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const double ee = __dsub_rn(r[i], (double)c[i]);
-            d = __dadd_rn(d, __dmul_rn(ee, ee));
-          }
-          insert(d, kb | (q << shift));
-        }
+        const uint32_t q = 8 * nt + 2 * qd;
+        if (e0 <= bound && q < K) collect(b, q);
+        if (e1 <= bound && q + 1 < K) collect(b, q + 1);
       }
     } else {
       // Pass 1, binary32 and branch-free: the estimate d_fl = sum_i (fl32(r_i) - c_i)^2 of every extension.  With
@@ -356,27 +377,28 @@ __global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p)
                               ? theta
                               : theta + 4.0f * (2.3841858e-7f /* 2^-22 */ * sqrtf(theta * r2max) + 9.5367432e-7f /* 2^-20 */ * theta) +
                                     1e-37f;
-      // Pass 2: the same estimates again (bit for bit); the few extensions within the bound are scored in binary64
-      // and kept in this lane's sorted list
+      // Pass 2: the same estimates again (bit for bit); the few extensions within the bound go on the list
       for (int b = 0; b < n_kept; ++b) {
         const float4 ra = *reinterpret_cast<const float4*>(&my_resid_f[b * 8]);
         const float4 rb = *reinterpret_cast<const float4*>(&my_resid_f[b * 8 + 4]);
-        uint32_t kb = kept_key[0];
-#pragma unroll
-        for (int x = 1; x < kMxBeam; ++x)
-          if (x == b) kb = kept_key[x];
-        const double* r = &my_resid[b * 8];
-        for (uint32_t q = lane; q < K; q += 32) {
-          const float* c = &book[((size_t)m * K + q) * 8];
-          if (!(estimate(ra, rb, c) <= bound)) continue;
-          double d = 0.0;
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const double ee = __dsub_rn(r[i], (double)c[i]);
-            d = __dadd_rn(d, __dmul_rn(ee, ee));
-          }
-          insert(d, kb | (q << shift));
+        for (uint32_t q = lane; q < K; q += 32)
+          if (estimate(ra, rb, &book[((size_t)m * K + q) * 8]) <= bound) collect((uint32_t)b, q);
+      }
+    }
+
+    // binary64 scores of the listed extensions, one per lane and round; a list that overflowed (many equal
+    // codewords, or fewer extensions than `keep`) is replaced by all extensions
+    __syncwarp();
+    {
+      const uint32_t n_cand = *my_cand_n;
+      if (n_cand <= (uint32_t)kMxCand) {
+        for (uint32_t i = lane; i < n_cand; i += 32) {
+          const uint32_t e = my_cand[i];
+          score_exact(e >> 8, e & 0xffu, i < 32u);
         }
+      } else {
+        for (uint32_t b = 0; b < (uint32_t)n_kept; ++b)
+          for (uint32_t q = lane; q < K; q += 32) score_exact(b, q, false);
       }
     }
 
@@ -465,6 +487,7 @@ __global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p)
 template <int M, bool CB_F16>
 cudaError_t launch_m(const MxParams& p, cudaStream_t stream) {
   const size_t smem = (size_t)M * p.K * 32 + (size_t)kMxWarps * kMxBeam * 8 * (sizeof(double) + sizeof(float)) +
+                      (size_t)kMxWarps * (kMxCand * sizeof(uint16_t) + sizeof(uint32_t)) +
                       (CB_F16 ? mx_image_bytes(M) : 0);
   cudaError_t e = cudaFuncSetAttribute(encode_mx_kernel<M, CB_F16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)smem);
