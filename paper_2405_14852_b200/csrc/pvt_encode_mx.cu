@@ -79,7 +79,10 @@ __global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p)
   // per warp: the extensions that pass the filter of a stage, (kept tuple << 8 | code), and their count
   uint16_t* cand = reinterpret_cast<uint16_t*>(resid_f + kMxWarps * kMxBeam * 8);
   uint32_t* cand_n = reinterpret_cast<uint32_t*>(cand + kMxWarps * kMxCand);
-  uint32_t* bfrag = cand_n + kMxWarps;
+  // per warp: the kept partial tuples and the target
+  uint32_t* kept_sm = cand_n + kMxWarps;
+  float* t_sm = reinterpret_cast<float*>(kept_sm + kMxWarps * kMxBeam);
+  uint32_t* bfrag = reinterpret_cast<uint32_t*>(t_sm + kMxWarps * 8);
   float* hnorm = reinterpret_cast<float*>(bfrag + M * (kMxPadK / 8) * 32);
   uint32_t* n2max_bits = reinterpret_cast<uint32_t*>(hnorm + M * kMxPadK);
   const uint32_t K = p.K;
@@ -150,14 +153,18 @@ __global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p)
   float* my_resid_f = resid_f + (size_t)warp * kMxBeam * 8;
   uint16_t* my_cand = cand + (size_t)warp * kMxCand;
   uint32_t* my_cand_n = cand_n + warp;
+  uint32_t* my_kept = kept_sm + (size_t)warp * kMxBeam;
+  float* my_t = t_sm + (size_t)warp * 8;
   const int beam = p.beam;
 
   // kept partial tuples: key = code_1 << 24 | code_2 << 16 | ... (lexicographic order of tuples = numeric order)
-  uint32_t kept_key[kMxBeam];
+  // (they live in shared memory: every use picks one by a run-time index)
   int n_kept = 1;
-  kept_key[0] = 0;
-#pragma unroll
-  for (int b = 1; b < kMxBeam; ++b) kept_key[b] = 0;
+  if (lane == 0) {
+    my_kept[0] = 0u;
+    *reinterpret_cast<float4*>(my_t) = make_float4(t[0], t[1], t[2], t[3]);
+    *reinterpret_cast<float4*>(my_t + 4) = make_float4(t[4], t[5], t[6], t[7]);
+  }
   double best_d = __longlong_as_double(kInfBits);
   uint32_t best_key = kNoKey;
 
@@ -167,14 +174,8 @@ __global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p)
     __syncwarp();
     for (int item = lane; item < n_kept * 8; item += 32) {
       const int b = item >> 3, i = item & 7;
-      uint32_t key = kept_key[0];
-#pragma unroll
-      for (int q = 1; q < kMxBeam; ++q)
-        if (q == b) key = kept_key[q];
-      double r = (double)t[0];
-#pragma unroll
-      for (int q = 1; q < 8; ++q)
-        if (q == i) r = (double)t[q];
+      const uint32_t key = my_kept[b];
+      double r = (double)my_t[i];
       for (int q = 0; q < m; ++q) {
         const uint32_t code = (key >> (24 - 8 * q)) & 0xffu;
         r = __dsub_rn(r, (double)book[((size_t)q * K + code) * 8 + i]);
@@ -227,11 +228,7 @@ __global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p)
         const double ee = __dsub_rn(r[i], (double)c[i]);
         d = __dadd_rn(d, __dmul_rn(ee, ee));
       }
-      uint32_t kb = kept_key[0];
-#pragma unroll
-      for (int x = 1; x < kMxBeam; ++x)
-        if ((uint32_t)x == b) kb = kept_key[x];
-      const uint32_t key = kb | (q << shift);
+      const uint32_t key = my_kept[b] | (q << shift);
       if (first) {  // the list is still empty
         ld[0] = d;
         lk[0] = key;
@@ -268,7 +265,12 @@ __global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p)
       // below 2^-17 S + 2^-22 2^-e C in all.
       const uint32_t g8 = (uint32_t)lane >> 2, qd = (uint32_t)lane & 3u;
       const uint32_t nk = (uint32_t)n_kept;
-      const uint32_t b = g8 % nk, rep = g8 / nk, nrep = (7u - b) / nk + 1u;  // copies of residual b among the 8 rows
+      uint32_t b = g8, rep = 0u, nrep = 1u;  // copies of residual b among the 8 rows (nk = 8: one each)
+      if (nk == 1u) {
+        b = 0u, rep = g8, nrep = 8u;
+      } else if (nk != 8u) {
+        b = g8 % nk, rep = g8 / nk, nrep = (7u - b) / nk + 1u;
+      }
       const float2 rv = *reinterpret_cast<const float2*>(&my_resid_f[b * 8 + 2 * qd]);
       float rr = 0.0f;
       {
@@ -302,6 +304,7 @@ __global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p)
       float m0 = __uint_as_float(0x7f800000u), m1 = m0;
       {
         uint32_t next = rep;
+#pragma unroll 4
         for (uint32_t nt = 0; nt < n_tiles; ++nt) {
           const float2 hh = *reinterpret_cast<const float2*>(hn + 8 * nt);
           float d0, d1;
@@ -328,6 +331,7 @@ __global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p)
                               : theta + 3.0517578e-5f /* 2^-15 */ * reach * reach + 9.5367432e-7f /* 2^-20 */ * inv * cmax + 1e-37f;
       // pass 2: the same estimates again (bit for bit); the few extensions within the bound go on the list
       uint32_t next = rep;
+#pragma unroll 4
       for (uint32_t nt = 0; nt < n_tiles; ++nt) {
         const float2 hh = *reinterpret_cast<const float2*>(hn + 8 * nt);
         float d0, d1;
@@ -389,8 +393,8 @@ __global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p)
     // binary64 scores of the listed extensions, one per lane and round; a list that overflowed (many equal
     // codewords, or fewer extensions than `keep`) is replaced by all extensions
     __syncwarp();
+    const uint32_t n_cand = *my_cand_n;
     {
-      const uint32_t n_cand = *my_cand_n;
       if (n_cand <= (uint32_t)kMxCand) {
         for (uint32_t i = lane; i < n_cand; i += 32) {
           const uint32_t e = my_cand[i];
@@ -402,43 +406,50 @@ __global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p)
       }
     }
 
-    // the warp's `keep` smallest: repeated minimum over the lanes' current heads
-    int head = 0;
-    uint32_t new_key[kMxBeam];
-#pragma unroll
-    for (int x = 0; x < kMxBeam; ++x) new_key[x] = 0;
+    // the warp's `keep` smallest under (score, tuple): repeated warp minimum over the lanes' current heads; with
+    // at most one listed extension per lane the head is the lane's only entry
+    __syncwarp();  // every lane has read the kept tuples it needed: they are replaced now
     int n_new = 0;
+    const bool single = n_cand <= 32u;
+    int head = 0;
     for (int round = 0; round < keep; ++round) {
-      double hd = __longlong_as_double(kInfBits);
-      uint32_t hk = kNoKey;
+      double hd = ld[0];
+      uint32_t hk = lk[0];
+      if (!single) {
 #pragma unroll
-      for (int x = 0; x < kMxBeam; ++x)
-        if (x == head) {
-          hd = ld[x];
-          hk = lk[x];
+        for (int x = 1; x < kMxBeam; ++x)
+          if (x == head) {
+            hd = ld[x];
+            hk = lk[x];
+          }
+        if (head >= kMxBeam) {
+          hd = __longlong_as_double(kInfBits);
+          hk = kNoKey;
         }
+      }
       const uint64_t bits = (uint64_t)__double_as_longlong(hd);
       const uint32_t hi = (uint32_t)(bits >> 32), lo = (uint32_t)bits;
       const uint32_t mhi = __reduce_min_sync(0xffffffffu, hi);
       const uint32_t mlo = __reduce_min_sync(0xffffffffu, hi == mhi ? lo : 0xffffffffu);
       const uint32_t mk = __reduce_min_sync(0xffffffffu, (hi == mhi && lo == mlo) ? hk : kNoKey);
       if (mhi == 0x7ff00000u && mlo == 0u) break;  // fewer candidates than `keep` (warp-uniform)
-      if (hi == mhi && lo == mlo && hk == mk) ++head;  // keys are unique: exactly one lane pops
+      if (hi == mhi && lo == mlo && hk == mk) {  // keys are unique: exactly one lane pops
+        if (single) {
+          ld[0] = __longlong_as_double(kInfBits);
+          lk[0] = kNoKey;
+        } else {
+          ++head;
+        }
+      }
       if (m == M - 1) {
         best_d = __longlong_as_double((long long)(((uint64_t)mhi << 32) | mlo));
         best_key = mk;
       } else {
-#pragma unroll
-        for (int x = 0; x < kMxBeam; ++x)
-          if (x == n_new) new_key[x] = mk;
+        if (lane == 0) my_kept[n_new] = mk;
         ++n_new;
       }
     }
-    if (m < M - 1) {
-#pragma unroll
-      for (int x = 0; x < kMxBeam; ++x) kept_key[x] = new_key[x];
-      n_kept = n_new;
-    }
+    if (m < M - 1) n_kept = n_new;
   }
 
   // the previous tuple joins the pool (Lemma 3.3: the step never raises the error)
@@ -487,7 +498,7 @@ __global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p)
 template <int M, bool CB_F16>
 cudaError_t launch_m(const MxParams& p, cudaStream_t stream) {
   const size_t smem = (size_t)M * p.K * 32 + (size_t)kMxWarps * kMxBeam * 8 * (sizeof(double) + sizeof(float)) +
-                      (size_t)kMxWarps * (kMxCand * sizeof(uint16_t) + sizeof(uint32_t)) +
+                      (size_t)kMxWarps * (kMxCand * sizeof(uint16_t) + sizeof(uint32_t) + kMxBeam * 4 + 8 * 4) +
                       (CB_F16 ? mx_image_bytes(M) : 0);
   cudaError_t e = cudaFuncSetAttribute(encode_mx_kernel<M, CB_F16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)smem);
