@@ -406,6 +406,38 @@ def test_three_and_four_codebooks_match_checker(M, K, f16, rows, cols, k, beam):
     assert band == 0  # every decision is taken on the checker's own binary64 values
 
 
+@pytest.mark.parametrize("M", [2, 3, 4])
+@pytest.mark.parametrize("f16", [True, False])
+def test_beam_search_with_targets_of_very_different_magnitude(M, f16):
+    """Rows of W scaled over twelve decades while the row scales stay put: neighbouring selected groups
+    (which share a warp, and on fp16 codebooks one power-of-two scale of the tensor-pipe operands) have
+    targets from 1e-6 to 1e6 times the codewords."""
+    rows, cols = 48, 256
+    L = synth.make_layer(rows, cols, cfg=230 + M, num_codebooks=M, codebook_size=256, codebook_fp16=f16,
+                         nearest=oracle_nearest)
+    decades = np.random.default_rng(231).uniform(-6.0, 6.0, size=(rows, 1))
+    L.W = (L.W * (10.0 ** decades)).astype(np.float32)
+    # every fourth group: consecutive selected groups come from different rows every few entries
+    idx = np.arange(0, L.num_groups, 5, dtype=np.uint32)
+    exact, band = check_encode(L, idx)
+    assert exact >= len(idx) - max(4, len(idx) // 100)
+
+
+@pytest.mark.parametrize("M", [2, 3, 4])
+def test_beam_search_with_a_codebook_of_equal_codewords(M):
+    """The second codebook holds one codeword 256 times: every extension of a stage ties exactly, far more than
+    any shortlist holds, and the lowest tuple must win on both sides."""
+    L = synth.make_layer(32, 256, cfg=240 + M, num_codebooks=M, codebook_size=256, codebook_fp16=True,
+                         nearest=oracle_nearest)
+    L.codebooks[1, :] = L.codebooks[1, 7]
+    idx = np.arange(L.num_groups, dtype=np.uint32)
+    t = oracle.targets(L.W, L.g, L.scale, L.eta, idx)
+    enc = oracle.encode(t, L.codebooks, L.codes.reshape(-1, M), L.beam)
+    got, err, status = run_encode(L, idx)
+    assert status == 0
+    assert np.array_equal(got.reshape(-1, M), enc.codes.reshape(-1, M))
+
+
 @pytest.mark.parametrize("M,K,f16,rows,cols", [(3, 100, True, 96, 136), (4, 256, True, 64, 512), (4, 50, False, 33, 72)])
 @pytest.mark.parametrize("out_f16", [False, True])
 def test_dequant_three_and_four_codebooks_bit_exact(M, K, f16, rows, cols, out_f16):
