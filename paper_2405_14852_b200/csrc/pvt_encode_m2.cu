@@ -5,7 +5,7 @@
 // pair in the pool).
 //
 // A warp handles four targets at a time; both codebooks live in shared memory;
-// two CTAs (16 warps) share an SM.
+// three CTAs (24 warps) share an SM.
 //   stage 1 (per target, the whole warp): lane l owns codewords l, l+32, ..., l+224
 //            of codebook 1: score1 = ||c1||^2/2 - <t, c1> for 256 codewords (8 per
 //            lane, packed f32x2); the `beam` smallest are extracted with warp-wide
@@ -34,6 +34,7 @@ size_t encode_m2_workspace_bytes() { return kWsHeaderBytes; }
 namespace {
 
 constexpr int kM2Threads = 256;
+constexpr int kM2CtasPerSm = 3;  // resident CTAs per SM the kernel is compiled for (registers) and launched as
 constexpr int kM2K = 256;  // codebooks are padded to this many codewords
 constexpr float kPadHalfNorm = 3.0e38f;
 constexpr float kInf = __builtin_huge_valf();
@@ -146,7 +147,7 @@ __device__ __forceinline__ float load_cb(const void* books, int f16, uint32_t m,
 
 // TC2: stage 2 on the tensor cores (fp16 codebooks: the codewords are exact halves), else on the FP32 pipe.
 template <bool TC2>
-__global__ void __launch_bounds__(kM2Threads, 2) encode_m2_kernel(const EncM2Params p) {
+__global__ void __launch_bounds__(kM2Threads, kM2CtasPerSm) encode_m2_kernel(const EncM2Params p) {
   __shared__ M2Smem sm;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
@@ -622,7 +623,7 @@ cudaError_t launch_encode_m2(const pvt_layer& L, uint64_t G, const uint32_t* idx
   const uint64_t warps_per_cta = kM2Threads / 32;
   const uint64_t groups = (k + kM2Group - 1) / kM2Group;
   uint64_t ctas = (groups + warps_per_cta - 1) / warps_per_cta;
-  if (ctas > 2 * (uint64_t)sm_count) ctas = 2 * (uint64_t)sm_count;  // two CTAs (16 warps) per SM
+  if (ctas > kM2CtasPerSm * (uint64_t)sm_count) ctas = kM2CtasPerSm * (uint64_t)sm_count;  // persistent: the resident CTAs
   timing_begin(kKernEncodeMain, stream);
   if (p.cb_f16)
     encode_m2_kernel<true><<<(unsigned)ctas, kM2Threads, 0, stream>>>(p);

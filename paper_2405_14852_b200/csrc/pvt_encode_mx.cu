@@ -70,7 +70,7 @@ __host__ __device__ constexpr size_t mx_image_bytes(int M) {
 }
 
 template <int M, bool CB_F16>
-__global__ void __launch_bounds__(kMxThreads) encode_mx_kernel(const MxParams p) {
+__global__ void __launch_bounds__(kMxThreads, M == 3 ? 4 : 3) encode_mx_kernel(const MxParams p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   float* book = reinterpret_cast<float*>(smem_raw);                               // [M][K][8]
   double* resid = reinterpret_cast<double*>(smem_raw + (size_t)M * p.K * 32);     // [warps][beam][8]
