@@ -37,7 +37,7 @@ template <int M, bool CB_F16, bool CODE_U16, bool OUT_F16, bool SMEM_BOOK, int P
 __global__ void __launch_bounds__(kDqThreads) dequant_kernel(const void* __restrict__ codebooks,
                                                               const void* __restrict__ codes,
                                                               const float* __restrict__ scale, uint64_t G,
-                                                              uint32_t gpr, uint32_t K, void* __restrict__ W_hat,
+                                                              FastDiv gpr, uint32_t K, void* __restrict__ W_hat,
                                                               uint32_t* status) {
   constexpr int kCwBytes = (CB_F16 ? 8 : 16) * PARTS;
   __shared__ __align__(16) unsigned char sh_book[SMEM_BOOK ? kDqSmemCodewords * kCwBytes : 16];
@@ -103,7 +103,7 @@ __global__ void __launch_bounds__(kDqThreads) dequant_kernel(const void* __restr
         v[u].z = __fadd_rn(v[u].z, v2.z);
         v[u].w = __fadd_rn(v[u].w, v2.w);
       }
-      s[u] = h < H ? __ldg(scale + j / gpr) : 0.0f;  // G < 2^32: a 32-bit division
+      s[u] = h < H ? __ldg(scale + fast_div(j, gpr)) : 0.0f;  // row of group j (G < 2^32)
     }
 #pragma unroll
     for (int u = 0; u < kDqUnroll; ++u) {
@@ -138,7 +138,7 @@ cudaError_t launch_t(const pvt_layer& L, uint64_t G, void* W_hat, uint32_t* stat
   const uint64_t want = (PARTS * G + per_block - 1) / per_block;
   const uint64_t cap = (uint64_t)sm_count * (uint64_t)per_sm;
   const unsigned blocks = (unsigned)(want < cap ? want : cap);
-  const uint32_t gpr = (uint32_t)(L.cols / (4 * PARTS));
+  const FastDiv gpr = make_fast_div((uint32_t)(L.cols / (4 * PARTS)));  // groups per row
   const uint32_t K = (uint32_t)L.codebook_size;
   if (smem_book)
     dequant_kernel<M, CB_F16, CODE_U16, OUT_F16, true, PARTS>

@@ -152,6 +152,29 @@ cudaError_t launch_trust_after_search(const pvt_layer& L, uint64_t G, uint64_t k
 cudaError_t launch_refine(const pvt_layer& L, uint64_t G, const uint32_t* idx, uint64_t k, int max_moves,
                           float* err_out, uint32_t* moves_out, uint32_t* status, cudaStream_t stream);
 
+// ---- division by an invariant 32-bit divisor ---------------------------------------------------------------
+// n / d for every 32-bit n as one multiply-high, a subtraction, an addition and two shifts (Granlund and
+// Montgomery, "Division by invariant integers using multiplication", 1994, unsigned case): with l = ceil(log2 d),
+// mul = floor(2^32 (2^l - d) / d) + 1, t = mulhi(mul, n):  n / d = (t + ((n - t) >> min(l, 1))) >> max(l - 1, 0).
+struct FastDiv {
+  uint32_t mul, s1, s2;
+};
+inline FastDiv make_fast_div(uint32_t d) {
+  uint32_t l = 0;
+  while (l < 32 && ((uint64_t)1 << l) < d) ++l;
+  FastDiv f;
+  f.mul = (uint32_t)((((uint64_t)1 << 32) * (((uint64_t)1 << l) - d)) / d + 1);
+  f.s1 = l < 1 ? l : 1;
+  f.s2 = l > 1 ? l - 1 : 0;
+  return f;
+}
+#ifdef __CUDACC__
+__device__ __forceinline__ uint32_t fast_div(uint32_t n, const FastDiv& f) {
+  const uint32_t t = __umulhi(f.mul, n);
+  return (t + ((n - t) >> f.s1)) >> f.s2;
+}
+#endif
+
 // ---- programmatic dependent launch --------------------------------------------------------------------
 // Consecutive kernels of a call depend on one another, so between two of them the GPU would idle for a launch
 // latency.  A kernel launched with launch_dependent() may be scheduled while the kernel before it on the stream
