@@ -95,6 +95,9 @@ def check_encode(L, idx_np, beam=None):
     (1, 65536, True, 512, 1024),
     (2, 256, True, 96, 136),       # ragged
     (2, 64, False, 33, 72),
+    (1, 16, True, 300, 8),         # one group per row
+    (1, 64, True, 70, 24),         # three groups per row
+    (2, 16, True, 9, 8248),        # 1031 groups per row (a prime)
 ])
 @pytest.mark.parametrize("out_f16", [False, True])
 def test_dequant_bit_exact(M, K, f16, rows, cols, out_f16):
