@@ -15,7 +15,8 @@
 // kept residuals are the rows of a 16 x 16 fp16 tile [ -hi(2^e r) | -lo(2^e r) ], the codewords the columns
 // [ c | c ], the accumulator starts at 2^e ||c||^2 / 2 (mma.sync m16n8k16, fp32 accumulation); with fewer than
 // eight kept residuals the rows repeat them and the copies share the codebook between them.  For binary32
-// codebooks the estimate is sum_i (fl32(r_i) - c_i)^2 on the FP32 pipe.
+// codebooks, and for a stage with one or two kept residuals (the first), the estimate is
+// sum_i (fl32(r_i) - c_i)^2 on the FP32 pipe.
 #include <cuda_fp16.h>
 
 #include "pvt_internal.h"
@@ -254,7 +255,7 @@ __global__ void __launch_bounds__(kMxThreads, M == 3 ? 4 : 3) encode_mx_kernel(c
       }
       return theta_bits;
     };
-    if (CB_F16) {
+    if (CB_F16 && n_kept >= 3) {  // with one or two kept residuals (the first stage) the FP32 pipe is cheaper
       // Estimates from the tensor pipe.  Row rho of the A tile (rho = lane / 4) holds kept residual b = rho mod
       // n_kept; the copies of a residual take the n-tiles of the codebook in turn.  A thread sees, per n-tile of
       // eight codewords, the estimates of its row against codewords 8 nt + 2 (lane % 4) and the next one:
