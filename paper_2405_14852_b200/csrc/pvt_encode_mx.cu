@@ -11,12 +11,11 @@
 // over fast estimates of all extensions: the first finds a threshold (the keep-th smallest of the lanes' minima),
 // the second gives every extension within the estimates' error bound of it its binary64 score and keeps the
 // lane's `beam` smallest in registers (sorted by insertion); the warp then extracts the overall `beam` smallest by
-// repeated warp minimum over the lanes' heads.  For fp16 codebooks the estimates come from the tensor pipe: the
-// kept residuals are the rows of a 16 x 16 fp16 tile [ -hi(2^e r) | -lo(2^e r) ], the codewords the columns
-// [ c | c ], the accumulator starts at 2^e ||c||^2 / 2 (mma.sync m16n8k16, fp32 accumulation); with fewer than
-// eight kept residuals the rows repeat them and the copies share the codebook between them.  For binary32
-// codebooks, and for a stage with one or two kept residuals (the first), the estimate is
-// sum_i (fl32(r_i) - c_i)^2 on the FP32 pipe.
+// repeated warp minimum over the lanes' heads.  For fp16 codebooks the estimates come from the tensor pipe: 16
+// codewords are the rows [ c | c ] of an fp16 tile, the kept residuals its columns [ -hi(2^e r) | -lo(2^e r) ],
+// the accumulator starts at 2^e ||c||^2 / 2 (mma.sync m16n8k16, fp32 accumulation): 16 instructions per pass over
+// 256 codewords.  For binary32 codebooks, and for a stage with one or two kept residuals (the first), the estimate
+// is sum_i (fl32(r_i) - c_i)^2 on the FP32 pipe.
 #include <cuda_fp16.h>
 
 #include "pvt_internal.h"
@@ -54,15 +53,15 @@ constexpr int kMxCand = 256;              // capacity of a warp's candidate list
 constexpr int kMxPadK = 256;              // codewords per codebook in the tensor-pipe image (padded)
 constexpr float kMxPadHalfNorm = 3.0e38f;  // half norm of a padding codeword: never within any bound
 
-// D = A (16 x 16, rows = residuals) x B (16 x 8, columns = codewords) + C, fp16 operands, fp32 accumulation;
-// rows 8..15 of A are zero
-__device__ __forceinline__ void mma_rows8(float& d0, float& d1, uint32_t a_hi, uint32_t a_lo, uint32_t b, float c0,
-                                          float c1) {
-  float d2 __attribute__((unused)), d3 __attribute__((unused));  // rows 8..15: nothing
-  asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %5}, {%7, %7}, "
-      "{%8, %9, %8, %9};"
-      : "=f"(d0), "=f"(d1), "=f"(d2), "=f"(d3)
-      : "r"(a_hi), "r"(0u), "r"(a_lo), "r"(b), "f"(c0), "f"(c1));
+// D = A (16 x 16, rows = codewords, each [ c | c ]) x B (16 x 8, columns = residuals, each [ -hi | -lo ]) + C,
+// fp16 operands, fp32 accumulation.  A thread passes the words of rows lane/4 and lane/4 + 8 (the same word serves
+// both halves of the depth) and the half norms of those two codewords as the start of the accumulator.
+__device__ __forceinline__ void mma_cw16(float (&d)[4], uint32_t a_row, uint32_t a_row8, uint32_t b_hi, uint32_t b_lo,
+                                         float c_row, float c_row8) {
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %4, %5}, {%6, %7}, "
+      "{%8, %8, %9, %9};"
+      : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+      : "r"(a_row), "r"(a_row8), "r"(b_hi), "r"(b_lo), "f"(c_row), "f"(c_row8));
 }
 
 // bytes of the tensor-pipe image of the codebooks: B fragments, half norms, largest norm per codebook
@@ -76,7 +75,8 @@ __global__ void __launch_bounds__(kMxThreads, M == 3 ? 4 : 3) encode_mx_kernel(c
   float* book = reinterpret_cast<float*>(smem_raw);                               // [M][K][8]
   double* resid = reinterpret_cast<double*>(smem_raw + (size_t)M * p.K * 32);     // [warps][beam][8]
   float* resid_f = reinterpret_cast<float*>(resid + kMxWarps * kMxBeam * 8);      // the same, rounded to binary32
-  // fp16 codebooks only: word [m][n-tile][lane] = halves (c[8 nt + lane/4][2 (lane%4)], [.. + 1]); ||c||^2/2; max ||c||^2
+  // fp16 codebooks only: A fragments, words [m][tile][lane][2] = halves (c[16 tile + lane/4 (+ 8)][2 (lane%4)], [.. + 1]);
+  // ||c||^2/2 as [m][tile][lane/4][2]; max ||c||^2
   // per warp: the extensions that pass the filter of a stage, (kept tuple << 8 | code), and their count
   uint16_t* cand = reinterpret_cast<uint16_t*>(resid_f + kMxWarps * kMxBeam * 8);
   uint32_t* cand_n = reinterpret_cast<uint32_t*>(cand + kMxWarps * kMxCand);
@@ -119,12 +119,14 @@ __global__ void __launch_bounds__(kMxThreads, M == 3 ? 4 : 3) encode_mx_kernel(c
       float n2 = 0.0f;
 #pragma unroll
       for (int i = 0; i < 8; ++i) n2 = fmaf(c[i], c[i], n2);
-      hnorm[m * kMxPadK + kap] = 0.5f * n2;
+      // 16 codewords per tile: codeword 16 mt + r sits in row r; a thread of the warp reads rows g and g + 8
+      const uint32_t mt = kap >> 4, g = kap & 7u, upper = (kap >> 3) & 1u;
+      hnorm[((m * (kMxPadK / 16) + mt) * 8 + g) * 2 + upper] = 0.5f * n2;
       atomicMax(&n2max_bits[m], __float_as_uint(n2));  // non-negative: bits order like values
 #pragma unroll
       for (int qq = 0; qq < 4; ++qq) {
         const __half2 v = __floats2half2_rn(c[2 * qq], c[2 * qq + 1]);  // exact: the codebook is fp16
-        bfrag[(m * (kMxPadK / 8) + (kap >> 3)) * 32 + 4 * (kap & 7u) + qq] = *reinterpret_cast<const uint32_t*>(&v);
+        bfrag[((m * (kMxPadK / 16) + mt) * 32 + 4 * g + qq) * 2 + upper] = *reinterpret_cast<const uint32_t*>(&v);
       }
     }
   }
@@ -256,9 +258,9 @@ __global__ void __launch_bounds__(kMxThreads, M == 3 ? 4 : 3) encode_mx_kernel(c
       return theta_bits;
     };
     if (CB_F16 && n_kept >= 3) {  // with one or two kept residuals (the first stage) the FP32 pipe is cheaper
-      // Estimates from the tensor pipe.  Row rho of the A tile (rho = lane / 4) holds kept residual b = rho mod
-      // n_kept; the copies of a residual take the n-tiles of the codebook in turn.  A thread sees, per n-tile of
-      // eight codewords, the estimates of its row against codewords 8 nt + 2 (lane % 4) and the next one:
+      // Estimates from the tensor pipe.  The kept residuals are the columns of B (column n = residual n, as
+      // [ -hi(2^e r) | -lo(2^e r) ]), 16 codewords the rows of A.  A thread sees, per tile of 16 codewords, the
+      // estimates of residuals 2 (lane % 4) and the next one against codewords 16 mt + lane / 4 and that + 8:
       //   est = ||r_f||^2 + 2 * 2^-e * D,   D = 2^e (||c||^2/2 - <r_f, c>)  up to rounding.
       // Error against the binary64 score d (R = largest residual norm, C = largest codeword norm, S = (R + C)^2):
       // rounding r to binary32 2^-23 sqrt(d) R; the halves 2^-21 R C, or 2^-24 2^-e sqrt(8) C where the low half is
@@ -266,59 +268,58 @@ __global__ void __launch_bounds__(kMxThreads, M == 3 ? 4 : 3) encode_mx_kernel(c
       // below 2^-17 S + 2^-22 2^-e C in all.
       const uint32_t g8 = (uint32_t)lane >> 2, qd = (uint32_t)lane & 3u;
       const uint32_t nk = (uint32_t)n_kept;
-      uint32_t b = g8, rep = 0u, nrep = 1u;  // copies of residual b among the 8 rows (nk = 8: one each)
-      if (nk == 1u) {
-        b = 0u, rep = g8, nrep = 8u;
-      } else if (nk != 8u) {
-        b = g8 % nk, rep = g8 / nk, nrep = (7u - b) / nk + 1u;
-      }
-      const float2 rv = *reinterpret_cast<const float2*>(&my_resid_f[b * 8 + 2 * qd]);
-      float rr = 0.0f;
-      {
+      // the column this thread contributes to B: residual g8, elements 2 qd and 2 qd + 1
+      float2 rv = make_float2(0.0f, 0.0f);
+      if (g8 < nk) rv = *reinterpret_cast<const float2*>(&my_resid_f[g8 * 8 + 2 * qd]);
+      // the two residuals whose estimates this thread receives, and their squared norms
+      const uint32_t b0 = 2u * qd, b1 = 2u * qd + 1u;
+      const bool valid0 = b0 < nk, valid1 = b1 < nk;
+      auto sq_norm = [&](uint32_t b) {
         const float4 ra = *reinterpret_cast<const float4*>(&my_resid_f[b * 8]);
         const float4 rb = *reinterpret_cast<const float4*>(&my_resid_f[b * 8 + 4]);
-        rr = ra.x * ra.x;
+        float rr = ra.x * ra.x;
         rr = fmaf(ra.y, ra.y, rr); rr = fmaf(ra.z, ra.z, rr); rr = fmaf(ra.w, ra.w, rr);
         rr = fmaf(rb.x, rb.x, rr); rr = fmaf(rb.y, rb.y, rr); rr = fmaf(rb.z, rb.z, rr); rr = fmaf(rb.w, rb.w, rr);
-      }
+        return rr;
+      };
+      const float inf_f = __uint_as_float(0x7f800000u);
+      const float rr0 = valid0 ? sq_norm(b0) : inf_f, rr1 = valid1 ? sq_norm(b1) : inf_f;  // inf: never within a bound
       const float rmax = fmaxf(fabsf(rv.x), fabsf(rv.y));
       const uint32_t rbits = __reduce_max_sync(0xffffffffu, __float_as_uint(rmax));
-      const float r2max = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(rr)));
+      const float r2max = __uint_as_float(
+          __reduce_max_sync(0xffffffffu, __float_as_uint(fmaxf(valid0 ? rr0 : 0.0f, valid1 ? rr1 : 0.0f))));
       int e = 126 - (int)((rbits >> 23) & 0xffu);
       e = e > 15 ? 15 : (e < -100 ? -100 : e);
       const float sc = __uint_as_float((uint32_t)(e + 127) << 23), inv = __uint_as_float((uint32_t)(127 - e) << 23);
-      uint32_t a_hi, a_lo;
+      uint32_t b_hi, b_lo;
       {
         const float x = -rv.x * sc, y = -rv.y * sc;  // exact
         const __half2 hi = __floats2half2_rn(x, y);
         const float2 back = __half22float2(hi);
         const __half2 lo = __floats2half2_rn(x - back.x, y - back.y);
-        a_hi = *reinterpret_cast<const uint32_t*>(&hi);
-        a_lo = *reinterpret_cast<const uint32_t*>(&lo);
+        b_hi = *reinterpret_cast<const uint32_t*>(&hi);
+        b_lo = *reinterpret_cast<const uint32_t*>(&lo);
       }
-      const uint32_t* bf = bfrag + (size_t)m * (kMxPadK / 8) * 32 + lane;
-      const float* hn = hnorm + (size_t)m * kMxPadK + 2 * qd;
+      const uint2* af = reinterpret_cast<const uint2*>(bfrag) + (size_t)m * (kMxPadK / 16) * 32 + lane;
+      const float2* hn = reinterpret_cast<const float2*>(hnorm) + (size_t)m * (kMxPadK / 16) * 8 + g8;
       const float two_inv = 2.0f * inv;
-      const uint32_t n_tiles = (K + 7u) >> 3;
-      // pass 1: this lane's two smallest estimates (all of a lane's extensions belong to one residual, so the
-      // best residual's lanes must be able to offer more than one each)
-      float m0 = __uint_as_float(0x7f800000u), m1 = m0;
-      {
-        uint32_t next = rep;
+      const uint32_t n_tiles = (K + 15u) >> 4;
+      // pass 1: this lane's two smallest estimates
+      float m0 = inf_f, m1 = inf_f;
 #pragma unroll 4
-        for (uint32_t nt = 0; nt < n_tiles; ++nt) {
-          const float2 hh = *reinterpret_cast<const float2*>(hn + 8 * nt);
-          float d0, d1;
-          mma_rows8(d0, d1, a_hi, a_lo, bf[32 * nt], hh.x * sc, hh.y * sc);
-          if (nt == next) {
-            next += nrep;
-            const float e0 = fmaf(d0, two_inv, rr), e1 = fmaf(d1, two_inv, rr);
-            const float lo = fminf(e0, e1), hi = fmaxf(e0, e1);
-            const float t0 = fmaxf(m0, lo);
-            m0 = fminf(m0, lo);
-            m1 = fminf(fminf(m1, hi), t0);
-          }
-        }
+      for (uint32_t mt = 0; mt < n_tiles; ++mt) {
+        const uint2 a = af[32 * mt];
+        const float2 hh = hn[8 * mt];
+        float d[4];
+        mma_cw16(d, a.x, a.y, b_hi, b_lo, hh.x * sc, hh.y * sc);
+        const float e00 = fmaf(d[0], two_inv, rr0), e01 = fmaf(d[1], two_inv, rr1);
+        const float e10 = fmaf(d[2], two_inv, rr0), e11 = fmaf(d[3], two_inv, rr1);
+        // the two smallest of the four, then of those and (m0, m1)
+        const float lo_a = fminf(e00, e01), hi_a = fmaxf(e00, e01), lo_b = fminf(e10, e11), hi_b = fmaxf(e10, e11);
+        const float t0 = fminf(lo_a, lo_b), t1 = fminf(fmaxf(lo_a, lo_b), fminf(hi_a, hi_b));
+        const float n0 = fminf(m0, t0);
+        m1 = fminf(fmaxf(m0, t0), fminf(m1, t1));
+        m0 = n0;
       }
       // an estimate can come out slightly negative; the order of the bit patterns needs non-negative values
       const uint32_t theta_bits =
@@ -331,18 +332,21 @@ __global__ void __launch_bounds__(kMxThreads, M == 3 ? 4 : 3) encode_mx_kernel(c
                               ? theta
                               : theta + 3.0517578e-5f /* 2^-15 */ * reach * reach + 9.5367432e-7f /* 2^-20 */ * inv * cmax + 1e-37f;
       // pass 2: the same estimates again (bit for bit); the few extensions within the bound go on the list
-      uint32_t next = rep;
 #pragma unroll 4
-      for (uint32_t nt = 0; nt < n_tiles; ++nt) {
-        const float2 hh = *reinterpret_cast<const float2*>(hn + 8 * nt);
-        float d0, d1;
-        mma_rows8(d0, d1, a_hi, a_lo, bf[32 * nt], hh.x * sc, hh.y * sc);
-        if (nt != next) continue;
-        next += nrep;
-        const float e0 = fmaf(d0, two_inv, rr), e1 = fmaf(d1, two_inv, rr);
-        const uint32_t q = 8 * nt + 2 * qd;
-        if (e0 <= bound && q < K) collect(b, q);
-        if (e1 <= bound && q + 1 < K) collect(b, q + 1);
+      for (uint32_t mt = 0; mt < n_tiles; ++mt) {
+        const uint2 a = af[32 * mt];
+        const float2 hh = hn[8 * mt];
+        float d[4];
+        mma_cw16(d, a.x, a.y, b_hi, b_lo, hh.x * sc, hh.y * sc);
+        const float e00 = fmaf(d[0], two_inv, rr0), e01 = fmaf(d[1], two_inv, rr1);
+        const float e10 = fmaf(d[2], two_inv, rr0), e11 = fmaf(d[3], two_inv, rr1);
+        const uint32_t q = 16u * mt + g8;
+        if (fminf(fminf(e00, e01), fminf(e10, e11)) <= bound) {
+          if (valid0 && e00 <= bound && q < K) collect(b0, q);
+          if (valid1 && e01 <= bound && q < K) collect(b1, q);
+          if (valid0 && e10 <= bound && q + 8u < K) collect(b0, q + 8u);
+          if (valid1 && e11 <= bound && q + 8u < K) collect(b1, q + 8u);
+        }
       }
     } else {
       // Pass 1, binary32 and branch-free: the estimate d_fl = sum_i (fl32(r_i) - c_i)^2 of every extension.  With
