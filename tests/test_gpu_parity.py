@@ -400,6 +400,9 @@ def test_two_codebook_ragged_target_counts(k):
     (4, 32, False, 33, 72, 297, 8),     # every group, ragged sizes
     (4, 256, True, 32, 512, 300, 4),
     (3, 16, True, 32, 128, 512, 1),     # greedy
+    (3, 100, True, 64, 256, 900, 8),    # codebook sizes that leave the last tile of 16 codewords ragged
+    (4, 23, True, 48, 128, 500, 8),
+    (3, 5, True, 32, 128, 300, 8),      # fewer codewords than the beam: three to eight kept tuples per stage
 ])
 def test_three_and_four_codebooks_match_checker(M, K, f16, rows, cols, k, beam):
     L = synth.make_layer(rows, cols, cfg=210 + M, num_codebooks=M, codebook_size=K, codebook_fp16=f16,
