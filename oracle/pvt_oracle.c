@@ -29,7 +29,10 @@
  * nearest-centroid routine (the V step with phi = ||x - z||^2 is the K-means
  * assignment step, Section 3.1), the expansion ||x-B||^2 = ||x||^2 - 2<x,B> +
  * ||B||^2 (Appendix D), beam >= K equals exhaustive search, beam = 1 equals
- * greedy residual quantisation, zero second codebook reduces to M = 1,
+ * greedy residual quantisation (two, three and four codebooks), narrow beams
+ * over three and four codebooks against an independent stage-by-stage search
+ * (tuples and distances equal, exact ties among partial tuples included), zero
+ * second codebook reduces to M = 1,
  * monotonicity (Lemma 3.3), locality, fixed point, full-sort selection with
  * crafted ties, closed-form dequantisation.  No end-to-end V-step result on a
  * real layer is printed in the paper, so beyond these pins parity is unpinned.

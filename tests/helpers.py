@@ -118,3 +118,54 @@ def check_codes_against_oracle(t, codebooks, got_codes, enc, rel=1e-6):
         ok = np.abs(d_got - d_ref) <= rel * np.maximum(d_got, d_ref)
         assert ok.all(), "reconstruction error differs by more than the relative tolerance inside the gap band"
     return int(same.sum()), int(band.sum())
+
+
+def stagewise_beam(t, codebooks, beam, prev=None):
+    """Greedy residual beam search written stage by stage on whole arrays (numpy, fp64), with no call
+    into the CPU checker: after stage m the `beam` partial tuples with the smallest
+    ||t - c^1 - ... - c^m||^2 are kept, ties resolved towards the lexicographically smaller tuple; the
+    last stage's extensions (plus `prev`, if given) form the pool, whose smallest member under
+    (distance, tuple) is returned.  The residual is carried codebook by codebook and the squared
+    distance summed element by element, so that equal operands give the checker's binary64 values.
+    Returns (tuples int64 [k, M], distances float64 [k])."""
+    t = np.asarray(t, dtype=np.float32).astype(np.float64)
+    books = np.asarray(codebooks).astype(np.float32).astype(np.float64)
+    M, K, dg = books.shape
+    out_codes = np.zeros((t.shape[0], M), dtype=np.int64)
+    out_dist = np.zeros(t.shape[0])
+    for n in range(t.shape[0]):
+        partial = [((), t[n].copy())]  # (tuple so far, residual)
+        scored = []
+        for m in range(M):
+            scored = []
+            for tup, res in partial:
+                diff = res[None, :] - books[m]
+                d = np.zeros(K)
+                for i in range(dg):  # element order, one rounding per addition
+                    d = d + diff[:, i] * diff[:, i]
+                for q in range(K):
+                    scored.append((float(d[q]), tup + (q,)))
+            if m == M - 1:
+                break
+            scored.sort()  # python tuples compare as (distance, then code tuple) -- the stated order
+            partial = []
+            for d_, tup in scored[:beam]:
+                res = t[n].copy()
+                for mm, q in enumerate(tup):
+                    res = res - books[mm, q]
+                partial.append((tup, res))
+        if prev is not None:
+            p = tuple(int(x) for x in np.asarray(prev)[n])
+            if p not in {tup for _, tup in scored}:
+                res = t[n].copy()
+                for mm in range(M - 1):
+                    res = res - books[mm, p[mm]]
+                diff = res - books[M - 1, p[M - 1]]
+                d = 0.0
+                for i in range(dg):
+                    d = d + diff[i] * diff[i]
+                scored.append((float(d), p))
+        best = min(scored)
+        out_codes[n] = best[1]
+        out_dist[n] = best[0]
+    return out_codes, out_dist

@@ -294,6 +294,81 @@ def test_three_codebooks_with_wide_beam_equal_enumeration():
     assert np.array_equal(enc.codes, best)
 
 
+def _residual_books(seed, M, K, dg=8, decay=0.5):
+    r = _rng(seed)
+    return np.stack([(decay ** m) * r.normal(size=(K, dg)) for m in range(M)]).astype(np.float32)
+
+
+@pytest.mark.parametrize("M", [3, 4])
+@pytest.mark.parametrize("K", [4, 7, 12])
+@pytest.mark.parametrize("beam", [1, 2, 3, 5])
+def test_narrow_beam_over_three_and_four_codebooks_against_a_stagewise_search(M, K, beam):
+    """Beams that really drop partial tuples at the second and third stage (beam < kept x K): every tuple
+    and distance against an independent stage-by-stage search that shares nothing with the checker."""
+    books = _residual_books(100 + 10 * M + K, M, K)
+    r = _rng(200 + beam)
+    t = r.normal(size=(25, 8)).astype(np.float32)
+    prev = r.integers(0, K, size=(25, M))
+    enc = oracle.encode(t, books, prev, beam=beam)
+    want_codes, want_d = helpers.stagewise_beam(t, books, beam, prev)
+    assert np.array_equal(enc.codes, want_codes)
+    assert np.array_equal(enc.d_best, want_d)
+    # without the previous tuple in the pool (previous tuple := the result, which adds nothing)
+    free_codes, free_d = helpers.stagewise_beam(t, books, beam)
+    enc_free = oracle.encode(t, books, free_codes, beam=beam)
+    assert np.array_equal(enc_free.codes, free_codes)
+    assert np.array_equal(enc_free.d_best, free_d)
+
+
+def test_narrow_beam_really_truncates_and_is_a_heuristic():
+    """The cases above are not secretly exhaustive: with three codebooks of 7 and beam 2 some targets end
+    above the enumerated optimum, and widening the beam to all tuples reaches it."""
+    books = _residual_books(131, 3, 7, decay=0.9)
+    t = _rng(132).normal(size=(60, 8)).astype(np.float32)
+    narrow, d_narrow = helpers.stagewise_beam(t, books, 2)
+    best, d_best = helpers.brute_force_tuples(t, books)
+    assert (d_narrow > d_best * (1 + 1e-9)).any()
+    enc = oracle.encode(t, books, narrow, beam=2)
+    assert np.array_equal(enc.codes, narrow)
+    wide = oracle.encode(t, books, narrow, beam=49)
+    assert np.array_equal(wide.codes, best)
+
+
+@pytest.mark.parametrize("M", [3, 4])
+def test_beam_one_over_more_codebooks_equals_greedy_residual_quantisation(M):
+    K = 9
+    books = _residual_books(140 + M, M, K)
+    t = _rng(150 + M).normal(size=(120, 8)).astype(np.float32)
+    res = t.astype(np.float64)
+    greedy = []
+    for m in range(M):
+        km = ((res[:, None] - books[m].astype(np.float64)[None]) ** 2).sum(-1).argmin(1)
+        res = res - books[m].astype(np.float64)[km]
+        greedy.append(km)
+    greedy = np.stack(greedy, 1)
+    enc = oracle.encode(t, books, greedy, beam=1)
+    assert np.array_equal(enc.codes, greedy)
+    assert np.allclose(enc.d_best, (res ** 2).sum(1), rtol=1e-13, atol=0)
+
+
+def test_equal_partial_distances_keep_the_smaller_tuple_at_a_truncating_stage():
+    """Duplicate codewords make exact ties among partial tuples; the kept ones must be the
+    lexicographically smaller tuples, which decides the final code when the beam is narrow."""
+    r = _rng(160)
+    b1 = r.normal(size=(6, 8)).astype(np.float32)
+    b1[4] = b1[1]  # codes 1 and 4 of the first codebook are the same vector
+    b2 = (0.5 * r.normal(size=(6, 8))).astype(np.float32)
+    b2[5] = b2[2]
+    b3 = (0.25 * r.normal(size=(6, 8))).astype(np.float32)
+    books = np.stack([b1, b2, b3])
+    t = (b1[1] + b2[2] + 0.01 * r.normal(size=(30, 8))).astype(np.float32)
+    for beam in (1, 2, 3):
+        want_codes, want_d = helpers.stagewise_beam(t, books, beam)
+        enc = oracle.encode(t, books, want_codes, beam=beam)
+        assert np.array_equal(enc.codes, want_codes)
+        assert np.all(enc.codes[:, 0] != 4)  # the duplicate with the larger code never wins
+
+
 def test_tuple_error_matches_independent_formula():
     books = _two_books(21, 16)
     t = _rng(22).normal(size=(30, 8)).astype(np.float32)
