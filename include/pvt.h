@@ -8,12 +8,12 @@
  * discrete codes (V step):
  *
  *     update = W - eta * g                  (Eq. 8: y - (1/L_S) Z(grad phi(y)))
- *     S      = choose_subspace(update, tau) (Algorithm 2: arg top-tau; Section
- *                                            3.4: largest update norm per matrix)
- *     codes[S] = find_nearest(update[S])    (Appendix C / Appendix J: try every
- *                                            code, or beam search for additive
- *                                            codebooks; codes outside S stay,
- *                                            Section 3.3)
+ *     S      = choose_subspace(update, tau) (Algorithm 2: top-tau selection; Section
+ *                                            3.4: by update size, per matrix)
+ *     codes[S] = find_nearest(update[S])    (Appendix C / Appendix J: exhaustive
+ *                                            search of one codebook, beam search
+ *                                            for additive codebooks; codes
+ *                                            outside S stay, Section 3.3)
  *
  * and the next step starts with dequantize_weights (Algorithm 3, first line).
  * This library is those three calls.
@@ -25,7 +25,10 @@
  *   - Every pointer is DEVICE memory owned by the caller (16-byte aligned where
  *     stated; index, error, move-count and status arrays 4-byte aligned; codes
  *     2-byte aligned when they are two-byte codes or pairs of one-byte codes).
- *     The library allocates nothing and keeps no state between calls.
+ *     The library allocates nothing.  It keeps no per-layer state between calls; the
+ *     only process-wide settings are the ones made through pvt_set_m1_search,
+ *     pvt_timing_enable and pvt_test_wait_limit (all off / automatic by default),
+ *     and pvt_vstep_select_noalloc remembers the address of its built-in scratch.
  *   - Every call only enqueues work on `cuda_stream` (a cudaStream_t passed as
  *     void*; NULL = the legacy default stream) and returns without synchronising,
  *     except pvt_status.  Calls on one stream execute in order.
@@ -105,8 +108,8 @@ size_t pvt_workspace_bytes(const pvt_layer* layer, uint64_t k);
 int pvt_workspace_init(void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
- * Subspace choice (Algorithm 2, "arg top tau"; Section 3.4, "largest update norm
- * within each weight matrix"; Algorithm 3, choose_subspace).
+ * Subspace choice (the top-tau selection of Algorithm 2; Section 3.4 ranks by the size
+ * of the update, separately for every weight matrix; choose_subspace of Algorithm 3).
  *   n_j = ||eta * g_j||^2 per group, in binary32: u_i = eta*g_i rounded once,
  *   acc = fma(u_i, u_i, acc) for i = 0..7 from acc = 0.
  *   idx_out[0..k) = the k groups with the largest n_j, ties at the threshold
@@ -134,11 +137,16 @@ int pvt_vstep_select(const pvt_layer* layer, uint64_t k, uint32_t* idx_out, void
  * Limits and rules
  *   - At most PVT_NOALLOC_MAX_GROUPS groups (2^21, e.g. one 4096 x 4096 layer);
  *     a larger layer is rejected with PVT_ETOOLARGE before anything is enqueued.
- *   - The array (about 10.03 MiB) is resident on every GPU that loads the library,
- *     from load until the process exits, whether or not this call is ever used.
- *   - The first call on each device looks up the array's device address (a
+ *   - The array (about 10.03 MiB) is held on every GPU on which the library's
+ *     device code has been loaded, until the process exits.  The CUDA runtime may
+ *     load that code lazily: then it is the first call of this function on a
+ *     device that makes the array resident (and that load may synchronise the
+ *     device and needs those 10 MiB to be free).
+ *   - The first call on each device also looks up the array's device address (a
  *     host-side runtime query; the device must be current).  Make that first
- *     call outside any stream capture.  The address is kept for the life of
+ *     call at start-up -- before the memory is handed out completely and outside
+ *     any stream capture; a call on a tiny layer will do.  From the second call
+ *     on nothing is loaded or looked up.  The address is kept for the life of
  *     the process: a cudaDeviceReset unloads the array and leaves that address
  *     dangling, so a process that resets a device must not call this
  *     afterwards on that device.
@@ -147,8 +155,9 @@ int pvt_vstep_select(const pvt_layer* layer, uint64_t k, uint32_t* idx_out, void
  *     and give wrong results: issue them on one stream, or order them yourself.
  *     What must start at zero is cleared at the start of every call; nothing
  *     else of a previous call is relied upon.
- *   - The call itself performs no allocation of any kind (no cudaMalloc /
- *     cudaFree, no allocating library routine) and does not synchronise.
+ *   - The call issues no cudaMalloc / cudaFree and no allocating library routine,
+ *     and apart from what the first call on a device may trigger (above) it does
+ *     not synchronise.
  * status_out: NULL, or a device uint32 that receives the PVT_DEV_* bits of this
  * call (written by a copy enqueued after the kernels).
  * Other arguments and return codes as pvt_vstep_select.
@@ -182,12 +191,12 @@ int pvt_vstep_encode(const pvt_layer* layer, const uint32_t* idx, uint64_t k, fl
                      size_t ws_bytes, void* cuda_stream);
 
 /*
- * V step whose subspace size comes from a trust ratio (Section 4.3: tau = "the
- * number of weights such that the update satisfies ||x_new - x_old|| / ||x_old||
- * <= 0.01"; Appendix J, "Hyperparameter tuning": the largest such number, found
- * by re-encoding a hundredth of the weights at a time in the order of decreasing
- * update norm and undoing codes from the end of the last portion; one weight is
- * always allowed to change).  x is the dequantised matrix W_hat of this layer.
+ * V step whose subspace size comes from a trust ratio (Section 4.3 sets tau so that the
+ * relative change ||x_new - x_old|| / ||x_old|| of a step stays at one per cent; the
+ * hyper-parameter paragraph of Appendix J takes the largest such count, found by
+ * re-encoding a hundredth of the weights at a time in the order of decreasing update
+ * norm and undoing codes from the end of the last portion, and always lets one weight
+ * change).  x is the dequantised matrix W_hat of this layer.
  *
  * What is computed: the k_max groups of largest ||eta*g_j||^2 are ranked by
  * (norm descending, index ascending) and all re-encoded as by pvt_vstep_encode.
@@ -279,7 +288,7 @@ int pvt_adam_update(float* param, void* param_f16, const double* grad, float* ex
 /*
  * Update direction of the V step as the paper runs it (Section 3.4: grad phi(y) of Eq. 8 is
  * replaced by a single Adam update, and the subspace is chosen by the magnitude of that
- * update; Algorithm 3, V-step line "update = adam(grad_phi) ...").  Per weight, binary32,
+ * update; the update line of Algorithm 3's V step).  Per weight, binary32,
  * every operation rounded once:
  *   m = fma(beta1, m, (1 - beta1) * g)        v = fma(beta2, v, ((1 - beta2) * g) * g)
  *   dir = (m / bias1) / (sqrt(v / bias2) + eps)
@@ -290,6 +299,14 @@ int pvt_adam_update(float* param, void* param_f16, const double* grad, float* ex
  */
 int pvt_adam_direction(const float* grad, float* exp_avg, float* exp_avg_sq, float* dir, uint64_t n, float beta1,
                        float beta2, float eps, float bias1, float bias2, void* cuda_stream);
+
+/*
+ * Bias corrections of Adam's step t >= 1 as the two calls above take them (Section 3.4; Appendix J
+ * betas): bias = 1 - beta^t, the power taken in binary64 from the binary32 beta, the difference
+ * rounded once to binary32.  Host arithmetic only; bias1_out, bias2_out: host.  PVT_EINVAL for
+ * step = 0, a beta outside [0, 1) or a null pointer.
+ */
+int pvt_adam_bias(uint64_t step, float beta1, float beta2, float* bias1_out, float* bias2_out);
 
 /*
  * Synchronises the stream, returns the PVT_DEV_* bits accumulated in the
@@ -342,6 +359,19 @@ int pvt_probe_fp32_tflops(float* scratch, size_t scratch_floats, float* tflops_o
 /* Kernels this process has launched through the library so far (memsets not counted). */
 unsigned long long pvt_launch_count(void);
 int pvt_timing_read(int kernel_id, float* total_ms, int* launches);
+
+/*
+ * Test hook for the give-up path of the on-chip waits (no counterpart in the paper).  Every wait of
+ * the single-codebook search kernels on an on-chip barrier polls a bounded number of times; when
+ * the bound is reached the kernel stops, lets the copies and tensor-core work it has issued finish,
+ * frees its tensor memory and returns, and pvt_status reports PVT_DEV_WAIT_EXPIRED (the codes of
+ * that call are then not written, and PVT_DEV_INTERNAL is set as well).  In normal operation the
+ * bound (2^22 polls) is never reached.  This call lowers it to max_polls (0 restores the default)
+ * and, if withhold_copy >= 0, makes every thread block leave out the codebook copy with that
+ * sequence number, so that a wait provably runs out without anything being left in flight.
+ * Process-wide; affects calls enqueued afterwards.  Never use it outside tests.
+ */
+void pvt_test_wait_limit(uint32_t max_polls, int64_t withhold_copy);
 
 #ifdef __cplusplus
 }

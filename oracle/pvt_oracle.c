@@ -5,18 +5,18 @@
  * check and the benchmark's CPU-baseline leg may call it.
  *
  * Every function follows one passage of the paper:
- *   - group update norm and arg-top-tau choice: Algorithm 2 ("find tau
- *     largest"), Section 3.4 ("largest update norm within each weight matrix"),
- *     Algorithm 3 ("choose_subspace(update, tau)");
+ *   - group update norm and arg-top-tau choice: the selection step of
+ *     Algorithm 2, Section 3.4 (ranking by update size, matrix by matrix),
+ *     choose_subspace of Algorithm 3;
  *   - target of the search: Eq. (8), y - (1/L) Z(grad phi(y)), in the scaled
- *     space of the codebooks (Appendix J, "per-channel trainable scales");
- *   - M = 1 search: Appendix C / Appendix J ("try every code in the codebook
- *     and choose the one that minimises" the squared error);
+ *     space of the codebooks (Appendix J: one trainable scale per channel);
+ *   - M = 1 search: Appendix C / Appendix J (all codewords are tried and the
+ *     one with the smallest squared error is taken);
  *   - M >= 2 search: Appendix C / Appendix J (beam search, beam size 8, target =
  *     gradient-updated dequantised weight), greedy residual form;
  *   - untouched codes outside the subspace: Section 3.3 (x+_i = y_i for i not
  *     in S^k);
- *   - dequantisation: Algorithm 3 ("dequantize_weights").
+ *   - dequantisation: dequantize_weights of Algorithm 3.
  *
  * Arithmetic: the norm, the target and the dequantised weight are sequences of
  * single IEEE binary32 operations (stated at each function) so that a GPU can
@@ -410,7 +410,7 @@ void pvt_oracle_pstep_grad(const float* g, const float* scale, const int32_t* co
   }
 }
 
-/* One Adam update of n binary32 parameters (Kingma & Ba; Algorithm 3 "adam(grad_codebooks)").  The
+/* One Adam update of n binary32 parameters (Kingma & Ba; the codebook update of Algorithm 3's P step).  The
  * gradient arrives in binary64 and is rounded once to binary32; then, all in binary32, each operation
  * rounded once, in this order:
  *     m = fmaf(beta1, m, (1 - beta1) * gr)          v = fmaf(beta2, v, ((1 - beta2) * gr) * gr)
@@ -433,7 +433,7 @@ void pvt_oracle_adam(float* param, const double* grad, float* exp_avg, float* ex
 }
 
 /* Update direction of the V step as the paper runs it (Section 3.4: grad phi(y) in Eq. 8 is replaced by a single
- * Adam update; Algorithm 3, V-step line "update = adam(grad_phi) ..."; the subspace is then chosen by the
+ * Adam update; the update line of Algorithm 3's V step; the subspace is then chosen by the
  * magnitude of this update).  Moments as in Adam; the direction is the bias-corrected ratio, all in binary32,
  * every operation rounded once:
  *     m = fmaf(beta1, m, (1 - beta1) * g)        v = fmaf(beta2, v, ((1 - beta2) * g) * g)
@@ -454,7 +454,7 @@ void pvt_oracle_adam_direction(const float* grad, float* exp_avg, float* exp_avg
   }
 }
 
-/* ---- subspace size from a trust ratio (Section 4.3; Appendix J, "Hyperparameter tuning") --------------------
+/* ---- subspace size from a trust ratio (Section 4.3; Appendix J, hyper-parameter paragraph) --------------------
  * The experiments behind Tables 1-2 do not fix tau: they take the largest number of weights, in the order of
  * decreasing update norm, whose re-encoding keeps ||x_new - x_old|| / ||x_old|| below 0.01, x being the
  * dequantised weights of one matrix.  The procedure the appendix describes -- re-encode a hundredth of the

@@ -90,6 +90,10 @@ def lib():
         L.pvt_adam_update.argtypes = [vp, vp, vp, vp, vp, u64, fl, fl, fl, fl, fl, fl, vp]
         L.pvt_adam_direction.restype = ctypes.c_int
         L.pvt_adam_direction.argtypes = [vp, vp, vp, vp, u64, fl, fl, fl, fl, fl, vp]
+        L.pvt_adam_bias.restype = ctypes.c_int
+        L.pvt_adam_bias.argtypes = [u64, fl, fl, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float)]
+        L.pvt_test_wait_limit.restype = None
+        L.pvt_test_wait_limit.argtypes = [ctypes.c_uint32, ctypes.c_int64]
         L.pvt_status.restype = ctypes.c_int
         L.pvt_status.argtypes = [vp, vp]
         L.pvt_strerror.restype = ctypes.c_char_p
@@ -231,10 +235,11 @@ def pvt_pstep_grad(layer: pvt_layer, grad_codebooks: torch.Tensor, grad_scale: O
                                 _stream_ptr(stream)), "pvt_pstep_grad")
 
 
-def adam_bias(step: int, beta1: float, beta2: float):
+def pvt_adam_bias(step: int, beta1: float, beta2: float):
     """Bias corrections 1 - beta^t of step t >= 1 as the binary32 numbers pvt_adam_update takes."""
-    f32 = lambda x: ctypes.c_float(x).value
-    return f32(1.0 - f32(beta1) ** step), f32(1.0 - f32(beta2) ** step)
+    b1, b2 = ctypes.c_float(0.0), ctypes.c_float(0.0)
+    _check(lib().pvt_adam_bias(step, beta1, beta2, ctypes.byref(b1), ctypes.byref(b2)), "pvt_adam_bias")
+    return b1.value, b2.value
 
 
 def pvt_adam_update(param: torch.Tensor, grad: torch.Tensor, exp_avg: torch.Tensor, exp_avg_sq: torch.Tensor,
@@ -244,7 +249,7 @@ def pvt_adam_update(param: torch.Tensor, grad: torch.Tensor, exp_avg: torch.Tens
     assert param.dtype == torch.float32 and grad.dtype == torch.float64
     assert exp_avg.dtype == torch.float32 and exp_avg_sq.dtype == torch.float32
     assert param_f16 is None or param_f16.dtype == torch.float16
-    bias1, bias2 = adam_bias(step, beta1, beta2)
+    bias1, bias2 = pvt_adam_bias(step, beta1, beta2)
     _check(lib().pvt_adam_update(param.data_ptr(), _ptr(param_f16), grad.data_ptr(), exp_avg.data_ptr(),
                                  exp_avg_sq.data_ptr(), param.numel(), lr, beta1, beta2, eps, bias1, bias2,
                                  _stream_ptr(stream)), "pvt_adam_update")
@@ -255,7 +260,7 @@ def pvt_adam_direction(grad: torch.Tensor, exp_avg: torch.Tensor, exp_avg_sq: to
     """Adam-normalised update direction of the V step (all float32; moments updated in place)."""
     for t in (grad, exp_avg, exp_avg_sq, out):
         assert t.dtype == torch.float32 and t.is_contiguous()
-    bias1, bias2 = adam_bias(step, beta1, beta2)
+    bias1, bias2 = pvt_adam_bias(step, beta1, beta2)
     _check(lib().pvt_adam_direction(grad.data_ptr(), exp_avg.data_ptr(), exp_avg_sq.data_ptr(), out.data_ptr(),
                                     grad.numel(), beta1, beta2, eps, bias1, bias2, _stream_ptr(stream)),
            "pvt_adam_direction")
@@ -285,6 +290,12 @@ def pvt_probe_fp32_tflops(stream=None) -> float:
     _check(lib().pvt_probe_fp32_tflops(scratch.data_ptr(), scratch.numel(), ctypes.byref(out), _stream_ptr(stream)),
            "pvt_probe_fp32_tflops")
     return float(out.value)
+
+
+def pvt_test_wait_limit(max_polls: int = 0, withhold_copy: int = -1) -> None:
+    """Test hook: poll limit of the search kernels' on-chip waits (0 = default) and the sequence number of a
+    codebook copy that every thread block leaves out (-1 = none).  Process-wide."""
+    lib().pvt_test_wait_limit(max_polls, withhold_copy)
 
 
 def pvt_launch_count() -> int:

@@ -1,6 +1,10 @@
-"""Build libpvt.so (the CUDA library behind the C ABI) in-tree with nvcc for sm_100a."""
+"""Build libpvt.so (the CUDA library behind the C ABI) in-tree with nvcc for sm_100a.
+
+Every ``csrc/*.cu`` is compiled to an object of its own (in parallel, only when it or a header is newer than
+the object) under ``_build/`` and the objects are linked into ``libpvt.so`` next to this file."""
 from __future__ import annotations
 
+import concurrent.futures
 import glob
 import os
 import subprocess
@@ -9,30 +13,51 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 LIB = os.path.join(HERE, "libpvt.so")
+OBJ_DIR = os.path.join(HERE, "_build")
 
 
 def sources():
     return sorted(glob.glob(os.path.join(HERE, "csrc", "*.cu")))
 
 
+def headers():
+    return (glob.glob(os.path.join(HERE, "csrc", "*.h")) + glob.glob(os.path.join(HERE, "csrc", "*.cuh")) +
+            glob.glob(os.path.join(ROOT, "include", "*.h")))
+
+
 def needs_build() -> bool:
     if not os.path.exists(LIB):
         return True
-    deps = sources() + glob.glob(os.path.join(HERE, "csrc", "*.h")) + glob.glob(os.path.join(ROOT, "include", "*.h"))
-    return max(os.path.getmtime(d) for d in deps) > os.path.getmtime(LIB)
+    return max(os.path.getmtime(d) for d in sources() + headers()) > os.path.getmtime(LIB)
+
+
+def _flags(verbose: bool):
+    flags = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+             "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", os.path.join(HERE, "csrc")]
+    if verbose:
+        flags += ["-Xptxas", "-v"]
+    return flags
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not needs_build():
         return LIB
     nvcc = os.environ.get("NVCC", "nvcc")
-    cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-           "-Xcompiler", "-fPIC", "-shared", "-cudart", "static",
-           "-I", os.path.join(ROOT, "include"), "-I", os.path.join(HERE, "csrc"), "-o", LIB]
-    if verbose:
-        cmd += ["-Xptxas", "-v"]
-    cmd += sources()
-    subprocess.run(cmd, check=True)
+    os.makedirs(OBJ_DIR, exist_ok=True)
+    newest_header = max(os.path.getmtime(h) for h in headers())
+    jobs = []
+    objects = []
+    for src in sources():
+        obj = os.path.join(OBJ_DIR, os.path.splitext(os.path.basename(src))[0] + ".o")
+        objects.append(obj)
+        stale = force or not os.path.exists(obj) or os.path.getmtime(obj) < max(os.path.getmtime(src), newest_header)
+        if stale:
+            jobs.append([nvcc] + _flags(verbose) + ["-c", src, "-o", obj])
+    with concurrent.futures.ThreadPoolExecutor(max_workers=max(1, min(len(jobs), os.cpu_count() or 1))) as pool:
+        for done in pool.map(lambda cmd: subprocess.run(cmd, check=True), jobs):
+            pass
+    subprocess.run([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-cudart", "static",
+                    "-Xcompiler", "-fPIC", "-o", LIB] + objects, check=True)
     return LIB
 
 

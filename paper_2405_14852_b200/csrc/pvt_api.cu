@@ -2,9 +2,11 @@
 // optional per-kernel timing.  Everything here runs on the host and only enqueues
 // work; the arithmetic of the V step lives in the kernels of the other files.
 #include <atomic>
+#include <cmath>
 #include <mutex>
 #include <vector>
 
+#include "pvt_encode_m1.cuh"
 #include "pvt_internal.h"
 
 namespace pvt {
@@ -362,6 +364,20 @@ void pvt_set_m1_search(int mode) {
 }
 
 unsigned long long pvt_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+void pvt_test_wait_limit(uint32_t max_polls, int64_t withhold_copy) {
+  m1::set_wait_test_hook(max_polls == 0 ? m1::kMaxSpins : max_polls,
+                         withhold_copy < 0 ? m1::kNoWithhold : (uint32_t)withhold_copy);
+}
+
+int pvt_adam_bias(uint64_t step, float beta1, float beta2, float* bias1_out, float* bias2_out) {
+  if (step < 1 || !bias1_out || !bias2_out || !(beta1 >= 0.0f && beta1 < 1.0f) || !(beta2 >= 0.0f && beta2 < 1.0f))
+    return PVT_EINVAL;
+  // beta^t in binary64 from the binary32 beta widened exactly (the C library's pow), one rounding to binary32
+  *bias1_out = (float)(1.0 - std::pow((double)beta1, (double)step));
+  *bias2_out = (float)(1.0 - std::pow((double)beta2, (double)step));
+  return PVT_OK;
+}
 
 int pvt_probe_fp32_tflops(float* scratch, size_t scratch_floats, float* tflops_out, void* cuda_stream) {
   if (!scratch || !tflops_out) return PVT_EINVAL;

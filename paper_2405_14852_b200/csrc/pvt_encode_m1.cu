@@ -1,5 +1,5 @@
 // Exhaustive nearest-codeword search of the V step for one codebook (Appendix C /
-// Appendix J: "try every code in the codebook"; Appendix D: the score
+// Appendix J: all codewords of the codebook are tried; Appendix D: the score
 // ||c||^2 - 2 <t, c>; Eq. 8 for the target t = (W - eta g) / s).
 //
 // Two kernels.
@@ -183,8 +183,9 @@ __global__ void __launch_bounds__(kEncThreads + 32, 1) encode_m1_kernel(const En
         for (uint32_t c = c_lo; c < c_hi && alive; ++c, ++it) {
           const uint32_t s = it % kEncStages;
           if (it >= kEncStages)
-            alive = mbar_wait(smem_u32(&sm.empty_bar[s]), ((it / kEncStages) - 1) & 1, abort_flag, p.status);
+            alive = mbar_wait(smem_u32(&sm.empty_bar[s]), ((it / kEncStages) - 1) & 1, abort_flag, p.status, p.max_spins);
           if (!alive) break;
+          if (it == p.withhold_copy) continue;  // test hook: this chunk never arrives, its consumers' wait runs out
           const uint32_t fb = smem_u32(&sm.full_bar[s]);
           mbar_expect_tx(fb, kChunkBytes);
           bulk_g2s(smem_u32(&sm.stage[s][0]), reinterpret_cast<const char*>(p.cbx) + (size_t)c * kChunkBytes,
@@ -195,8 +196,9 @@ __global__ void __launch_bounds__(kEncThreads + 32, 1) encode_m1_kernel(const En
         // drain: let every copy that was issued land before the CTA may exit
         for (uint32_t back = 1; back <= kEncStages && back <= it; ++back) {
           const uint32_t j = it - back;
+          if (j == p.withhold_copy) continue;  // never issued
           const uint32_t fb = smem_u32(&sm.full_bar[j % kEncStages]);
-          for (uint32_t spin = 0; spin < kMaxSpins; ++spin) {
+          for (uint32_t spin = 0; spin < p.max_spins; ++spin) {
             if (mbar_try_wait(fb, (j / kEncStages) & 1)) break;
             __nanosleep(64);
           }
@@ -248,7 +250,7 @@ __global__ void __launch_bounds__(kEncThreads + 32, 1) encode_m1_kernel(const En
     // 2.-4. stream the codebook chunks of this slice
     for (uint32_t c = c_lo; c < c_hi; ++c, ++it) {
       const uint32_t st = it % kEncStages;
-      mbar_wait(smem_u32(&sm.full_bar[st]), (it / kEncStages) & 1, abort_flag, p.status);
+      mbar_wait(smem_u32(&sm.full_bar[st]), (it / kEncStages) & 1, abort_flag, p.status, p.max_spins);
       const unsigned char* stage = &sm.stage[st][0];
 #pragma unroll 1
       for (int sub = 0; sub < kChunkCodewords / kSubCodewords; ++sub) {
@@ -526,6 +528,9 @@ cudaError_t launch_encode_m1(const pvt_layer& L, uint64_t G, const uint32_t* idx
   p.code_u16 = L.code_dtype == PVT_U16;
   p.err_out = err_out;
   p.status = reinterpret_cast<uint32_t*>(base);
+  const WaitTestHook hook = wait_test_hook();
+  p.max_spins = hook.max_spins;
+  p.withhold_copy = hook.withhold_copy;
 
   cudaError_t err = cudaMemsetAsync(base + lay.n2max_off, 0, sizeof(uint32_t), stream);
   if (err != cudaSuccess) return err;

@@ -10,7 +10,17 @@
 namespace pvt {
 namespace m1 {
 
-constexpr uint32_t kMaxSpins = 1u << 22;
+constexpr uint32_t kMaxSpins = 1u << 22;     // polls after which a wait on an on-chip barrier gives up
+constexpr uint32_t kNoWithhold = 0xffffffffu;
+
+// Test hook for the give-up path of the waits (host side, process-wide): the poll limit the search kernels
+// run with, and the number of one codebook copy that the producer leaves out so that a wait really runs out.
+struct WaitTestHook {
+  uint32_t max_spins;      // kMaxSpins unless a test lowered it
+  uint32_t withhold_copy;  // kNoWithhold, or the per-CTA sequence number of the copy that is never issued
+};
+WaitTestHook wait_test_hook();
+void set_wait_test_hook(uint32_t max_spins, uint32_t withhold_copy);
 
 struct EncM1Params {
   const float* W;
@@ -36,6 +46,8 @@ struct EncM1Params {
   int code_u16;
   float* err_out;
   uint32_t* status;
+  uint32_t max_spins;      // poll limit of every wait on an on-chip barrier
+  uint32_t withhold_copy;  // kNoWithhold; otherwise the producer skips its copy of this sequence number (test hook)
 };
 
 // order-preserving map binary32 -> u32 (and back)
@@ -111,11 +123,11 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
                "l"(src), "r"(bytes), "r"(bar)
                : "memory");
 }
-// Bounded wait.  Gives up after kMaxSpins polls (or as soon as another thread gave
+// Bounded wait.  Gives up after max_spins polls (or as soon as another thread gave
 // up), flags the CTA as aborted and reports through the status word.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                          uint32_t* status) {
-  for (uint32_t spin = 0; spin < kMaxSpins; ++spin) {
+                                          uint32_t* status, uint32_t max_spins) {
+  for (uint32_t spin = 0; spin < max_spins; ++spin) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
     if (spin > 4096) __nanosleep(64);  // try_wait itself suspends the thread for a short while

@@ -1,5 +1,5 @@
 // Exhaustive nearest-codeword search of the V step for one fp16 codebook on the
-// tensor cores (Appendix C / Appendix J: "try every code in the codebook";
+// tensor cores (Appendix C / Appendix J: all codewords of the codebook are tried;
 // Appendix D: the score ||c||^2 - 2 <t, c>; Eq. 8 for the target).
 //
 // The score matrix S[n][kappa] = 2^e_n (<t_n, c_kappa> - ||c_kappa||^2 / 2) is a
@@ -96,7 +96,19 @@ constexpr float kNegInf = -__builtin_huge_valf();
 
 namespace {
 std::atomic<int> g_m1_search{PVT_M1_AUTO};
+std::atomic<uint32_t> g_max_spins{m1::kMaxSpins};
+std::atomic<uint32_t> g_withhold_copy{m1::kNoWithhold};
 }
+
+namespace m1 {
+WaitTestHook wait_test_hook() {
+  return WaitTestHook{g_max_spins.load(std::memory_order_relaxed), g_withhold_copy.load(std::memory_order_relaxed)};
+}
+void set_wait_test_hook(uint32_t max_spins, uint32_t withhold_copy) {
+  g_max_spins.store(max_spins, std::memory_order_relaxed);
+  g_withhold_copy.store(withhold_copy, std::memory_order_relaxed);
+}
+}  // namespace m1
 
 void set_m1_search(int mode) { g_m1_search.store(mode, std::memory_order_relaxed); }
 
@@ -379,12 +391,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
           const uint32_t fb = smem_u32(&sm.full_bar[s]);
           if (sub == 0) {
             if (grp >= (uint32_t)kTcStages)
-              alive = mbar_wait(smem_u32(&sm.empty_bar[s]), ((grp / kTcStages) - 1) & 1, abort_flag, p.status);
+              alive = mbar_wait(smem_u32(&sm.empty_bar[s]), ((grp / kTcStages) - 1) & 1, abort_flag, p.status, p.max_spins);
             if (!alive) break;
             const uint32_t left = total - it;
             mbar_expect_tx(fb, (left < (uint32_t)kTcGroupSteps ? left : (uint32_t)kTcGroupSteps) * kStepBytes);
           }
-          bulk_g2s(smem_u32(&sm.b[s][sub][0]), bimg + (size_t)st * kStepBytes, kStepBytes, fb);
+          // test hook: a step that is never copied leaves its stage's barrier incomplete, so the MMA warps' wait
+          // for that stage runs out
+          if (it != p.withhold_copy) bulk_g2s(smem_u32(&sm.b[s][sub][0]), bimg + (size_t)st * kStepBytes, kStepBytes, fb);
         }
       }
       if (!alive) {
@@ -392,8 +406,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
         const uint32_t groups = (it + kTcGroupSteps - 1) / kTcGroupSteps;
         for (uint32_t back = 1; back <= (uint32_t)kTcStages && back <= groups; ++back) {
           const uint32_t j = groups - back;
+          if (p.withhold_copy / kTcGroupSteps == j) continue;  // incomplete on purpose; its other copies landed long ago
           const uint32_t fb = smem_u32(&sm.full_bar[j % kTcStages]);
-          for (uint32_t spin = 0; spin < kMaxSpins; ++spin) {
+          for (uint32_t spin = 0; spin < p.max_spins; ++spin) {
             if (mbar_try_wait(fb, (j / kTcStages) & 1)) break;
             __nanosleep(64);
           }
@@ -421,13 +436,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
       for (uint64_t u = blockIdx.x; u < units && alive; u += gridDim.x, ++unit_i) {
         uint32_t s_lo, s_hi;
         slice_units(p, (uint32_t)(u % p.n_slices), &s_lo, &s_hi);
-        alive = mbar_wait(smem_u32(&sm.a_ready), unit_i & 1, abort_flag, p.status);
+        alive = mbar_wait(smem_u32(&sm.a_ready), unit_i & 1, abort_flag, p.status, p.max_spins);
         tc_fence_after();
         for (uint32_t st = s_lo; st < s_hi && alive; ++st, ++it) {
           const uint32_t grp = it / kTcGroupSteps, sub = it % kTcGroupSteps, s = grp % kTcStages, buf = it & 1;
           if (sub == 0 || it == 0)
-            alive = mbar_wait(smem_u32(&sm.full_bar[s]), (grp / kTcStages) & 1, abort_flag, p.status);
-          if (alive) alive = mbar_wait(buf ? empty1 : empty0, ((it >> 1) & 1) ^ 1, abort_flag, p.status);
+            alive = mbar_wait(smem_u32(&sm.full_bar[s]), (grp / kTcStages) & 1, abort_flag, p.status, p.max_spins);
+          if (alive) alive = mbar_wait(buf ? empty1 : empty0, ((it >> 1) & 1) ^ 1, abort_flag, p.status, p.max_spins);
           if (!alive) break;
           tc_fence_after();
           const uint64_t b_desc = b_desc0 + (uint64_t)((s * kTcGroupSteps + sub) * (kStepBytes >> 4));
@@ -445,7 +460,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
       if (!alive) {
         // wait (bounded) for whatever was issued before tensor memory is released
         umma_commit(smem_u32(&sm.drain_bar[q]));
-        for (uint32_t spin = 0; spin < kMaxSpins; ++spin) {
+        for (uint32_t spin = 0; spin < kMaxSpins; ++spin) {  // always the full limit: these MMAs do complete
           if (mbar_try_wait(smem_u32(&sm.drain_bar[q]), 0)) break;
           __nanosleep(64);
         }
@@ -562,7 +577,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
           // one lane polls (256 threads polling one barrier slow every barrier operation of the CTA
           // down); the warp-wide exchange orders the other lanes after its observation
           bool ok = true;
-          if (lane == 0) ok = mbar_wait(smem_u32(&sm.tmem_full[buf][rb]), (it >> 1) & 1, abort_flag, p.status);
+          if (lane == 0) ok = mbar_wait(smem_u32(&sm.tmem_full[buf][rb]), (it >> 1) & 1, abort_flag, p.status, p.max_spins);
           alive = __shfl_sync(0xffffffffu, ok, 0);
           if (!alive) break;
           tc_fence_after();
@@ -688,6 +703,9 @@ cudaError_t launch_encode_m1_tc(const pvt_layer& L, uint64_t G, const uint32_t* 
   p.code_u16 = L.code_dtype == PVT_U16;
   p.err_out = err_out;
   p.status = reinterpret_cast<uint32_t*>(base);
+  const WaitTestHook hook = wait_test_hook();
+  p.max_spins = hook.max_spins;
+  p.withhold_copy = hook.withhold_copy;
 
   cudaError_t err = cudaMemsetAsync(stats, 0, sizeof(TcStats), stream);
   if (err != cudaSuccess) return err;

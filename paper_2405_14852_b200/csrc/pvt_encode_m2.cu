@@ -1,5 +1,5 @@
 // Greedy residual beam search of the V step for two additive codebooks
-// (Appendix C: "find the best combination of codes via beam search"; Appendix J:
+// (Appendix C: the code combination is found by beam search; Appendix J:
 // two 8-bit codebooks, group size 8, beam size 8, target = gradient-updated
 // dequantised weight; Eq. 8 for the target; Lemma 3.3 for keeping the previous
 // pair in the pool).

@@ -1,5 +1,5 @@
-// Subspace choice of the V step (Algorithm 2 "arg top tau"; Section 3.4 "largest
-// update norm within each weight matrix"): squared update norm per weight group,
+// Subspace choice of the V step (the top-tau selection of Algorithm 2; Section 3.4 ranks by
+// update size, separately for every weight matrix): squared update norm per weight group,
 // then an exact top-k by radix select on the binary32 bit patterns, ties at the
 // threshold resolved towards the lowest group index, result in ascending order.
 //

@@ -1,4 +1,4 @@
-// V step whose subspace size follows from a trust ratio (Section 4.3; Appendix J, "Hyperparameter tuning"):
+// V step whose subspace size follows from a trust ratio (Section 4.3; Appendix J, hyper-parameter paragraph):
 // the groups are taken in the order of decreasing update norm and re-encoded, and the longest prefix of that
 // order is kept whose total squared change of the dequantised weights stays below ratio^2 * ||W_hat||^2; the
 // other groups get their previous codes back; one group always keeps its new code.

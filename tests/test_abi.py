@@ -106,3 +106,18 @@ def test_misaligned_index_and_output_pointers_are_rejected():
     assert lib.pvt_vstep_refine(ctypes.byref(L), 0x2000, 4, 1, None, 0x3001, None, None) == B.PVT_EINVAL
     assert lib.pvt_vstep_select_noalloc(ctypes.byref(L), 4, 0x2002, None, None) == B.PVT_EINVAL
     assert lib.pvt_dequant(ctypes.byref(_layer(num_codebooks=2, codes=0x1001)), 0x4000, B.PVT_F32, None, None) == B.PVT_EINVAL
+
+
+def test_adam_bias_is_computed_in_the_library_and_equals_the_checkers():
+    """Host arithmetic of the library (no GPU): 1 - beta^t for the betas of Appendix J over many steps, bit for
+    bit what the CPU checker uses, plus the closed values of the first step."""
+    from oracle import pvt_oracle as oracle
+    for step in list(range(1, 200)) + [1000, 12345, 10 ** 6]:
+        for b1, b2 in ((0.9, 0.95), (0.9, 0.999), (0.0, 0.5)):
+            assert B.pvt_adam_bias(step, b1, b2) == oracle.adam_bias(step, b1, b2)
+    one = ctypes.c_float
+    assert B.pvt_adam_bias(1, 0.9, 0.95) == (one(1.0 - one(0.9).value).value, one(1.0 - one(0.95).value).value)
+    b1, b2 = ctypes.c_float(), ctypes.c_float()
+    assert B.lib().pvt_adam_bias(0, 0.9, 0.95, ctypes.byref(b1), ctypes.byref(b2)) == B.PVT_EINVAL
+    assert B.lib().pvt_adam_bias(3, 1.0, 0.95, ctypes.byref(b1), ctypes.byref(b2)) == B.PVT_EINVAL
+    assert B.lib().pvt_adam_bias(3, 0.9, 0.95, None, ctypes.byref(b2)) == B.PVT_EINVAL

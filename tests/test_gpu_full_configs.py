@@ -34,6 +34,19 @@ CASES = [
     (5, 1, "0.01", torch.float32),
     (5, 3, "0.01", torch.float32),
     (5, 1, "1.0", torch.float32),   # every group re-encoded (1 048 576 targets): the selection is the index list
+    # the remaining workload lines of the benchmark's table
+    (3, 0, "0.001", torch.float32),
+    (3, 0, "0.1", torch.float32),   # 563 609 targets: the compute-bound two-codebook case
+    (3, 1, "0.01", torch.float32),
+    (3, 1, "0.1", torch.float32),
+    (4, 3, "0.01", torch.float16),
+    (4, 4, "0.01", torch.float16),
+    (4, 5, "0.01", torch.float16),
+    (5, 0, "0.01", torch.float32),
+    (5, 0, "1.0", torch.float32),   # 8 388 608 targets
+    (5, 2, "0.01", torch.float32),
+    (5, 2, "1.0", torch.float32),   # 29 360 128 targets
+    (5, 3, "1.0", torch.float32),
 ]
 
 
@@ -79,6 +92,34 @@ def test_full_size_step_against_checker(cfg, which, tau, wdtype):
         assert got_W.tobytes() == want_W.astype(np.float16).tobytes()
     else:
         assert got_W.tobytes() == want_W.tobytes()
+
+
+@pytest.mark.parametrize("K,f16", [(256, False), (512, True)])
+def test_fp32_engine_with_eight_targets_per_thread(K, f16):
+    """More than 148 x 8192 targets on the FP32 engine: the variant of the search kernel that keeps eight
+    targets per thread (tiles of 2048 targets).  4096 x 4096, every group re-encoded, a small codebook so that
+    the checker evaluates every pair: all 2 097 152 codes compared."""
+    from paper_2405_14852_b200 import binding as B
+    L = synth.make_layer(4096, 4096, cfg=7, codebook_size=K, codebook_fp16=f16)
+    G = L.num_groups
+    assert G >= 148 * 8192 * 1.3
+    B.pvt_set_m1_search(B.PVT_M1_FP32)
+    try:
+        dev = VStepLayer.from_host(L)
+        idx = torch.arange(G, dtype=torch.int32, device="cuda")
+        err = torch.empty(G, dtype=torch.float32, device="cuda")
+        dev.encode(idx, err)
+        torch.cuda.synchronize()
+        assert dev.status() == 0
+    finally:
+        B.pvt_set_m1_search(B.PVT_M1_AUTO)
+    sel = np.arange(G, dtype=np.uint32)
+    t = oracle.targets(L.W, L.g, L.scale, L.eta, sel)
+    enc = oracle.encode(t, L.codebooks, L.codes.reshape(G, 1))
+    got = dev.codes.cpu().numpy().reshape(G, 1)
+    exact, band = helpers.check_codes_against_oracle(t, L.codebooks, got, enc, REL)
+    assert exact >= G - G // 500
+    assert np.allclose(err.cpu().numpy(), enc.d_best, rtol=1e-5, atol=1e-30)
 
 
 def test_full_size_trust_step_against_checker():

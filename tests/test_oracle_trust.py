@@ -1,4 +1,4 @@
-"""Pins of the CPU checker's trust-ratio subspace rule (Section 4.3 and Appendix J, "Hyperparameter tuning"):
+"""Pins of the CPU checker's trust-ratio subspace rule (Section 4.3 and the hyper-parameter paragraph of Appendix J):
 a worked example done by hand, the bound and its maximality recomputed from dequantised matrices, the limits
 ratio -> 0 and ratio -> infinity, and independence of the portion size.  No GPU needed."""
 import numpy as np

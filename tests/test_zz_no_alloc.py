@@ -63,6 +63,33 @@ def test_noalloc_select_with_crafted_ties_after_a_previous_call():
     assert torch.equal(out.cpu(), torch.arange(300, dtype=torch.int32))
 
 
+@pytest.mark.gpu
+def test_noalloc_select_at_its_largest_layer_against_the_checker():
+    """4096 x 4096 = 2^21 groups, the most the built-in scratch takes: the index list against the CPU
+    checker's full sort, and no device memory taken or returned by the call (the first call on a device may
+    make the array resident, so the free memory is compared across a second call)."""
+    from oracle import pvt_oracle as oracle
+    rows = cols = 4096
+    assert rows * (cols // 8) == B.PVT_NOALLOC_MAX_GROUPS
+    g_host = _g(rows, cols, 14)
+    k = 20971
+    want = oracle.select(oracle.group_norms(g_host, 1.0), k)
+    g = torch.from_numpy(g_host).cuda()
+    desc = _desc(g, rows, cols)
+    got = torch.empty(k, dtype=torch.int32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B.pvt_vstep_select_noalloc(desc, k, got, status)
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    got.fill_(-1)
+    B.pvt_vstep_select_noalloc(desc, k, got, status)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
+    assert int(status.item()) == 0
+    assert np.array_equal(got.cpu().numpy().astype(np.uint32), want)
+
+
 def test_noalloc_select_rejects_layers_beyond_the_built_in_scratch():
     """Host-side check only: nothing is enqueued, so this runs without a GPU."""
     rows, cols = 4096, 4096 + 8  # one column group more than 2^21 groups
