@@ -3,20 +3,29 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
 
-One "step" is one whole V step over one layer: pvt_vstep_select, pvt_vstep_encode
-and pvt_dequant through the C ABI.  Default workload: a 4096 x 4096 fp32 layer,
-one fp16 codebook of 65536 codewords (group size 8), tau = 0.01.  With N > 1
-(launched by torch.distributed.run) every rank steps its own layer of the same
-shape (layers are independent problems: no collective on the data path); the
-reported value is the work of all ranks over the slowest rank's time.
+One "step" is one whole V step over the workload: for every layer of it, pvt_vstep_select,
+pvt_vstep_encode and pvt_dequant through the C ABI, all on one stream.  The default workload is
+the largest one of the benchmark table that one GPU holds: the seven linear layers of one
+Llama-2-70B decoder block (2 x 8192x8192, 2 x 8192x1024, 2 x 28672x8192, 8192x28672; fp32 weights
+and update, one fp16 codebook of 65536 codewords per layer, groups of 8) with every group
+re-encoded (tau = 1.0): 106 954 752 groups, 7.0e12 codeword pairs per step.  The single-layer
+workloads of the table are available by name (--list).  With N > 1 (launched by
+torch.distributed.run) every rank steps its own copy of the workload (layers are independent
+problems: no collective on the data path); the reported value is the work of all ranks over the
+slowest rank's time.
 
-Prints ONE JSON line on rank 0.
+Besides the headline, the line carries `sub` (the 4096x4096, tau = 0.01 layer with the search on
+the tensor cores and on the FP32 pipe) and `sweep` (every single-layer workload of the table,
+briefly).  Prints ONE JSON line on rank 0.
 """
 from __future__ import annotations
 
 import argparse
+import concurrent.futures
+import hashlib
 import json
 import os
+import re
 import subprocess
 import sys
 import threading
@@ -30,19 +39,23 @@ METRIC = "vstep_reencoded_groups_per_s"
 UNIT = "groups/s"
 FP32_LANES_PER_SM = 128  # FP32 FMA lanes of one sm_100 multiprocessor
 FLOP_PER_PAIR = 16       # one codeword-pair evaluation = a dot product of 8 elements
+BLOCK_PREFIX = "llama2_70b_block_1x16"
+DEFAULT_WORKLOAD = BLOCK_PREFIX + "_tau1.0"
+SUB_WORKLOAD = "llama2_7b_attn_4096x4096_1x16_tau0.01"
+GRAPH_BELOW_MS = 5.0     # steps shorter than this are timed as CUDA graph replays (launch gaps matter there)
 
 
 def workloads():
+    """name -> ("layer", cfg, entry, tau) or ("block", tau)."""
     from paper_2405_14852_b200 import synth
     out = {}
     for cfg, entries in synth.CONFIGS.items():
         for which, e in enumerate(entries):
             for tau in e[7]:
-                out[f"{e[0]}_tau{tau}"] = (cfg, which, tau)
+                out[f"{e[0]}_tau{tau}"] = ("layer", cfg, which, tau)
+    for tau in ("0.01", "1.0"):
+        out[f"{BLOCK_PREFIX}_tau{tau}"] = ("block", tau)
     return out
-
-
-DEFAULT_WORKLOAD = "llama2_7b_attn_4096x4096_1x16_tau0.01"
 
 
 # --------------------------------------------------------------------------- clocks
@@ -83,7 +96,7 @@ class ClockSampler:
         except subprocess.TimeoutExpired:
             self.proc.kill()
         self.thread.join(timeout=2)
-        sm, smax, reasons = [], None, set()
+        sm, smax, reasons, power = [], None, set(), []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in self.lines:
             f = [x.strip() for x in line.split(",")]
@@ -92,27 +105,356 @@ class ClockSampler:
             try:
                 sm.append(float(f[0]))
                 smax = float(f[1])
+                power.append(float(f[2]))
             except ValueError:
                 continue
             for name, v in zip(names, f[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(name)
         sm.sort()
-        # the busy samples are the upper half: idle gaps between steps pull the clock down
-        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": smax, "samples": len(sm),
-                "reasons": sorted(reasons)}
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": smax, "sm_mhz_min": sm[0] if sm else None,
+                "samples": len(sm), "power_w_max": max(power) if power else None, "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------- layers on the device
+
+
+class DeviceLayer:
+    """One synthetic layer: pinned host arrays, device arrays, descriptor, index buffer, outputs."""
+
+    def __init__(self, L, tau, dev, out_dtype, keep_host=True):
+        import numpy as np
+        import torch
+
+        from paper_2405_14852_b200 import binding as B
+        from paper_2405_14852_b200 import synth
+        self.L = L
+        self.name = L.name
+        self.rows, self.cols, self.M, self.K = L.rows, L.cols, L.num_codebooks, L.codebook_size
+        self.G = L.num_groups
+        self.tau = tau
+        self.k = synth.subspace_size(tau, self.G)
+        self.pairs = self.k * L.pairs_per_group()
+        self.h = {}
+        self.d = {}
+        for n in ("W", "g", "scale", "codebooks", "codes"):
+            a = np.ascontiguousarray(getattr(L, n))
+            t = torch.from_numpy(a)
+            if keep_host:
+                pinned = torch.empty(t.shape, dtype=t.dtype, pin_memory=True)
+                pinned.copy_(t)
+                self.h[n] = pinned
+                self.d[n] = pinned.to(dev, non_blocking=True)
+            else:
+                self.d[n] = t.to(dev)
+        torch.cuda.synchronize()
+        self.codes0 = self.d["codes"].clone()
+        self.W_hat = torch.empty(self.rows, self.cols, dtype=out_dtype, device=dev)
+        self.idx = torch.empty(self.k, dtype=torch.int32, device=dev)
+        self.desc = B.make_layer(self.rows, self.cols, self.d["W"], self.d["g"], self.d["scale"], self.d["codebooks"],
+                                 self.d["codes"], eta=L.eta, beam=L.beam)
+        self.ws_bytes = B.pvt_workspace_bytes(self.desc, self.k)
+        self.code_bytes = L.codes.dtype.itemsize * self.M
+        self.h2d_bytes = sum(t.numel() * t.element_size() for t in self.d.values())
+
+    def set_tau(self, tau, dev):
+        import torch
+
+        from paper_2405_14852_b200 import binding as B
+        from paper_2405_14852_b200 import synth
+        self.tau = tau
+        self.k = synth.subspace_size(tau, self.G)
+        self.pairs = self.k * self.L.pairs_per_group()
+        self.idx = torch.empty(self.k, dtype=torch.int32, device=dev)
+        self.ws_bytes = B.pvt_workspace_bytes(self.desc, self.k)
+
+
+class Runner:
+    """Steps a list of DeviceLayers through the three C-ABI calls and times them."""
+
+    def __init__(self, layers, dev, world=1):
+        import torch
+
+        from paper_2405_14852_b200 import binding as B
+        self.B = B
+        self.torch = torch
+        self.layers = layers
+        self.dev = dev
+        self.world = world
+        # one workspace serves every layer: the calls of a step run one after the other on one stream
+        self.ws = torch.empty(max(l.ws_bytes for l in layers), dtype=torch.uint8, device=dev)
+        B.pvt_workspace_init(self.ws)
+        self.k = sum(l.k for l in layers)
+        self.pairs = sum(l.pairs for l in layers)
+        self.G = sum(l.G for l in layers)
+
+    def step(self):
+        B = self.B
+        for l in self.layers:
+            B.pvt_vstep_select(l.desc, l.k, l.idx, self.ws)
+            B.pvt_vstep_encode(l.desc, l.idx, l.k, None, self.ws)
+            B.pvt_dequant(l.desc, l.W_hat)
+
+    def restore_codes(self):
+        for l in self.layers:
+            l.d["codes"].copy_(l.codes0)
+
+    def barrier(self):
+        import torch.distributed as dist
+        self.torch.cuda.synchronize()
+        if self.world > 1:
+            dist.barrier()
+        self.torch.cuda.synchronize()
+
+    def check_status(self, where):
+        st = self.B.pvt_status(self.ws)
+        if st != 0:
+            raise SystemExit(f"bench.py: device status word {st} {where}")
+
+    def timed(self, steps, warmup, flush_l2, allow_graph=True):
+        """W warm-up steps, then K timed steps (L2 flushed and the previous codes restored before each, both
+        untimed): eager launches with the library's per-kernel events, and -- when a step is short enough for
+        launch gaps to matter -- the same step replayed from a CUDA graph.  Returns a dict of timings."""
+        torch, B = self.torch, self.B
+        for _ in range(max(warmup, 3)):
+            self.restore_codes()
+            self.step()
+        torch.cuda.synchronize()
+        self.check_status("after warm-up")
+        B.pvt_timing_enable(True)
+        for kid in range(9):
+            B.pvt_timing_read(kid)
+        launches0 = B.pvt_launch_count()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        self.barrier()
+        for a, b in ev:
+            self.restore_codes()
+            flush_l2()
+            a.record()
+            self.step()
+            b.record()
+        self.barrier()
+        launches = B.pvt_launch_count() - launches0
+        eager_ms = sum(a.elapsed_time(b) for a, b in ev)
+        kern = {kid: B.pvt_timing_read(kid) for kid in range(5)}
+        B.pvt_timing_enable(False)
+        out = {"eager_ms_per_step": eager_ms / steps, "ms_per_step": eager_ms / steps, "graphed": False,
+               "launches": int(launches), "kern": kern}
+        if allow_graph and eager_ms / steps < GRAPH_BELOW_MS:
+            try:
+                side = torch.cuda.Stream(device=self.dev)
+                side.wait_stream(torch.cuda.current_stream())
+                with torch.cuda.stream(side):
+                    self.step()
+                torch.cuda.current_stream().wait_stream(side)
+                torch.cuda.synchronize()
+                gph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(gph):
+                    self.step()
+                for _ in range(3):
+                    self.restore_codes()
+                    gph.replay()
+                self.barrier()
+                launches0 = B.pvt_launch_count()
+                for a, b in ev:
+                    self.restore_codes()
+                    flush_l2()
+                    a.record()
+                    gph.replay()
+                    b.record()
+                self.barrier()
+                out["ms_per_step"] = sum(a.elapsed_time(b) for a, b in ev) / steps
+                out["graphed"] = True
+            except RuntimeError as exc:  # capture not possible: report the eager timing and say so
+                print(f"bench.py: CUDA graph capture failed ({exc}); eager launches are timed", file=sys.stderr)
+        self.check_status("after the timed region")
+        return out
+
+    def e2e(self, steps):
+        """The same step with host buffers: every layer's W, g, scale, codebook and codes copied from pinned
+        host memory inside the timed region, the selected indices and the new codes copied back."""
+        torch = self.torch
+        h_idx = [torch.empty(l.k, dtype=torch.int32, pin_memory=True) for l in self.layers]
+        h_codes = [torch.empty(l.h["codes"].shape, dtype=l.h["codes"].dtype, pin_memory=True) for l in self.layers]
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        h2d = sum(l.h2d_bytes for l in self.layers)
+        d2h = sum(t.numel() * t.element_size() for t in h_idx + h_codes)
+        B = self.B
+        self.barrier()
+        for a, b in ev:
+            a.record()
+            for l, hi, hc in zip(self.layers, h_idx, h_codes):
+                for n in ("W", "g", "scale", "codebooks", "codes"):
+                    l.d[n].copy_(l.h[n], non_blocking=True)
+                B.pvt_vstep_select(l.desc, l.k, l.idx, self.ws)
+                B.pvt_vstep_encode(l.desc, l.idx, l.k, None, self.ws)
+                B.pvt_dequant(l.desc, l.W_hat)
+                hi.copy_(l.idx, non_blocking=True)
+                hc.copy_(l.d["codes"], non_blocking=True)
+            b.record()
+            b.synchronize()
+        self.barrier()
+        return sum(a.elapsed_time(b) for a, b in ev) / steps, h2d, d2h
+
+
+def make_flush(dev):
+    import torch
+    flush = torch.empty(64 << 20, dtype=torch.int32, device=dev)  # 256 MiB, twice the L2
+
+    def flush_l2():
+        # write, then read: the write evicts every line of the step's arrays, the read leaves the L2 full of
+        # clean lines, so that no write-back of the flush buffer is charged to the step that follows
+        flush.fill_(1)
+        flush.sum()
+    return flush_l2
+
+
+def build_layers(kind, rank, dev, out_dtype, keep_host=True):
+    """Host generation (in parallel threads: the generators release the interpreter lock) + upload."""
+    from paper_2405_14852_b200 import synth
+    if kind[0] == "block":
+        tau = kind[1]
+        n = len(synth.BLOCK_70B)
+        with concurrent.futures.ThreadPoolExecutor(max_workers=min(n, os.cpu_count() or 1)) as pool:
+            host = list(pool.map(lambda i: synth.make_block_layer(i, seed_offset=100 * rank), range(n)))
+        out = []
+        for L in host:
+            out.append(DeviceLayer(L, tau, dev, out_dtype, keep_host))
+        return out
+    _, cfg, which, tau = kind
+    name, rows, cols, M, K, f16, rowmax, _ = synth.CONFIGS[cfg][which]
+    L = synth.make_layer(rows, cols, cfg=rank_layer_seed(cfg, rank), num_codebooks=M, codebook_size=K,
+                         codebook_fp16=f16, row_max_scale=rowmax, nearest=_nearest_on_gpu, name=name)
+    return [DeviceLayer(L, tau, dev, out_dtype, keep_host)]
+
+
+# --------------------------------------------------------------------------- rooflines
+
+
+def device_peaks(local, clocks=None):
+    import torch
+    peaks = _measured_peaks()
+    props = torch.cuda.get_device_properties(local)
+    sm_max_mhz = (clocks or {}).get("sm_max_mhz") or peaks.get("sm_max_mhz") or 1965.0
+    peaks["sm_count"] = props.multi_processor_count
+    peaks["sm_max_mhz_used"] = sm_max_mhz
+    peaks["alu_tflops"] = props.multi_processor_count * FP32_LANES_PER_SM * 2 * sm_max_mhz * 1e6 / 1e12
+    peaks["epilogue_pairs_per_s"] = props.multi_processor_count * 128 * sm_max_mhz * 1e6
+    return peaks
+
+
+def search_roofline(engine, pairs_per_step, enc_ms, enc_n, steps, peaks, traffic):
+    """Roofline record of the search kernel: algorithmic flops of the launches of one step over their summed
+    duration (CUDA events inside the library, around every launch, on the launching stream)."""
+    per_step_ms = enc_ms / max(steps, 1)
+    achieved = FLOP_PER_PAIR * pairs_per_step / (per_step_ms * 1e-3) / 1e12
+    common = {"achieved": achieved, "unit": "TFLOP/s", "flop_per_pair": FLOP_PER_PAIR,
+              "launches": enc_n, "avg_launch_ms": enc_ms / max(enc_n, 1), "kernel_ms_per_step": per_step_ms,
+              "pairs_per_s": pairs_per_step / (per_step_ms * 1e-3), "traffic": traffic}
+    if engine == "tensor":
+        tpeak = peaks.get("bf16_tflops_sustained" if per_step_ms > 50.0 else "bf16_tflops") or peaks.get("bf16_tflops")
+        which = "sustained" if per_step_ms > 50.0 and peaks.get("bf16_tflops_sustained") else "burst"
+        r = {"kernel": "encode_m1_tc_kernel (exhaustive search, tcgen05)", "bound": "tensor", "peak": tpeak,
+             "frac": achieved / tpeak,
+             "peak_is": (f"measured bf16 matmul, {which} figure (fp16 operands run at the same rate)"
+                         if not peaks.get("fallback") else "fallback of the profiling recipe"),
+             "frac_of_fp32_alu_roofline": achieved / peaks["alu_tflops"],
+             "frac_of_epilogue_bound": common["pairs_per_s"] / peaks["epilogue_pairs_per_s"],
+             "epilogue_bound_is": "one accumulator read per pair: 128 lanes per SM per clock at the maximum SM clock"}
+    else:
+        r = {"kernel": "encode_m1_kernel (exhaustive search, FP32 pipe)" if engine == "fp32"
+             else "encode_m2_kernel (beam search)", "bound": "alu", "peak": peaks["alu_tflops"],
+             "frac": achieved / peaks["alu_tflops"],
+             "peak_is": f"{peaks['sm_count']} SMs x 128 FP32 lanes x 2 flop x {peaks['sm_max_mhz_used']:.0f} MHz "
+                        f"(derived; no measured FP32 peak)"}
+        if engine == "beam":
+            r["note"] = ("issue-bound; stage 2 (2048 of 2304 pairs per group) on the tensor pipe for fp16 codebooks; "
+                         "the search as written needs 16 (K1 + K2) + 2 B K2 flop per group (B.K2 cross terms reuse "
+                         "<t, c2>), the 16 flop per pair of the metric count every pair as a full dot product")
+    r.update(common)
+    return r
+
+
+def engine_of(layer, search):
+    if layer.M != 1:
+        return "beam"
+    f16 = layer.L.codebooks.dtype.itemsize == 2
+    if f16 and (search == "tensor" or (search == "auto" and layer.K >= 1024)):
+        return "tensor"
+    return "fp32"
+
+
+_PROFILE_OF = {"tensor": ("encode_m1_tc_kernel_8192x1024_1x16_tau1.0.md", ["pvt_encode_m1_tc.cu", "pvt_encode_m1.cuh"]),
+               "fp32": ("encode_m1_fp32_kernel_4096x4096_1x16_tau0.01.md", ["pvt_encode_m1.cu", "pvt_encode_m1.cuh"])}
+
+
+def kernel_source_hash(files):
+    h = hashlib.sha256()
+    for f in files:
+        with open(os.path.join(ROOT, "paper_2405_14852_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic(engine, targets_per_step):
+    """DRAM bytes of the search kernel per step from the committed ncu summary, scaled by the number of targets
+    (the traffic is the gathered W, g rows and the per-target records: proportional to the targets).  None when
+    there is no summary or the kernel's source has changed since the counters were taken."""
+    if engine not in _PROFILE_OF:
+        return None
+    name, files = _PROFILE_OF[engine]
+    try:
+        text = open(os.path.join(ROOT, "profiles", name)).read()
+    except OSError:
+        return None
+    m_hash = re.search(r"kernel_source_sha256_16:\s*([0-9a-f]{16})", text)
+    m_bytes = re.search(r"dram_bytes_per_target:\s*([0-9.eE+]+)", text)
+    if not m_hash or not m_bytes or m_hash.group(1) != kernel_source_hash(files):
+        return None
+    return float(m_bytes.group(1)) * targets_per_step
+
+
+def stage_record(runner, t, steps, peaks, out_itemsize):
+    kern = t["kern"]
+    B = runner.B
+    hbm = peaks.get("hbm_gbs")
+
+    def per_step(kid):
+        ms, n = kern[kid]
+        return ms / max(steps, 1), n
+
+    sel_ms, _ = per_step(B.PVT_KERNEL_SELECT)
+    enc_ms, _ = per_step(B.PVT_KERNEL_ENCODE_MAIN)
+    aux_ms, _ = per_step(B.PVT_KERNEL_ENCODE_AUX)
+    dq_ms, _ = per_step(B.PVT_KERNEL_DEQUANT)
+    rs_ms, _ = per_step(B.PVT_KERNEL_ENCODE_RESCORE)
+    sel_bytes = sum(l.G * 32 + 4 * l.k for l in runner.layers)
+    dq_bytes = sum(l.G * (l.code_bytes + 8 * out_itemsize) for l in runner.layers)
+    st = {"select": {"ms": sel_ms, "algorithmic_bytes": sel_bytes, "gbs": sel_bytes / (sel_ms * 1e-3) / 1e9 if sel_ms else None},
+          "encode_search": {"ms": enc_ms, "pairs": runner.pairs, "pairs_per_s": runner.pairs / (enc_ms * 1e-3) if enc_ms else None},
+          "encode_codebook_prep": {"ms": aux_ms},
+          "encode_rescore": {"ms": rs_ms},
+          "dequant": {"ms": dq_ms, "algorithmic_bytes": dq_bytes, "gbs": dq_bytes / (dq_ms * 1e-3) / 1e9 if dq_ms else None}}
+    if hbm:
+        for s in ("select", "dequant"):
+            if st[s]["gbs"]:
+                st[s]["frac_of_measured_hbm"] = st[s]["gbs"] / hbm
+    t_enc_call = (aux_ms + enc_ms + rs_ms) * 1e-3
+    if t_enc_call > 0:
+        st["rates"] = {"groups_per_s_encode": runner.k / t_enc_call,
+                       "groups_per_s_select_plus_encode": runner.k / (t_enc_call + sel_ms * 1e-3),
+                       "pairs_per_s_encode": runner.pairs / t_enc_call}
+    return st
 
 
 # --------------------------------------------------------------------------- our arm
 
 
 def run_ours(args):
-    import numpy as np
     import torch
     import torch.distributed as dist
 
     from paper_2405_14852_b200 import binding as B
-    from paper_2405_14852_b200 import synth
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -124,283 +466,207 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
-    cfg, which, tau = workloads()[args.workload]
-    name, rows, cols, M, K, f16, rowmax, _ = synth.CONFIGS[cfg][which]
-    B.pvt_set_m1_search({"auto": B.PVT_M1_AUTO, "fp32": B.PVT_M1_FP32, "tensor": B.PVT_M1_TENSOR}[args.search])
-    tensor_engine = M == 1 and f16 and (args.search == "tensor" or (args.search == "auto" and K >= 1024))
-
-    def gpu_nearest(X, C):  # only the recipe of a second codebook needs it: the library's own search
-        return _nearest_on_gpu(X, C)
-
-    # every rank draws its own layer (seed offset): independent problems, no exchange
-    L = synth.make_layer(rows, cols, cfg=rank_layer_seed(cfg, rank), num_codebooks=M, codebook_size=K, codebook_fp16=f16,
-                         row_max_scale=rowmax, nearest=gpu_nearest, name=name)
-    G = L.num_groups
-    k = synth.subspace_size(tau, G)
-    pairs_per_group = L.pairs_per_group()
-
-    # host side (pinned) and device side of every array
-    def pin(a):
-        t = torch.from_numpy(np.ascontiguousarray(a))
-        return t.pin_memory()
-
-    h = {n: pin(getattr(L, n)) for n in ("W", "g", "scale", "codebooks", "codes")}
-    d = {n: t.to(dev) for n, t in h.items()}
-    codes0 = d["codes"].clone()
+    kind = workloads()[args.workload]
+    search_mode = {"auto": B.PVT_M1_AUTO, "fp32": B.PVT_M1_FP32, "tensor": B.PVT_M1_TENSOR}
+    B.pvt_set_m1_search(search_mode[args.search])
     out_dtype = torch.float16 if args.dequant_fp16 else torch.float32
-    W_hat = torch.empty(rows, cols, dtype=out_dtype, device=dev)
-    idx = torch.empty(k, dtype=torch.int32, device=dev)
-    h_idx = torch.empty(k, dtype=torch.int32).pin_memory()
-    h_codes_out = torch.empty_like(h["codes"]).pin_memory()
-    desc = B.make_layer(rows, cols, d["W"], d["g"], d["scale"], d["codebooks"], d["codes"], eta=L.eta, beam=L.beam)
-    ws = B.new_workspace(desc, k, device=dev)
-    flush = torch.empty(64 << 20, dtype=torch.int32, device=dev)  # 256 MiB, twice the L2
+    t0 = time.perf_counter()
+    layers = build_layers(kind, rank, dev, out_dtype)
+    setup_s = time.perf_counter() - t0
+    runner = Runner(layers, dev, world)
+    flush_l2 = make_flush(dev)
+    engine = engine_of(layers[0], args.search)
+    steps = args.steps
 
-    def flush_l2():
-        # write, then read: the write evicts every line of the step's arrays, the read leaves the L2 full of
-        # clean lines, so that no write-back of the flush buffer is charged to the step that follows
-        flush.fill_(1)
-        flush.sum()
-
-    def step():
-        B.pvt_vstep_select(desc, k, idx, ws)
-        B.pvt_vstep_encode(desc, idx, k, None, ws)
-        B.pvt_dequant(desc, W_hat)
-
-    def barrier():
-        torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    # ---- warm-up
-    for _ in range(max(args.warmup, 3)):
-        d["codes"].copy_(codes0)
-        step()
-    torch.cuda.synchronize()
-    st = B.pvt_status(ws)
-    if st != 0:
-        raise SystemExit(f"bench.py: device status word {st} after warm-up")
-
-    # ---- device-resident timing: K steps, L2 flushed before each, per-kernel events inside the library
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    B.pvt_timing_enable(True)
-    for kid in range(7):
-        B.pvt_timing_read(kid)
-    launches0 = B.pvt_launch_count()
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    barrier()
-    for a, b in ev:
-        d["codes"].copy_(codes0)  # same previous codes every step (untimed)
-        flush_l2()                # evict W, g and the codebook from L2 (untimed)
-        a.record()
-        step()
-        b.record()
-    barrier()
-    launches = B.pvt_launch_count() - launches0
-    eager_ms = sum(a.elapsed_time(b) for a, b in ev)
-    kern = {kid: B.pvt_timing_read(kid) for kid in range(5)}
-    B.pvt_timing_enable(False)
-
-    # ---- the same step as a CUDA graph (the three C-ABI calls captured once, replayed K times): the launch
-    # gaps between the step's nine short kernels and four memsets disappear; this is the headline timing
-    graphed = False
-    total_ms = eager_ms
-    if not args.no_graph:
-        try:
-            side = torch.cuda.Stream(device=dev)
-            side.wait_stream(torch.cuda.current_stream())
-            with torch.cuda.stream(side):
-                step()
-            torch.cuda.current_stream().wait_stream(side)
-            torch.cuda.synchronize()
-            gph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(gph):
-                step()
-            for _ in range(3):
-                d["codes"].copy_(codes0)
-                gph.replay()
-            barrier()
-            for a, b in ev:
-                d["codes"].copy_(codes0)
-                flush_l2()
-                a.record()
-                gph.replay()
-                b.record()
-            barrier()
-            total_ms = sum(a.elapsed_time(b) for a, b in ev)
-            graphed = True
-        except RuntimeError as exc:  # capture not possible: report the eager timing and say so
-            print(f"bench.py: CUDA graph capture failed ({exc}); eager launches are timed", file=sys.stderr)
-    B.pvt_timing_enable(True)
-    # the P-step kernels that share the V step's inputs (not part of the timed step): same flush, own events
-    gb = torch.empty((M, K, 8), dtype=torch.float64, device=dev)
-    gs = torch.empty(rows, dtype=torch.float64, device=dev)
-    master = d["codebooks"].float().reshape(-1).clone()
-    adam_m, adam_v = torch.zeros_like(master), torch.zeros_like(master)
-    scratch16 = torch.empty(master.numel(), dtype=torch.float16, device=dev)
-    for i in range(min(args.steps, 10)):
-        flush_l2()
-        B.pvt_pstep_grad(desc, gb, gs)
-        B.pvt_adam_update(master, gb.reshape(-1), adam_m, adam_v, i + 1, 3e-4, param_f16=scratch16)
-    torch.cuda.synchronize()
-    kern[B.PVT_KERNEL_PSTEP_GRAD] = B.pvt_timing_read(B.PVT_KERNEL_PSTEP_GRAD)
-    kern[B.PVT_KERNEL_ADAM] = B.pvt_timing_read(B.PVT_KERNEL_ADAM)
-    B.pvt_timing_enable(False)
-    st = B.pvt_status(ws)
-    if st != 0:
-        raise SystemExit(f"bench.py: device status word {st} after the timed region")
-
-    # ---- end to end: host buffers in, host buffers out, copies inside the timed region
-    e2e_steps = max(3, min(args.steps, 10))
-    ev2 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(e2e_steps)]
-    h2d = sum(t.numel() * t.element_size() for t in h.values())
-    d2h = h_idx.numel() * 4 + h_codes_out.numel() * h_codes_out.element_size()
-    barrier()
-    for a, b in ev2:
-        a.record()
-        for n in ("W", "g", "scale", "codebooks", "codes"):
-            d[n].copy_(h[n], non_blocking=True)
-        step()
-        h_idx.copy_(idx, non_blocking=True)
-        h_codes_out.copy_(d["codes"], non_blocking=True)
-        b.record()
-        b.synchronize()
-    barrier()
-    e2e_ms = sum(a.elapsed_time(b) for a, b in ev2) / e2e_steps
+    t = runner.timed(steps, args.warmup, flush_l2, allow_graph=not args.no_graph)
+    e2e_steps = max(3, min(steps, 5))
+    e2e_ms, h2d, d2h = runner.e2e(e2e_steps)
     clocks = sampler.stop() if rank == 0 else None
 
-    # reference point for the streaming kernels at this size: a library fill of the dequantised matrix (the bytes
-    # pvt_dequant writes), cold L2, timed the same way.  Outside the timed region; rank 0 only.
-    fill_ms = None
+    total_ms, e2e_ms = slowest_rank([t["ms_per_step"], e2e_ms], dev, world)
+    ms_per_step = total_ms
+
     if rank == 0:
+        peaks = device_peaks(local, clocks)
+        ffma_measured = B.pvt_probe_fp32_tflops()  # the FP32 pipe, measured in this job
+        enc_ms, enc_n = t["kern"][B.PVT_KERNEL_ENCODE_MAIN]
+        roofline = search_roofline(engine, runner.pairs, enc_ms, enc_n, steps, peaks,
+                                   recorded_traffic(engine, runner.k))
+        roofline["fp32_fma_microbenchmark_tflops"] = ffma_measured
+        stages = stage_record(runner, t, steps, peaks, runner.layers[0].W_hat.element_size())
+        # reference point for the streaming kernels: a library fill of the dequantised matrices (the bytes
+        # pvt_dequant writes), cold L2, timed the same way, outside the timed region
         spans = []
-        for _ in range(5):
+        for _ in range(3):
             flush_l2()
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record()
-            W_hat.fill_(0)
+            for l in runner.layers:
+                l.W_hat.fill_(0)
             b.record()
             b.synchronize()
             spans.append(a.elapsed_time(b))
-        fill_ms = sorted(spans)[len(spans) // 2]
+        stages["dequant"]["library_fill_of_the_same_output_ms"] = sorted(spans)[1]
 
-    total_ms, e2e_ms = slowest_rank([total_ms, e2e_ms], dev, world)
-    ms_per_step = total_ms / args.steps
-
-    if rank == 0:
-        peaks = _measured_peaks()
-        props = torch.cuda.get_device_properties(local)
-        sm_max_mhz = (clocks or {}).get("sm_max_mhz") or peaks.get("sm_max_mhz") or 1965.0
-        alu_peak = props.multi_processor_count * FP32_LANES_PER_SM * 2 * sm_max_mhz * 1e6 / 1e12  # TFLOP/s
-        ffma_measured = B.pvt_probe_fp32_tflops()  # the same pipe, measured in this job
-        enc_ms, enc_n = kern[B.PVT_KERNEL_ENCODE_MAIN]
-        enc_avg_ms = enc_ms / max(enc_n, 1)
-        pairs = k * pairs_per_group
-        achieved = FLOP_PER_PAIR * pairs / (enc_avg_ms * 1e-3) / 1e12
-        hbm = peaks.get("hbm_gbs")
-        stages = {}
-        sel_ms, sel_n = kern[B.PVT_KERNEL_SELECT]
-        aux_ms, aux_n = kern[B.PVT_KERNEL_ENCODE_AUX]
-        dq_ms, dq_n = kern[B.PVT_KERNEL_DEQUANT]
-        code_bytes = L.codes.dtype.itemsize * M
-        dq_bytes = G * (code_bytes + 8 * W_hat.element_size())
-        sel_bytes = G * 32 + 4 * k
-        stages["select"] = {"ms": sel_ms / max(sel_n, 1), "algorithmic_bytes": sel_bytes,
-                            "gbs": sel_bytes / (sel_ms / max(sel_n, 1) * 1e-3) / 1e9 if sel_n else None}
-        stages["encode_search"] = {"ms": enc_avg_ms, "pairs": pairs,
-                                   "pairs_per_s": pairs / (enc_avg_ms * 1e-3)}
-        stages["encode_codebook_prep"] = {"ms": aux_ms / max(aux_n, 1)}
-        rs_ms, rs_n = kern[B.PVT_KERNEL_ENCODE_RESCORE]
-        stages["encode_rescore"] = {"ms": rs_ms / max(rs_n, 1)}
-        stages["dequant"] = {"ms": dq_ms / max(dq_n, 1), "algorithmic_bytes": dq_bytes,
-                             "gbs": dq_bytes / (dq_ms / max(dq_n, 1) * 1e-3) / 1e9 if dq_n else None}
-        stages["dequant"]["library_fill_of_the_same_output_ms"] = fill_ms
-        # per-stage rates: the whole encode call (codebook preparation + search + rescoring), alone and with
-        # the selection in front of it
-        t_enc_call = (aux_ms / max(aux_n, 1) + enc_avg_ms + rs_ms / max(rs_n, 1)) * 1e-3
-        t_sel_call = sel_ms / max(sel_n, 1) * 1e-3
-        stages["rates"] = {"groups_per_s_encode": k / t_enc_call if t_enc_call > 0 else None,
-                           "groups_per_s_select_plus_encode": k / (t_enc_call + t_sel_call) if t_enc_call > 0 else None,
-                           "pairs_per_s_encode": pairs / t_enc_call if t_enc_call > 0 else None}
-        pg_ms, pg_n = kern[B.PVT_KERNEL_PSTEP_GRAD]
-        ad_ms, ad_n = kern[B.PVT_KERNEL_ADAM]
-        pg_bytes = G * (32 + code_bytes) + M * K * 8 * 8 + rows * 12
-        ad_bytes = M * K * 8 * (8 + 4 * 6 + 2)
-        stages["pstep_grad"] = {"ms": pg_ms / max(pg_n, 1), "algorithmic_bytes": pg_bytes,
-                                "gbs": pg_bytes / (pg_ms / max(pg_n, 1) * 1e-3) / 1e9 if pg_n else None,
-                                "note": "not part of the timed V step"}
-        stages["adam"] = {"ms": ad_ms / max(ad_n, 1), "algorithmic_bytes": ad_bytes,
-                          "gbs": ad_bytes / (ad_ms / max(ad_n, 1) * 1e-3) / 1e9 if ad_n else None,
-                          "note": "not part of the timed V step"}
-        if hbm:
-            for s in ("select", "dequant", "pstep_grad", "adam"):
-                if stages[s]["gbs"]:
-                    stages[s]["frac_of_measured_hbm"] = stages[s]["gbs"] / hbm
-        if tensor_engine:
-            # dense contraction on the tensor cores: algorithmic flops against the measured fp16/bf16 peak
-            tpeak = peaks.get("bf16_tflops")
-            roofline = {"kernel": "encode search (M=1, tcgen05)", "bound": "tensor", "achieved": achieved,
-                        "peak": tpeak, "unit": "TFLOP/s", "frac": achieved / tpeak,
-                        "peak_is": ("measured bf16 matmul (fp16 operands run at the same rate)"
-                                    if not peaks.get("fallback") else "fallback of the profiling recipe"),
-                        "flop_per_pair": FLOP_PER_PAIR, "avg_launch_ms": enc_avg_ms, "launches": enc_n,
-                        "executed_tflops": achieved * 4.0,  # operands are padded from depth 8 to depth 32
-                        "frac_of_fp32_alu_roofline": achieved / alu_peak,
-                        "fp32_fma_microbenchmark_tflops": ffma_measured,
-                        "frac_of_epilogue_bound": (pairs / (enc_avg_ms * 1e-3)) /
-                                                  (props.multi_processor_count * 128 * sm_max_mhz * 1e6),
-                        "epilogue_bound_is": "one accumulator read per pair: 128 lanes per SM per clock",
-                        # dram__bytes_read + dram__bytes_write of one launch (ncu, this kernel, default workload)
-                        "traffic": 7.64e6 if args.workload == DEFAULT_WORKLOAD else None}
-        else:
-            roofline = {"kernel": "encode search (M=1, fp32 pipe)" if M == 1 else "encode beam search (M=2)",
-                        "bound": "alu", "achieved": achieved, "peak": alu_peak, "unit": "TFLOP/s",
-                        "frac": achieved / alu_peak,
-                        "peak_is": f"{props.multi_processor_count} SMs x 128 FP32 lanes x 2 flop x "
-                                   f"{sm_max_mhz:.0f} MHz (derived; no measured FP32 peak)",
-                        "flop_per_pair": FLOP_PER_PAIR, "avg_launch_ms": enc_avg_ms, "launches": enc_n,
-                        "fp32_fma_microbenchmark_tflops": ffma_measured,
-                        # dram__bytes_read + dram__bytes_write of one launch (ncu, FP32 engine, default workload)
-                        "traffic": 7.87e6 if (M == 1 and args.workload == DEFAULT_WORKLOAD) else None}
-            if M == 2:
-                # the kernel is bound by instruction issue; the pair evaluations of stage 2 themselves run on the
-                # tensor pipe when the codebooks are fp16, so the FP32-pipe roofline is a yardstick, not a ceiling
-                roofline["note"] = ("issue-bound; stage 2 (2048 of 2304 pairs per group) on the tensor pipe for fp16 "
-                                    "codebooks, the FP32-pipe roofline is the yardstick the 16 flop per pair refer to")
+        L0 = runner.layers[0]
+        config = {"workload": args.workload,
+                  "layers": [{"name": l.name, "rows": l.rows, "cols": l.cols, "groups": l.G, "k": l.k} for l in runner.layers],
+                  "group_dim": 8, "groups": runner.G, "num_codebooks": L0.M, "codebook_size": L0.K,
+                  "codebook_dtype": "f16" if L0.L.codebooks.dtype.itemsize == 2 else "f32",
+                  "tau": L0.tau, "k": runner.k, "pairs_per_step": runner.pairs,
+                  "search_engine": engine, "dequant_dtype": "f16" if args.dequant_fp16 else "f32",
+                  "l2": "flushed before every timed step (256 MiB written, then read)",
+                  "launch": ("CUDA graph replay of the step's C-ABI calls" if t["graphed"]
+                             else "eager launches of pvt_vstep_select + pvt_vstep_encode + pvt_dequant per layer, one stream"),
+                  "parallelism": f"independent workloads x{world}"}
         line = {
-            "metric": METRIC, "value": job_value(k, world, ms_per_step), "unit": UNIT,
-            "pairs_per_s": world * pairs / (ms_per_step * 1e-3),
-            "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
-            "ms_per_step_eager_launches": eager_ms / args.steps,
+            "metric": METRIC, "value": job_value(runner.k, world, ms_per_step), "unit": UNIT,
+            "pairs_per_s": world * runner.pairs / (ms_per_step * 1e-3),
+            "n_gpus": world, "steps": steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
+            "ms_per_step_eager_launches": t["eager_ms_per_step"],
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f32", "data": "synthetic",
-            "config": {"workload": args.workload, "rows": rows, "cols": cols, "group_dim": 8, "groups": G,
-                       "num_codebooks": M, "codebook_size": K, "codebook_dtype": "f16" if f16 else "f32",
-                       "tau": tau, "k": k, "pairs_per_group": pairs_per_group,
-                       "search_engine": ("tensor" if tensor_engine else "fp32") if M == 1 else "beam",
-                       "dequant_dtype": "f16" if args.dequant_fp16 else "f32",
-                       "l2": "flushed before every timed step (256 MiB written, then read)",
-                       "launch": ("CUDA graph replay of pvt_vstep_select + pvt_vstep_encode + pvt_dequant" if graphed
-                                  else "eager launches"),
-                       "parallelism": f"independent layers x{world}"},
-            "e2e": {"value": world * k / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+            "dtype": "f32", "data": "synthetic", "config": config,
+            "e2e": {"value": world * runner.k / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "what": "pinned host W, g, scale, codebook, codes -> device; select+encode+dequant; "
+                    "what": "per layer: pinned host W, g, scale, codebook, codes -> device; select+encode+dequant; "
                             "idx and codes -> pinned host"},
-            "gpu_launches": int(launches),
-            "roofline": roofline,
-            "stages": stages,
-            "clocks": clocks,
+            "gpu_launches": t["launches"],
+            "roofline": roofline, "stages": stages, "clocks": clocks, "setup_s": setup_s,
         }
+        del runner
+        if not args.no_sub:
+            line["sub"] = sub_record(args, dev, local, peaks, flush_l2, layers)
+        if not args.no_sweep:
+            line["sweep"] = sweep_record(args, dev, peaks, flush_l2, layers if kind[0] == "block" else None)
+        if not args.no_next:
+            line["stages"].update(pstep_record(dev, peaks, flush_l2))
         if not args.no_cpu_baseline and world == 1:
-            line["cpu_baseline"] = cpu_baseline(L, k, tau, budget_s=args.cpu_seconds)
+            line["cpu_baseline"] = cpu_baseline(layers, budget_s=args.cpu_seconds)
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def sub_record(args, dev, local, peaks, flush_l2, resident_layers):
+    """The 4096 x 4096, one codebook of 65 536, tau = 0.01 layer with the exhaustive search on either engine."""
+    import torch
+
+    from paper_2405_14852_b200 import binding as B
+    kind = workloads()[SUB_WORKLOAD]
+    layers = build_layers(kind, 0, dev, torch.float32, keep_host=False)
+    out = {"workload": SUB_WORKLOAD, "k": layers[0].k, "pairs": layers[0].pairs}
+    for engine, mode in (("tensor", B.PVT_M1_TENSOR), ("fp32", B.PVT_M1_FP32)):
+        B.pvt_set_m1_search(mode)
+        for l in layers:
+            l.set_tau(l.tau, dev)
+        runner = Runner(layers, dev)
+        steps = 20
+        t = runner.timed(steps, 3, flush_l2)
+        enc_ms, enc_n = t["kern"][B.PVT_KERNEL_ENCODE_MAIN]
+        r = search_roofline(engine, runner.pairs, enc_ms, enc_n, steps, peaks, recorded_traffic(engine, runner.k)
+                            if engine == "fp32" else recorded_traffic(engine, runner.k))
+        st = stage_record(runner, t, steps, peaks, 4)
+        out[engine] = {"ms_per_step": t["ms_per_step"], "groups_per_s": runner.k / (t["ms_per_step"] * 1e-3),
+                       "pairs_per_s": runner.pairs / (t["ms_per_step"] * 1e-3), "graph_replay": t["graphed"],
+                       "roofline": r,
+                       "stages_ms": {k: v["ms"] for k, v in st.items() if isinstance(v, dict) and "ms" in v},
+                       "select_frac_of_measured_hbm": st["select"].get("frac_of_measured_hbm"),
+                       "dequant_frac_of_measured_hbm": st["dequant"].get("frac_of_measured_hbm")}
+        del runner
+    B.pvt_set_m1_search({"auto": B.PVT_M1_AUTO, "fp32": B.PVT_M1_FP32, "tensor": B.PVT_M1_TENSOR}[args.search])
+    return out
+
+
+def sweep_record(args, dev, peaks, flush_l2, block_layers):
+    """Every single-layer workload of the table, briefly (3 timed steps each after 3 warm-up steps): step time,
+    rates and the search kernel's fraction of its bound.  The 70B shapes reuse the block's resident layers."""
+    import torch
+
+    from paper_2405_14852_b200 import binding as B
+    from paper_2405_14852_b200 import synth
+    rows_out = []
+    by_shape = {}
+    if block_layers:
+        for l in block_layers:
+            by_shape.setdefault((l.rows, l.cols), l)
+    for cfg, entries in synth.CONFIGS.items():
+        for which, e in enumerate(entries):
+            name, rows, cols, M, K, f16, rowmax, taus = e
+            layer = by_shape.get((rows, cols)) if cfg == 5 else None
+            own = layer is None
+            if own:
+                layer = build_layers(("layer", cfg, which, taus[0]), 0, dev,
+                                     torch.float16 if cfg == 4 else torch.float32, keep_host=False)[0]
+            saved_tau = layer.tau
+            for tau in taus:
+                layer.set_tau(tau, dev)
+                runner = Runner([layer], dev)
+                t = runner.timed(3, 3, flush_l2)
+                engine = engine_of(layer, args.search)
+                enc_ms, enc_n = t["kern"][B.PVT_KERNEL_ENCODE_MAIN]
+                r = search_roofline(engine, runner.pairs, enc_ms, enc_n, 3, peaks, None)
+                st = stage_record(runner, t, 3, peaks, layer.W_hat.element_size())
+                rec = {"workload": f"{name}_tau{tau}", "k": layer.k, "ms_per_step": t["ms_per_step"],
+                       "graph_replay": t["graphed"],
+                       "groups_per_s": layer.k / (t["ms_per_step"] * 1e-3),
+                       "pairs_per_s": layer.pairs / (t["ms_per_step"] * 1e-3),
+                       "select_ms": st["select"]["ms"], "search_ms": st["encode_search"]["ms"],
+                       "rescore_ms": st["encode_rescore"]["ms"], "dequant_ms": st["dequant"]["ms"],
+                       "select_frac_hbm": st["select"].get("frac_of_measured_hbm"),
+                       "dequant_frac_hbm": st["dequant"].get("frac_of_measured_hbm"),
+                       "search_bound": r["bound"], "search_frac": r["frac"]}
+                if engine == "tensor":
+                    rec["search_frac_of_epilogue_bound"] = r["frac_of_epilogue_bound"]
+                    rec["search_frac_of_fp32_alu_roofline"] = r["frac_of_fp32_alu_roofline"]
+                rows_out.append(rec)
+                del runner
+            if own:
+                del layer
+                torch.cuda.empty_cache()
+            else:
+                layer.set_tau(saved_tau, dev)
+    return rows_out
+
+
+def pstep_record(dev, peaks, flush_l2):
+    """The P-step kernels that share the V step's inputs (not part of the timed step), on the 4096 x 4096 layer."""
+    import torch
+
+    from paper_2405_14852_b200 import binding as B
+    layer = build_layers(workloads()[SUB_WORKLOAD], 0, dev, torch.float32, keep_host=False)[0]
+    M, K, rows, G = layer.M, layer.K, layer.rows, layer.G
+    B.pvt_timing_enable(True)
+    for kid in (B.PVT_KERNEL_PSTEP_GRAD, B.PVT_KERNEL_ADAM):
+        B.pvt_timing_read(kid)
+    gb = torch.empty((M, K, 8), dtype=torch.float64, device=dev)
+    gs = torch.empty(rows, dtype=torch.float64, device=dev)
+    master = layer.d["codebooks"].float().reshape(-1).clone()
+    adam_m, adam_v = torch.zeros_like(master), torch.zeros_like(master)
+    scratch16 = torch.empty(master.numel(), dtype=torch.float16, device=dev)
+    n = 10
+    for i in range(n):
+        flush_l2()
+        B.pvt_pstep_grad(layer.desc, gb, gs)
+        B.pvt_adam_update(master, gb.reshape(-1), adam_m, adam_v, i + 1, 3e-4, param_f16=scratch16)
+    torch.cuda.synchronize()
+    pg_ms, pg_n = B.pvt_timing_read(B.PVT_KERNEL_PSTEP_GRAD)
+    ad_ms, ad_n = B.pvt_timing_read(B.PVT_KERNEL_ADAM)
+    B.pvt_timing_enable(False)
+    hbm = peaks.get("hbm_gbs")
+    pg_bytes = G * (32 + layer.code_bytes) + M * K * 8 * 8 + rows * 12
+    ad_bytes = M * K * 8 * (8 + 4 * 6 + 2)
+    out = {}
+    for key, ms, cnt, nbytes in (("pstep_grad", pg_ms, pg_n, pg_bytes), ("adam", ad_ms, ad_n, ad_bytes)):
+        rec = {"ms": ms / max(cnt, 1), "algorithmic_bytes": nbytes, "gbs": nbytes / (ms / max(cnt, 1) * 1e-3) / 1e9 if cnt else None,
+               "note": f"not part of the timed V step; {SUB_WORKLOAD}'s layer"}
+        if hbm and rec["gbs"]:
+            rec["frac_of_measured_hbm"] = rec["gbs"] / hbm
+        out[key] = rec
+    return out
 
 
 def rank_layer_seed(cfg: int, rank: int) -> int:
@@ -452,50 +718,10 @@ def _measured_peaks():
         with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
             return json.load(f)
     except OSError:
-        return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "fallback": True}
+        return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "fallback": True}
 
 
 # --------------------------------------------------------------------------- CPU arm
-
-
-def cpu_baseline(L, k, tau, budget_s=15.0):
-    """The CPU checker, as it stands, on a bounded sample of the same layer: norms and
-    selection over all groups, the search on the first n selected groups (n sized for
-    about `budget_s` seconds), dequantisation of the whole layer.  The search time is
-    scaled to all k groups; the value is k over that estimated whole-step time."""
-    import numpy as np
-
-    from oracle import pvt_oracle as oracle
-    threads = oracle.num_threads()
-    t0 = time.perf_counter()
-    norms = oracle.group_norms(L.g, L.eta)
-    idx = oracle.select(norms, k)
-    t_sel = time.perf_counter() - t0
-    codes2 = L.codes.reshape(-1, L.num_codebooks)
-    # calibrate on a small probe, then size the sample
-    n0 = min(k, 256)
-    t_probe = _time_oracle_encode(oracle, L, idx[:n0], codes2)
-    n = int(min(k, max(n0, n0 * budget_s / max(t_probe, 1e-6))))
-    t_enc = _time_oracle_encode(oracle, L, idx[:n], codes2)
-    t0 = time.perf_counter()
-    oracle.dequant(L.codes, L.codebooks, L.scale, L.rows, L.cols)
-    t_deq = time.perf_counter() - t0
-    t_step = t_sel + t_enc * (k / n) + t_deq
-    # the same search on one thread, on a sample smaller by the thread count (a few seconds)
-    one_thread = None
-    if threads > 1:
-        n1 = max(1, min(n, n // threads))
-        oracle.set_num_threads(1)
-        try:
-            t1 = _time_oracle_encode(oracle, L, idx[:n1], codes2)
-        finally:
-            oracle.set_num_threads(threads)
-        one_thread = {"pairs_per_s": n1 * L.pairs_per_group() / t1, "sample_groups": n1, "seconds": t1}
-    return {"value": k / t_step, "unit": UNIT, "cores": threads, "kind": "oracle", "search_on_one_thread": one_thread,
-            "sample": f"norms+selection over all {L.num_groups} groups ({t_sel:.2f} s), search of the first {n} of "
-                      f"{k} selected groups ({t_enc:.2f} s, scaled by k/n), dequantisation of the whole layer "
-                      f"({t_deq:.2f} s)",
-            "pairs_per_s": n * L.pairs_per_group() / t_enc, "estimated_step_s": t_step}
 
 
 def _time_oracle_encode(oracle, L, idx, codes2):
@@ -506,55 +732,147 @@ def _time_oracle_encode(oracle, L, idx, codes2):
     return time.perf_counter() - t0
 
 
-def run_reference(args):
-    """The CPU checker timed as the reference arm: every step is one bounded sample of
-    the workload (selection over all groups, search of n selected groups, whole-layer
-    dequantisation); value = groups re-encoded per second of that step."""
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
-        return
+def _oracle_sample(oracle, L, k, search_budget_s, probe=256):
+    """The CPU checker, as it stands, on one layer: norms and selection over all its groups, the search on the
+    first n selected groups (n sized for about `search_budget_s` seconds), dequantisation of the whole layer."""
+    t0 = time.perf_counter()
+    idx = oracle.select(oracle.group_norms(L.g, L.eta), k)
+    t_sel = time.perf_counter() - t0
+    codes2 = L.codes.reshape(-1, L.num_codebooks)
+    n0 = min(k, probe)
+    t_probe = _time_oracle_encode(oracle, L, idx[:n0], codes2)
+    n = int(min(k, max(n0, n0 * search_budget_s / max(t_probe, 1e-6))))
+    t_enc = _time_oracle_encode(oracle, L, idx[:n], codes2)
+    t0 = time.perf_counter()
+    oracle.dequant(L.codes, L.codebooks, L.scale, L.rows, L.cols)
+    t_deq = time.perf_counter() - t0
+    return idx, codes2, n, t_sel, t_enc, t_deq
+
+
+def _extrapolate(sample_layer, k_sample, n, t_sel, t_enc, t_deq, G_total, k_total, pairs_total):
+    """Whole-workload step time of the checker from its timings on one layer: selection and dequantisation
+    scale with the groups, the search with the codeword pairs."""
+    pairs_n = n * sample_layer.pairs_per_group()
+    return (t_sel + t_deq) * (G_total / sample_layer.num_groups) + t_enc * (pairs_total / pairs_n)
+
+
+def _pick_sample_layer(layers):
+    """The smallest layer of the workload stands for it on the CPU."""
+    return min(layers, key=lambda l: l.G)
+
+
+def cpu_baseline(layers, budget_s=12.0):
+    from oracle import pvt_oracle as oracle
+    threads = oracle.num_threads()
+    dl = _pick_sample_layer(layers)
+    L = dl.L
+    G_total, k_total, pairs_total = sum(l.G for l in layers), sum(l.k for l in layers), sum(l.pairs for l in layers)
+    idx, codes2, n, t_sel, t_enc, t_deq = _oracle_sample(oracle, L, dl.k, budget_s)
+    t_step = _extrapolate(L, dl.k, n, t_sel, t_enc, t_deq, G_total, k_total, pairs_total)
+    one_thread = None
+    if threads > 1:
+        n1 = max(1, min(n, n // threads))
+        oracle.set_num_threads(1)
+        try:
+            t1 = _time_oracle_encode(oracle, L, idx[:n1], codes2)
+        finally:
+            oracle.set_num_threads(threads)
+        one_thread = {"pairs_per_s": n1 * L.pairs_per_group() / t1, "sample_groups": n1, "seconds": t1}
+    whole = len(layers) == 1 and n == dl.k
+    return {"value": k_total / t_step, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "search_on_one_thread": one_thread,
+            "sample": (f"layer {L.name}: norms+selection over its {L.num_groups} groups ({t_sel:.2f} s), search of the "
+                       f"first {n} of its {dl.k} selected groups ({t_enc:.2f} s), dequantisation of the layer "
+                       f"({t_deq:.2f} s); " + ("measured on the whole workload" if whole else
+                       f"extrapolated to the workload's {G_total} groups (selection, dequantisation) and "
+                       f"{pairs_total:.3e} codeword pairs (search), linearly")),
+            "extrapolated": not whole,
+            "pairs_per_s": n * L.pairs_per_group() / t_enc, "estimated_step_s": t_step}
+
+
+def host_layers(kind):
+    """Host arrays for the CPU arm: only the layer that is sampled is generated."""
     import numpy as np
 
     from oracle import pvt_oracle as oracle
     from paper_2405_14852_b200 import synth
-    cfg, which, tau = workloads()[args.workload]
-    name, rows, cols, M, K, f16, rowmax, _ = synth.CONFIGS[cfg][which]
 
     def nearest(X, C):
         return oracle.encode(X, C[None], np.zeros((X.shape[0], 1))).codes[:, 0]
 
+    class HL:  # the fields of DeviceLayer that the CPU arm reads
+        def __init__(self, L, tau):
+            self.L, self.G, self.tau = L, L.num_groups, tau
+            self.k = synth.subspace_size(tau, self.G)
+            self.pairs = self.k * L.pairs_per_group()
+            self.name, self.rows, self.cols, self.M, self.K = L.name, L.rows, L.cols, L.num_codebooks, L.codebook_size
+
+    class Shape(HL):  # a layer that is only counted, never generated
+        def __init__(self, name, rows, cols, M, K, tau):
+            self.L = None
+            self.G = rows * (cols // 8)
+            self.tau = tau
+            self.k = synth.subspace_size(tau, self.G)
+            self.pairs = self.k * K
+            self.name, self.rows, self.cols, self.M, self.K = name, rows, cols, M, K
+
+    if kind[0] == "block":
+        tau = kind[1]
+        shapes = synth.block_layer_shapes()
+        smallest = min(range(len(shapes)), key=lambda i: shapes[i][1] * shapes[i][2])
+        out = []
+        for i, (name, rows, cols, M, K, f16, rowmax) in enumerate(shapes):
+            out.append(HL(synth.make_block_layer(i), tau) if i == smallest else
+                       Shape(f"llama2_70b_{name}_{rows}x{cols}_1x16", rows, cols, M, K, tau))
+        return out
+    _, cfg, which, tau = kind
+    name, rows, cols, M, K, f16, rowmax, _ = synth.CONFIGS[cfg][which]
     L = synth.make_layer(rows, cols, cfg=cfg, num_codebooks=M, codebook_size=K, codebook_fp16=f16,
                          row_max_scale=rowmax, nearest=nearest, name=name)
-    k = synth.subspace_size(tau, L.num_groups)
-    codes2 = L.codes.reshape(-1, M)
+    return [HL(L, tau)]
+
+
+def run_reference(args):
+    """The CPU checker timed as the reference arm: every step is one bounded sample of the workload (selection
+    over all groups of its smallest layer, search of n of that layer's selected groups for about two seconds,
+    dequantisation of that layer), extrapolated linearly to the whole workload; value = groups re-encoded per
+    second of that step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import pvt_oracle as oracle
+    kind = workloads()[args.workload]
+    layers = host_layers(kind)
+    dl = min((l for l in layers if l.L is not None), key=lambda l: l.G)
+    L = dl.L
+    G_total, k_total, pairs_total = sum(l.G for l in layers), sum(l.k for l in layers), sum(l.pairs for l in layers)
     threads = oracle.num_threads()
-    # sample size: about 2 s of search per step
-    idx_full = oracle.select(oracle.group_norms(L.g, L.eta), k)
-    n0 = min(k, 128)
-    t_probe = _time_oracle_encode(oracle, L, idx_full[:n0], codes2)
-    n = int(min(k, max(n0, n0 * 2.0 / max(t_probe, 1e-6))))
     warm = max(args.warmup, 1)
     times = []
+    n = None
     for i in range(warm + args.steps):
-        t0 = time.perf_counter()
-        idx = oracle.select(oracle.group_norms(L.g, L.eta), k)
-        t_sel = time.perf_counter() - t0
-        t_enc = _time_oracle_encode(oracle, L, idx[:n], codes2)
-        t0 = time.perf_counter()
-        oracle.dequant(L.codes, L.codebooks, L.scale, L.rows, L.cols)
-        t_deq = time.perf_counter() - t0
+        idx, codes2, n, t_sel, t_enc, t_deq = _oracle_sample(oracle, L, dl.k, 2.0, probe=128)
         if i >= warm:
-            times.append(t_sel + t_enc * (k / n) + t_deq)
+            times.append(_extrapolate(L, dl.k, n, t_sel, t_enc, t_deq, G_total, k_total, pairs_total))
     t_step = sum(times) / len(times)
-    value = k / t_step
-    sample = (f"per step: norms+selection over all {L.num_groups} groups, search of the first {n} of {k} selected "
-              f"groups (time scaled by k/n), dequantisation of the whole layer")
+    value = k_total / t_step
+    whole = len(layers) == 1 and n == dl.k
+    sample = (f"per step, layer {L.name}: norms+selection over its {L.num_groups} groups, search of the first {n} of "
+              f"its {dl.k} selected groups, dequantisation of the layer; " +
+              ("the whole workload" if whole else f"extrapolated linearly to {G_total} groups and {pairs_total:.3e} pairs"))
+    first = layers[0]
+    config = {"workload": args.workload,
+              "layers": [{"name": l.name, "rows": l.rows, "cols": l.cols, "groups": l.G, "k": l.k} for l in layers],
+              "group_dim": 8, "groups": G_total, "num_codebooks": first.M, "codebook_size": first.K,
+              "codebook_dtype": "f16" if first.K > 256 or first.M > 1 else "f32",
+              "tau": first.tau, "k": k_total, "pairs_per_step": pairs_total,
+              "search_engine": "cpu checker (binary64)", "dequant_dtype": "f32",
+              "l2": "not applicable", "launch": "host threads", "parallelism": "host cores"}
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": warm, "ms_per_step": t_step * 1e3, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": args.workload, "rows": rows, "cols": cols, "groups": L.num_groups,
-                       "num_codebooks": M, "codebook_size": K, "tau": tau, "k": k},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": config,
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample,
+                             "extrapolated": not whole},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
@@ -566,7 +884,6 @@ def run_reference(args):
 def run_next_rows(args):
     """Times the calls that widen the path (trust-ratio step, local search, three and four codebooks, groups of
     16 weights) on synthetic layers of the benchmark shapes and prints one JSON line.  Not the headline metric."""
-    import numpy as np
     import torch
 
     from paper_2405_14852_b200 import binding as B
@@ -593,7 +910,7 @@ def run_next_rows(args):
 
     out = {"what": "median of 5 cold-L2 calls each, CUDA events; synthetic layers of the benchmark shapes"}
 
-    # trust-ratio step on the default workload's layer (its random previous codes make every change large, so
+    # trust-ratio step on the 4096 x 4096 layer (its random previous codes make every change large, so
     # the cut falls early; the cost is that of ranking and re-encoding k_max groups either way)
     L = synth.make_layer(4096, 4096, cfg=2, codebook_size=65536, codebook_fp16=True)
     dev = VStepLayer.from_host(L)
@@ -644,7 +961,7 @@ def run_next_rows(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
@@ -652,13 +969,19 @@ def main():
                     help="engine of the single-codebook search")
     ap.add_argument("--dequant-fp16", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of a CUDA graph replay")
+    ap.add_argument("--no-graph", action="store_true", help="never time a CUDA graph replay")
+    ap.add_argument("--no-sub", action="store_true", help="leave out the 4096x4096 record with both search engines")
+    ap.add_argument("--no-sweep", action="store_true", help="leave out the sweep over the single-layer workloads")
+    ap.add_argument("--no-next", action="store_true", help="leave out the P-step kernels' timings")
+    ap.add_argument("--only", action="store_true", help="the headline workload only (no sub, sweep, P step, CPU leg)")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--list", action="store_true")
     ap.add_argument("--next-rows", action="store_true",
                     help="time the calls beyond the V step proper (trust-ratio step, local search, 3-4 codebooks, "
                          "groups of 16) instead of the headline metric")
     args = ap.parse_args()
+    if args.only:
+        args.no_sub = args.no_sweep = args.no_next = args.no_cpu_baseline = True
     if args.list:
         print("\n".join(workloads()))
         return

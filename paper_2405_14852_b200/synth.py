@@ -177,6 +177,26 @@ CONFIGS = {
 }
 
 
+# One transformer block of the largest model of the benchmark table: the seven linear layers of a
+# Llama-2-70B decoder block (grouped-query attention: key / value projections are 8192 x 1024), as
+# (layer name, entry of CONFIGS[5]).
+BLOCK_70B = (("q_proj", 0), ("o_proj", 0), ("k_proj", 1), ("v_proj", 1), ("gate_proj", 2), ("up_proj", 2),
+             ("down_proj", 3))
+BLOCK_SEED_BASE = 50  # layer i of the block draws from the seed family cfg = BLOCK_SEED_BASE + i
+
+
+def block_layer_shapes():
+    """(name, rows, cols, M, K, fp16 codebook, row-max scale) of every layer of the block."""
+    return [(name,) + tuple(CONFIGS[5][which][1:7]) for name, which in BLOCK_70B]
+
+
+def make_block_layer(i: int, *, seed_offset: int = 0) -> SynthLayer:
+    """Layer i of the 70B block (its own seed family, so no two layers share weights or codebooks)."""
+    name, rows, cols, M, K, f16, rowmax = block_layer_shapes()[i]
+    return make_layer(rows, cols, cfg=BLOCK_SEED_BASE + i + seed_offset, num_codebooks=M, codebook_size=K,
+                      codebook_fp16=f16, row_max_scale=rowmax, name=f"llama2_70b_{name}_{rows}x{cols}_1x16")
+
+
 def make_config_layer(cfg: int, which: int = 0, *, nearest=None) -> SynthLayer:
     name, rows, cols, M, K, f16, rowmax, _ = CONFIGS[cfg][which]
     return make_layer(rows, cols, cfg=cfg, num_codebooks=M, codebook_size=K, codebook_fp16=f16,

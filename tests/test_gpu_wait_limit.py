@@ -27,7 +27,7 @@ pytestmark = pytest.mark.gpu
     ("fp32", 65536, 0),
 ])
 def test_a_wait_that_runs_out_is_reported_and_the_next_call_is_correct(engine, K, withhold):
-    L = synth.make_layer(256, 1024, cfg=61, codebook_size=K, codebook_fp16=True)
+    L = synth.make_layer(1024, 1024, cfg=61, codebook_size=K, codebook_fp16=True)
     k = 3000
     idx_np = oracle.select(oracle.group_norms(L.g, L.eta), k)
     idx = torch.from_numpy(idx_np.astype(np.int32)).cuda()
