@@ -574,3 +574,93 @@ int pvt_oracle_local_search(const float* t, int64_t k, int32_t dg, int32_t M, in
   }
   return bad ? -1 : 0;
 }
+
+/* ---- straight-through buffer (Appendix E; Section 3.4 and the "PV + STE" rows of Table 1) -------------------
+ * Straight-through estimation keeps an auxiliary, non-quantised copy of the weights.  Every step moves it by the
+ * update computed at the quantised weights, and the codes are then chosen to approximate the buffer: updates that
+ * are too small to change a code are not lost but add up in the buffer until the stored code stops being the
+ * nearest one.  Combined with the subspace V step (the reading taken here): the buffer takes the step of every
+ * weight, the subspace is still chosen by the size of this step's update, and the chosen groups are re-encoded
+ * against the buffer (the V step's search with W := buffer and a zero step).
+ *     buffer_i = fmaf(-eta, g_i, buffer_i)        binary32, one fused operation per weight
+ * Pins: a scalar example worked by hand in which four equal small updates flip a code that the plain V step
+ * (which restarts from the dequantised weight every time) never flips; eta = 0 leaves the buffer bit for bit;
+ * exact rationals for single elements.
+ */
+void pvt_oracle_ste_accumulate(float* buffer, const float* g, int64_t n, float eta) {
+  for (int64_t i = 0; i < n; ++i) buffer[i] = fmaf(-eta, g[i], buffer[i]);
+}
+
+/* ---- random subspaces (appendix on small-scale experiments: besides the greedy choice, subspaces drawn
+ * uniformly at random, or at random in proportion to the size of the gradient entries) ----------------------
+ * Every group j gets a 32-bit random word from a counter-based generator, Philox-4x32 with 10 rounds (Salmon,
+ * Moraes, Dror, Shaw: "Parallel random numbers: as easy as 1, 2, 3", SC 2011): counter (j mod 2^32, j div 2^32,
+ * 0, 0), key (seed mod 2^32, seed div 2^32), first output word r_j.  The k groups with the largest sampling key
+ * are taken, ties towards the lowest index (the same selection rule as the greedy choice):
+ *   uniform:       key_j = (float)(r_j >> 8)                  (24 random bits, exact in binary32): a uniformly
+ *                  random k-subset.
+ *   proportional:  key_j = (float)(w_j / E_j),  E_j = -ln u_j,  u_j = (r_j + 1/2) 2^-32,  w_j = the group's
+ *                  squared update norm: the groups with the k earliest arrivals of independent exponential
+ *                  clocks of rates w_j, i.e. k draws without replacement, each in proportion to w among the
+ *                  groups not yet drawn (Efraimidis and Spirakis, "Weighted random sampling with a reservoir",
+ *                  2006).  Groups of weight 0 get key 0.
+ * -ln u is evaluated by a fixed sequence of binary64 operations so that it can be reproduced bit for bit:
+ *   x = r + 1/2 = m 2^e with m in [1, 2); if m > sqrt 2: m = m/2, e = e + 1;  z = (m - 1)/(m + 1);
+ *   p = 1 + z^2/3 + ... + z^20/21 by Horner's rule in z^2 with one fused operation per coefficient;
+ *   E = fma(32 - e, ln 2, -(2z * p)).
+ * Pins: the generator's published known-answer vectors; E against the C library's logarithm; a k-subset of
+ * distinct indices for every k; k = G; inclusion frequencies over many seeds against k/G (uniform) and against
+ * w_j / sum w for k = 1 (proportional) within binomial bounds; zero weights never drawn; equal weights behave
+ * like the uniform rule in distribution.
+ */
+void pvt_oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]) {
+  uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3], k0 = key[0], k1 = key[1];
+  for (int round = 0; round < 10; ++round) {
+    const uint64_t p0 = (uint64_t)0xD2511F53u * c0, p1 = (uint64_t)0xCD9E8D57u * c2;
+    const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0, n1 = (uint32_t)p1;
+    const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1, n3 = (uint32_t)p0;
+    c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+/* -ln((r + 1/2) 2^-32), the fixed binary64 sequence described above */
+double pvt_oracle_neglog_u32(uint32_t r) {
+  int e = -1;
+  if (r) {
+    e = 31;
+    while (!(r >> e)) --e;
+  }
+  double m = ldexp((double)r + 0.5, -e); /* exact: in [1, 2) */
+  if (m > 1.4142135623730951) {
+    m = m * 0.5;
+    e = e + 1;
+  }
+  const double z = (m - 1.0) / (m + 1.0), z2 = z * z;
+  double p = 1.0 / 21.0;
+  for (int d = 19; d >= 1; d -= 2) p = fma(p, z2, 1.0 / (double)d);
+  const double lnm = (2.0 * z) * p;
+  return fma((double)(32 - e), 0.6931471805599453, -lnm);
+}
+
+/* Sampling keys of all G groups.  mode 0: uniform; mode 1: proportional to norms[j] (binary32, >= 0). */
+int pvt_oracle_sample_keys(const float* norms, int64_t G, int32_t mode, uint64_t seed, float* keys_out) {
+  if (mode != 0 && mode != 1) return -1;
+  if (mode == 1 && !norms) return -1;
+  const uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+  for (int64_t j = 0; j < G; ++j) {
+    const uint32_t ctr[4] = {(uint32_t)j, (uint32_t)((uint64_t)j >> 32), 0u, 0u};
+    uint32_t out[4];
+    pvt_oracle_philox4x32_10(ctr, key, out);
+    if (mode == 0) {
+      keys_out[j] = (float)(out[0] >> 8);
+    } else {
+      const float w = norms[j];
+      if (!(w >= 0.0f) || !isfinite(w)) return -1;
+      keys_out[j] = w > 0.0f ? (float)((double)w / pvt_oracle_neglog_u32(out[0])) : 0.0f;
+    }
+  }
+  return 0;
+}

@@ -42,6 +42,9 @@ def lib():
         L.pvt_oracle_encode.restype = ctypes.c_int
         L.pvt_oracle_rank.restype = ctypes.c_int
         L.pvt_oracle_local_search.restype = ctypes.c_int
+        L.pvt_oracle_sample_keys.restype = ctypes.c_int
+        L.pvt_oracle_neglog_u32.restype = ctypes.c_double
+        L.pvt_oracle_neglog_u32.argtypes = [ctypes.c_uint32]
         _lib = L
     return _lib
 
@@ -350,3 +353,61 @@ def local_search(t, codebooks, codes, max_moves: int = 64):
     if rc != 0:
         raise ValueError("pvt_oracle_local_search rejected its arguments")
     return out, d, moves
+
+
+SAMPLE_UNIFORM, SAMPLE_PROPORTIONAL = 0, 1
+
+
+def ste_accumulate(buffer, g, eta: float) -> np.ndarray:
+    """Straight-through buffer after one step: fmaf(-eta, g, buffer) per weight (Appendix E); returns a new array."""
+    out = np.ascontiguousarray(buffer, dtype=np.float32).copy()
+    g = _f32(g)
+    assert out.shape == g.shape
+    lib().pvt_oracle_ste_accumulate(_p(out, ctypes.c_float), _p(g, ctypes.c_float), ctypes.c_int64(out.size),
+                                    ctypes.c_float(eta))
+    return out
+
+
+def philox4x32_10(ctr, key) -> np.ndarray:
+    """One block of the Philox-4x32-10 generator: four 32-bit words."""
+    c = np.ascontiguousarray(ctr, dtype=np.uint32)
+    k = np.ascontiguousarray(key, dtype=np.uint32)
+    assert c.size == 4 and k.size == 2
+    out = np.zeros(4, dtype=np.uint32)
+    lib().pvt_oracle_philox4x32_10(_p(c, ctypes.c_uint32), _p(k, ctypes.c_uint32), _p(out, ctypes.c_uint32))
+    return out
+
+
+def neglog_u32(r: int) -> float:
+    """-ln((r + 1/2) 2^-32) by the sampler's fixed binary64 sequence."""
+    return float(lib().pvt_oracle_neglog_u32(ctypes.c_uint32(r)))
+
+
+def sample_keys(num_groups: int, mode: int, seed: int, norms=None) -> np.ndarray:
+    """Sampling keys (binary32, >= 0) of every group for the random subspace rules."""
+    keys = np.empty(num_groups, dtype=np.float32)
+    nptr = None
+    if norms is not None:
+        norms = _f32(norms)
+        assert norms.size == num_groups
+        nptr = _p(norms, ctypes.c_float)
+    rc = lib().pvt_oracle_sample_keys(nptr, ctypes.c_int64(num_groups), ctypes.c_int32(mode), ctypes.c_uint64(seed),
+                                      _p(keys, ctypes.c_float))
+    if rc != 0:
+        raise ValueError("pvt_oracle_sample_keys rejected its arguments")
+    return keys
+
+
+def sample_subspace(num_groups: int, k: int, mode: int, seed: int, norms=None) -> np.ndarray:
+    """A random subspace of k groups (uniform, or in proportion to the squared update norms), ascending uint32 [k]."""
+    return select(sample_keys(num_groups, mode, seed, norms), k)
+
+
+def vstep_ste(buffer, g, scale, codebooks, codes, eta: float, k: int, beam: int = 8):
+    """Subspace V step combined with a straight-through buffer: the buffer takes the whole step, the subspace is
+    chosen by the size of this step's update, the chosen groups are re-encoded against the buffer.  Returns
+    (new buffer, VStepResult)."""
+    dg = np.asarray(codebooks).shape[2]
+    new_buffer = ste_accumulate(buffer, g, eta)
+    idx = select(group_norms(g, eta, dg), k)
+    return new_buffer, vstep(new_buffer, g, scale, codebooks, codes, 0.0, k, beam, idx=idx)
