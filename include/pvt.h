@@ -167,6 +167,47 @@ int pvt_vstep_select_noalloc(const pvt_layer* layer, uint64_t k, uint32_t* idx_o
                              void* cuda_stream);
 
 /*
+ * Subspace choice combined with a straight-through buffer (Appendix E: an auxiliary, non-quantised
+ * copy of the weights that takes every update, so that updates too small to change a code add up
+ * until they do; Section 3.4 and the "PV + STE" rows of Table 1 combine it with the subspace V step).
+ * One pass over g does both:
+ *   buffer[r, c] = fma(-eta, g[r, c], buffer[r, c])   for every weight (binary32, one fused operation),
+ *   idx_out      = exactly what pvt_vstep_select returns (the k groups of largest ||eta g_j||^2).
+ * The V step is then completed by pvt_vstep_encode on a descriptor with W = buffer and eta = 0: the
+ * chosen groups are re-encoded against buffer / scale.  (Reading of the paper, which does not spell
+ * the combination out: the buffer takes the step of every weight, the subspace is chosen by the size
+ * of this step's update.)
+ * buffer: device, rows x cols floats, 16-byte aligned, updated in place, must not alias g.  With
+ * k = G the buffer is still updated.  Other arguments, workspace and return codes as pvt_vstep_select.
+ */
+int pvt_vstep_select_ste(const pvt_layer* layer, float* buffer, uint64_t k, uint32_t* idx_out, void* ws,
+                         size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Random subspaces (the small-scale experiments' appendix: instead of the greedy choice, S^k drawn
+ * uniformly at random, or at random in proportion to the size of the gradient entries).  Every group
+ * j gets the first output word r_j of the counter-based generator Philox-4x32 with 10 rounds (Salmon,
+ * Moraes, Dror, Shaw, SC 2011) at counter (j mod 2^32, j div 2^32, 0, 0) and key (seed mod 2^32, seed
+ * div 2^32); the k groups with the largest sampling key are returned in ascending order, ties towards
+ * the lowest index:
+ *   PVT_SAMPLE_UNIFORM       key_j = (float)(r_j >> 8): a uniformly random k-subset; g is not read.
+ *   PVT_SAMPLE_PROPORTIONAL  key_j = (float)(n_j / E_j), n_j = ||eta g_j||^2 as in pvt_vstep_select,
+ *                            E_j = -ln((r_j + 1/2) 2^-32): k draws without replacement, each in
+ *                            proportion to n_j among the groups not yet drawn (exponential clocks);
+ *                            groups with n_j = 0 get key 0.  E_j is a fixed sequence of binary64
+ *                            operations (x = r + 1/2 = m 2^e, m in [1, 2), halved when above sqrt 2;
+ *                            z = (m - 1)/(m + 1); p = 1 + z^2/3 + ... + z^20/21 by Horner's rule with
+ *                            one fused operation per coefficient; E = fma(32 - e, ln 2, -(2 z p))),
+ *                            the quotient is taken in binary64 and rounded once to binary32.
+ * The same seed gives the same subspace on every device and run.  Workspace, idx_out and return
+ * codes as pvt_vstep_select; PVT_EINVAL for an unknown rule.
+ */
+#define PVT_SAMPLE_UNIFORM 0
+#define PVT_SAMPLE_PROPORTIONAL 1
+int pvt_vstep_sample(const pvt_layer* layer, uint64_t k, int32_t rule, uint64_t seed, uint32_t* idx_out, void* ws,
+                     size_t ws_bytes, void* cuda_stream);
+
+/*
  * Re-encode the k groups listed in idx (Eq. 8; Appendix C / Appendix J;
  * Appendix D for the score ||c||^2 - 2 <t, c>).
  *   target (binary32): t_i = fma(-eta, g_i, W_i) / scale[r].

@@ -25,6 +25,7 @@ PVT_KERNEL_SELECT, PVT_KERNEL_ENCODE_MAIN, PVT_KERNEL_ENCODE_AUX, PVT_KERNEL_DEQ
 PVT_KERNEL_ENCODE_RESCORE = 4
 PVT_KERNEL_PSTEP_GRAD, PVT_KERNEL_ADAM, PVT_KERNEL_TRUST, PVT_KERNEL_REFINE = 5, 6, 7, 8
 PVT_M1_AUTO, PVT_M1_FP32, PVT_M1_TENSOR = 0, 1, 2
+PVT_SAMPLE_UNIFORM, PVT_SAMPLE_PROPORTIONAL = 0, 1
 
 
 class pvt_layer(ctypes.Structure):
@@ -74,6 +75,10 @@ def lib():
         L.pvt_vstep_select.argtypes = [lp, u64, vp, vp, sz, vp]
         L.pvt_vstep_select_noalloc.restype = ctypes.c_int
         L.pvt_vstep_select_noalloc.argtypes = [lp, u64, vp, vp, vp]
+        L.pvt_vstep_select_ste.restype = ctypes.c_int
+        L.pvt_vstep_select_ste.argtypes = [lp, vp, u64, vp, vp, sz, vp]
+        L.pvt_vstep_sample.restype = ctypes.c_int
+        L.pvt_vstep_sample.argtypes = [lp, u64, ctypes.c_int32, u64, vp, vp, sz, vp]
         L.pvt_vstep_encode.restype = ctypes.c_int
         L.pvt_vstep_encode.argtypes = [lp, vp, u64, vp, vp, sz, vp]
         L.pvt_trust_workspace_bytes.restype = sz
@@ -182,6 +187,23 @@ def pvt_vstep_select_noalloc(layer: pvt_layer, k: int, idx_out: torch.Tensor,
     calls that could overlap on the GPU must be ordered by the caller."""
     _check(lib().pvt_vstep_select_noalloc(ctypes.byref(layer), k, idx_out.data_ptr(), _ptr(status_out),
                                           _stream_ptr(stream)), "pvt_vstep_select_noalloc")
+
+
+def pvt_vstep_select_ste(layer: pvt_layer, buffer: torch.Tensor, k: int, idx_out: torch.Tensor, ws: torch.Tensor,
+                         stream=None) -> None:
+    """pvt_vstep_select that also lets the straight-through buffer (float32 [rows, cols], in place) take the
+    step -eta * g (Appendix E)."""
+    if buffer.dtype != torch.float32 or not buffer.is_cuda or not buffer.is_contiguous():
+        raise ValueError("buffer must be a contiguous float32 CUDA tensor")
+    _check(lib().pvt_vstep_select_ste(ctypes.byref(layer), buffer.data_ptr(), k, idx_out.data_ptr(), ws.data_ptr(),
+                                      ws.numel() * ws.element_size(), _stream_ptr(stream)), "pvt_vstep_select_ste")
+
+
+def pvt_vstep_sample(layer: pvt_layer, k: int, rule: int, seed: int, idx_out: torch.Tensor, ws: torch.Tensor,
+                     stream=None) -> None:
+    """A random subspace of k groups: PVT_SAMPLE_UNIFORM or PVT_SAMPLE_PROPORTIONAL (to the squared update norm)."""
+    _check(lib().pvt_vstep_sample(ctypes.byref(layer), k, rule, seed, idx_out.data_ptr(), ws.data_ptr(),
+                                  ws.numel() * ws.element_size(), _stream_ptr(stream)), "pvt_vstep_sample")
 
 
 def pvt_vstep_encode(layer: pvt_layer, idx: torch.Tensor, k: int, err_out: Optional[torch.Tensor],

@@ -183,6 +183,39 @@ int pvt_vstep_select(const pvt_layer* layer, uint64_t k, uint32_t* idx_out, void
   return e == cudaSuccess ? PVT_OK : fail_cuda(e);
 }
 
+int pvt_vstep_select_ste(const pvt_layer* layer, float* buffer, uint64_t k, uint32_t* idx_out, void* ws,
+                         size_t ws_bytes, void* cuda_stream) {
+  uint64_t G = 0;
+  int rc = check_layer(layer, &G);
+  if (rc != PVT_OK) return rc;
+  if (k < 1 || k > G) return PVT_EINVAL;
+  if (!layer->g || !aligned16(layer->g) || !buffer || !aligned16(buffer) || !idx_out || !aligned4(idx_out) || !ws)
+    return PVT_EINVAL;
+  if (static_cast<const void*>(buffer) == static_cast<const void*>(layer->g)) return PVT_EINVAL;
+  if (reinterpret_cast<uintptr_t>(ws) & (kWsAlign - 1)) return PVT_EINVAL;
+  if (ws_bytes < select_layout(G).bytes) return PVT_EWORKSPACE;
+  const cudaError_t e = launch_select_keyed(*layer, G, k, idx_out, ws, sm_count(),
+                                            static_cast<cudaStream_t>(cuda_stream), 1, buffer, 0);
+  return e == cudaSuccess ? PVT_OK : fail_cuda(e);
+}
+
+int pvt_vstep_sample(const pvt_layer* layer, uint64_t k, int32_t rule, uint64_t seed, uint32_t* idx_out, void* ws,
+                     size_t ws_bytes, void* cuda_stream) {
+  uint64_t G = 0;
+  int rc = check_layer(layer, &G);
+  if (rc != PVT_OK) return rc;
+  if (rule != PVT_SAMPLE_UNIFORM && rule != PVT_SAMPLE_PROPORTIONAL) return PVT_EINVAL;
+  if (k < 1 || k > G) return PVT_EINVAL;
+  if (rule == PVT_SAMPLE_PROPORTIONAL && (!layer->g || !aligned16(layer->g))) return PVT_EINVAL;
+  if (!idx_out || !aligned4(idx_out) || !ws) return PVT_EINVAL;
+  if (reinterpret_cast<uintptr_t>(ws) & (kWsAlign - 1)) return PVT_EINVAL;
+  if (ws_bytes < select_layout(G).bytes) return PVT_EWORKSPACE;
+  const cudaError_t e = launch_select_keyed(*layer, G, k, idx_out, ws, sm_count(),
+                                            static_cast<cudaStream_t>(cuda_stream),
+                                            rule == PVT_SAMPLE_UNIFORM ? 2 : 3, nullptr, seed);
+  return e == cudaSuccess ? PVT_OK : fail_cuda(e);
+}
+
 int pvt_vstep_encode(const pvt_layer* layer, const uint32_t* idx, uint64_t k, float* err_out, void* ws,
                      size_t ws_bytes, void* cuda_stream) {
   uint64_t G = 0;

@@ -104,6 +104,10 @@ EncodeM1TcLayout encode_m1_tc_layout(uint32_t K, uint64_t k, int sm_count, int g
 // launchers (each returns a cudaError_t) --------------------------------------
 cudaError_t launch_select(const pvt_layer& L, uint64_t G, uint64_t k, uint32_t* idx_out, void* ws, int sm_count,
                           cudaStream_t stream);
+// the same selection on other keys: 0 squared update norm, 1 the same while a straight-through buffer takes the
+// step, 2 uniformly random keys, 3 keys of a draw in proportion to the squared update norm (seeded)
+cudaError_t launch_select_keyed(const pvt_layer& L, uint64_t G, uint64_t k, uint32_t* idx_out, void* ws, int sm_count,
+                                cudaStream_t stream, int key_mode, float* buffer, uint64_t seed);
 cudaError_t launch_encode_m1(const pvt_layer& L, uint64_t G, const uint32_t* idx, uint64_t k, float* err_out,
                              void* ws, int sm_count, cudaStream_t stream);
 cudaError_t launch_encode_m1_tc(const pvt_layer& L, uint64_t G, const uint32_t* idx, uint64_t k, float* err_out,

@@ -115,10 +115,57 @@ __device__ __forceinline__ float norm_chain(float acc, const float4& a, float et
   return acc;
 }
 
-template <int LP>
+// ---- random subspace rules (appendix on small-scale experiments: subspaces drawn uniformly at random, or at
+// random in proportion to the size of the gradient entries) --------------------------------------------------
+// Every group gets the first output word of Philox-4x32 with 10 rounds (Salmon et al., SC 2011) at counter
+// (j mod 2^32, j div 2^32, 0, 0) under the key (seed mod 2^32, seed div 2^32).
+__device__ __forceinline__ uint32_t philox_first_word(uint64_t j, uint64_t seed) {
+  uint32_t c0 = (uint32_t)j, c1 = (uint32_t)(j >> 32), c2 = 0u, c3 = 0u;
+  uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
+#pragma unroll
+  for (int round = 0; round < 10; ++round) {
+    const uint32_t h0 = __umulhi(0xD2511F53u, c0), l0 = 0xD2511F53u * c0;
+    const uint32_t h1 = __umulhi(0xCD9E8D57u, c2), l1 = 0xCD9E8D57u * c2;
+    const uint32_t n0 = h1 ^ c1 ^ k0, n2 = h0 ^ c3 ^ k1;
+    c0 = n0; c1 = l1; c2 = n2; c3 = l0;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  return c0;
+}
+
+// E = -ln((r + 1/2) 2^-32) by a fixed sequence of binary64 operations (each rounded once, none contracted):
+// r + 1/2 = m 2^e, m in [1, 2), m halved and e raised when m > sqrt 2; z = (m - 1)/(m + 1);
+// p = 1 + z^2/3 + ... + z^20/21 by Horner's rule, one fused operation per coefficient; E = fma(32 - e, ln 2, -(2z p)).
+__device__ __forceinline__ double neglog_u32(uint32_t r) {
+  int e = r ? 31 - __clz((int)r) : -1;
+  // (r + 1/2) 2^-e, exact: the significand of r + 1/2 with the exponent field set to that of 1.0
+  const double x = __dadd_rn((double)r, 0.5);
+  double m = __longlong_as_double((__double_as_longlong(x) & 0x000fffffffffffffll) | 0x3ff0000000000000ll);
+  if (m > 1.4142135623730951) {
+    m = __dmul_rn(m, 0.5);
+    e = e + 1;
+  }
+  const double z = __ddiv_rn(__dadd_rn(m, -1.0), __dadd_rn(m, 1.0)), z2 = __dmul_rn(z, z);
+  double p = 1.0 / 21.0;
+#pragma unroll
+  for (int d = 19; d >= 1; d -= 2) p = __fma_rn(p, z2, 1.0 / (double)d);
+  const double lnm = __dmul_rn(__dmul_rn(2.0, z), p);
+  return __fma_rn((double)(32 - e), 0.6931471805599453, -lnm);
+}
+
+// What the first pass computes per group (everything after the keys is the same top-k):
+//   kKeyNorm          key = squared update norm (the greedy rule of the V step)
+//   kKeyNormBuffer    the same, and the straight-through buffer takes the step: buffer = fma(-eta, g, buffer)
+//   kKeyUniform       key = the top 24 bits of the group's random word, as a binary32 number
+//   kKeyProportional  key = (float)(norm / E), E the exponential clock of the group's random word
+enum KeyMode { kKeyNorm = 0, kKeyNormBuffer = 1, kKeyUniform = 2, kKeyProportional = 3 };
+
+template <int LP, int MODE>
 __global__ void __launch_bounds__(kSelThreads) norm_hist_kernel(const float* __restrict__ g, uint64_t G, float eta,
                                                                  uint64_t k, uint32_t* __restrict__ keys,
-                                                                 uint32_t* __restrict__ hist0, SelectState* st) {
+                                                                 uint32_t* __restrict__ hist0, SelectState* st,
+                                                                 float* __restrict__ buffer, uint64_t seed) {
   pdl_trigger();
   pdl_wait();
   constexpr int kTile = kSelThreads * kNormPer / LP;  // groups per block and iteration
@@ -127,6 +174,7 @@ __global__ void __launch_bounds__(kSelThreads) norm_hist_kernel(const float* __r
   for (int b = threadIdx.x; b < kSelBins0; b += kSelThreads) sh_hist[b] = 0;
   __syncthreads();
   const float4* g4 = reinterpret_cast<const float4*>(g);
+  float4* buf4 = reinterpret_cast<float4*>(buffer);
   const uint64_t F = (uint64_t)LP * G;  // 16-byte pieces
   const uint32_t n_tiles = (uint32_t)((G + kTile - 1) / kTile);
   const int q = threadIdx.x & (LP - 1);  // position of this lane within its group
@@ -136,7 +184,23 @@ __global__ void __launch_bounds__(kSelThreads) norm_hist_kernel(const float* __r
 #pragma unroll
     for (int i = 0; i < kNormPer; ++i) {  // all loads of the iteration first
       const uint64_t f = f0 + (uint64_t)i * kSelThreads;
-      a[i] = f < F ? __ldcs(g4 + f) : make_float4(0.f, 0.f, 0.f, 0.f);
+      a[i] = (MODE != kKeyUniform && f < F) ? __ldcs(g4 + f) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    if (MODE == kKeyNormBuffer) {  // the straight-through buffer takes the step of every weight (Appendix E)
+      float4 b[kNormPer];
+#pragma unroll
+      for (int i = 0; i < kNormPer; ++i) {
+        const uint64_t f = f0 + (uint64_t)i * kSelThreads;
+        b[i] = f < F ? __ldcs(buf4 + f) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+      const float neg_eta = -eta;
+#pragma unroll
+      for (int i = 0; i < kNormPer; ++i) {
+        const uint64_t f = f0 + (uint64_t)i * kSelThreads;
+        if (f < F)
+          __stcs(buf4 + f, make_float4(__fmaf_rn(neg_eta, a[i].x, b[i].x), __fmaf_rn(neg_eta, a[i].y, b[i].y),
+                                       __fmaf_rn(neg_eta, a[i].z, b[i].z), __fmaf_rn(neg_eta, a[i].w, b[i].w)));
+      }
     }
 #pragma unroll
     for (int i = 0; i < kNormPer; ++i) {
@@ -149,7 +213,12 @@ __global__ void __launch_bounds__(kSelThreads) norm_hist_kernel(const float* __r
         acc = q >= r ? next : acc;
       }
       if (q == LP - 1 && f < F) {
-        const uint32_t key = __float_as_uint(acc);
+        uint32_t key = __float_as_uint(acc);
+        if (MODE == kKeyUniform) key = __float_as_uint((float)(philox_first_word(f / LP, seed) >> 8));
+        if (MODE == kKeyProportional)
+          key = acc > 0.0f ? __float_as_uint(__double2float_rn(
+                                 __ddiv_rn((double)acc, neglog_u32(philox_first_word(f / LP, seed)))))
+                           : 0u;
         keys[f / LP] = key;
         atomicAdd(&sh_hist[key >> 20], 1u);
       }
@@ -403,11 +472,46 @@ __global__ void iota_kernel(uint32_t* idx_out, uint64_t k) {
 
 }  // namespace
 
+namespace {
+
+template <int LP, int MODE>
+cudaError_t launch_norm(const pvt_layer& L, uint64_t G, uint64_t k, uint32_t* keys, uint32_t* hist0, SelectState* st,
+                        float* buffer, uint64_t seed, int sm_count, cudaStream_t stream) {
+  int per_sm = 0;
+  cudaError_t err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, norm_hist_kernel<LP, MODE>, kSelThreads, 0);
+  if (err != cudaSuccess) return err;
+  const uint64_t tile = (uint64_t)kSelThreads * kNormPer / LP;
+  const uint64_t tiles = (G + tile - 1) / tile;
+  const uint64_t resident = (uint64_t)sm_count * (uint64_t)(per_sm > 0 ? per_sm : 1);  // a persistent grid
+  norm_hist_kernel<LP, MODE><<<(unsigned)(tiles < resident ? tiles : resident), kSelThreads, 0, stream>>>(
+      L.g, G, L.eta, k, keys, hist0, st, buffer, seed);
+  return cudaGetLastError();
+}
+
+template <int LP>
+cudaError_t launch_norm_mode(int mode, const pvt_layer& L, uint64_t G, uint64_t k, uint32_t* keys, uint32_t* hist0,
+                             SelectState* st, float* buffer, uint64_t seed, int sm_count, cudaStream_t stream) {
+  switch (mode) {
+    case kKeyNormBuffer: return launch_norm<LP, kKeyNormBuffer>(L, G, k, keys, hist0, st, buffer, seed, sm_count, stream);
+    case kKeyUniform: return launch_norm<LP, kKeyUniform>(L, G, k, keys, hist0, st, buffer, seed, sm_count, stream);
+    case kKeyProportional:
+      return launch_norm<LP, kKeyProportional>(L, G, k, keys, hist0, st, buffer, seed, sm_count, stream);
+    default: return launch_norm<LP, kKeyNorm>(L, G, k, keys, hist0, st, buffer, seed, sm_count, stream);
+  }
+}
+
+}  // namespace
+
 cudaError_t launch_select(const pvt_layer& L, uint64_t G, uint64_t k, uint32_t* idx_out, void* ws, int sm_count,
                           cudaStream_t stream) {
+  return launch_select_keyed(L, G, k, idx_out, ws, sm_count, stream, kKeyNorm, nullptr, 0);
+}
+
+cudaError_t launch_select_keyed(const pvt_layer& L, uint64_t G, uint64_t k, uint32_t* idx_out, void* ws, int sm_count,
+                                cudaStream_t stream, int key_mode, float* buffer, uint64_t seed) {
   timing_begin(kKernSelect, stream);
   cudaError_t err = cudaSuccess;
-  if (k == G) {  // every group is taken: the ascending index list itself
+  if (k == G && key_mode != kKeyNormBuffer) {  // every group is taken: the ascending index list itself
     iota_kernel<<<(unsigned)((k + 255) / 256), 256, 0, stream>>>(idx_out, k);
     err = cudaGetLastError();
     count_launches(1);
@@ -431,26 +535,16 @@ cudaError_t launch_select(const pvt_layer& L, uint64_t G, uint64_t k, uint32_t* 
     return err;
   uint32_t* cand = reinterpret_cast<uint32_t*>(base + lay.cand_off);
   // persistent grids: exactly the blocks that are resident at once
-  int norm_per_sm = 0, mid_per_sm = 0;
-  const int lp = L.group_dim / 4;  // lanes per group in the norm pass: 2 or 4
-  if ((err = (lp == 2 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&norm_per_sm, norm_hist_kernel<2>, kSelThreads, 0)
-                      : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&norm_per_sm, norm_hist_kernel<4>, kSelThreads,
-                                                                      0))) !=
-          cudaSuccess ||
-      (err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&mid_per_sm, refine_mid_kernel, kSelThreads, 0)) !=
-          cudaSuccess)
+  int mid_per_sm = 0;
+  if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&mid_per_sm, refine_mid_kernel, kSelThreads, 0)) !=
+      cudaSuccess)
     return err;
-  const uint64_t norm_tile = (uint64_t)kSelThreads * kNormPer / lp;
-  const uint64_t norm_tiles = (G + norm_tile - 1) / norm_tile;
-  const uint64_t norm_res = (uint64_t)sm_count * (uint64_t)(norm_per_sm > 0 ? norm_per_sm : 1);
-  const unsigned norm_grid = (unsigned)(norm_tiles < norm_res ? norm_tiles : norm_res);
   const uint64_t quad_blocks = ((G + 3) / 4 + 2 * kSelThreads - 1) / (2 * kSelThreads);
   const uint64_t mid_res = (uint64_t)sm_count * (uint64_t)(mid_per_sm > 0 ? mid_per_sm : 1);
   const unsigned mid_grid = (unsigned)(quad_blocks < mid_res ? quad_blocks : mid_res);
-  if (lp == 2)
-    norm_hist_kernel<2><<<norm_grid, kSelThreads, 0, stream>>>(L.g, G, L.eta, k, keys, hist0, st);
-  else
-    norm_hist_kernel<4><<<norm_grid, kSelThreads, 0, stream>>>(L.g, G, L.eta, k, keys, hist0, st);
+  err = L.group_dim == 16 ? launch_norm_mode<4>(key_mode, L, G, k, keys, hist0, st, buffer, seed, sm_count, stream)
+                          : launch_norm_mode<2>(key_mode, L, G, k, keys, hist0, st, buffer, seed, sm_count, stream);
+  if (err != cudaSuccess) return err;
   err = launch_dependent(refine_mid_kernel, mid_grid, kSelThreads, 0, stream, keys, G, hist1, cand, lay.cand_cap, st);
   if (err != cudaSuccess) return err;
   const unsigned low_grid = (unsigned)(lay.cand_cap / 8192 < (uint32_t)sm_count ? lay.cand_cap / 8192 + 1 : sm_count);

@@ -56,6 +56,29 @@ class VStepLayer:
         B.pvt_vstep_select(self.desc, k, idx_out, ws)
         return idx_out
 
+    def select_ste(self, buffer: torch.Tensor, k: int, idx_out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """Selection while the straight-through buffer takes the step (Appendix E): buffer -= eta * g in place."""
+        ws = self.reserve(k)
+        if idx_out is None:
+            idx_out = torch.empty(k, dtype=torch.int32, device=self.W.device)
+        B.pvt_vstep_select_ste(self.desc, buffer, k, idx_out, ws)
+        return idx_out
+
+    def sample(self, k: int, rule: int, seed: int, idx_out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """A random subspace (B.PVT_SAMPLE_UNIFORM / B.PVT_SAMPLE_PROPORTIONAL) instead of the greedy one."""
+        ws = self.reserve(k)
+        if idx_out is None:
+            idx_out = torch.empty(k, dtype=torch.int32, device=self.W.device)
+        B.pvt_vstep_sample(self.desc, k, rule, seed, idx_out, ws)
+        return idx_out
+
+    def encode_against(self, buffer: torch.Tensor, idx: torch.Tensor, err_out: Optional[torch.Tensor] = None) -> None:
+        """Re-encode the listed groups against buffer / scale (the V step's search with W = buffer, zero step)."""
+        k = int(idx.numel())
+        desc = B.make_layer(self.rows, self.cols, buffer, self.g, self.scale, self.codebooks, self.codes, eta=0.0,
+                            beam=self.beam, group_dim=self.group_dim)
+        B.pvt_vstep_encode(desc, idx, k, err_out, self.reserve(k))
+
     def encode(self, idx: torch.Tensor, err_out: Optional[torch.Tensor] = None) -> None:
         k = int(idx.numel())
         B.pvt_vstep_encode(self.desc, idx, k, err_out, self.reserve(k))

@@ -121,3 +121,19 @@ def test_adam_bias_is_computed_in_the_library_and_equals_the_checkers():
     assert B.lib().pvt_adam_bias(0, 0.9, 0.95, ctypes.byref(b1), ctypes.byref(b2)) == B.PVT_EINVAL
     assert B.lib().pvt_adam_bias(3, 1.0, 0.95, ctypes.byref(b1), ctypes.byref(b2)) == B.PVT_EINVAL
     assert B.lib().pvt_adam_bias(3, 0.9, 0.95, None, ctypes.byref(b2)) == B.PVT_EINVAL
+
+
+def test_buffer_and_sampling_calls_reject_bad_arguments():
+    L = _layer()
+    lib = B.lib()
+    big = 1 << 30
+    assert lib.pvt_vstep_select_ste(ctypes.byref(L), None, 4, 0x2000, 0x4000, big, None) == B.PVT_EINVAL
+    assert lib.pvt_vstep_select_ste(ctypes.byref(L), 0x3004, 4, 0x2000, 0x4000, big, None) == B.PVT_EINVAL  # alignment
+    assert lib.pvt_vstep_select_ste(ctypes.byref(L), 0x1000, 4, 0x2000, 0x4000, big, None) == B.PVT_EINVAL  # buffer == g
+    assert lib.pvt_vstep_select_ste(ctypes.byref(L), 0x3000, 0, 0x2000, 0x4000, big, None) == B.PVT_EINVAL
+    assert lib.pvt_vstep_select_ste(ctypes.byref(L), 0x3000, 4, 0x2000, 0x4000, 256, None) == B.PVT_EWORKSPACE
+    assert lib.pvt_vstep_sample(ctypes.byref(L), 4, 7, 1, 0x2000, 0x4000, big, None) == B.PVT_EINVAL  # unknown rule
+    assert lib.pvt_vstep_sample(ctypes.byref(L), 0, B.PVT_SAMPLE_UNIFORM, 1, 0x2000, 0x4000, big, None) == B.PVT_EINVAL
+    assert lib.pvt_vstep_sample(ctypes.byref(_layer(g=None)), 4, B.PVT_SAMPLE_PROPORTIONAL, 1, 0x2000, 0x4000, big,
+                                None) == B.PVT_EINVAL
+    assert lib.pvt_vstep_sample(ctypes.byref(L), 4, B.PVT_SAMPLE_UNIFORM, 1, 0x2000, 0x4000, 256, None) == B.PVT_EWORKSPACE
