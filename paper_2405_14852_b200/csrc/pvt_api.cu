@@ -135,7 +135,7 @@ namespace {
 
 // workspace of pvt_vstep_encode for k groups of this layer
 size_t encode_bytes(const pvt_layer& L, uint64_t k, int sms) {
-  if (L.num_codebooks >= 3) return kWsHeaderBytes;
+  if (L.num_codebooks >= 3) return encode_m2_workspace_bytes();  // header + the codebooks' image
   if (L.group_dim == 16)
     return encode_m1_use_tc(L, k) ? encode_m1_tc_layout((uint32_t)L.codebook_size, k, sms, 16).bytes : kWsHeaderBytes;
   if (L.num_codebooks != 1) return encode_m2_workspace_bytes();
@@ -250,7 +250,7 @@ int pvt_vstep_encode(const pvt_layer* layer, const uint32_t* idx, uint64_t k, fl
     e = launch_encode_m2(*layer, G, idx, k, err_out, ws, sms, static_cast<cudaStream_t>(cuda_stream));
   } else {
     if (layer->beam < 1 || layer->beam > 8) return PVT_EUNSUPPORTED;
-    if (ws_bytes < kWsHeaderBytes) return PVT_EWORKSPACE;
+    if (ws_bytes < encode_m2_workspace_bytes()) return PVT_EWORKSPACE;
     e = launch_encode_mx(*layer, G, idx, k, err_out, ws, static_cast<cudaStream_t>(cuda_stream));
   }
   return e == cudaSuccess ? PVT_OK : fail_cuda(e);

@@ -29,7 +29,8 @@
 
 namespace pvt {
 
-size_t encode_m2_workspace_bytes() { return kWsHeaderBytes; }
+// header + the image of the codebooks (two codebooks: under 40 KiB; up to four: under 56 KiB)
+size_t encode_m2_workspace_bytes() { return kWsHeaderBytes + 57344; }
 
 namespace {
 
@@ -57,7 +58,10 @@ struct EncM2Params {
 
 constexpr int kM2Group = 4;  // targets per warp iteration: 4 targets x 8 beam entries = 32 lanes
 
-struct M2Smem {
+// Everything the kernel derives from the two codebooks, in the byte order it has in shared memory.  One small
+// kernel writes it once per call into the workspace; every CTA of the search fetches it with a single bulk copy
+// (cp.async.bulk, completion on an mbarrier; no multicast).
+struct M2Image {
   alignas(16) float c1[kM2K][8];
   alignas(16) float c2[kM2K][8];
   alignas(16) uint64_t p1[4][8][32];  // stage-1 operands: (c1[l+64q][i], c1[l+64q+32][i])
@@ -67,18 +71,22 @@ struct M2Smem {
       alignas(16) float x2[kM2K / 2][16];  // FP32 stage 2: pair p holds (c2[2p][0], c2[2p+1][0], c2[2p][1], ...)
       alignas(8) float hx2[kM2K / 2][2];   // (||c2||^2/2) of the pair
     };
-    struct {
-      // tensor stage 2: B fragments of codebook 2, word [n-tile][lane] = halves (c2[8 nt + lane/4][2 (lane%4)], [.. + 1]);
-      // and the sub-chunk minima of a warp's 32 residual rows on their way to the lanes that own the rows
-      uint32_t b2[kM2K / 8][32];
-      alignas(16) float wmin[kM2Threads / 32][32][8];
-    };
+    // tensor stage 2: B fragments of codebook 2, word [n-tile][lane] = halves (c2[8 nt + lane/4][2 (lane%4)], [.. + 1])
+    uint32_t b2[kM2K / 8][32];
   };
   alignas(8) float h2[kM2K];
+  float n1max, n2max;
+  float pad_[2];
+};
+static_assert(sizeof(M2Image) % 16 == 0, "the bulk copy moves multiples of 16 bytes");
+
+struct M2Smem {
+  M2Image img;
+  // the sub-chunk minima of a warp's 32 residual rows on their way to the lanes that own the rows (tensor stage 2)
+  alignas(16) float wmin[kM2Threads / 32][32][8];
   alignas(16) float wt[kM2Threads / 32][kM2Group][8];     // the targets of a warp's group
   alignas(16) uint32_t wk[kM2Threads / 32][kM2Group][8];  // their beam entries (codes of codebook 1)
-  float red[kM2Threads / 32][2];
-  float n1max, n2max;
+  alignas(8) uint64_t img_bar;                            // completion of the image copy
 };
 
 __device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
@@ -145,13 +153,52 @@ __device__ __forceinline__ float load_cb(const void* books, int f16, uint32_t m,
   return f16 ? __half2float(reinterpret_cast<const __half*>(books)[off]) : reinterpret_cast<const float*>(books)[off];
 }
 
+// ---- PTX helpers of the image copy ----------------------------------------------------------------------------
+constexpr uint32_t kM2MaxSpins = 1u << 22;  // polls after which the wait for the image gives up
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ bool mbar_try_wait0(uint32_t bar) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar)
+      : "memory");
+  return ok != 0;
+}
+// One bulk copy global -> shared of the whole image (16-byte aligned on both sides, a multiple of 16 bytes),
+// issued by one thread; every thread then waits, a bounded number of polls, for its completion.  Returns false
+// (after recording PVT_DEV_WAIT_EXPIRED) if the copy has not landed by then: the CTA must leave without reading it.
+__device__ __forceinline__ bool fetch_image(void* dst, const void* src, uint32_t bytes, uint64_t* bar, uint32_t* status) {
+  const uint32_t b = smem_addr(bar);
+  if (threadIdx.x == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(b));
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(b), "r"(bytes) : "memory");
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_addr(dst)),
+                 "l"(src), "r"(bytes), "r"(b)
+                 : "memory");
+  }
+  __syncthreads();  // the barrier is initialised before anybody polls it
+  bool ok = false;
+  for (uint32_t spin = 0; spin < kM2MaxSpins && !ok; ++spin) {
+    ok = mbar_try_wait0(b);
+    if (!ok && spin > 4096) __nanosleep(64);
+  }
+  if (!ok) atomicOr(status, PVT_DEV_WAIT_EXPIRED);
+  // everybody agrees (a thread that gave up makes the whole CTA leave)
+  return __syncthreads_and(ok) != 0;
+}
+
+// ---- the codebook image: one block, one codeword per thread (K <= 256 = block size) ----
 // TC2: stage 2 on the tensor cores (fp16 codebooks: the codewords are exact halves), else on the FP32 pipe.
 template <bool TC2>
-__global__ void __launch_bounds__(kM2Threads, kM2CtasPerSm) encode_m2_kernel(const EncM2Params p) {
-  __shared__ M2Smem sm;
+__global__ void __launch_bounds__(kM2Threads) m2_image_kernel(const EncM2Params p, M2Image* __restrict__ img_out) {
+  __shared__ float red[kM2Threads / 32][2];
+  M2Image& sm = *img_out;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-
-  // ---- stage the codebooks: one codeword per thread (K <= 256 = block size) ----
   {
     float c1[8], c2[8], n1 = 0.0f, n2 = 0.0f;
     const bool real = (uint32_t)tid < p.K;
@@ -191,21 +238,30 @@ __global__ void __launch_bounds__(kM2Threads, kM2CtasPerSm) encode_m2_kernel(con
       m2 = fmaxf(m2, __shfl_xor_sync(0xffffffffu, m2, o));
     }
     if (lane == 0) {
-      sm.red[warp][0] = m1;
-      sm.red[warp][1] = m2;
+      red[warp][0] = m1;
+      red[warp][1] = m2;
     }
     __syncthreads();
     if (tid == 0) {
       float a = 0.0f, b = 0.0f;
       for (int w = 0; w < kM2Threads / 32; ++w) {
-        a = fmaxf(a, sm.red[w][0]);
-        b = fmaxf(b, sm.red[w][1]);
+        a = fmaxf(a, red[w][0]);
+        b = fmaxf(b, red[w][1]);
       }
       sm.n1max = a;
       sm.n2max = b;
+      sm.pad_[0] = sm.pad_[1] = 0.0f;
     }
-    __syncthreads();
   }
+}
+
+template <bool TC2>
+__global__ void __launch_bounds__(kM2Threads, kM2CtasPerSm) encode_m2_kernel(const EncM2Params p,
+                                                                              const M2Image* __restrict__ image) {
+  __shared__ M2Smem smem;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (!fetch_image(&smem.img, image, (uint32_t)sizeof(M2Image), &smem.img_bar, p.status)) return;
+  M2Image& sm = smem.img;
   const float n1max = sm.n1max, n2max = sm.n2max;
   const float s1max = sqrtf(n1max), s2max = sqrtf(n2max);
   const uint32_t B = p.beam;  // already min(beam, K)
@@ -232,7 +288,7 @@ __global__ void __launch_bounds__(kM2Threads, kM2CtasPerSm) encode_m2_kernel(con
         lane_prev = p.codes[lane_j];
         tv = __fdiv_rn(__fmaf_rn(-p.eta, gv, wv), sc);
       }
-      sm.wt[warp][my_q][my_b] = tv;
+      smem.wt[warp][my_q][my_b] = tv;
     }
     __syncwarp();
 
@@ -249,8 +305,8 @@ __global__ void __launch_bounds__(kM2Threads, kM2CtasPerSm) encode_m2_kernel(con
       }
       float t[8];
       {
-        const float4 ta = *reinterpret_cast<const float4*>(&sm.wt[warp][q][0]);
-        const float4 tb = *reinterpret_cast<const float4*>(&sm.wt[warp][q][4]);
+        const float4 ta = *reinterpret_cast<const float4*>(&smem.wt[warp][q][0]);
+        const float4 tb = *reinterpret_cast<const float4*>(&smem.wt[warp][q][4]);
         t[0] = ta.x, t[1] = ta.y, t[2] = ta.z, t[3] = ta.w, t[4] = tb.x, t[5] = tb.y, t[6] = tb.z, t[7] = tb.w;
       }
       float nt2 = 0.0f;
@@ -362,8 +418,8 @@ __global__ void __launch_bounds__(kM2Threads, kM2CtasPerSm) encode_m2_kernel(con
       }
       // hand the target and its beam to the lanes of stage 2
       if (lane == 0) {
-        *reinterpret_cast<uint4*>(&sm.wk[warp][q][0]) = make_uint4(beam_code[0], beam_code[1], beam_code[2], beam_code[3]);
-        *reinterpret_cast<uint4*>(&sm.wk[warp][q][4]) = make_uint4(beam_code[4], beam_code[5], beam_code[6], beam_code[7]);
+        *reinterpret_cast<uint4*>(&smem.wk[warp][q][0]) = make_uint4(beam_code[0], beam_code[1], beam_code[2], beam_code[3]);
+        *reinterpret_cast<uint4*>(&smem.wk[warp][q][4]) = make_uint4(beam_code[4], beam_code[5], beam_code[6], beam_code[7]);
       }
       if (my_q == q) {
         my_j = j;
@@ -378,10 +434,10 @@ __global__ void __launch_bounds__(kM2Threads, kM2CtasPerSm) encode_m2_kernel(con
     float t[8], c1v[8], r[8];
     uint32_t k1 = 0;
     {
-      const float4 ta = *reinterpret_cast<const float4*>(&sm.wt[warp][my_q][0]);
-      const float4 tb = *reinterpret_cast<const float4*>(&sm.wt[warp][my_q][4]);
+      const float4 ta = *reinterpret_cast<const float4*>(&smem.wt[warp][my_q][0]);
+      const float4 tb = *reinterpret_cast<const float4*>(&smem.wt[warp][my_q][4]);
       t[0] = ta.x; t[1] = ta.y; t[2] = ta.z; t[3] = ta.w; t[4] = tb.x; t[5] = tb.y; t[6] = tb.z; t[7] = tb.w;
-      k1 = active ? sm.wk[warp][my_q][my_b] : 0u;
+      k1 = active ? smem.wk[warp][my_q][my_b] : 0u;
       const float4 ca = *reinterpret_cast<const float4*>(&sm.c1[k1][0]);
       const float4 cb = *reinterpret_cast<const float4*>(&sm.c1[k1][4]);
       c1v[0] = ca.x; c1v[1] = ca.y; c1v[2] = ca.z; c1v[3] = ca.w; c1v[4] = cb.x; c1v[5] = cb.y; c1v[6] = cb.z; c1v[7] = cb.w;
@@ -407,8 +463,8 @@ __global__ void __launch_bounds__(kM2Threads, kM2CtasPerSm) encode_m2_kernel(con
         const uint32_t row = 16u * (r4 >> 1) + 8u * (r4 & 1) + g8, tq = row >> 3, b = row & 7u;
         const uint32_t tj = __shfl_sync(0xffffffffu, my_j, 8 * tq);
         const bool valid = tj != 0xffffffffu && b < B;
-        const uint32_t kr = valid ? sm.wk[warp][tq][b] : 0u;  // the beam of a skipped target was never written
-        const float2 tt = *reinterpret_cast<const float2*>(&sm.wt[warp][tq][2 * qd]);
+        const uint32_t kr = valid ? smem.wk[warp][tq][b] : 0u;  // the beam of a skipped target was never written
+        const float2 tt = *reinterpret_cast<const float2*>(&smem.wt[warp][tq][2 * qd]);
         const float2 cc = *reinterpret_cast<const float2*>(&sm.c1[kr][2 * qd]);
         nr[r4].x = valid ? __fsub_rn(cc.x, tt.x) : 0.0f;  // -(t - c1), exactly
         nr[r4].y = valid ? __fsub_rn(cc.y, tt.y) : 0.0f;
@@ -452,13 +508,13 @@ __global__ void __launch_bounds__(kM2Threads, kM2CtasPerSm) encode_m2_kernel(con
         }
         if (qd == 0) {
 #pragma unroll
-          for (int r4 = 0; r4 < 4; ++r4) sm.wmin[warp][16 * (r4 >> 1) + 8 * (r4 & 1) + g8][sub] = m[r4];
+          for (int r4 = 0; r4 < 4; ++r4) smem.wmin[warp][16 * (r4 >> 1) + 8 * (r4 & 1) + g8][sub] = m[r4];
         }
       }
       __syncwarp();
       {
-        const float4 ma = *reinterpret_cast<const float4*>(&sm.wmin[warp][lane][0]);
-        const float4 mb = *reinterpret_cast<const float4*>(&sm.wmin[warp][lane][4]);
+        const float4 ma = *reinterpret_cast<const float4*>(&smem.wmin[warp][lane][0]);
+        const float4 mb = *reinterpret_cast<const float4*>(&smem.wmin[warp][lane][4]);
         const float mm[8] = {ma.x, ma.y, ma.z, ma.w, mb.x, mb.y, mb.z, mb.w};
 #pragma unroll
         for (int sub = 0; sub < 8; ++sub) sub_min[sub] = active ? __fmaf_rn(mm[sub], inv, rho) : kInf;
@@ -528,7 +584,7 @@ __global__ void __launch_bounds__(kM2Threads, kM2CtasPerSm) encode_m2_kernel(con
           hhi &= hhi - 1u;
         }
         const uint32_t hb = pos >> 3, hsub = pos & 7u;
-        const uint32_t hk1 = work ? sm.wk[warp][my_q][hb] : 0u;
+        const uint32_t hk1 = work ? smem.wk[warp][my_q][hb] : 0u;
         float sc1[8], sr[8], srho = 0.0f;
         {
           const float4 ca = *reinterpret_cast<const float4*>(&sm.c1[hk1][0]);
@@ -624,12 +680,22 @@ cudaError_t launch_encode_m2(const pvt_layer& L, uint64_t G, const uint32_t* idx
   const uint64_t groups = (k + kM2Group - 1) / kM2Group;
   uint64_t ctas = (groups + warps_per_cta - 1) / warps_per_cta;
   if (ctas > kM2CtasPerSm * (uint64_t)sm_count) ctas = kM2CtasPerSm * (uint64_t)sm_count;  // persistent: the resident CTAs
+  static_assert(sizeof(M2Image) <= 40960, "the workspace reserves 40 KiB for the image");
+  M2Image* image = reinterpret_cast<M2Image*>(static_cast<char*>(ws) + kWsHeaderBytes);
+  timing_begin(kKernEncodeAux, stream);
+  if (p.cb_f16)
+    m2_image_kernel<true><<<1, kM2Threads, 0, stream>>>(p, image);
+  else
+    m2_image_kernel<false><<<1, kM2Threads, 0, stream>>>(p, image);
+  timing_end(kKernEncodeAux, stream);
+  cudaError_t err = cudaGetLastError();
+  if (err != cudaSuccess) return err;
   timing_begin(kKernEncodeMain, stream);
   if (p.cb_f16)
-    encode_m2_kernel<true><<<(unsigned)ctas, kM2Threads, 0, stream>>>(p);
+    encode_m2_kernel<true><<<(unsigned)ctas, kM2Threads, 0, stream>>>(p, image);
   else
-    encode_m2_kernel<false><<<(unsigned)ctas, kM2Threads, 0, stream>>>(p);
-  count_launches(1);
+    encode_m2_kernel<false><<<(unsigned)ctas, kM2Threads, 0, stream>>>(p, image);
+  count_launches(2);
   timing_end(kKernEncodeMain, stream);
   return cudaGetLastError();
 }

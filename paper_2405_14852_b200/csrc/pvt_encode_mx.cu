@@ -69,31 +69,30 @@ __host__ __device__ constexpr size_t mx_image_bytes(int M) {
   return (size_t)M * (kMxPadK / 8) * 32 * 4 + (size_t)M * kMxPadK * 4 + 16;
 }
 
+// bytes of everything the kernel derives from the codebooks (binary32 copy, and for fp16 codebooks the tensor-pipe
+// image), in the byte order it has at the start of shared memory: a multiple of 16
+__host__ __device__ constexpr size_t mx_staged_bytes(int M, uint32_t K, bool f16) {
+  return (size_t)M * K * 32 + (f16 ? mx_image_bytes(M) : 0);
+}
+
+// Writes that image into the workspace, once per call (one block).
+//   book   [M][K][8] binary32
+//   fp16 codebooks only: A fragments, words [m][tile][lane][2] = halves (c[16 tile + lane/4 (+ 8)][2 (lane%4)], [.. + 1]);
+//   ||c||^2/2 as [m][tile][lane/4][2]; max ||c||^2 per codebook (bit patterns)
 template <int M, bool CB_F16>
-__global__ void __launch_bounds__(kMxThreads, M == 3 ? 4 : 3) encode_mx_kernel(const MxParams p) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  float* book = reinterpret_cast<float*>(smem_raw);                               // [M][K][8]
-  double* resid = reinterpret_cast<double*>(smem_raw + (size_t)M * p.K * 32);     // [warps][beam][8]
-  float* resid_f = reinterpret_cast<float*>(resid + kMxWarps * kMxBeam * 8);      // the same, rounded to binary32
-  // fp16 codebooks only: A fragments, words [m][tile][lane][2] = halves (c[16 tile + lane/4 (+ 8)][2 (lane%4)], [.. + 1]);
-  // ||c||^2/2 as [m][tile][lane/4][2]; max ||c||^2
-  // per warp: the extensions that pass the filter of a stage, (kept tuple << 8 | code), and their count
-  uint16_t* cand = reinterpret_cast<uint16_t*>(resid_f + kMxWarps * kMxBeam * 8);
-  uint32_t* cand_n = reinterpret_cast<uint32_t*>(cand + kMxWarps * kMxCand);
-  // per warp: the kept partial tuples and the target
-  uint32_t* kept_sm = cand_n + kMxWarps;
-  float* t_sm = reinterpret_cast<float*>(kept_sm + kMxWarps * kMxBeam);
-  uint32_t* bfrag = reinterpret_cast<uint32_t*>(t_sm + kMxWarps * 8);
+__global__ void __launch_bounds__(kMxThreads) mx_image_kernel(const MxParams p, unsigned char* __restrict__ out) {
+  const uint32_t K = p.K;
+  float* book = reinterpret_cast<float*>(out);
+  uint32_t* bfrag = reinterpret_cast<uint32_t*>(out + (size_t)M * K * 32);
   float* hnorm = reinterpret_cast<float*>(bfrag + M * (kMxPadK / 8) * 32);
   uint32_t* n2max_bits = reinterpret_cast<uint32_t*>(hnorm + M * kMxPadK);
-  const uint32_t K = p.K;
   if (CB_F16) {
     for (uint32_t e = threadIdx.x; e < (uint32_t)M * kMxPadK; e += kMxThreads) {
       hnorm[e] = kMxPadHalfNorm;
 #pragma unroll
       for (int qq = 0; qq < 4; ++qq) bfrag[4 * e + qq] = 0u;
     }
-    if (threadIdx.x < M) n2max_bits[threadIdx.x] = 0u;
+    if (threadIdx.x < 4) n2max_bits[threadIdx.x] = 0u;
     __syncthreads();
   }
   for (uint32_t row = threadIdx.x; row < M * K; row += kMxThreads) {
@@ -130,15 +129,67 @@ __global__ void __launch_bounds__(kMxThreads, M == 3 ? 4 : 3) encode_mx_kernel(c
       }
     }
   }
-  __syncthreads();
+}
+
+constexpr uint32_t kMxMaxSpins = 1u << 22;  // polls after which the wait for the image gives up
+
+template <int M, bool CB_F16>
+__global__ void __launch_bounds__(kMxThreads, M == 3 ? 4 : 3) encode_mx_kernel(const MxParams p,
+                                                                                const unsigned char* __restrict__ image) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const uint32_t K = p.K;
+  const size_t staged = mx_staged_bytes(M, K, CB_F16);
+  // the codebooks' image, fetched with one bulk copy (cp.async.bulk, completion on an mbarrier; no multicast)
+  float* book = reinterpret_cast<float*>(smem_raw);                               // [M][K][8]
+  uint32_t* bfrag = reinterpret_cast<uint32_t*>(smem_raw + (size_t)M * K * 32);
+  float* hnorm = reinterpret_cast<float*>(bfrag + M * (kMxPadK / 8) * 32);
+  uint32_t* n2max_bits = reinterpret_cast<uint32_t*>(hnorm + M * kMxPadK);
+  // scratch behind it
+  double* resid = reinterpret_cast<double*>(smem_raw + staged);                   // [warps][beam][8]
+  float* resid_f = reinterpret_cast<float*>(resid + kMxWarps * kMxBeam * 8);      // the same, rounded to binary32
+  // per warp: the extensions that pass the filter of a stage, (kept tuple << 8 | code), and their count
+  uint16_t* cand = reinterpret_cast<uint16_t*>(resid_f + kMxWarps * kMxBeam * 8);
+  uint32_t* cand_n = reinterpret_cast<uint32_t*>(cand + kMxWarps * kMxCand);
+  // per warp: the kept partial tuples and the target
+  uint32_t* kept_sm = cand_n + kMxWarps;
+  float* t_sm = reinterpret_cast<float*>(kept_sm + kMxWarps * kMxBeam);
+  uint64_t* img_bar = reinterpret_cast<uint64_t*>(t_sm + kMxWarps * 8);
+  {
+    const uint32_t b = (uint32_t)__cvta_generic_to_shared(img_bar);
+    if (threadIdx.x == 0) {
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(b));
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(b), "r"((uint32_t)staged) : "memory");
+      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                       (uint32_t)__cvta_generic_to_shared(smem_raw)),
+                   "l"(image), "r"((uint32_t)staged), "r"(b)
+                   : "memory");
+    }
+    __syncthreads();  // the barrier is initialised before anybody polls it
+    uint32_t ok = 0;
+    for (uint32_t spin = 0; spin < kMxMaxSpins && !ok; ++spin) {
+      asm volatile(
+          "{\n\t.reg .pred q;\n\t"
+          "mbarrier.try_wait.parity.shared::cta.b64 q, [%1], 0;\n\t"
+          "selp.u32 %0, 1, 0, q;\n\t}"
+          : "=r"(ok)
+          : "r"(b)
+          : "memory");
+      if (!ok && spin > 4096) __nanosleep(64);
+    }
+    if (!ok) atomicOr(p.status, PVT_DEV_WAIT_EXPIRED);
+    if (!__syncthreads_and((int)ok)) return;  // the image has not landed: nobody reads it
+  }
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const uint64_t n = (uint64_t)blockIdx.x * kMxWarps + warp;
-  if (n >= p.k) return;
+  // persistent: the resident warps share out the targets
+#pragma unroll 1
+  for (uint64_t n = (uint64_t)blockIdx.x * kMxWarps + warp; n < p.k; n += (uint64_t)gridDim.x * kMxWarps) {
+  __syncwarp();  // the warp's scratch of the previous target is no longer read
   const uint32_t j = __ldg(p.idx + n);
   if (j >= p.G) {
     if (lane == 0) atomicOr(p.status, PVT_DEV_BAD_INDEX);
-    return;
+    continue;
   }
   // target (Eq. 8 in the scaled space): one fma and one division per element, binary32
   float t[8];
@@ -498,19 +549,27 @@ __global__ void __launch_bounds__(kMxThreads, M == 3 ? 4 : 3) encode_mx_kernel(c
       if (p.err_out) p.err_out[n] = (float)best_d;
     }
   }
+  }  // targets of this warp
 }
 
 template <int M, bool CB_F16>
-cudaError_t launch_m(const MxParams& p, cudaStream_t stream) {
-  const size_t smem = (size_t)M * p.K * 32 + (size_t)kMxWarps * kMxBeam * 8 * (sizeof(double) + sizeof(float)) +
-                      (size_t)kMxWarps * (kMxCand * sizeof(uint16_t) + sizeof(uint32_t) + kMxBeam * 4 + 8 * 4) +
-                      (CB_F16 ? mx_image_bytes(M) : 0);
+cudaError_t launch_m(const MxParams& p, unsigned char* image, int sm_count, cudaStream_t stream) {
+  const size_t smem = mx_staged_bytes(M, p.K, CB_F16) +
+                      (size_t)kMxWarps * kMxBeam * 8 * (sizeof(double) + sizeof(float)) +
+                      (size_t)kMxWarps * (kMxCand * sizeof(uint16_t) + sizeof(uint32_t) + kMxBeam * 4 + 8 * 4) + 16;
   cudaError_t e = cudaFuncSetAttribute(encode_mx_kernel<M, CB_F16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)smem);
   if (e != cudaSuccess) return e;
-  const unsigned blocks = (unsigned)((p.k + kMxWarps - 1) / kMxWarps);
-  encode_mx_kernel<M, CB_F16><<<blocks, kMxThreads, smem, stream>>>(p);
-  count_launches(1);
+  mx_image_kernel<M, CB_F16><<<1, kMxThreads, 0, stream>>>(p, image);
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  int per_sm = 0;
+  if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, encode_mx_kernel<M, CB_F16>, kMxThreads, smem)) !=
+      cudaSuccess)
+    return e;
+  const uint64_t needed = (p.k + kMxWarps - 1) / kMxWarps;
+  const uint64_t resident = (uint64_t)sm_count * (uint64_t)(per_sm > 0 ? per_sm : 1);
+  encode_mx_kernel<M, CB_F16><<<(unsigned)(needed < resident ? needed : resident), kMxThreads, smem, stream>>>(p, image);
+  count_launches(2);
   return cudaGetLastError();
 }
 
@@ -536,10 +595,12 @@ cudaError_t launch_encode_mx(const pvt_layer& L, uint64_t G, const uint32_t* idx
   const bool f16 = L.codebook_dtype == PVT_F16;
   timing_begin(kKernEncodeMain, stream);
   cudaError_t e;
+  unsigned char* image = static_cast<unsigned char*>(ws) + kWsHeaderBytes;
+  const int sms = device_sm_count();
   if (L.num_codebooks == 3)
-    e = f16 ? launch_m<3, true>(p, stream) : launch_m<3, false>(p, stream);
+    e = f16 ? launch_m<3, true>(p, image, sms, stream) : launch_m<3, false>(p, image, sms, stream);
   else
-    e = f16 ? launch_m<4, true>(p, stream) : launch_m<4, false>(p, stream);
+    e = f16 ? launch_m<4, true>(p, image, sms, stream) : launch_m<4, false>(p, image, sms, stream);
   timing_end(kKernEncodeMain, stream);
   return e;
 }
