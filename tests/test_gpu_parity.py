@@ -177,6 +177,57 @@ def test_select_denormal_and_zero_norms():
     assert np.array_equal(run_select(L, 77), want)
 
 
+def _layer_with_a_block_of_equal_norms(rows, cols, gd, seed):
+    """Norms: the first two fifths of the groups (at random positions) far above a value v, one fifth exactly v,
+    the rest far below it."""
+    G = rows * cols // gd
+    r = np.random.default_rng(seed)
+    g = np.zeros((G, gd), dtype=np.float32)
+    perm = r.permutation(G)
+    top, tie, low = perm[:2 * G // 5], perm[2 * G // 5:3 * G // 5], perm[3 * G // 5:]
+    g[top] = r.uniform(2e-3, 4e-3, size=(top.size, gd)).astype(np.float32)
+    g[tie] = np.float32(1e-3)
+    g[low] = r.uniform(1e-5, 5e-4, size=(low.size, gd)).astype(np.float32)
+    L = synth.SynthLayer(rows=rows, cols=cols, group_dim=gd, num_codebooks=1, codebook_size=2, beam=8, eta=1.0,
+                         W=np.zeros((1, gd), np.float32), g=g.reshape(rows, cols), scale=np.ones(rows, np.float32),
+                         codebooks=np.zeros((1, 2, gd), np.float16), codes=np.zeros((G, 1), np.uint8))
+    return L, G
+
+
+@pytest.mark.parametrize("rows,cols,gd", [(4096, 4096, 8), (2048, 8192, 16)])
+def test_select_with_a_large_block_of_equal_norms_around_the_threshold(rows, cols, gd):
+    """A fifth of a large layer shares one norm and the subspace ends just inside, at, or just beyond that block:
+    the threshold bucket then holds far more keys than the candidate list takes, and hundreds of thousands of
+    ties must be split by index.  The exact index set must come out, ties towards the lowest index."""
+    L, G = _layer_with_a_block_of_equal_norms(rows, cols, gd, 55)
+    norms = oracle.group_norms(L.g, L.eta, gd)
+    g_dev = torch.from_numpy(L.g).cuda()
+    dev = VStepLayer(rows, cols, g_dev, g_dev, torch.ones(rows, device="cuda"),
+                     torch.zeros(1, 2, gd, dtype=torch.float16, device="cuda"),
+                     torch.zeros(G, 1, dtype=torch.uint8, device="cuda"), group_dim=gd)
+    top = 2 * G // 5
+    for k in (top + G // 1000, top - G // 1000, top + G // 10, top, top + 1, 3 * G // 5 + G // 1000):
+        want = oracle.select(norms, k)
+        got = dev.select(k)
+        torch.cuda.synchronize()
+        assert dev.status() == 0
+        assert np.array_equal(to_np(got).astype(np.uint32), want), k
+
+
+def test_select_many_sizes_against_the_checker():
+    """Subspace sizes from one group to all but one on three mid-size layers (one with a ragged last tile)."""
+    for rows, cols in ((128, 1016), (129, 1024), (640, 1024)):
+        L = select_only_layer(rows, cols, 56)
+        G = L.num_groups
+        norms = oracle.group_norms(L.g, L.eta)
+        dev = VStepLayer.from_host(L)
+        for k in (1, 2, 7, G // 1000 + 1, G // 100, G // 10, G // 3, G // 2, G - G // 100, G - 1):
+            got = dev.select(k)
+            torch.cuda.synchronize()
+            assert dev.status() == 0
+            assert np.array_equal(to_np(got).astype(np.uint32), oracle.select(norms, k)), (rows, cols, k)
+
+
 # ------------------------------------------------------------------ M = 1 search
 
 
