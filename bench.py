@@ -428,7 +428,8 @@ def stage_record(runner, t, steps, peaks, out_itemsize):
     aux_ms, _ = per_step(B.PVT_KERNEL_ENCODE_AUX)
     dq_ms, _ = per_step(B.PVT_KERNEL_DEQUANT)
     rs_ms, _ = per_step(B.PVT_KERNEL_ENCODE_RESCORE)
-    sel_bytes = sum(l.G * 32 + 4 * l.k for l in runner.layers)
+    # the selection reads g once (32 B per group) and writes the indices; with k = G it is the index list itself
+    sel_bytes = sum((l.G * 32 if l.k < l.G else 0) + 4 * l.k for l in runner.layers)
     dq_bytes = sum(l.G * (l.code_bytes + 8 * out_itemsize) for l in runner.layers)
     st = {"select": {"ms": sel_ms, "algorithmic_bytes": sel_bytes, "gbs": sel_bytes / (sel_ms * 1e-3) / 1e9 if sel_ms else None},
           "encode_search": {"ms": enc_ms, "pairs": runner.pairs, "pairs_per_s": runner.pairs / (enc_ms * 1e-3) if enc_ms else None},
