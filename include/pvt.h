@@ -296,6 +296,22 @@ int pvt_vstep_refine(const pvt_layer* layer, const uint32_t* idx, uint64_t k, in
 int pvt_dequant(const pvt_layer* layer, void* W_hat, int32_t out_dtype, uint32_t* status, void* cuda_stream);
 
 /*
+ * The V step over every linear layer of a model block in one call (Algorithm 3, V-step lines: the loop over
+ * the quantised weights; the subspace is chosen inside each weight matrix, Section 3.4, so the layers are
+ * independent): for i = 0 .. n_layers-1, in order, on the one stream,
+ *     pvt_vstep_select(layers[i], k[i]) -> idx_out[i];  pvt_vstep_encode(layers[i], idx_out[i], k[i]);
+ *     pvt_dequant(layers[i]) -> W_hat[i]   (skipped when W_hat or W_hat[i] is NULL).
+ * A convenience that adds no arithmetic of its own.  layers, k, idx_out, W_hat: HOST arrays of n_layers
+ * entries (descriptors, subspace sizes, device pointers to k[i] uint32, device pointers to rows x cols of
+ * out_dtype).  ws: one device workspace shared by all layers, at least pvt_block_workspace_bytes (the largest
+ * per-layer need), header cleared by pvt_workspace_init; status bits of all layers accumulate in it.
+ * Every layer is validated before anything is enqueued; return codes as the three calls.
+ */
+size_t pvt_block_workspace_bytes(const pvt_layer* layers, const uint64_t* k, int32_t n_layers);
+int pvt_vstep_block(const pvt_layer* layers, const uint64_t* k, int32_t n_layers, uint32_t* const* idx_out,
+                    void* const* W_hat, int32_t out_dtype, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
  * P step, the half that shares its inputs with the V step (Algorithm 3, P-step lines:
  * grad_codebooks = backprop(grad_phi)).  Chain rule through dequantize_weights,
  * W_hat[r, 8c+i] = scale[r] * v[j][i], v[j] = sum_m C_m[codes[j][m]] (the binary32 sum

@@ -87,6 +87,11 @@ def lib():
         L.pvt_vstep_trust.argtypes = [lp, u64, fl, vp, vp, vp, vp, sz, vp]
         L.pvt_vstep_refine.restype = ctypes.c_int
         L.pvt_vstep_refine.argtypes = [lp, vp, u64, ctypes.c_int32, vp, vp, vp, vp]
+        L.pvt_block_workspace_bytes.restype = sz
+        L.pvt_block_workspace_bytes.argtypes = [lp, ctypes.POINTER(u64), ctypes.c_int32]
+        L.pvt_vstep_block.restype = ctypes.c_int
+        L.pvt_vstep_block.argtypes = [lp, ctypes.POINTER(u64), ctypes.c_int32, ctypes.POINTER(vp), ctypes.POINTER(vp),
+                                      ctypes.c_int32, vp, sz, vp]
         L.pvt_dequant.restype = ctypes.c_int
         L.pvt_dequant.argtypes = [lp, vp, ctypes.c_int32, vp, vp]
         L.pvt_pstep_grad.restype = ctypes.c_int
@@ -247,6 +252,40 @@ def pvt_dequant(layer: pvt_layer, W_hat: torch.Tensor, status: Optional[torch.Te
     out_dtype = {torch.float32: PVT_F32, torch.float16: PVT_F16}[W_hat.dtype]
     _check(lib().pvt_dequant(ctypes.byref(layer), W_hat.data_ptr(), out_dtype, _ptr(status), _stream_ptr(stream)),
            "pvt_dequant")
+
+
+class Block:
+    """Host arrays for pvt_vstep_block: the layers of one model block, their subspace sizes and output pointers
+    (marshalled once; the tensors must stay alive while the block is used)."""
+
+    def __init__(self, layers, ks, idx_outs, W_hats=None):
+        n = len(layers)
+        self.n = n
+        self.layers = (pvt_layer * n)(*layers)
+        self.k = (ctypes.c_uint64 * n)(*[int(x) for x in ks])
+        self.idx = (ctypes.c_void_p * n)(*[t.data_ptr() for t in idx_outs])
+        self.W_hat = None
+        self.out_dtype = PVT_F32
+        if W_hats is not None:
+            self.W_hat = (ctypes.c_void_p * n)(*[None if t is None else t.data_ptr() for t in W_hats])
+            dts = {t.dtype for t in W_hats if t is not None}
+            if len(dts) > 1:
+                raise ValueError("the dequantised matrices of a block share one dtype")
+            if dts:
+                self.out_dtype = {torch.float32: PVT_F32, torch.float16: PVT_F16}[dts.pop()]
+        self._keep = (list(idx_outs), list(W_hats) if W_hats is not None else None)
+
+    def workspace_bytes(self) -> int:
+        need = int(lib().pvt_block_workspace_bytes(self.layers, self.k, self.n))
+        if need == 0:
+            raise PvtError(PVT_EINVAL, "pvt_block_workspace_bytes")
+        return need
+
+
+def pvt_vstep_block(block: Block, ws: torch.Tensor, stream=None) -> None:
+    """select -> encode -> dequantise over every layer of the block, one C call."""
+    _check(lib().pvt_vstep_block(block.layers, block.k, block.n, block.idx, block.W_hat, block.out_dtype, ws.data_ptr(),
+                                 ws.numel() * ws.element_size(), _stream_ptr(stream)), "pvt_vstep_block")
 
 
 def pvt_pstep_grad(layer: pvt_layer, grad_codebooks: torch.Tensor, grad_scale: Optional[torch.Tensor] = None,

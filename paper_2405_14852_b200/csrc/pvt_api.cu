@@ -324,6 +324,50 @@ int pvt_dequant(const pvt_layer* layer, void* W_hat, int32_t out_dtype, uint32_t
   return e == cudaSuccess ? PVT_OK : fail_cuda(e);
 }
 
+size_t pvt_block_workspace_bytes(const pvt_layer* layers, const uint64_t* k, int32_t n_layers) {
+  if (!layers || !k || n_layers < 1) return 0;
+  size_t need = 0;
+  for (int32_t i = 0; i < n_layers; ++i) {
+    const size_t b = pvt_workspace_bytes(&layers[i], k[i]);
+    if (b == 0) return 0;
+    if (b > need) need = b;
+  }
+  return need;
+}
+
+int pvt_vstep_block(const pvt_layer* layers, const uint64_t* k, int32_t n_layers, uint32_t* const* idx_out,
+                    void* const* W_hat, int32_t out_dtype, void* ws, size_t ws_bytes, void* cuda_stream) {
+  if (!layers || !k || !idx_out || n_layers < 1) return PVT_EINVAL;
+  // every layer is checked before anything is enqueued: the block is taken whole or not at all
+  const size_t need = pvt_block_workspace_bytes(layers, k, n_layers);
+  if (need == 0) {
+    // find out which complaint it is: the per-layer calls below report it without launching (bad layers come first)
+    for (int32_t i = 0; i < n_layers; ++i) {
+      uint64_t G = 0;
+      int rc = check_layer(&layers[i], &G);
+      if (rc == PVT_OK) rc = check_quantiser(&layers[i]);
+      if (rc != PVT_OK) return rc;
+      if (k[i] < 1 || k[i] > G) return PVT_EINVAL;
+    }
+    return PVT_EINVAL;
+  }
+  if (ws_bytes < need) return PVT_EWORKSPACE;
+  for (int32_t i = 0; i < n_layers; ++i) {
+    const pvt_layer& L = layers[i];
+    if (!idx_out[i] || !aligned4(idx_out[i]) || !L.W || !L.g || !L.scale || !L.codebooks || !L.codes) return PVT_EINVAL;
+    if (!aligned16(L.W) || !aligned16(L.g) || !aligned16(L.codebooks) || !codes_aligned(&L)) return PVT_EINVAL;
+    if (W_hat && W_hat[i] && !aligned16(W_hat[i])) return PVT_EINVAL;
+  }
+  if (W_hat && out_dtype != PVT_F32 && out_dtype != PVT_F16) return PVT_EINVAL;
+  for (int32_t i = 0; i < n_layers; ++i) {
+    int rc = pvt_vstep_select(&layers[i], k[i], idx_out[i], ws, ws_bytes, cuda_stream);
+    if (rc == PVT_OK) rc = pvt_vstep_encode(&layers[i], idx_out[i], k[i], nullptr, ws, ws_bytes, cuda_stream);
+    if (rc == PVT_OK && W_hat && W_hat[i]) rc = pvt_dequant(&layers[i], W_hat[i], out_dtype, nullptr, cuda_stream);
+    if (rc != PVT_OK) return rc;
+  }
+  return PVT_OK;
+}
+
 int pvt_pstep_grad(const pvt_layer* layer, double* grad_codebooks, double* grad_scale, uint32_t* status,
                    void* cuda_stream) {
   uint64_t G = 0;

@@ -137,3 +137,23 @@ def test_buffer_and_sampling_calls_reject_bad_arguments():
     assert lib.pvt_vstep_sample(ctypes.byref(_layer(g=None)), 4, B.PVT_SAMPLE_PROPORTIONAL, 1, 0x2000, 0x4000, big,
                                 None) == B.PVT_EINVAL
     assert lib.pvt_vstep_sample(ctypes.byref(L), 4, B.PVT_SAMPLE_UNIFORM, 1, 0x2000, 0x4000, 256, None) == B.PVT_EWORKSPACE
+
+
+def test_block_call_validates_every_layer_before_launching():
+    lib = B.lib()
+    good, bad = _layer(), _layer(cols=60)
+    n = 2
+    arr = (B.pvt_layer * n)(good, bad)
+    ks = (ctypes.c_uint64 * n)(4, 4)
+    idx = (ctypes.c_void_p * n)(0x2000, 0x3000)
+    assert lib.pvt_block_workspace_bytes(arr, ks, n) == 0
+    assert lib.pvt_vstep_block(arr, ks, n, idx, None, B.PVT_F32, 0x4000, 1 << 30, None) == B.PVT_EINVAL
+    arr = (B.pvt_layer * n)(good, _layer(rows=64, cols=256))
+    need = lib.pvt_block_workspace_bytes(arr, ks, n)
+    assert need == max(B.pvt_workspace_bytes(arr[0], 4), B.pvt_workspace_bytes(arr[1], 4))
+    assert lib.pvt_vstep_block(arr, ks, n, idx, None, B.PVT_F32, 0x4000, need - 1, None) == B.PVT_EWORKSPACE
+    ks_bad = (ctypes.c_uint64 * n)(4, 0)
+    assert lib.pvt_vstep_block(arr, ks_bad, n, idx, None, B.PVT_F32, 0x4000, 1 << 30, None) == B.PVT_EINVAL
+    idx_bad = (ctypes.c_void_p * n)(0x2000, None)
+    assert lib.pvt_vstep_block(arr, ks, n, idx_bad, None, B.PVT_F32, 0x4000, 1 << 30, None) == B.PVT_EINVAL
+    assert lib.pvt_vstep_block(arr, ks, 0, idx, None, B.PVT_F32, 0x4000, 1 << 30, None) == B.PVT_EINVAL
