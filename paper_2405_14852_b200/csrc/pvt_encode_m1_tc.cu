@@ -293,6 +293,22 @@ __device__ __forceinline__ void tmem_ld_wait(uint32_t* v) {
                : "memory");
 }
 
+// non-blocking test of a phase by lane 0 alone, without a branch (the other lanes get 0); try_wait may suspend the
+// thread for a while when the phase is not complete, test_wait does not
+__device__ __forceinline__ uint32_t mbar_test_wait_lane0(uint32_t bar, uint32_t parity, uint32_t lane) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.eq.u32 q, %3, 0;\n\t"
+      "setp.ne.u32 p, %3, %3;\n\t"
+      "@q mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity), "r"(lane)
+      : "memory");
+  return ok;
+}
+
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float d;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -417,13 +433,19 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
     }
   } else if (warp >= 9) {
     // ------------------------------------------------------------ MMA issuers: warp 9 -> A block 0, warp 10 -> A block 1
-    if (lane == 0) {
+    // The whole warp runs the loop, so that everything the instructions need (descriptors, addresses, parities) is
+    // computed once per warp in converged code; one lane issues.  A thread on its own runs one dependent instruction
+    // after the other at several cycles each, a wait costs 100-150 cycles even on a finished phase and an MMA or a
+    // commit about 50, and the loop is part of the hand-over ring of the accumulators.  So it is kept to the bare
+    // sequence: a codebook stage (four steps) is one trip, its steps are unrolled with constant buffer numbers,
+    // parities and descriptor offsets, and a wait that is already over costs a single poll.
+    {
       const uint32_t q = (uint32_t)warp - 9u;
-      const uint64_t a_desc = smem_desc(smem_u32(&sm.a[q][0]), D::kAGroupBytes);
-      // A lone thread pays about 150 cycles for a wait on an mbarrier (even on a finished phase) and about
-      // 50 per MMA or commit, and its loop is part of the hand-over ring of the accumulators: per step one wait
-      // (accumulator free), two MMAs, one commit; the codebook stage costs a wait and a commit per four steps.
-      uint32_t it = 0, unit_i = 0, total = 0;
+      uint64_t a_desc[D::kMmas];
+#pragma unroll
+      for (int m = 0; m < D::kMmas; ++m)
+        a_desc[m] = smem_desc(smem_u32(&sm.a[q][0]), D::kAGroupBytes) + (uint64_t)(D::a_chunk(m) * (128 >> 4));
+      uint32_t total = 0;  // steps of this CTA
       for (uint64_t u = blockIdx.x; u < units; u += gridDim.x) {
         uint32_t s_lo, s_hi;
         slice_units(p, (uint32_t)(u % p.n_slices), &s_lo, &s_hi);
@@ -432,32 +454,59 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
       const uint64_t b_desc0 = smem_desc(smem_u32(&sm.b[0][0][0]), D::kBGroupBytes);
       const uint32_t full0 = smem_u32(&sm.tmem_full[0][q]), full1 = smem_u32(&sm.tmem_full[1][q]);
       const uint32_t empty0 = smem_u32(&sm.tmem_empty[0][q]), empty1 = smem_u32(&sm.tmem_empty[1][q]);
+      const uint32_t d0 = tmem_base + q * 128, d1 = d0 + 256;
+      const uint32_t a_ready = smem_u32(&sm.a_ready);
+      // a wait whose answer is the same in every lane: one poll by all of them when the phase is already over,
+      // otherwise lane 0 polls (bounded) and tells the others
+      auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
+        if (__all_sync(0xffffffffu, mbar_try_wait(bar, parity))) return true;
+        bool ok = true;
+        if (lane == 0) ok = mbar_wait(bar, parity, abort_flag, p.status, p.max_spins);
+        return __shfl_sync(0xffffffffu, ok, 0);
+      };
       bool alive = true;
-      for (uint64_t u = blockIdx.x; u < units && alive; u += gridDim.x, ++unit_i) {
-        uint32_t s_lo, s_hi;
-        slice_units(p, (uint32_t)(u % p.n_slices), &s_lo, &s_hi);
-        alive = mbar_wait(smem_u32(&sm.a_ready), unit_i & 1, abort_flag, p.status, p.max_spins);
-        tc_fence_after();
-        for (uint32_t st = s_lo; st < s_hi && alive; ++st, ++it) {
-          const uint32_t grp = it / kTcGroupSteps, sub = it % kTcGroupSteps, s = grp % kTcStages, buf = it & 1;
-          if (sub == 0 || it == 0)
-            alive = mbar_wait(smem_u32(&sm.full_bar[s]), (grp / kTcStages) & 1, abort_flag, p.status, p.max_spins);
-          if (alive) alive = mbar_wait(buf ? empty1 : empty0, ((it >> 1) & 1) ^ 1, abort_flag, p.status, p.max_spins);
-          if (!alive) break;
-          tc_fence_after();
-          const uint64_t b_desc = b_desc0 + (uint64_t)((s * kTcGroupSteps + sub) * (kStepBytes >> 4));
-          // two K chunks per instruction (see TcDim for which chunks of A meet which chunks of B)
-          const uint32_t d = tmem_base + buf * 256 + q * 128;
+      uint64_t u = blockIdx.x;
+      uint32_t it = 0, unit_i = 0, left = 0;  // steps issued; units begun; steps left in the unit
+      uint32_t s = 0, stage_par = 0;          // codebook stage of the trip and the parity of its barrier
+      while (it < total && alive) {
+        alive = wait_all(smem_u32(&sm.full_bar[s]), stage_par);
+        const uint64_t b_s = b_desc0 + (uint64_t)(s * kTcGroupSteps * (kStepBytes >> 4));
 #pragma unroll
-          for (int m = 0; m < D::kMmas; ++m)
-            umma_f16(d, a_desc + (uint64_t)(D::a_chunk(m) * (128 >> 4)), b_desc + (uint64_t)(D::b_chunk(m) * (128 >> 4)),
-                     kIdesc, m > 0);
-          umma_commit(buf ? full1 : full0);  // the accumulator is ready
-          if (sub == (uint32_t)kTcGroupSteps - 1 && it + 1 < total)
-            umma_commit(smem_u32(&sm.empty_bar[s]));  // this warp has read the whole stage
+        for (int sub = 0; sub < kTcGroupSteps; ++sub) {
+          if (it < total && alive) {
+            if (left == 0) {  // the next unit begins: its A rows must be in place
+              uint32_t s_lo, s_hi;
+              slice_units(p, (uint32_t)(u % p.n_slices), &s_lo, &s_hi);
+              left = s_hi - s_lo;
+              u += gridDim.x;
+              alive = wait_all(a_ready, unit_i & 1);
+              ++unit_i;
+            }
+            // step 4 g + sub uses buffer sub & 1, for the (2 g + sub / 2)-th time
+            if (alive) alive = wait_all((sub & 1) ? empty1 : empty0, sub < 2 ? 1u : 0u);
+            if (alive) {
+              tc_fence_after();
+              if (lane == 0) {
+                // two K chunks per instruction (see TcDim for which chunks of A meet which chunks of B)
+#pragma unroll
+                for (int m = 0; m < D::kMmas; ++m)
+                  umma_f16((sub & 1) ? d1 : d0, a_desc[m],
+                           b_s + (uint64_t)(sub * (kStepBytes >> 4) + D::b_chunk(m) * (128 >> 4)), kIdesc, m > 0);
+                umma_commit((sub & 1) ? full1 : full0);  // the accumulator is ready
+              }
+              __syncwarp();
+              ++it;
+              --left;
+            }
+          }
         }
+        // this warp has read the whole stage (the last stage is not reused)
+        if (alive && it < total && lane == 0) umma_commit(smem_u32(&sm.empty_bar[s]));
+        __syncwarp();
+        s = (s == (uint32_t)kTcStages - 1) ? 0 : s + 1;
+        if (s == 0) stage_par ^= 1;
       }
-      if (!alive) {
+      if (!alive && lane == 0) {
         // wait (bounded) for whatever was issued before tensor memory is released
         umma_commit(smem_u32(&sm.drain_bar[q]));
         for (uint32_t spin = 0; spin < kMaxSpins; ++spin) {  // always the full limit: these MMAs do complete
@@ -549,10 +598,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
                            4.76837158203125e-7f /* 2^-21 */ * cnmax + 1e-30f;
       float best = kNegInf, thr = kNegInf;
 
-      // Software-pipelined epilogue.  The 128 columns of a step are read as two halves into
-      // two register sets; the first half of step i+1 is requested (if its MMAs are done)
-      // before the maximum of the second half of step i is computed, and a buffer goes back
-      // to the MMA warp as soon as both halves are in registers.
+      // Software-pipelined epilogue.  The 128 columns of a step are read as two halves into two register sets, and
+      // nothing that has to wait for a result is asked for right after it was requested: the second half is
+      // requested before the maxima of the first, the barrier of the next step is tested (without blocking) before
+      // those maxima and the answer used after them, and a maximum is compared with the threshold one half later,
+      // together with its successor.  A buffer goes back to the MMA warp as soon as both halves are in registers.
       uint32_t v[64], w[64];
       bool pending = false;  // the first half of step `st` is already in flight
       // the list of remembered sub-chunks lives in shared memory, its fill count and the largest evicted maximum
@@ -570,6 +620,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
           thr = best - margin;
         }
       };
+      float mx_prev = kNegInf;  // maximum of the previous step's second half, not yet compared
+      uint32_t sub_prev = 0;
       for (uint32_t st = s_lo; st < s_hi; ++st, ++it) {
         const uint32_t buf = it & 1;
         const uint32_t taddr = tmem_base + lane_base + buf * 256 + rb * 128;
@@ -585,24 +637,30 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
         }
         tmem_ld_wait(v);
         tmem_ld64(taddr + 64, w);
-        note(max64(v), 2 * st);
+        const uint32_t nbuf = (it + 1) & 1;
+        uint32_t early = 0;  // is the next step's accumulator complete?  asked now, looked at after the maxima
+        if (st + 1 < s_hi)
+          early = mbar_test_wait_lane0(smem_u32(&sm.tmem_full[nbuf][rb]), ((it + 1) >> 1) & 1, (uint32_t)lane);
+        const float mv = max64(v);
         tmem_ld_wait(w);
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&sm.tmem_empty[buf][rb]));
         pending = false;
-        if (st + 1 < s_hi) {
-          const uint32_t nbuf = (it + 1) & 1;
-          bool ready = false;
-          if (lane == 0) ready = mbar_try_wait(smem_u32(&sm.tmem_full[nbuf][rb]), ((it + 1) >> 1) & 1);
-          if (__shfl_sync(0xffffffffu, ready, 0)) {
-            tc_fence_after();
-            tmem_ld64(tmem_base + lane_base + nbuf * 256 + rb * 128, v);
-            pending = true;
-          }
+        if (__any_sync(0xffffffffu, early != 0)) {
+          tc_fence_after();
+          tmem_ld64(tmem_base + lane_base + nbuf * 256 + rb * 128, v);
+          pending = true;
         }
-        note(max64(w), 2 * st + 1);
+        const float mw = max64(w);
+        if (fmaxf(mx_prev, mv) >= thr) {
+          note(mx_prev, sub_prev);
+          note(mv, 2 * st);
+        }
+        mx_prev = mw;
+        sub_prev = 2 * st + 1;
       }
+      if (alive) note(mx_prev, sub_prev);
 
       // leave the candidates of this (tile, slice) for the rescoring kernel (minimum convention: -S)
       if (alive && have) {
