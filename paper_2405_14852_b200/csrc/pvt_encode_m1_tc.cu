@@ -293,22 +293,18 @@ __device__ __forceinline__ void tmem_ld_wait(uint32_t* v) {
                : "memory");
 }
 
-// non-blocking test of a phase by lane 0 alone, without a branch (the other lanes get 0); try_wait may suspend the
-// thread for a while when the phase is not complete, test_wait does not
-__device__ __forceinline__ uint32_t mbar_test_wait_lane0(uint32_t bar, uint32_t parity, uint32_t lane) {
+// non-blocking test of a phase (try_wait may suspend the thread for a while when the phase is not complete)
+__device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
-      "{\n\t.reg .pred p, q;\n\t"
-      "setp.eq.u32 q, %3, 0;\n\t"
-      "setp.ne.u32 p, %3, %3;\n\t"
-      "@q mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(bar), "r"(parity), "r"(lane)
+      : "r"(bar), "r"(parity)
       : "memory");
   return ok;
 }
-
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float d;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -628,10 +624,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
         if (!pending) {
           // one lane polls (256 threads polling one barrier slow every barrier operation of the CTA
           // down); the warp-wide exchange orders the other lanes after its observation
-          bool ok = true;
-          if (lane == 0) ok = mbar_wait(smem_u32(&sm.tmem_full[buf][rb]), (it >> 1) & 1, abort_flag, p.status, p.max_spins);
-          alive = __shfl_sync(0xffffffffu, ok, 0);
-          if (!alive) break;
+          const uint32_t fbar = smem_u32(&sm.tmem_full[buf][rb]), fpar = (it >> 1) & 1;
+          if (!__all_sync(0xffffffffu, mbar_try_wait(fbar, fpar))) {
+            bool ok = true;
+            if (lane == 0) ok = mbar_wait(fbar, fpar, abort_flag, p.status, p.max_spins);
+            alive = __shfl_sync(0xffffffffu, ok, 0);
+            if (!alive) break;
+          }
           tc_fence_after();
           tmem_ld64(taddr, v);
         }
@@ -640,14 +639,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
         const uint32_t nbuf = (it + 1) & 1;
         uint32_t early = 0;  // is the next step's accumulator complete?  asked now, looked at after the maxima
         if (st + 1 < s_hi)
-          early = mbar_test_wait_lane0(smem_u32(&sm.tmem_full[nbuf][rb]), ((it + 1) >> 1) & 1, (uint32_t)lane);
+          early = mbar_test_wait(smem_u32(&sm.tmem_full[nbuf][rb]), ((it + 1) >> 1) & 1);
         const float mv = max64(v);
         tmem_ld_wait(w);
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&sm.tmem_empty[buf][rb]));
         pending = false;
-        if (__any_sync(0xffffffffu, early != 0)) {
+        if (__all_sync(0xffffffffu, early != 0)) {
           tc_fence_after();
           tmem_ld64(tmem_base + lane_base + nbuf * 256 + rb * 128, v);
           pending = true;
