@@ -33,13 +33,17 @@
 // SM, persistent over (tile, slice) units.  Warps 0-7: own one target per thread,
 // build A, run the epilogue (warp w reads tensor-memory lanes 32 (w % 4) .. of the
 // accumulator of A block w / 4).  Warp 8: bulk-copy producer (stages of four steps).
-// Warps 9 and 10: one thread each issues the MMAs of one A block, warp 9 also
-// allocates tensor memory.  Tensor memory: 2 buffers x 2 accumulators x 128 columns =
-// 512 columns, so the MMAs of step i+1 overlap the epilogue of step i.  The pace is set
-// by the hand-over ring of an accumulator buffer (issue -> execute -> completion seen ->
-// read out -> release seen) and tensor memory holds only two such buffers; a lone
-// thread pays about 150 cycles per mbarrier wait and 50 per MMA or commit, so the
-// issuing threads do as little as possible per step.
+// Warps 9 and 10: each runs the issue loop of one A block as a whole warp (so that
+// descriptors and addresses are warp-uniform values) with one lane issuing the MMAs;
+// warp 9 also allocates tensor memory.  Tensor memory: 2 buffers x 2 accumulators x
+// 128 columns = 512 columns, so the MMAs of step i+1 overlap the epilogue of step i.
+// The pace is set by fixed costs per hand-over of an accumulator (issue -> execute ->
+// completion seen -> read out -> release seen), not by a pipe: a wait on an mbarrier
+// costs 100-150 cycles even on a finished phase, an MMA or a commit about 50, a
+// tensor-memory load about 100 while MMAs are writing, and a thread that runs alone
+// in divergent code pays several cycles per dependent instruction.  Hence: converged
+// issue loops with constant parities and offsets, every result asked for well before
+// it is used, and as few barrier operations per step as possible.
 //
 // Codewords whose half squared norm exceeds the fp16 range get a sentinel row
 // that can never win and are listed as "exceptions": the rescoring kernel always
@@ -364,7 +368,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
     for (int b = 0; b < 2; ++b) {
       for (int q = 0; q < 2; ++q) {
         mbar_init(smem_u32(&sm.tmem_full[b][q]), 1);
-        mbar_init(smem_u32(&sm.tmem_empty[b][q]), kTcEpiThreads / 64);  // the four warps of the block
+        mbar_init(smem_u32(&sm.tmem_empty[b][q]), kTcEpiThreads / 2);  // every thread of the block's four warps
       }
     }
     mbar_init(smem_u32(&sm.a_ready), kTcEpiThreads);
@@ -643,8 +647,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
         const float mv = max64(v);
         tmem_ld_wait(w);
         tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&sm.tmem_empty[buf][rb]));
+        mbar_arrive(smem_u32(&sm.tmem_empty[buf][rb]));
         pending = false;
         if (__all_sync(0xffffffffu, early != 0)) {
           tc_fence_after();
