@@ -32,7 +32,7 @@
 // CTA = 256 targets (two 128-row A blocks) x a slice of the codebook, one CTA per
 // SM, persistent over (tile, slice) units.  Warps 0-7: own one target per thread,
 // build A, run the epilogue (warp w reads tensor-memory lanes 32 (w % 4) .. of the
-// accumulator of A block w / 4).  Warp 8: bulk-copy producer (stages of four steps).
+// accumulator of A block w / 4).  Warp 8: bulk-copy producer (two stages of eight steps).
 // Warps 9 and 10: each runs the issue loop of one A block as a whole warp (so that
 // descriptors and addresses are warp-uniform values) with one lane issuing the MMAs;
 // warp 9 also allocates tensor memory.  Tensor memory: 2 buffers x 2 accumulators x
@@ -88,8 +88,8 @@ struct TcDim {
 };
 constexpr int kTcStepBytes = TcDim<8>::kStepBytes;
 constexpr int kTcSubCw = 64;            // tracking granularity of the running maximum
-constexpr int kTcGroupSteps = 4;        // steps per codebook stage: the MMA threads wait for the codebook once per four steps
-constexpr int kTcStages = 3;            // codebook stages (four steps each: 16 KB, or 32 KB for groups of 16)
+constexpr int kTcGroupSteps = 8;        // steps per codebook stage: the MMA warps wait for the codebook once per eight steps
+constexpr int kTcStages = 2;            // codebook stages (eight steps each: 32 KB, or 64 KB for groups of 16)
 constexpr int kTcEpiThreads = 256;
 constexpr int kTcThreads = kTcEpiThreads + 96;  // + producer warp + one MMA warp per A block
 constexpr uint32_t kTmemCols = 512;
@@ -437,7 +437,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
     // computed once per warp in converged code; one lane issues.  A thread on its own runs one dependent instruction
     // after the other at several cycles each, a wait costs 100-150 cycles even on a finished phase and an MMA or a
     // commit about 50, and the loop is part of the hand-over ring of the accumulators.  So it is kept to the bare
-    // sequence: a codebook stage (four steps) is one trip, its steps are unrolled with constant buffer numbers,
+    // sequence: a codebook stage (eight steps) is one trip, its steps are unrolled with constant buffer numbers,
     // parities and descriptor offsets, and a wait that is already over costs a single poll.
     {
       const uint32_t q = (uint32_t)warp - 9u;
@@ -482,8 +482,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
               alive = wait_all(a_ready, unit_i & 1);
               ++unit_i;
             }
-            // step 4 g + sub uses buffer sub & 1, for the (2 g + sub / 2)-th time
-            if (alive) alive = wait_all((sub & 1) ? empty1 : empty0, sub < 2 ? 1u : 0u);
+            // step 8 g + sub uses buffer sub & 1, for the (4 g + sub / 2)-th time
+            if (alive) alive = wait_all((sub & 1) ? empty1 : empty0, ((sub >> 1) & 1) ? 0u : 1u);
             if (alive) {
               tc_fence_after();
               if (lane == 0) {
