@@ -348,6 +348,8 @@ struct TcSmem {
   uint32_t abort_flag;
 };
 
+// (The bound is the launch size itself: with 384 the register limit drops from 184 to 168, which the epilogue loop
+// needs in full, and the same source runs 18 % slower.)
 template <int DG>
 __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1Params p,
                                                                       const unsigned char* __restrict__ bimg,
@@ -389,7 +391,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
 
   if (warp == 8) {
     // ------------------------------------------------------------ bulk-copy producer
-    if (lane == 0) {
+    // (the whole warp runs the loop, lane 0 issues the copies: no lane waits at the final barrier meanwhile)
+    {
       // total number of steps of this CTA (for the byte count of the last, partial stage)
       uint32_t total = 0;
       for (uint64_t u = blockIdx.x; u < units; u += gridDim.x) {
@@ -406,18 +409,27 @@ __global__ void __launch_bounds__(kTcThreads, 1) encode_m1_tc_kernel(const EncM1
           const uint32_t grp = it / kTcGroupSteps, sub = it % kTcGroupSteps, s = grp % kTcStages;
           const uint32_t fb = smem_u32(&sm.full_bar[s]);
           if (sub == 0) {
-            if (grp >= (uint32_t)kTcStages)
-              alive = mbar_wait(smem_u32(&sm.empty_bar[s]), ((grp / kTcStages) - 1) & 1, abort_flag, p.status, p.max_spins);
+            if (grp >= (uint32_t)kTcStages) {
+              const uint32_t eb = smem_u32(&sm.empty_bar[s]), ep = ((grp / kTcStages) - 1) & 1;
+              if (!__all_sync(0xffffffffu, mbar_try_wait(eb, ep))) {
+                bool ok = true;
+                if (lane == 0) ok = mbar_wait(eb, ep, abort_flag, p.status, p.max_spins);
+                alive = __shfl_sync(0xffffffffu, ok, 0);
+              }
+            }
             if (!alive) break;
             const uint32_t left = total - it;
-            mbar_expect_tx(fb, (left < (uint32_t)kTcGroupSteps ? left : (uint32_t)kTcGroupSteps) * kStepBytes);
+            if (lane == 0)
+              mbar_expect_tx(fb, (left < (uint32_t)kTcGroupSteps ? left : (uint32_t)kTcGroupSteps) * kStepBytes);
+            __syncwarp();
           }
           // test hook: a step that is never copied leaves its stage's barrier incomplete, so the MMA warps' wait
           // for that stage runs out
-          if (it != p.withhold_copy) bulk_g2s(smem_u32(&sm.b[s][sub][0]), bimg + (size_t)st * kStepBytes, kStepBytes, fb);
+          if (lane == 0 && it != p.withhold_copy)
+            bulk_g2s(smem_u32(&sm.b[s][sub][0]), bimg + (size_t)st * kStepBytes, kStepBytes, fb);
         }
       }
-      if (!alive) {
+      if (!alive && lane == 0) {
         // let every copy that was issued land before the CTA may exit
         const uint32_t groups = (it + kTcGroupSteps - 1) / kTcGroupSteps;
         for (uint32_t back = 1; back <= (uint32_t)kTcStages && back <= groups; ++back) {
